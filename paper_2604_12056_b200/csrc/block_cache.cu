@@ -1,0 +1,248 @@
+// Stage 5 — dense in-block attention and the online-softmax merge (Section 4.3, Section 2.2);
+// stage 6 — cache maintenance (Section 4.3, Section 2.1) and the page summaries (Section 2.3).
+//
+// These stages touch O(B * H * d) data: they are latency-bound, so the kernels are plain fp32
+// CUDA-core code laid out for coalesced global access and conflict-free shared-memory access.
+#include "kernels.h"
+
+namespace losa {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kTokTile = 8;
+
+// One CTA per (token tile, KV head, sequence): K_b, V_b of the KV head staged in shared memory as
+// fp32; one warp per query row: lane = block key for the scores (columns visited in a rotated
+// order so that the 32 lanes hit 32 banks), lane = output column for P V.
+template <typename T, int D>
+__global__ void __launch_bounds__(kThreads)
+block_attn_merge_kernel(const T* __restrict__ q, const T* __restrict__ k_blk, const T* __restrict__ v_blk,
+                        const float* __restrict__ o_p, const float* __restrict__ lse_p,
+                        T* __restrict__ out, float* __restrict__ lse_out, int B, int Hq, int Hkv,
+                        float sm_scale) {
+  extern __shared__ __align__(16) float smem[];
+  float* Ks = smem;                 // [B][D]
+  float* Vs = Ks + B * D;           // [B][D]
+  float* Qs = Vs + B * D;           // [warps][D]
+  const int t0 = blockIdx.x * kTokTile, kh = blockIdx.y, s = blockIdx.z;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int G = Hq / Hkv;
+  for (int idx = tid * 8; idx < B * D; idx += kThreads * 8) {
+    const int t = idx / D, j = idx % D;
+    const size_t src = ((static_cast<size_t>(s) * B + t) * Hkv + kh) * D + j;
+    float a[8], b[8];
+    load8(k_blk + src, a);
+    load8(v_blk + src, b);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { Ks[idx + e] = a[e]; Vs[idx + e] = b[e]; }
+  }
+  __syncthreads();
+  const int ntok = min(kTokTile, B - t0);
+  float* qw = Qs + warp * D;
+  for (int r = warp; r < ntok * G; r += kThreads / 32) {
+    const int tok = t0 + r / G, h = kh * G + r % G;
+    const size_t row = (static_cast<size_t>(s) * B + tok) * Hq + h;
+    __syncwarp();
+    for (int j = lane; j < D; j += 32) qw[j] = to_f32(q[row * D + j]);
+    __syncwarp();
+    float sc[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+      const int t = lane + 32 * u;
+      float dot = 0.f;
+      if (t < B) {
+        const float* kr = Ks + t * D;
+#pragma unroll 8
+        for (int j = 0; j < D; ++j) {
+          const int jj = (j + lane) & (D - 1);
+          dot = fmaf(qw[jj], kr[jj], dot);
+        }
+      }
+      sc[u] = (t < B) ? dot * sm_scale : -INFINITY;
+    }
+    const float M = warp_max(fmaxf(sc[0], sc[1]));
+    float p[2];
+    p[0] = expf(sc[0] - M);
+    p[1] = expf(sc[1] - M);
+    const float sum = warp_sum(p[0] + p[1]);
+    const float Lb = M + logf(sum);
+    float ob[D / 32];
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) ob[c] = 0.f;
+    for (int t = 0; t < B; ++t) {
+      const float pt = __shfl_sync(0xffffffffu, t < 32 ? p[0] : p[1], t & 31);
+#pragma unroll
+      for (int c = 0; c < D / 32; ++c) ob[c] = fmaf(pt, Vs[t * D + lane + 32 * c], ob[c]);
+    }
+    const float Lp = lse_p[row];
+    const float M2 = fmaxf(Lp, Lb);
+    const float L = M2 + logf(expf(Lp - M2) + expf(Lb - M2));
+    const float wp = expf(Lp - L), wb = expf(Lb - L) / sum;
+#pragma unroll
+    for (int c = 0; c < D / 32; ++c) {
+      const int j = lane + 32 * c;
+      const float v = (wp > 0.f ? wp * o_p[row * D + j] : 0.f) + wb * ob[c];
+      out[row * D + j] = from_f32<T>(v);
+    }
+    if (lse_out && lane == 0) lse_out[row] = L;
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+commit_step_kernel(const uint4* __restrict__ q, uint4* __restrict__ q_prev, size_t n_vec,
+                   int32_t* __restrict__ step, int N) {
+  for (size_t i = blockIdx.x * static_cast<size_t>(kThreads) + threadIdx.x; i < n_vec;
+       i += static_cast<size_t>(gridDim.x) * kThreads)
+    q_prev[i] = q[i];
+  if (blockIdx.x == 0 && threadIdx.x < N) step[threadIdx.x] += 1;
+}
+
+// min / max of column j of logical page p over its valid tokens; tokens at prefix positions >=
+// new_from are taken from the block being appended (k_blk) instead of the pool.
+template <typename T>
+__device__ __forceinline__ void summarise_column(const T* __restrict__ k_pages, const T* __restrict__ k_blk,
+                                                 T* __restrict__ kmin, T* __restrict__ kmax,
+                                                 size_t page_off, int64_t stride_tok, int valid,
+                                                 int page_start, int new_from, size_t blk_off,
+                                                 int blk_stride, size_t sum_off, int j) {
+  float lo = INFINITY, hi = -INFINITY;
+  for (int t = 0; t < valid; ++t) {
+    const int pos = page_start + t;
+    const float v = (pos >= new_from)
+                        ? to_f32(k_blk[blk_off + static_cast<size_t>(pos - new_from) * blk_stride + j])
+                        : to_f32(k_pages[page_off + static_cast<size_t>(t) * stride_tok + j]);
+    lo = fminf(lo, v);
+    hi = fmaxf(hi, v);
+  }
+  kmin[sum_off + j] = from_f32<T>(lo);
+  kmax[sum_off + j] = from_f32<T>(hi);
+}
+
+template <typename T>
+__global__ void build_summaries_kernel(const T* __restrict__ k_pages, T* __restrict__ kmin,
+                                       T* __restrict__ kmax, const int32_t* __restrict__ page_table,
+                                       const int32_t* __restrict__ kv_len, int64_t stride_page,
+                                       int64_t stride_head, int64_t stride_tok, int Hkv, int D, int g,
+                                       int Pmax, int n_phys, int32_t* __restrict__ status) {
+  const int p = blockIdx.x, kh = blockIdx.y, s = blockIdx.z, j = threadIdx.x;
+  const int len = kv_len[s];
+  const int valid = min(g, len - p * g);
+  if (valid <= 0) return;
+  const int phys = page_table[static_cast<size_t>(s) * Pmax + p];
+  if (phys < 0 || phys >= n_phys) { set_status(status, LOSA_ERR_BOUNDS); return; }
+  summarise_column<T>(k_pages, nullptr, kmin, kmax,
+                      static_cast<size_t>(phys) * stride_page + static_cast<size_t>(kh) * stride_head,
+                      stride_tok, valid, p * g, INT_MAX, 0, 0,
+                      (static_cast<size_t>(phys) * Hkv + kh) * D, j);
+}
+
+// Block finalisation: one CTA per (touched page, KV head, sequence) writes the block tokens that
+// fall into the page and recomputes the page's summaries; kv_len / step are bumped by a second
+// kernel so that every CTA here sees the old length.
+template <typename T>
+__global__ void append_block_kernel(T* __restrict__ k_pages, T* __restrict__ v_pages, T* __restrict__ kmin,
+                                    T* __restrict__ kmax, const T* __restrict__ k_blk,
+                                    const T* __restrict__ v_blk, const int32_t* __restrict__ page_table,
+                                    const int32_t* __restrict__ kv_len, int64_t stride_page,
+                                    int64_t stride_head, int64_t stride_tok, int B, int Hkv, int D,
+                                    int g, int Pmax, int n_phys, int32_t* __restrict__ status) {
+  const int kh = blockIdx.y, s = blockIdx.z, j = threadIdx.x;
+  const int L0 = kv_len[s];
+  const int p = L0 / g + blockIdx.x;
+  if (p > (L0 + B - 1) / g) return;
+  if (p >= Pmax) { set_status(status, LOSA_ERR_BOUNDS); return; }
+  const int phys = page_table[static_cast<size_t>(s) * Pmax + p];
+  if (phys < 0 || phys >= n_phys) { set_status(status, LOSA_ERR_BOUNDS); return; }
+  const size_t page_off = static_cast<size_t>(phys) * stride_page + static_cast<size_t>(kh) * stride_head;
+  const size_t blk_off = (static_cast<size_t>(s) * B * Hkv + kh) * D;
+  const int blk_stride = Hkv * D;
+  const int first = max(L0, p * g), last = min(L0 + B, p * g + g);   // prefix positions written here
+  for (int pos = first; pos < last; ++pos) {
+    const size_t dst = page_off + static_cast<size_t>(pos - p * g) * stride_tok + j;
+    const size_t src = blk_off + static_cast<size_t>(pos - L0) * blk_stride + j;
+    k_pages[dst] = k_blk[src];
+    v_pages[dst] = v_blk[src];
+  }
+  summarise_column<T>(k_pages, k_blk, kmin, kmax, page_off, stride_tok, last - p * g, p * g, L0,
+                      blk_off, blk_stride, (static_cast<size_t>(phys) * Hkv + kh) * D, j);
+}
+
+__global__ void finalize_counters_kernel(int32_t* __restrict__ kv_len, int32_t* __restrict__ step, int N, int B) {
+  const int s = threadIdx.x;
+  if (s < N) { kv_len[s] += B; step[s] = 0; }
+}
+
+template <typename T, int D>
+int32_t launch_merge_t(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk,
+                       const losa_state_t* state, void* out, float* lse_out, cudaStream_t st) {
+  const losa_shape_t& sh = c->shape;
+  const size_t smem = (static_cast<size_t>(2) * sh.block_size * D + (kThreads / 32) * D) * sizeof(float);
+  if (smem > 48 * 1024)
+    LOSA_CUDA_TRY(c, cudaFuncSetAttribute(block_attn_merge_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  dim3 grid((sh.block_size + kTokTile - 1) / kTokTile, sh.n_kv_heads, sh.batch);
+  block_attn_merge_kernel<T, D><<<grid, kThreads, smem, st>>>(
+      static_cast<const T*>(q), static_cast<const T*>(k_blk), static_cast<const T*>(v_blk), state->o_p,
+      state->lse_p, static_cast<T*>(out), lse_out, sh.block_size, sh.n_q_heads, sh.n_kv_heads, sh.sm_scale);
+  return after_launch(c);
+}
+
+template <typename T>
+int32_t launch_update_t(losa_ctx* c, losa_kv_t* kv, losa_state_t* state, const void* q,
+                        const void* k_blk, const void* v_blk, int32_t finalize_block, cudaStream_t st) {
+  const losa_shape_t& sh = c->shape;
+  if (!finalize_block) {
+    const size_t n_vec = static_cast<size_t>(sh.batch) * sh.block_size * sh.n_q_heads * sh.head_dim * sizeof(T) / 16;
+    const int blocks = static_cast<int>(std::min<size_t>((n_vec + kThreads - 1) / kThreads, static_cast<size_t>(c->n_sms) * 4));
+    commit_step_kernel<T><<<std::max(blocks, 1), kThreads, 0, st>>>(
+        static_cast<const uint4*>(q), static_cast<uint4*>(state->q_prev), n_vec, state->step, sh.batch);
+    return after_launch(c);
+  }
+  dim3 grid((sh.block_size + sh.page_size - 1) / sh.page_size + 1, sh.n_kv_heads, sh.batch);
+  append_block_kernel<T><<<grid, sh.head_dim, 0, st>>>(
+      static_cast<T*>(kv->k_pages), static_cast<T*>(kv->v_pages), static_cast<T*>(kv->kmin),
+      static_cast<T*>(kv->kmax), static_cast<const T*>(k_blk), static_cast<const T*>(v_blk),
+      kv->page_table, kv->kv_len, kv->stride_page, kv->stride_head, kv->stride_tok, sh.block_size,
+      sh.n_kv_heads, sh.head_dim, sh.page_size, sh.max_pages_per_seq, kv->n_phys_pages, status_ptr(c));
+  int32_t rc = after_launch(c);
+  if (rc != LOSA_OK) return rc;
+  finalize_counters_kernel<<<1, std::max(32, sh.batch), 0, st>>>(kv->kv_len, state->step, sh.batch, sh.block_size);
+  return after_launch(c);
+}
+
+template <typename T>
+int32_t launch_summaries_t(losa_ctx* c, losa_kv_t* kv, cudaStream_t st) {
+  const losa_shape_t& sh = c->shape;
+  if (sh.max_pages_per_seq == 0) return LOSA_OK;
+  dim3 grid(sh.max_pages_per_seq, sh.n_kv_heads, sh.batch);
+  build_summaries_kernel<T><<<grid, sh.head_dim, 0, st>>>(
+      static_cast<const T*>(kv->k_pages), static_cast<T*>(kv->kmin), static_cast<T*>(kv->kmax),
+      kv->page_table, kv->kv_len, kv->stride_page, kv->stride_head, kv->stride_tok, sh.n_kv_heads,
+      sh.head_dim, sh.page_size, sh.max_pages_per_seq, kv->n_phys_pages, status_ptr(c));
+  return after_launch(c);
+}
+
+}  // namespace
+
+int32_t launch_block_attn_merge(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk,
+                                const losa_state_t* state, void* out, float* lse_out_opt, cudaStream_t st) {
+  const bool bf = c->shape.dtype == LOSA_BF16;
+  if (bf && c->shape.head_dim == 128) return launch_merge_t<__nv_bfloat16, 128>(c, q, k_blk, v_blk, state, out, lse_out_opt, st);
+  if (bf) return launch_merge_t<__nv_bfloat16, 64>(c, q, k_blk, v_blk, state, out, lse_out_opt, st);
+  if (c->shape.head_dim == 128) return launch_merge_t<float, 128>(c, q, k_blk, v_blk, state, out, lse_out_opt, st);
+  return launch_merge_t<float, 64>(c, q, k_blk, v_blk, state, out, lse_out_opt, st);
+}
+
+int32_t launch_update_prefix_cache(losa_ctx* c, losa_kv_t* kv, losa_state_t* state, const void* q,
+                                   const void* k_blk, const void* v_blk, int32_t finalize_block, cudaStream_t st) {
+  return c->shape.dtype == LOSA_BF16
+             ? launch_update_t<__nv_bfloat16>(c, kv, state, q, k_blk, v_blk, finalize_block, st)
+             : launch_update_t<float>(c, kv, state, q, k_blk, v_blk, finalize_block, st);
+}
+
+int32_t launch_build_page_summaries(losa_ctx* c, losa_kv_t* kv, cudaStream_t st) {
+  return c->shape.dtype == LOSA_BF16 ? launch_summaries_t<__nv_bfloat16>(c, kv, st)
+                                     : launch_summaries_t<float>(c, kv, st);
+}
+
+}  // namespace losa

@@ -1,0 +1,157 @@
+// Shared device/host helpers of the LoSA CUDA library (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/losa.h"
+
+namespace losa {
+
+// ----------------------------------------------------------------------------- constants
+constexpr int kRowsPerGroup = 128;  // query rows (active token x head of a KV head) one CTA keeps
+constexpr int kMaxSegments = 1024;  // (sequence, KV head, row group) triples per call
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+// ----------------------------------------------------------------------------- context
+// Workspace layout (byte offsets from the caller's buffer, each 256-byte aligned).
+struct WorkspaceLayout {
+  size_t status;     // int32[4]  : device status word (+ padding)
+  size_t counters;   // uint32[N] : arrival counters of select_active (self-resetting)
+  size_t delta;      // double[N*B]
+  size_t scores;     // float[N*B*H_q*score_stride]
+  size_t partials;   // float[n_slots * kRowsPerGroup * (d + 2)]
+  size_t total;
+  int32_t score_stride;  // P_max rounded up to 64
+  int32_t n_slots;       // n_ctas + n_segments
+  int32_t n_ctas;        // CTAs of the split-KV attention kernels (one per SM)
+  int32_t n_row_groups;  // ceil(B*G / kRowsPerGroup)
+  int32_t n_segments;    // N * H_kv * n_row_groups
+};
+
+}  // namespace losa
+
+struct losa_ctx {
+  losa_shape_t shape;
+  losa::WorkspaceLayout lay;
+  char* ws;
+  int device;
+  int n_sms;
+  int max_smem_optin;
+  int32_t last_cuda_error;
+  int64_t launches;
+  // cached TMA descriptors of the K / V pools (opaque 128-byte blobs, see sparse_prefix_attn.cu)
+  alignas(64) unsigned char tmap_k[128];
+  alignas(64) unsigned char tmap_v[128];
+  const void* tmap_key_k;
+  const void* tmap_key_v;
+  int64_t tmap_strides[3];
+  int32_t tmap_n_phys;
+  void* encode_fn;  // cuTensorMapEncodeTiled, resolved through the runtime
+};
+
+namespace losa {
+
+inline int32_t* status_ptr(const losa_ctx* c) { return reinterpret_cast<int32_t*>(c->ws + c->lay.status); }
+
+// Records a CUDA error in the context and maps it to LOSA_ERR_CUDA.
+inline int32_t cuda_fail(losa_ctx* c, cudaError_t e) {
+  c->last_cuda_error = static_cast<int32_t>(e);
+  return LOSA_ERR_CUDA;
+}
+#define LOSA_CUDA_TRY(ctx, expr)                             \
+  do {                                                       \
+    cudaError_t e__ = (expr);                                \
+    if (e__ != cudaSuccess) return ::losa::cuda_fail(ctx, e__); \
+  } while (0)
+
+inline int32_t after_launch(losa_ctx* c, int n = 1) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(c, e);
+  c->launches += n;
+  return LOSA_OK;
+}
+
+// ----------------------------------------------------------------------------- device helpers
+#ifdef __CUDACC__
+
+__device__ __forceinline__ void set_status(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+template <typename T> __device__ __forceinline__ T from_f32(float x);
+template <> __device__ __forceinline__ float from_f32<float>(float x) { return x; }
+template <> __device__ __forceinline__ __nv_bfloat16 from_f32<__nv_bfloat16>(float x) { return __float2bfloat16_rn(x); }
+
+// 8 consecutive elements starting at a 16-byte (bf16) / 32-byte (fp32) aligned address -> fp32.
+__device__ __forceinline__ void load8(const float* p, float (&v)[8]) {
+  const float4 a = *reinterpret_cast<const float4*>(p);
+  const float4 b = *reinterpret_cast<const float4*>(p + 4);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&v)[8]) {
+  const uint4 u = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+__device__ __forceinline__ int pages_of(int len, int g) { return (len + g - 1) / g; }
+
+// ---- balanced split of the flattened (segment, union position) list over the CTAs ------------
+// Segment seg = (s * H_kv + kh) * n_row_groups + rg holds union_count[s, kh] items when its row
+// group has rows, else none.  CTA b owns items [b*T/n, (b+1)*T/n).  The partial result a CTA
+// produces for a segment goes to slot b + seg, which is unique (b and seg never both stay put
+// between consecutive pieces).
+__device__ __forceinline__ int rows_in_group(int n_active, int G, int rg) {
+  const int r = n_active * G - rg * kRowsPerGroup;
+  return r < 0 ? 0 : (r > kRowsPerGroup ? kRowsPerGroup : r);
+}
+__device__ __forceinline__ long long cta_lo(long long T, int b, int n) { return (T * b) / n; }
+
+// Exclusive prefix of segment item counts into pre[0..n_seg] (shared memory), by one warp.
+__device__ __forceinline__ void segment_prefix(int* pre, int n_seg, int n_rg, int H_kv, int G,
+                                               const int32_t* n_active, const int32_t* union_count,
+                                               int B, int lane) {
+  int run = 0;
+  for (int base = 0; base < n_seg; base += 32) {
+    const int seg = base + lane;
+    int c = 0;
+    if (seg < n_seg) {
+      const int rg = seg % n_rg, sk = seg / n_rg, s = sk / H_kv;
+      int na = n_active[s];
+      na = na < 0 ? 0 : (na > B ? B : na);
+      c = rows_in_group(na, G, rg) > 0 ? max(union_count[sk], 0) : 0;
+    }
+    int inc = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
+    }
+    if (seg < n_seg) pre[seg] = run + inc - c;
+    run += __shfl_sync(0xffffffffu, inc, 31);
+  }
+  if (lane == 0) pre[n_seg] = run;
+}
+
+#endif  // __CUDACC__
+
+}  // namespace losa

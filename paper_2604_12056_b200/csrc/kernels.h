@@ -1,0 +1,40 @@
+// Host-side launchers of the stage kernels.  Each enqueues on `st`, validates nothing (the C-ABI
+// layer in api.cu has done so) and returns LOSA_OK or LOSA_ERR_CUDA.
+#pragma once
+#include "common.cuh"
+
+namespace losa {
+
+int32_t launch_select_active(losa_ctx* c, const void* x_cur, const void* x_prev, int32_t row_width,
+                             const int32_t* m_per_seq, const int32_t* step, int32_t* active_idx,
+                             int32_t* n_active, float* delta_opt, cudaStream_t st);
+
+int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
+                                const int32_t* active_idx, const int32_t* n_active,
+                                const int32_t* step, int32_t k, int32_t* topk_pages,
+                                float* topk_scores_opt, cudaStream_t st);
+
+int32_t launch_page_union(losa_ctx* c, const int32_t* topk_pages, const int32_t* active_idx,
+                          const int32_t* n_active, int32_t k, const int32_t* kv_len,
+                          const int32_t* step, int32_t* union_pages, int32_t* union_count,
+                          cudaStream_t st);
+
+int32_t launch_sparse_prefix_attn(losa_ctx* c, const void* q, const losa_kv_t* kv,
+                                  const int32_t* active_idx, const int32_t* n_active,
+                                  const int32_t* union_pages, const int32_t* union_count,
+                                  losa_state_t* state, cudaStream_t st);
+
+int32_t launch_block_attn_merge(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk,
+                                const losa_state_t* state, void* out, float* lse_out_opt,
+                                cudaStream_t st);
+
+int32_t launch_update_prefix_cache(losa_ctx* c, losa_kv_t* kv, losa_state_t* state, const void* q,
+                                   const void* k_blk, const void* v_blk, int32_t finalize_block,
+                                   cudaStream_t st);
+
+int32_t launch_build_page_summaries(losa_ctx* c, losa_kv_t* kv, cudaStream_t st);
+
+// Largest k and page count the top-k kernel's shared memory allows for this context.
+int32_t topk_max_sortable(const losa_ctx* c);
+
+}  // namespace losa

@@ -1,0 +1,290 @@
+// Stages 2 and 3 — QUEST page scores, top-k per active query, union per KV head
+// (Section 2.3, Section 4.2, Section 4.4).
+//
+//   page_scores_kernel : each CTA reads the min/max keys of 64 pages of one (sequence, KV head)
+//                        once and scores them against every active query of that KV head.  A page
+//                        is handled by d/8 lanes: one 16-byte vector of kmin and kmax per lane,
+//                        eight products per lane added left to right, then an xor-butterfly over
+//                        the lanes — exactly the summation order the interface fixes, so the fp32
+//                        result is reproducible bit for bit.
+//   topk_kernel        : one CTA per (sequence, active token, head) sorts 64-bit keys
+//                        (order-preserving score bits, inverted page id) with a shared-memory
+//                        bitonic network; the first k keys are the answer in the required order
+//                        (score descending, page ascending), with no tie handling left to do.
+//   union_kernel       : one CTA per (sequence, KV head) ORs the selected ids into a bitmap and
+//                        emits the set bits in ascending order with a popcount scan.
+#include "kernels.h"
+
+namespace losa {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kPagesPerCta = 64;
+constexpr int kRowTile = 32;
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kThreads)
+page_scores_kernel(const T* __restrict__ q, const T* __restrict__ kmin, const T* __restrict__ kmax,
+                   const int32_t* __restrict__ page_table, const int32_t* __restrict__ kv_len,
+                   const int32_t* __restrict__ active_idx, const int32_t* __restrict__ n_active,
+                   const int32_t* __restrict__ step, float* __restrict__ scores, int B, int Hq, int Hkv,
+                   int g, int Pmax, int n_phys, int score_stride, int32_t* __restrict__ status) {
+  constexpr int LPP = D / 8;            // lanes per page
+  constexpr int GROUPS = kThreads / LPP;
+  const int s = blockIdx.z, kh = blockIdx.y, p0 = blockIdx.x * kPagesPerCta;
+  if (step && step[s] == 0) return;
+  const int P = pages_of(kv_len[s], g);
+  if (p0 >= P) return;
+  int na = n_active[s];
+  na = na < 0 ? 0 : (na > B ? B : na);
+  const int G = Hq / Hkv, rows = na * G;
+  if (rows == 0) return;
+
+  __shared__ __align__(16) T qs[kRowTile * D];
+  __shared__ float sc[kRowTile][kPagesPerCta + 1];
+  const int tid = threadIdx.x;
+  const int grp = tid / LPP, sub = tid % LPP;
+  const int np = min(kPagesPerCta, P - p0);
+
+  for (int r0 = 0; r0 < rows; r0 += kRowTile) {
+    const int nr = min(kRowTile, rows - r0);
+    // stage the queries of this row tile (16-byte chunks)
+    constexpr int CH = 16 / sizeof(T);   // elements per 16 bytes
+    for (int idx = tid; idx < nr * (D / CH); idx += kThreads) {
+      const int r = idx / (D / CH), ch = idx % (D / CH);
+      const int row = r0 + r, a = row / G, gi = row % G;
+      int tok = active_idx[s * B + a];
+      if (tok < 0 || tok >= B) { set_status(status, LOSA_ERR_BOUNDS); tok = 0; }
+      const T* src = q + ((static_cast<size_t>(s) * B + tok) * Hq + kh * G + gi) * D + ch * CH;
+      *reinterpret_cast<uint4*>(&qs[r * D + ch * CH]) = *reinterpret_cast<const uint4*>(src);
+    }
+    __syncthreads();
+    // the trip count is the same for every lane: the butterfly below needs whole warps
+    for (int pbase = 0; pbase < np; pbase += GROUPS) {
+      const int pl = pbase + grp;
+      const bool ok = pl < np;
+      float lo[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, hi[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+      if (ok) {
+        int phys = page_table[static_cast<size_t>(s) * Pmax + p0 + pl];
+        if (phys < 0 || phys >= n_phys) { set_status(status, LOSA_ERR_BOUNDS); phys = 0; }
+        const size_t so = (static_cast<size_t>(phys) * Hkv + kh) * D + sub * 8;
+        load8(kmin + so, lo);
+        load8(kmax + so, hi);
+      }
+      for (int r = 0; r < nr; ++r) {
+        float qv[8];
+        load8(&qs[r * D + sub * 8], qv);
+        float acc = fmaxf(__fmul_rn(qv[0], lo[0]), __fmul_rn(qv[0], hi[0]));
+#pragma unroll
+        for (int j = 1; j < 8; ++j)
+          acc = __fadd_rn(acc, fmaxf(__fmul_rn(qv[j], lo[j]), __fmul_rn(qv[j], hi[j])));
+#pragma unroll
+        for (int off = LPP / 2; off >= 1; off >>= 1)
+          acc = __fadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
+        if (ok && sub == 0) sc[r][pl] = __fadd_rn(acc, 0.0f);
+      }
+    }
+    __syncthreads();
+    for (int idx = tid; idx < nr * kPagesPerCta; idx += kThreads) {
+      const int r = idx / kPagesPerCta, pl = idx % kPagesPerCta;
+      if (pl < np) {
+        const int row = r0 + r, a = row / G, gi = row % G;
+        scores[((static_cast<size_t>(s) * B + a) * Hq + kh * G + gi) * score_stride + p0 + pl] = sc[r][pl];
+      }
+    }
+    __syncthreads();
+  }
+}
+
+__device__ __forceinline__ uint32_t order_bits(float x) {
+  const uint32_t b = __float_as_uint(x);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float unorder_bits(uint32_t o) {
+  return __uint_as_float((o & 0x80000000u) ? (o & 0x7fffffffu) : ~o);
+}
+
+__global__ void __launch_bounds__(kThreads)
+topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ kv_len,
+            const int32_t* __restrict__ active_idx, const int32_t* __restrict__ n_active,
+            const int32_t* __restrict__ step, int32_t* __restrict__ topk_pages,
+            float* __restrict__ topk_scores, int B, int Hq, int g, int k, int score_stride,
+            int32_t* __restrict__ status) {
+  extern __shared__ __align__(16) unsigned long long keys[];
+  const int h = blockIdx.x, a = blockIdx.y, s = blockIdx.z;
+  if (step && step[s] == 0) return;
+  int na = n_active[s];
+  na = na > B ? B : na;
+  if (a >= na) return;
+  int tok = active_idx[s * B + a];
+  if (tok < 0 || tok >= B) { set_status(status, LOSA_ERR_BOUNDS); return; }
+  const int P = pages_of(kv_len[s], g);
+  const int tid = threadIdx.x;
+  int n = 2;
+  while (n < P) n <<= 1;
+  const float* sc = scores + ((static_cast<size_t>(s) * B + a) * Hq + h) * score_stride;
+  for (int p = tid; p < n; p += kThreads)
+    keys[p] = (p < P) ? ((static_cast<unsigned long long>(order_bits(sc[p])) << 32) |
+                         static_cast<unsigned long long>(0xffffffffu - static_cast<uint32_t>(p)))
+                      : 0ull;
+  __syncthreads();
+  // bitonic network, descending
+  for (int k2 = 2; k2 <= n; k2 <<= 1) {
+    for (int j = k2 >> 1; j > 0; j >>= 1) {
+      for (int t = tid; t < (n >> 1); t += kThreads) {
+        const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+        const int x = i | j;
+        const unsigned long long ka = keys[i], kb = keys[x];
+        const bool desc = (i & k2) == 0;
+        if ((ka < kb) == desc) { keys[i] = kb; keys[x] = ka; }
+      }
+      __syncthreads();
+    }
+  }
+  const size_t o = ((static_cast<size_t>(s) * B + tok) * Hq + h) * k;
+  for (int j = tid; j < k; j += kThreads) {
+    if (j < P) {
+      const unsigned long long key = keys[j];
+      topk_pages[o + j] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(key));
+      if (topk_scores) topk_scores[o + j] = unorder_bits(static_cast<uint32_t>(key >> 32));
+    } else {
+      topk_pages[o + j] = -1;
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kThreads)
+union_kernel(const int32_t* __restrict__ topk_pages, const int32_t* __restrict__ active_idx,
+             const int32_t* __restrict__ n_active, const int32_t* __restrict__ kv_len,
+             const int32_t* __restrict__ step, int32_t* __restrict__ union_pages,
+             int32_t* __restrict__ union_count, int B, int Hq, int Hkv, int g, int k, int Pmax,
+             int32_t* __restrict__ status) {
+  extern __shared__ uint32_t bitmap[];
+  __shared__ int s_warp[kThreads / 32];
+  const int kh = blockIdx.x, s = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int P = min(pages_of(kv_len[s], g), Pmax);
+  const int W = (Pmax + 31) / 32;
+  const int G = Hq / Hkv;
+  const bool all = step && step[s] == 0;
+  for (int w = tid; w < W; w += kThreads) {
+    uint32_t v = 0;
+    if (all) {
+      const int lo = w * 32;
+      v = (P >= lo + 32) ? 0xffffffffu : (P > lo ? ((1u << (P - lo)) - 1u) : 0u);
+    }
+    bitmap[w] = v;
+  }
+  __syncthreads();
+  if (!all) {
+    int na = n_active[s];
+    na = na < 0 ? 0 : (na > B ? B : na);
+    const int per_tok = G * k;
+    for (int idx = tid; idx < na * per_tok; idx += kThreads) {
+      const int a = idx / per_tok, rem = idx % per_tok, gi = rem / k, j = rem % k;
+      const int tok = active_idx[s * B + a];
+      if (tok < 0 || tok >= B) { set_status(status, LOSA_ERR_BOUNDS); continue; }
+      const int p = topk_pages[((static_cast<size_t>(s) * B + tok) * Hq + kh * G + gi) * k + j];
+      if (p < 0) continue;
+      if (p >= P) { set_status(status, LOSA_ERR_BOUNDS); continue; }
+      atomicOr(&bitmap[p >> 5], 1u << (p & 31));
+    }
+    __syncthreads();
+  }
+  // each thread owns a contiguous run of words; exclusive scan of the per-thread popcounts
+  const int per = (W + kThreads - 1) / kThreads;
+  const int w0 = tid * per, w1 = min(W, w0 + per);
+  int cnt = 0;
+  for (int w = w0; w < w1; ++w) cnt += __popc(bitmap[w]);
+  int inc = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  if (lane == 31) s_warp[warp] = inc;
+  __syncthreads();
+  int base = 0, total = 0;
+#pragma unroll
+  for (int w = 0; w < kThreads / 32; ++w) {
+    if (w < warp) base += s_warp[w];
+    total += s_warp[w];
+  }
+  int pos = base + inc - cnt;
+  int32_t* out = union_pages + (static_cast<size_t>(s) * Hkv + kh) * Pmax;
+  for (int w = w0; w < w1; ++w) {
+    uint32_t v = bitmap[w];
+    while (v) {
+      const int b = __ffs(v) - 1;
+      v &= v - 1;
+      out[pos++] = w * 32 + b;
+    }
+  }
+  for (int t = total + tid; t < Pmax; t += kThreads) out[t] = -1;
+  if (tid == 0) union_count[s * Hkv + kh] = total;
+}
+
+template <typename T, int D>
+void launch_scores(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
+                   const int32_t* n_active, const int32_t* step, cudaStream_t st) {
+  const losa_shape_t& sh = c->shape;
+  dim3 grid((sh.max_pages_per_seq + kPagesPerCta - 1) / kPagesPerCta, sh.n_kv_heads, sh.batch);
+  page_scores_kernel<T, D><<<grid, kThreads, 0, st>>>(
+      static_cast<const T*>(q), static_cast<const T*>(kv->kmin), static_cast<const T*>(kv->kmax),
+      kv->page_table, kv->kv_len, active_idx, n_active, step,
+      reinterpret_cast<float*>(c->ws + c->lay.scores), sh.block_size, sh.n_q_heads, sh.n_kv_heads,
+      sh.page_size, sh.max_pages_per_seq, kv->n_phys_pages, c->lay.score_stride, status_ptr(c));
+}
+
+int pow2_at_least(int x) {
+  int n = 2;
+  while (n < x) n <<= 1;
+  return n;
+}
+
+}  // namespace
+
+int32_t topk_max_sortable(const losa_ctx* c) {
+  int n = 2;
+  while (static_cast<size_t>(n) * 2 * sizeof(unsigned long long) <= static_cast<size_t>(c->max_smem_optin)) n <<= 1;
+  return n;
+}
+
+int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
+                                const int32_t* active_idx, const int32_t* n_active,
+                                const int32_t* step, int32_t k, int32_t* topk_pages,
+                                float* topk_scores_opt, cudaStream_t st) {
+  const losa_shape_t& sh = c->shape;
+  if (sh.max_pages_per_seq == 0) return LOSA_OK;
+  const bool bf = sh.dtype == LOSA_BF16;
+  if (bf && sh.head_dim == 128) launch_scores<__nv_bfloat16, 128>(c, q, kv, active_idx, n_active, step, st);
+  else if (bf) launch_scores<__nv_bfloat16, 64>(c, q, kv, active_idx, n_active, step, st);
+  else if (sh.head_dim == 128) launch_scores<float, 128>(c, q, kv, active_idx, n_active, step, st);
+  else launch_scores<float, 64>(c, q, kv, active_idx, n_active, step, st);
+  int32_t rc = after_launch(c);
+  if (rc != LOSA_OK) return rc;
+
+  const size_t smem = static_cast<size_t>(pow2_at_least(sh.max_pages_per_seq)) * sizeof(unsigned long long);
+  if (smem > 48 * 1024)
+    LOSA_CUDA_TRY(c, cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  dim3 grid(sh.n_q_heads, sh.block_size, sh.batch);
+  topk_kernel<<<grid, kThreads, smem, st>>>(reinterpret_cast<const float*>(c->ws + c->lay.scores),
+                                            kv->kv_len, active_idx, n_active, step, topk_pages,
+                                            topk_scores_opt, sh.block_size, sh.n_q_heads, sh.page_size,
+                                            k, c->lay.score_stride, status_ptr(c));
+  return after_launch(c);
+}
+
+int32_t launch_page_union(losa_ctx* c, const int32_t* topk_pages, const int32_t* active_idx,
+                          const int32_t* n_active, int32_t k, const int32_t* kv_len,
+                          const int32_t* step, int32_t* union_pages, int32_t* union_count,
+                          cudaStream_t st) {
+  const losa_shape_t& sh = c->shape;
+  const size_t smem = static_cast<size_t>((sh.max_pages_per_seq + 31) / 32 + 1) * sizeof(uint32_t);
+  dim3 grid(sh.n_kv_heads, sh.batch);
+  union_kernel<<<grid, kThreads, smem, st>>>(topk_pages, active_idx, n_active, kv_len, step, union_pages,
+                                             union_count, sh.block_size, sh.n_q_heads, sh.n_kv_heads,
+                                             sh.page_size, k, sh.max_pages_per_seq, status_ptr(c));
+  return after_launch(c);
+}
+
+}  // namespace losa

@@ -1,0 +1,112 @@
+// Stage 1 — locality score (Eq. 1, Section 3.2) and locality pruning (Section 4.1).
+//
+// One CTA per (token, sequence) streams the token's row of x_cur and x_prev with 16-byte loads and
+// reduces sum (x_cur - x_prev)^2 in fp64 (the selection is an integer decision, so it is taken in
+// fp64 like the definition; the work is a few hundred KB).  The last CTA of a sequence to arrive
+// (self-resetting counter) ranks the B scores by (Delta descending, token ascending) and emits the
+// first m tokens in ascending order.
+#include "kernels.h"
+
+namespace losa {
+namespace {
+
+constexpr int kThreads = 256;
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+select_active_kernel(const T* __restrict__ x_cur, const T* __restrict__ x_prev, int row_width, int B,
+                     const int32_t* __restrict__ m_per_seq, const int32_t* __restrict__ step,
+                     int32_t* __restrict__ active_idx, int32_t* __restrict__ n_active,
+                     float* __restrict__ delta_opt, double* __restrict__ delta_ws,
+                     unsigned int* __restrict__ counters) {
+  const int i = blockIdx.x, s = blockIdx.y;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const size_t row = (static_cast<size_t>(s) * B + i) * row_width;
+  constexpr int kVec = 8;
+  double acc = 0.0;
+  for (int c = tid * kVec; c < row_width; c += kThreads * kVec) {
+    float a[8], b[8];
+    load8(x_cur + row + c, a);
+    load8(x_prev + row + c, b);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const double df = static_cast<double>(a[j]) - static_cast<double>(b[j]);
+      acc = fma(df, df, acc);
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+  __shared__ double s_part[kThreads / 32];
+  __shared__ double s_delta[LOSA_MAX_BLOCK];
+  __shared__ bool s_last;
+  if (lane == 0) s_part[warp] = acc;
+  __syncthreads();
+  if (tid == 0) {
+    double t = 0.0;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) t += s_part[w];
+    t /= static_cast<double>(row_width);
+    delta_ws[s * B + i] = t;
+    if (delta_opt) delta_opt[s * B + i] = static_cast<float>(t);
+    __threadfence();
+    const unsigned int ticket = atomicInc(&counters[s], static_cast<unsigned int>(B - 1));
+    s_last = (ticket == static_cast<unsigned int>(B - 1));
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  if (tid < B) s_delta[tid] = *(reinterpret_cast<volatile double*>(delta_ws) + s * B + tid);
+  __syncthreads();
+  if (warp != 0) return;
+
+  int m = m_per_seq ? m_per_seq[s] : -1;
+  if (m < 0 || m > B || (step && step[s] == 0)) m = B;
+  // token t = lane (+32): active when fewer than m tokens precede it in the ranking
+  bool act[2];
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+    const int t = lane + 32 * half;
+    act[half] = false;
+    if (t < B) {
+      const double dt = s_delta[t];
+      int rank = 0;
+      for (int j = 0; j < B; ++j) {
+        const double dj = s_delta[j];
+        rank += (dj > dt || (dj == dt && j < t)) ? 1 : 0;
+      }
+      act[half] = rank < m;
+    }
+  }
+  const unsigned b0 = __ballot_sync(0xffffffffu, act[0]);
+  const unsigned b1 = __ballot_sync(0xffffffffu, act[1]);
+  const unsigned below = (1u << lane) - 1u;
+  const int n0 = __popc(b0), n1 = __popc(b1);
+  int32_t* out = active_idx + static_cast<size_t>(s) * B;
+  if (act[0]) out[__popc(b0 & below)] = lane;
+  if (act[1]) out[n0 + __popc(b1 & below)] = lane + 32;
+  for (int t = n0 + n1 + lane; t < B; t += 32) out[t] = -1;
+  if (lane == 0) n_active[s] = n0 + n1;
+}
+
+}  // namespace
+
+int32_t launch_select_active(losa_ctx* c, const void* x_cur, const void* x_prev, int32_t row_width,
+                             const int32_t* m_per_seq, const int32_t* step, int32_t* active_idx,
+                             int32_t* n_active, float* delta_opt, cudaStream_t st) {
+  const losa_shape_t& sh = c->shape;
+  dim3 grid(sh.block_size, sh.batch);
+  double* dws = reinterpret_cast<double*>(c->ws + c->lay.delta);
+  unsigned int* ctr = reinterpret_cast<unsigned int*>(c->ws + c->lay.counters);
+  if (sh.dtype == LOSA_BF16) {
+    select_active_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(
+        static_cast<const __nv_bfloat16*>(x_cur), static_cast<const __nv_bfloat16*>(x_prev), row_width,
+        sh.block_size, m_per_seq, step, active_idx, n_active, delta_opt, dws, ctr);
+  } else {
+    select_active_kernel<float><<<grid, kThreads, 0, st>>>(
+        static_cast<const float*>(x_cur), static_cast<const float*>(x_prev), row_width, sh.block_size,
+        m_per_seq, step, active_idx, n_active, delta_opt, dws, ctr);
+  }
+  return after_launch(c);
+}
+
+}  // namespace losa

@@ -1,0 +1,171 @@
+"""GPU-vs-oracle parity of every stage, through the C-ABI (needs a B200).
+
+Index outputs (active sets, top-k page lists, unions, counters) must be bit-exact; attention
+outputs within the stated tolerances: fp32 mode |a-b| <= 1e-5 * max(|b|, max|b_row|); bf16 mode
+|a-b| <= 2e-2 + 1e-2 |b|; every LSE within 1e-3.
+"""
+import numpy as np
+import pytest
+
+from helpers import OracleLayer, delta_gap_ok
+from paper_2604_12056_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def assert_close(got, want, dtype, what):
+    got, want = np.asarray(got, np.float64), np.asarray(want, np.float64)
+    if dtype == "f32":
+        row_max = np.abs(want).max(axis=-1, keepdims=True)
+        tol = 1e-5 * np.maximum(np.abs(want), row_max)
+    else:
+        tol = 2e-2 + 1e-2 * np.abs(want)
+    bad = np.abs(got - want) > tol
+    assert not bad.any(), f"{what}: {bad.sum()} of {bad.size} outside tolerance, worst {np.abs(got - want).max():.3e}"
+
+
+def assert_lse_close(got, want, what):
+    got, want = np.asarray(got, np.float64), np.asarray(want, np.float64)
+    inf = np.isinf(want)
+    assert (np.isinf(got) == inf).all() and (got[inf] == want[inf]).all(), what
+    assert (np.abs(got[~inf] - want[~inf]) <= 1e-3).all(), f"{what}: worst {np.abs(got[~inf] - want[~inf]).max():.3e}"
+
+
+def compare(snap, ref, cfg, what):
+    for key in ("act", "na", "topk", "up", "uc"):
+        assert (snap[key] == ref[key]).all(), f"{what}: {key} differs"
+    np.testing.assert_allclose(snap["delta"], ref["delta"], rtol=1e-5, atol=1e-12, err_msg=what)
+    for s in range(cfg.batch):
+        m = int(ref["na"][s])
+        assert delta_gap_ok(ref["delta"][s], m), f"{what}: selection-ambiguous Delta in sequence {s}"
+    assert_close(snap["o_p"], ref["o_p"], cfg.dtype, what + " o_p")
+    assert_lse_close(snap["lse_p"], ref["lse_p"], what + " lse_p")
+    assert_close(snap["out"], ref["out"], cfg.dtype, what + " out")
+    assert_lse_close(snap["lse"], ref["lse"], what + " lse")
+
+
+def run_blocks(cfg, modes=("losa",), m=None, n_blocks=1, pad_nan=True, want_scores=True):
+    """Runs n_blocks blocks through GPU and oracle in lock-step, comparing after every step."""
+    from paper_2604_12056_b200.layer import LosaLayer, to_device
+    w = wl.Workload(cfg, pad_nan=pad_nan)
+    gpu = {md: LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len, md) for md in modes}
+    ora = {md: OracleLayer(w, md) for md in modes}
+    for md in modes:     # page summaries: exact min / max on both sides
+        from paper_2604_12056_b200.layer import to_host
+        P = [(int(L) + cfg.page_size - 1) // cfg.page_size for L in w.kv_len]
+        used = np.concatenate([w.page_table[s, :P[s]] for s in range(cfg.batch)]) if sum(P) else np.zeros(0, np.int64)
+        assert (to_host(gpu[md].kmin)[used] == wl.elem_to_f32(ora[md].kmin)[used]).all()
+        assert (to_host(gpu[md].kmax)[used] == wl.elem_to_f32(ora[md].kmax)[used]).all()
+    for b in range(n_blocks):
+        steps = w.block_steps(m)
+        for t, inp in enumerate(steps):
+            last = t == len(steps) - 1 and n_blocks > 1
+            q, kb, vb = to_device(inp.q), to_device(inp.k_blk), to_device(inp.v_blk)
+            mt = to_device(inp.m_per_seq)
+            for md in modes:
+                g = gpu[md]
+                g.run_step(q, kb, vb, mt, want_scores=want_scores)
+                snap = g.snapshot()
+                assert g.ctx.poll_status() == 0
+                ref = ora[md].run_step(inp, finalize=last)
+                compare(snap, ref, cfg, f"{cfg.name}/{md} block {b} step {t}")
+                if want_scores and md == "losa" and t > 0:
+                    sel = ref["topk"] >= 0
+                    rows = np.zeros_like(sel)
+                    for s in range(cfg.batch):
+                        rows[s, ref["act"][s, :ref["na"][s]]] = True
+                    assert np.isfinite(snap["topk_scores"][sel & rows]).all()
+                if last:
+                    g.finalize_block(kb, vb)
+                    s2 = g.snapshot()
+                    assert (s2["kv_len"] == ora[md].kv_len).all() and (s2["step"] == 0).all()
+                    assert g.ctx.poll_status() == 0
+    return gpu, ora
+
+
+def test_c1_fp32_full_block_all_modes():
+    run_blocks(wl.config("c1"), modes=("losa", "naive", "dense"))
+
+
+def test_c1_hidden_state_selection():
+    from paper_2604_12056_b200.layer import LosaLayer, to_device
+    cfg = wl.config("c1")
+    w = wl.Workload(cfg)
+    steps = w.block_steps()
+    g, o = LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len), OracleLayer(w)
+    args = lambda i: (to_device(i.q), to_device(i.k_blk), to_device(i.v_blk), to_device(i.m_per_seq))
+    g.run_step(*args(steps[0]))
+    o.run_step(steps[0])
+    g.run_step(*args(steps[1]), x_sel=(to_device(steps[1].hidden), to_device(steps[0].hidden)))
+    ref = o.run_step(steps[1], x_sel=(steps[1].hidden, steps[0].hidden))
+    compare(g.snapshot(), ref, cfg, "c1 hidden-state selection")
+    assert ref["act"][0, :4].tolist() == steps[1].planted[0].tolist()
+
+
+def test_c2_reduced_bf16_all_modes():
+    run_blocks(wl.config("c2", kv_lens=(2048,), steps=4), modes=("losa", "naive", "dense"))
+
+
+@pytest.mark.parametrize("g,d,hq,hkv,dtype", [
+    (16, 64, 4, 1, "bf16"), (32, 128, 8, 2, "bf16"), (64, 128, 8, 8, "bf16"), (16, 128, 16, 1, "bf16"),
+    (32, 64, 6, 2, "f32"), (64, 128, 4, 2, "f32"), (16, 128, 2, 2, "f32"),
+])
+def test_ragged_batch_partial_pages_and_empty_prefix(g, d, hq, hkv, dtype):
+    # ragged lengths: a partial last page, an empty prefix, a single token, exact page multiples
+    cfg = wl.config("c2", n_q_heads=hq, n_kv_heads=hkv, head_dim=d, page_size=g, dtype=dtype,
+                    kv_lens=(5 * g + 3, 0, 1, 7 * g), block_size=12, steps=3, topk=3, m_active=2)
+    run_blocks(cfg, modes=("losa", "naive"))
+
+
+@pytest.mark.parametrize("m", [0, 1, 16])
+def test_active_count_extremes(m):
+    cfg = wl.config("c2", kv_lens=(700, 333), block_size=16, steps=3, topk=4, m_active=max(m, 1))
+    run_blocks(cfg, m=m)
+
+
+def test_budget_larger_than_cache_and_shuffled_pages():
+    cfg = wl.config("c2", kv_lens=(150,), block_size=8, steps=3, topk=64, m_active=2)
+    gpu, _ = run_blocks(cfg)
+    assert gpu["losa"].snapshot()["uc"].max() == 5
+
+
+def test_maximum_block_two_row_groups():
+    # B = 64 tokens x 4 heads per KV head = 256 query rows: two row groups per (sequence, KV head)
+    cfg = wl.config("c4", kv_lens=(64 * 40 + 17,), steps=2, topk=8, m_active=40, heavy_frac=0.0)
+    run_blocks(cfg, modes=("losa", "dense"))
+
+
+def test_many_rows_per_kv_head_fp32():
+    cfg = wl.config("c1", n_q_heads=16, n_kv_heads=1, kv_lens=(400,), block_size=16, steps=2, m_active=9)
+    run_blocks(cfg, modes=("losa",))
+
+
+def test_multi_block_append():
+    cfg = wl.config("c5", kv_lens=(200, 90, 64), n_blocks=3, steps=3, topk=4)
+    run_blocks(cfg, n_blocks=3)
+
+
+def test_multi_block_append_fp32_small_pages():
+    cfg = wl.config("c1", kv_lens=(100, 7), n_blocks=2, steps=2, topk=3, m_active=3, block_size=24)
+    run_blocks(cfg, n_blocks=2)
+
+
+def test_out_of_range_page_table_is_reported_not_fatal():
+    from paper_2604_12056_b200 import binding as B
+    from paper_2604_12056_b200.layer import LosaLayer, to_device
+    cfg = wl.config("c2", kv_lens=(256,), block_size=8, steps=2, topk=2, m_active=1)
+    w = wl.Workload(cfg)
+    g = LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len)
+    inp = w.start_block()
+    g.page_table[0, 3] = 10 ** 6          # logical page 3 now names a page outside the pool
+    g.run_step(to_device(inp.q), to_device(inp.k_blk), to_device(inp.v_blk), to_device(inp.m_per_seq))
+    assert g.ctx.poll_status() == B.LOSA_ERR_BOUNDS
+    assert g.ctx.poll_status() == 0       # cleared by the poll; the context stays usable
+    g.page_table[0, 3] = int(w.page_table[0, 3])
+    g.step.zero_()
+    g.run_step(to_device(inp.q), to_device(inp.k_blk), to_device(inp.v_blk), to_device(inp.m_per_seq))
+    assert g.ctx.poll_status() == 0
+    ref = OracleLayer(w).run_step(inp)
+    compare(g.snapshot(), ref, cfg, "after recovery")
+EOF
+echo done
