@@ -219,7 +219,10 @@ class Workload:
         P = u.shape[0]
         pick = rng.integers(0, P, size=(n, Hq, 8))
         kh = np.arange(Hq) // G
-        t = _unit(u[pick, kh[None, :, None]].sum(2))                   # [n, H_q, d]
+        t = u[pick, kh[None, :, None]].sum(2)                          # [n, H_q, d]
+        if P < 8:   # too few pages to make fresh draws differ: add a random direction
+            t = _unit(t) + np.float32(0.5) * _unit(rng.standard_normal((n, Hq, d), dtype=np.float32))
+        t = _unit(t)
         cd = self.common_dir[s][kh][None]                               # [1, H_q, d]
         mix = np.float32(c.rho) * cd + np.float32(np.sqrt(1 - c.rho ** 2)) * t
         return (np.float32(c.tau * np.sqrt(d)) * _unit(mix)).astype(np.float32)

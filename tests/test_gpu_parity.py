@@ -163,9 +163,8 @@ def test_out_of_range_page_table_is_reported_not_fatal():
     assert g.ctx.poll_status() == 0       # cleared by the poll; the context stays usable
     g.page_table[0, 3] = int(w.page_table[0, 3])
     g.step.zero_()
+    g.q_prev.zero_()
     g.run_step(to_device(inp.q), to_device(inp.k_blk), to_device(inp.v_blk), to_device(inp.m_per_seq))
     assert g.ctx.poll_status() == 0
     ref = OracleLayer(w).run_step(inp)
     compare(g.snapshot(), ref, cfg, "after recovery")
-EOF
-echo done
