@@ -132,6 +132,14 @@ int32_t losa_last_cuda_error(const losa_ctx* ctx);
 /* Number of kernels this context has launched so far (host counter, for accounting). */
 int64_t losa_launch_count(const losa_ctx* ctx);
 
+/* Timing aid.  With `enable` != 0 every later losa_sparse_prefix_attn records a pair of CUDA events
+ * (owned by the context) on its stream immediately before and after its main kernel — not around
+ * the small combine kernel that follows.  losa_stage4_last_ms waits for the second event and
+ * returns the time between the two in milliseconds (host pointer).  Do not enable while a stream
+ * capture is in progress. */
+int32_t losa_profile_stage4(losa_ctx* ctx, int32_t enable);
+int32_t losa_stage4_last_ms(losa_ctx* ctx, float* out_ms);
+
 /* Stage 1 — locality score and locality pruning (Eq. 1 in Section 3.2; Section 4.1).
  *   x_cur, x_prev [N, B, row_width] (dtype): the representation whose change is measured, this
  *       step's and the previous step's (queries flattened over heads: row_width = H_q*d; hidden

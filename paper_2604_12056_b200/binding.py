@@ -28,6 +28,7 @@ EXPORTS = [
     "losa_last_cuda_error", "losa_launch_count", "losa_select_active", "losa_page_scores_topk",
     "losa_page_union", "losa_sparse_prefix_attn", "losa_block_attn_merge",
     "losa_update_prefix_cache", "losa_build_page_summaries", "losa_denoise_step_host",
+    "losa_profile_stage4", "losa_stage4_last_ms",
 ]
 
 
@@ -153,6 +154,14 @@ class Context:
 
     def launch_count(self) -> int:
         return int(lib().losa_launch_count(self._h))
+
+    def profile_stage4(self, enable: bool):
+        self._check("losa_profile_stage4", lib().losa_profile_stage4(self._h, C.c_int32(1 if enable else 0)))
+
+    def stage4_last_ms(self) -> float:
+        ms = C.c_float(0.0)
+        self._check("losa_stage4_last_ms", lib().losa_stage4_last_ms(self._h, C.byref(ms)))
+        return float(ms.value)
 
     def poll_status(self) -> int:
         return int(lib().losa_poll_status(self._h, _stream()))

@@ -119,6 +119,8 @@ int32_t losa_create(const losa_shape_t* shape, void* workspace, size_t workspace
 
 int32_t losa_destroy(losa_ctx* ctx) {
   if (!ctx) return LOSA_ERR_INVALID_ARG;
+  if (ctx->ev_begin) cudaEventDestroy(ctx->ev_begin);
+  if (ctx->ev_end) cudaEventDestroy(ctx->ev_end);
   delete ctx;
   return LOSA_OK;
 }
@@ -130,6 +132,23 @@ int32_t losa_poll_status(losa_ctx* ctx, void* stream) {
   LOSA_CUDA_TRY(ctx, cudaMemcpy(&st, status_ptr(ctx), sizeof(st), cudaMemcpyDeviceToHost));
   if (st != 0) LOSA_CUDA_TRY(ctx, cudaMemset(status_ptr(ctx), 0, sizeof(st)));
   return st;
+}
+
+int32_t losa_profile_stage4(losa_ctx* ctx, int32_t enable) {
+  if (!ctx) return LOSA_ERR_INVALID_ARG;
+  if (enable && !ctx->ev_begin) {
+    LOSA_CUDA_TRY(ctx, cudaEventCreate(&ctx->ev_begin));
+    LOSA_CUDA_TRY(ctx, cudaEventCreate(&ctx->ev_end));
+  }
+  ctx->profile = enable ? 1 : 0;
+  return LOSA_OK;
+}
+
+int32_t losa_stage4_last_ms(losa_ctx* ctx, float* out_ms) {
+  if (!ctx || !out_ms || !ctx->ev_begin) return LOSA_ERR_INVALID_ARG;
+  LOSA_CUDA_TRY(ctx, cudaEventSynchronize(ctx->ev_end));
+  LOSA_CUDA_TRY(ctx, cudaEventElapsedTime(out_ms, ctx->ev_begin, ctx->ev_end));
+  return LOSA_OK;
 }
 
 int32_t losa_last_cuda_error(const losa_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }

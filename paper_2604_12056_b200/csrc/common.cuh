@@ -50,6 +50,9 @@ struct losa_ctx {
   int64_t tmap_strides[3];
   int32_t tmap_n_phys;
   void* encode_fn;  // cuTensorMapEncodeTiled, resolved through the runtime
+  // optional timing of the stage-4 main kernel
+  int32_t profile;
+  cudaEvent_t ev_begin, ev_end;
 };
 
 namespace losa {

@@ -648,11 +648,17 @@ template <int D, int GP>
 int32_t launch_mma(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
   constexpr int smem = mma_smem_bytes<D, GP>();
   static_assert(n_stages<D, GP>() >= 3, "ring too shallow");
-  LOSA_CUDA_TRY(c, cudaFuncSetAttribute(attn_mma_kernel<D, GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+  static int attr_device = -1;   // the opt-in is per device and per kernel
+  if (attr_device != c->device) {
+    LOSA_CUDA_TRY(c, cudaFuncSetAttribute(attn_mma_kernel<D, GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    attr_device = c->device;
+  }
   CUtensorMap mk, mv;
   memcpy(&mk, c->tmap_k, sizeof(mk));
   memcpy(&mv, c->tmap_v, sizeof(mv));
+  if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_begin, st));
   attn_mma_kernel<D, GP><<<ap.n_ctas, kMmaThreads, smem, st>>>(mk, mv, ap);
+  if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_end, st));
   int32_t rc = after_launch(c);
   if (rc != LOSA_OK) return rc;
   attn_combine_kernel<D, true><<<dim3(ap.n_seg, kRowsPerGroup / 8), 256, 0, st>>>(ap);
@@ -664,7 +670,9 @@ int32_t launch_simt(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
   const size_t smem = (static_cast<size_t>(2) * GP * D + 2 * kRowsPerGroup * D + 2 * kRowsPerGroup) * sizeof(float) +
                       (ap.n_seg + 1) * sizeof(int);
   LOSA_CUDA_TRY(c, cudaFuncSetAttribute(attn_simt_kernel<T, D, GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_begin, st));
   attn_simt_kernel<T, D, GP><<<ap.n_ctas, 256, smem, st>>>(ap);
+  if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_end, st));
   int32_t rc = after_launch(c);
   if (rc != LOSA_OK) return rc;
   attn_combine_kernel<D, false><<<dim3(ap.n_seg, kRowsPerGroup / 8), 256, 0, st>>>(ap);
