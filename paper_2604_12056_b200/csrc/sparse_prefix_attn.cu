@@ -249,8 +249,8 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+__device__ __forceinline__ void mbar_arrive(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -276,6 +276,21 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
       return false;
     }
   }
+}
+// Bounded wait until the producer has tagged the stage with `round`.
+__device__ __forceinline__ bool wait_round(volatile int* tag, int round, volatile int* abort_flag,
+                                           int32_t* status) {
+  if (*tag == round) return true;
+  const long long t0 = clock64();
+  while (*tag != round) {
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitCycles) {
+      *abort_flag = 1;
+      set_status(status, LOSA_ERR_TIMEOUT);
+      return false;
+    }
+  }
+  return true;
 }
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
                                             int c1, int c2, int c3) {
@@ -333,7 +348,8 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   const uint32_t full0 = qs + q_region_bytes<D>();       // full[NSTAGE], then empty[NSTAGE]
   const uint32_t empty0 = full0 + 8 * NSTAGE;
   volatile int* meta = reinterpret_cast<volatile int*>(tail + 16 * NSTAGE);        // valid tokens per stage
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 16 * NSTAGE + 4 * NSTAGE);
+  volatile int* stage_round = meta + NSTAGE;   // which pass over the ring the stage's current page belongs to
+  volatile int* abort_flag = stage_round + NSTAGE;
   int* pre = reinterpret_cast<int*>(tail + 512);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -341,6 +357,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     for (int i = 0; i < NSTAGE; ++i) {
       mbar_init(full0 + 8 * i, 1);
       mbar_init(empty0 + 8 * i, kConsumerWarps);
+      stage_round[i] = -1;
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -382,6 +399,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
           const bool go = mbar_wait(empty0 + 8 * stage, (round & 1) ^ 1, abort_flag, p.status);
           if (go) {
             meta[stage] = vj;
+            stage_round[stage] = round;
             const uint32_t fb = full0 + 8 * stage, dst = stage0 + stage * STAGE;
             mbar_expect_tx(fb, STAGE);
 #pragma unroll
@@ -440,10 +458,16 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
     for (int n = 0; n < ND; ++n) { oacc[n][0] = oacc[n][1] = oacc[n][2] = oacc[n][3] = 0.f; }
 
-    for (int j = 0; j < npg; ++j) {
+    // Page j of the piece belongs to the warps of page slot j % ns (one warp per row tile).  Only
+    // they wait for it and release it, each with weight ns, so that a stage always collects
+    // kConsumerWarps arrivals and is refilled as soon as ITS readers are done with it.
+    for (int j = slot; j < npg; j += ns) {
       const int it = item + j - lo, stage = it % NSTAGE, round = it / NSTAGE;
-      const bool ready = mbar_wait(full0 + 8 * stage, round & 1, abort_flag, p.status);
-      if (ready && has_rows && (j % ns) == slot) {
+      // A parity wait is only meaningful once the stage is in this item's pass over the ring:
+      // this warp may get here while the stage's previous page is still in flight.
+      const bool ready = wait_round(stage_round + stage, round, abort_flag, p.status) &&
+                         mbar_wait(full0 + 8 * stage, round & 1, abort_flag, p.status);
+      if (ready && has_rows) {
         const int valid = meta[stage];
         const uint32_t kt = stage0 + stage * STAGE, vt = kt + KBYTES;
         if (valid < GP) {
@@ -526,7 +550,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
       }
       __syncwarp();
-      if (lane == 0) mbar_arrive(empty0 + 8 * stage);
+      if (ready && lane == 0) mbar_arrive(empty0 + 8 * stage, static_cast<uint32_t>(ns));
     }
 
     // ---- merge the page slots of each row tile through shared memory (tree), slot 0 keeps it

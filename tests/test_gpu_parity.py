@@ -168,3 +168,48 @@ def test_out_of_range_page_table_is_reported_not_fatal():
     assert g.ctx.poll_status() == 0
     ref = OracleLayer(w).run_step(inp)
     compare(g.snapshot(), ref, cfg, "after recovery")
+
+
+def test_full_size_c3_in_the_benchmark_configuration():
+    """The benchmark's workload (ragged 16K/24K/32K/32K batch, 3 active tokens, top-64 pages) at
+    full size.  Step 0 (dense): index outputs in full, attention on sampled tokens the oracle
+    computes one by one.  Step 1 (LoSA): everything in full — only the active tokens are
+    recomputed, so the oracle finishes in seconds."""
+    from oracle import oracle as orc
+    from paper_2604_12056_b200.layer import LosaLayer, to_device
+    cfg = wl.config("c3")
+    w = wl.Workload(cfg)
+    g = LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len)
+    o = OracleLayer(w)
+    inp0, inp1 = w.start_block(), w.next_step()
+    N, B = cfg.batch, cfg.block_size
+    # ---- step 0
+    g.run_step(to_device(inp0.q), to_device(inp0.k_blk), to_device(inp0.v_blk), to_device(inp0.m_per_seq))
+    s0 = g.snapshot()
+    assert g.ctx.poll_status() == 0
+    sh = o.sh
+    act, na, _ = orc.select_active(sh, inp0.q, o.q_prev, inp0.m_per_seq, o.step)
+    up, uc = orc.page_union(sh, o.topk, act, na, cfg.topk, o.kv_len, o.step)
+    for key, ref in (("act", act), ("na", na), ("up", up), ("uc", uc)):
+        assert (s0[key] == ref).all(), key
+    sample = np.array([0, 13, 31], np.int32)
+    act_s = np.full((N, B), -1, np.int32)
+    act_s[:, :3] = sample
+    o.o_p[:] = s0["o_p"]
+    o.lse_p[:] = s0["lse_p"]
+    orc.sparse_prefix_attn(sh, inp0.q, o.kv, act_s, np.full(N, 3, np.int32), up, uc, o.o_p, o.lse_p)
+    assert_close(s0["o_p"][:, sample], o.o_p[:, sample], cfg.dtype, "step 0 sampled o_p")
+    assert_lse_close(s0["lse_p"][:, sample], o.lse_p[:, sample], "step 0 sampled lse_p")
+    out, lse = orc.block_attn_merge(sh, inp0.q, inp0.k_blk, inp0.v_blk, o.o_p, o.lse_p)
+    assert_close(s0["out"], out, cfg.dtype, "step 0 out")
+    assert_lse_close(s0["lse"], lse, "step 0 lse")
+    orc.update_prefix_cache(sh, o.kv, o.q_prev, o.step, inp0.q, inp0.k_blk, inp0.v_blk, False)
+    # ---- step 1: the oracle state now holds GPU values for the non-sampled tokens (within tolerance)
+    g.run_step(to_device(inp1.q), to_device(inp1.k_blk), to_device(inp1.v_blk), to_device(inp1.m_per_seq))
+    s1 = g.snapshot()
+    assert g.ctx.poll_status() == 0
+    ref = o.run_step(inp1)
+    for s in range(N):
+        assert ref["act"][s, :3].tolist() == inp1.planted[s].tolist()
+    compare(s1, ref, cfg, "c3 full size, LoSA step")
+    assert 8 * 64 <= ref["uc"].sum() < 26624 // 2
