@@ -9,11 +9,14 @@ namespace losa {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kTokTile = 8;
+constexpr int kTokTile = 2;
 
-// One CTA per (token tile, KV head, sequence): K_b, V_b of the KV head staged in shared memory as
-// fp32; one warp per query row: lane = block key for the scores (columns visited in a rotated
-// order so that the 32 lanes hit 32 banks), lane = output column for P V.
+// One CTA per (pair of block tokens, KV head, sequence): K_b, V_b of the KV head staged in shared
+// memory as fp32; one warp per query row (the G heads of the two tokens).  Everything a row needs
+// from global memory (its query, cached L_p and o_p) is requested before the arithmetic starts, so
+// the kernel pays one memory latency, not one per operand.  Scores: lane = block key, columns
+// visited in a rotated order so that the 32 lanes hit 32 banks, four independent partial sums;
+// P V: lane = output column.
 template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 block_attn_merge_kernel(const T* __restrict__ q, const T* __restrict__ k_blk, const T* __restrict__ v_blk,
@@ -27,38 +30,59 @@ block_attn_merge_kernel(const T* __restrict__ q, const T* __restrict__ k_blk, co
   const int t0 = blockIdx.x * kTokTile, kh = blockIdx.y, s = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = Hq / Hkv;
+  const int ntok = min(kTokTile, B - t0);
+  constexpr int C = D / 32;
+  // this warp's first row: issue its loads before staging K_b / V_b
+  int r = warp;
+  bool have = r < ntok * G;
+  size_t row = 0;
+  float qv[C], opv[C], Lp = 0.f;
+  auto fetch = [&]() {
+    row = (static_cast<size_t>(s) * B + t0 + r / G) * Hq + kh * G + r % G;
+#pragma unroll
+    for (int c = 0; c < C; ++c) {
+      qv[c] = to_f32(q[row * D + lane + 32 * c]);
+      opv[c] = o_p[row * D + lane + 32 * c];
+    }
+    Lp = lse_p[row];
+  };
+  if (have) fetch();
   for (int idx = tid * 8; idx < B * D; idx += kThreads * 8) {
     const int t = idx / D, j = idx % D;
     const size_t src = ((static_cast<size_t>(s) * B + t) * Hkv + kh) * D + j;
     float a[8], b[8];
     load8(k_blk + src, a);
     load8(v_blk + src, b);
-#pragma unroll
-    for (int e = 0; e < 8; ++e) { Ks[idx + e] = a[e]; Vs[idx + e] = b[e]; }
+    *reinterpret_cast<float4*>(Ks + idx) = make_float4(a[0], a[1], a[2], a[3]);
+    *reinterpret_cast<float4*>(Ks + idx + 4) = make_float4(a[4], a[5], a[6], a[7]);
+    *reinterpret_cast<float4*>(Vs + idx) = make_float4(b[0], b[1], b[2], b[3]);
+    *reinterpret_cast<float4*>(Vs + idx + 4) = make_float4(b[4], b[5], b[6], b[7]);
   }
   __syncthreads();
-  const int ntok = min(kTokTile, B - t0);
   float* qw = Qs + warp * D;
-  for (int r = warp; r < ntok * G; r += kThreads / 32) {
-    const int tok = t0 + r / G, h = kh * G + r % G;
-    const size_t row = (static_cast<size_t>(s) * B + tok) * Hq + h;
+  while (have) {
     __syncwarp();
-    for (int j = lane; j < D; j += 32) qw[j] = to_f32(q[row * D + j]);
+#pragma unroll
+    for (int c = 0; c < C; ++c) qw[lane + 32 * c] = qv[c];
     __syncwarp();
     float sc[2];
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
       const int t = lane + 32 * u;
-      float dot = 0.f;
+      float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
       if (t < B) {
         const float* kr = Ks + t * D;
-#pragma unroll 8
-        for (int j = 0; j < D; ++j) {
-          const int jj = (j + lane) & (D - 1);
-          dot = fmaf(qw[jj], kr[jj], dot);
+#pragma unroll 4
+        for (int j = 0; j < D; j += 4) {
+          const int j0 = (j + lane) & (D - 1), j1 = (j + 1 + lane) & (D - 1);
+          const int j2 = (j + 2 + lane) & (D - 1), j3 = (j + 3 + lane) & (D - 1);
+          d0 = fmaf(qw[j0], kr[j0], d0);
+          d1 = fmaf(qw[j1], kr[j1], d1);
+          d2 = fmaf(qw[j2], kr[j2], d2);
+          d3 = fmaf(qw[j3], kr[j3], d3);
         }
       }
-      sc[u] = (t < B) ? dot * sm_scale : -INFINITY;
+      sc[u] = (t < B) ? ((d0 + d1) + (d2 + d3)) * sm_scale : -INFINITY;
     }
     const float M = warp_max(fmaxf(sc[0], sc[1]));
     float p[2];
@@ -66,25 +90,27 @@ block_attn_merge_kernel(const T* __restrict__ q, const T* __restrict__ k_blk, co
     p[1] = expf(sc[1] - M);
     const float sum = warp_sum(p[0] + p[1]);
     const float Lb = M + logf(sum);
-    float ob[D / 32];
+    float ob[C];
 #pragma unroll
-    for (int c = 0; c < D / 32; ++c) ob[c] = 0.f;
+    for (int c = 0; c < C; ++c) ob[c] = 0.f;
+#pragma unroll 4
     for (int t = 0; t < B; ++t) {
       const float pt = __shfl_sync(0xffffffffu, t < 32 ? p[0] : p[1], t & 31);
 #pragma unroll
-      for (int c = 0; c < D / 32; ++c) ob[c] = fmaf(pt, Vs[t * D + lane + 32 * c], ob[c]);
+      for (int c = 0; c < C; ++c) ob[c] = fmaf(pt, Vs[t * D + lane + 32 * c], ob[c]);
     }
-    const float Lp = lse_p[row];
     const float M2 = fmaxf(Lp, Lb);
     const float L = M2 + logf(expf(Lp - M2) + expf(Lb - M2));
     const float wp = expf(Lp - L), wb = expf(Lb - L) / sum;
 #pragma unroll
-    for (int c = 0; c < D / 32; ++c) {
-      const int j = lane + 32 * c;
-      const float v = (wp > 0.f ? wp * o_p[row * D + j] : 0.f) + wb * ob[c];
-      out[row * D + j] = from_f32<T>(v);
+    for (int c = 0; c < C; ++c) {
+      const float v = (wp > 0.f ? wp * opv[c] : 0.f) + wb * ob[c];
+      out[row * D + lane + 32 * c] = from_f32<T>(v);
     }
     if (lse_out && lane == 0) lse_out[row] = L;
+    r += kThreads / 32;
+    have = r < ntok * G;
+    if (have) fetch();
   }
 }
 
@@ -95,7 +121,8 @@ commit_step_kernel(const uint4* __restrict__ q, uint4* __restrict__ q_prev, size
   for (size_t i = blockIdx.x * static_cast<size_t>(kThreads) + threadIdx.x; i < n_vec;
        i += static_cast<size_t>(gridDim.x) * kThreads)
     q_prev[i] = q[i];
-  if (blockIdx.x == 0 && threadIdx.x < N) step[threadIdx.x] += 1;
+  if (blockIdx.x == 0)
+    for (int s = threadIdx.x; s < N; s += kThreads) step[s] += 1;
 }
 
 // min / max of column j of logical page p over its valid tokens; tokens at prefix positions >=

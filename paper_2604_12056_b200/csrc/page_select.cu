@@ -153,6 +153,157 @@ topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ kv_len
   }
 }
 
+// ---- top-k by threshold search: one warp per query, O(P) work --------------------------------
+// Keys are (order-preserving score bits, inverted page id), all distinct, so "the k largest keys"
+// is the required answer with ties already broken.  The warp histograms the score bits of the
+// still-undecided range into 256 equal-width bins, finds the bin holding the k-th largest, takes
+// every key above that bin, and either finishes by sorting "taken + threshold bin" (a few dozen
+// keys) or narrows the range to the threshold bin and repeats.  A range of one value means the
+// remaining candidates tie on the score: the lowest page ids win, taken in page order.
+constexpr int kSelWarps = 4;
+constexpr int kSelCap = 512;     // candidate keys a warp can sort; also the largest k of this path
+constexpr int kSelBins = 256;
+
+__device__ __forceinline__ unsigned long long make_key(uint32_t ob, int p) {
+  return (static_cast<unsigned long long>(ob) << 32) |
+         static_cast<unsigned long long>(0xffffffffu - static_cast<uint32_t>(p));
+}
+
+__global__ void __launch_bounds__(kSelWarps * 32)
+topk_select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ kv_len,
+                   const int32_t* __restrict__ active_idx, const int32_t* __restrict__ n_active,
+                   const int32_t* __restrict__ step, int32_t* __restrict__ topk_pages,
+                   float* __restrict__ topk_scores, int N, int B, int Hq, int g, int k, int score_stride,
+                   int32_t* __restrict__ status) {
+  __shared__ unsigned long long s_cand[kSelWarps][kSelCap];
+  __shared__ int s_hist[kSelWarps][kSelBins];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int qid = blockIdx.x * kSelWarps + warp;
+  const int h = qid % Hq, a = (qid / Hq) % B, s = qid / (Hq * B);
+  if (s >= N) return;
+  if (step && step[s] == 0) return;
+  int na = n_active[s];
+  na = na > B ? B : na;
+  if (a >= na) return;
+  const int tok = active_idx[s * B + a];
+  if (tok < 0 || tok >= B) { if (lane == 0) set_status(status, LOSA_ERR_BOUNDS); return; }
+  const int P = pages_of(kv_len[s], g);
+  const int kk = min(k, P);
+  const float* row = scores + ((static_cast<size_t>(s) * B + a) * Hq + h) * score_stride;
+  unsigned long long* cand = s_cand[warp];
+  int* hist = s_hist[warp];
+  const unsigned below = (1u << lane) - 1u;
+
+  uint32_t lo = 0xffffffffu, hi = 0u;
+  for (int p = lane; p < P; p += 32) {
+    const uint32_t ob = order_bits(row[p]);
+    lo = min(lo, ob);
+    hi = max(hi, ob);
+  }
+  lo = __reduce_min_sync(0xffffffffu, lo);
+  hi = __reduce_max_sync(0xffffffffu, hi);
+  int need = kk, ncand = 0;
+  while (need > 0) {
+    if (lo == hi) {
+      // every remaining candidate has the same score: lowest pages first, in page order
+      for (int base = 0; base < P && need > 0; base += 32) {
+        const int p = base + lane;
+        const bool hit = p < P && order_bits(row[p]) == lo;
+        const unsigned bal = __ballot_sync(0xffffffffu, hit);
+        const int rank = __popc(bal & below);
+        if (hit && rank < need) cand[ncand + rank] = make_key(lo, p);
+        const int taken = min(need, __popc(bal));
+        ncand += taken;
+        need -= taken;
+      }
+      break;
+    }
+    const int width = 32 - __clz(hi - lo);           // bits needed for hi - lo  (>= 1)
+    const int shift = width > 8 ? width - 8 : 0;      // (ob - lo) >> shift is in [0, 255]
+    for (int b = lane; b < kSelBins; b += 32) hist[b] = 0;
+    __syncwarp();
+    for (int p = lane; p < P; p += 32) {
+      const uint32_t ob = order_bits(row[p]);
+      if (ob >= lo && ob <= hi) atomicAdd(&hist[(ob - lo) >> shift], 1);
+    }
+    __syncwarp();
+    // lane owns bins [8*lane, 8*lane+8); suffix sums over lanes locate the threshold bin
+    int c[8], tot = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) { c[e] = hist[8 * lane + e]; tot += c[e]; }
+    int suf = tot;                                     // inclusive suffix: lanes >= this one
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_down_sync(0xffffffffu, suf, o);
+      if (lane + o < 32) suf += t;
+    }
+    const int above_lanes = suf - tot;
+    const bool owner = above_lanes < need && need <= suf;
+    int bstar = 0, cnt_above = 0, cnt_thr = 0;
+    if (owner) {
+      int run = above_lanes;
+#pragma unroll
+      for (int e = 7; e >= 0; --e) {
+        if (run < need && need <= run + c[e]) { bstar = 8 * lane + e; cnt_above = run; cnt_thr = c[e]; }
+        run += c[e];
+      }
+    }
+    const int src = __ffs(__ballot_sync(0xffffffffu, owner)) - 1;
+    bstar = __shfl_sync(0xffffffffu, bstar, src);
+    cnt_above = __shfl_sync(0xffffffffu, cnt_above, src);
+    cnt_thr = __shfl_sync(0xffffffffu, cnt_thr, src);
+    const bool finish = ncand + cnt_above + cnt_thr <= kSelCap;
+    // take the keys above the threshold bin (and, when finishing, the threshold bin itself)
+    for (int base = 0; base < P; base += 32) {
+      const int p = base + lane;
+      bool take = false;
+      uint32_t ob = 0;
+      if (p < P) {
+        ob = order_bits(row[p]);
+        if (ob >= lo && ob <= hi) {
+          const int bin = static_cast<int>((ob - lo) >> shift);
+          take = bin > bstar || (finish && bin == bstar);
+        }
+      }
+      const unsigned bal = __ballot_sync(0xffffffffu, take);
+      if (take) cand[ncand + __popc(bal & below)] = make_key(ob, p);
+      ncand += __popc(bal);
+    }
+    if (finish) break;
+    need -= cnt_above;
+    const uint32_t nlo = lo + (static_cast<uint32_t>(bstar) << shift);
+    const unsigned long long top = static_cast<unsigned long long>(nlo) + ((1ull << shift) - 1ull);
+    hi = top < hi ? static_cast<uint32_t>(top) : hi;
+    lo = nlo;
+  }
+  // sort the candidates (descending) and emit the first kk
+  int n2 = 2;
+  while (n2 < ncand) n2 <<= 1;
+  for (int i = ncand + lane; i < n2; i += 32) cand[i] = 0ull;
+  __syncwarp();
+  for (int k2 = 2; k2 <= n2; k2 <<= 1) {
+    for (int j = k2 >> 1; j > 0; j >>= 1) {
+      for (int t = lane; t < (n2 >> 1); t += 32) {
+        const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+        const int x = i | j;
+        const unsigned long long ka = cand[i], kb = cand[x];
+        if ((ka < kb) == ((i & k2) == 0)) { cand[i] = kb; cand[x] = ka; }
+      }
+      __syncwarp();
+    }
+  }
+  const size_t o = ((static_cast<size_t>(s) * B + tok) * Hq + h) * k;
+  for (int j = lane; j < k; j += 32) {
+    if (j < kk) {
+      const unsigned long long key = cand[j];
+      topk_pages[o + j] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(key));
+      if (topk_scores) topk_scores[o + j] = unorder_bits(static_cast<uint32_t>(key >> 32));
+    } else {
+      topk_pages[o + j] = -1;
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kThreads)
 union_kernel(const int32_t* __restrict__ topk_pages, const int32_t* __restrict__ active_idx,
              const int32_t* __restrict__ n_active, const int32_t* __restrict__ kv_len,
@@ -263,12 +414,20 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
   int32_t rc = after_launch(c);
   if (rc != LOSA_OK) return rc;
 
+  const float* sc = reinterpret_cast<const float*>(c->ws + c->lay.scores);
+  if (k <= kSelCap) {
+    const int queries = sh.batch * sh.block_size * sh.n_q_heads;
+    topk_select_kernel<<<(queries + kSelWarps - 1) / kSelWarps, kSelWarps * 32, 0, st>>>(
+        sc, kv->kv_len, active_idx, n_active, step, topk_pages, topk_scores_opt, sh.batch, sh.block_size,
+        sh.n_q_heads, sh.page_size, k, c->lay.score_stride, status_ptr(c));
+    return after_launch(c);
+  }
+  // budgets beyond what one warp can sort: whole-list bitonic sort, one CTA per query
   const size_t smem = static_cast<size_t>(pow2_at_least(sh.max_pages_per_seq)) * sizeof(unsigned long long);
   if (smem > 48 * 1024)
     LOSA_CUDA_TRY(c, cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   dim3 grid(sh.n_q_heads, sh.block_size, sh.batch);
-  topk_kernel<<<grid, kThreads, smem, st>>>(reinterpret_cast<const float*>(c->ws + c->lay.scores),
-                                            kv->kv_len, active_idx, n_active, step, topk_pages,
+  topk_kernel<<<grid, kThreads, smem, st>>>(sc, kv->kv_len, active_idx, n_active, step, topk_pages,
                                             topk_scores_opt, sh.block_size, sh.n_q_heads, sh.page_size,
                                             k, c->lay.score_stride, status_ptr(c));
   return after_launch(c);

@@ -45,7 +45,21 @@ struct AttnParams {
   int32_t* status;
   int B, Hq, Hkv, G, Pmax, n_phys, n_rg, n_seg, n_ctas;
   float sm_scale;
+#ifdef LOSA_TRACE
+  unsigned long long* trace;   // [n_ctas][8] timestamps, development builds only
+#endif
 };
+
+#ifdef LOSA_TRACE
+__device__ __forceinline__ unsigned long long gtime() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define LOSA_STAMP(slot) do { if (p.trace) p.trace[blockIdx.x * 8 + (slot)] = gtime(); } while (0)
+#else
+#define LOSA_STAMP(slot) do { } while (0)
+#endif
 
 __device__ __forceinline__ float* partial_base(float* partials, int slot, int D) {
   return partials + static_cast<size_t>(slot) * kRowsPerGroup * (D + 2);
@@ -171,17 +185,20 @@ __global__ void __launch_bounds__(256, 1) attn_simt_kernel(AttnParams p) {
 }
 
 // ===================================================================== combine kernel
-// grid (n_seg, 16): warp = one query row of the segment's row group.  LOG2 says whether the
-// partial maxima are in base-2 units (tensor-core kernel) or natural units (fp32 kernel).
+// grid (n_seg, 16): warp = one query row of the segment's row group.  The CTAs whose item range
+// meets the segment are consecutive; lanes take one piece each for the row maxima and sums, then
+// the warp walks the pieces with every load of a group of four issued together.  LOG2 says
+// whether the partial maxima are in base-2 units (tensor-core kernel) or natural units (fp32).
 template <int D, bool LOG2>
 __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
   __shared__ int pre[kMaxSegments + 1];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (warp == 0) segment_prefix(pre, p.n_seg, p.n_rg, p.Hkv, p.G, p.n_active, p.union_count, p.B, lane);
-  __syncthreads();
   const int sg = blockIdx.x, r = blockIdx.y * 8 + warp;
   const int rg = sg % p.n_rg, sk = sg / p.n_rg, s = sk / p.Hkv, kh = sk % p.Hkv;
   const int rows = rows_in_group(clamp_active(p.n_active[s], p.B), p.G, rg);
+  if (blockIdx.y * 8 >= rows) return;                 // whole CTA idle: skip the prefix as well
+  if (warp == 0) segment_prefix(pre, p.n_seg, p.n_rg, p.Hkv, p.G, p.n_active, p.union_count, p.B, lane);
+  __syncthreads();
   if (r >= rows) return;
   const int row = rg * kRowsPerGroup + r, a = row / p.G, gi = row % p.G;
   const int tok = p.active_idx[s * p.B + a];
@@ -189,36 +206,62 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
   const size_t orow = (static_cast<size_t>(s) * p.B + tok) * p.Hq + kh * p.G + gi;
   const int start = pre[sg], end = pre[sg + 1];
   const long long T_all = pre[p.n_seg];
-  float acc[D / 32];
+  constexpr int C = D / 32;
+  float acc[C];
 #pragma unroll
-  for (int c = 0; c < D / 32; ++c) acc[c] = 0.f;
+  for (int c = 0; c < C; ++c) acc[c] = 0.f;
   float M = -INFINITY, Lsum = 0.f;
   if (end > start) {
     int b0 = static_cast<int>((static_cast<long long>(start) * p.n_ctas) / T_all);
     while (b0 + 1 < p.n_ctas && cta_lo(T_all, b0 + 1, p.n_ctas) <= start) ++b0;
-    for (int pass = 0; pass < 2; ++pass) {
-      for (int b = b0; b < p.n_ctas; ++b) {
+    int b1 = static_cast<int>((static_cast<long long>(end - 1) * p.n_ctas) / T_all);   // last CTA that can meet it
+    while (b1 + 1 < p.n_ctas && cta_lo(T_all, b1 + 1, p.n_ctas) < end) ++b1;
+    // pass 1: the row maximum over the pieces
+    for (int base = b0; base <= b1; base += 32) {
+      const int b = base + lane;
+      float mj = -INFINITY;
+      if (b <= b1) {
         const long long lo = cta_lo(T_all, b, p.n_ctas), hi = cta_lo(T_all, b + 1, p.n_ctas);
-        if (lo >= end) break;
-        if (hi <= start || hi <= lo) continue;
-        const float* part = partial_base(p.partials, b + sg, D);
-        const float mj = part[r];
-        if (pass == 0) {
-          M = fmaxf(M, mj);
-        } else {
-          const float w = (mj == -INFINITY) ? 0.f : (LOG2 ? exp2f(mj - M) : expf(mj - M));
-          Lsum = fmaf(part[kRowsPerGroup + r], w, Lsum);
-#pragma unroll
-          for (int c = 0; c < D / 32; ++c)
-            acc[c] = fmaf(part[2 * kRowsPerGroup + r * D + lane + 32 * c], w, acc[c]);
+        if (lo < end && hi > start && hi > lo) mj = partial_base(p.partials, b + sg, D)[r];
+      }
+      M = fmaxf(M, warp_max(mj));
+    }
+    // pass 2: weights, sum and output
+    for (int base = b0; base <= b1; base += 32) {
+      const int b = base + lane;
+      float wj = 0.f, lj = 0.f;
+      if (b <= b1) {
+        const long long lo = cta_lo(T_all, b, p.n_ctas), hi = cta_lo(T_all, b + 1, p.n_ctas);
+        if (lo < end && hi > start && hi > lo) {
+          const float* part = partial_base(p.partials, b + sg, D);
+          const float mj = part[r];
+          wj = (mj == -INFINITY) ? 0.f : (LOG2 ? exp2f(mj - M) : expf(mj - M));
+          lj = part[kRowsPerGroup + r];
         }
+      }
+      Lsum += warp_sum(lj * wj);
+      const int n = min(32, b1 - base + 1);
+      for (int i0 = 0; i0 < n; i0 += 4) {
+        float w[4], v[4][C];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = i0 + u;
+          w[u] = (i < n) ? __shfl_sync(0xffffffffu, wj, i & 31) : 0.f;
+          const float* src = partial_base(p.partials, base + i + sg, D) + 2 * kRowsPerGroup + r * D + lane;
+#pragma unroll
+          for (int c = 0; c < C; ++c) v[u][c] = (w[u] != 0.f) ? src[32 * c] : 0.f;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+#pragma unroll
+          for (int c = 0; c < C; ++c) acc[c] = fmaf(v[u][c], w[u], acc[c]);
       }
     }
   }
   const bool empty = !(Lsum > 0.f);
   const float inv = empty ? 0.f : 1.f / Lsum;
 #pragma unroll
-  for (int c = 0; c < D / 32; ++c) p.o_p[orow * D + lane + 32 * c] = acc[c] * inv;
+  for (int c = 0; c < C; ++c) p.o_p[orow * D + lane + 32 * c] = acc[c] * inv;
   if (lane == 0) p.lse_p[orow] = empty ? -INFINITY : (LOG2 ? (M + log2f(Lsum)) * kLn2 : M + logf(Lsum));
 }
 
@@ -353,6 +396,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   int* pre = reinterpret_cast<int*>(tail + 512);
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) LOSA_STAMP(0);
   if (tid == 0) {
     for (int i = 0; i < NSTAGE; ++i) {
       mbar_init(full0 + 8 * i, 1);
@@ -371,6 +415,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   if (lo >= hi) return;
   int sg0 = 0;
   while (pre[sg0 + 1] <= lo) ++sg0;
+  if (tid == 0) LOSA_STAMP(1);
 
   if (warp == kConsumerWarps) {
     // ------------------------------------------------------------------ producer warp
@@ -398,6 +443,8 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
           const int it = b0 + j - lo, stage = it % NSTAGE, round = it / NSTAGE;
           const bool go = mbar_wait(empty0 + 8 * stage, (round & 1) ^ 1, abort_flag, p.status);
           if (go) {
+            if (it == 0) LOSA_STAMP(7);                  // about to issue the first copy
+            if (it == NSTAGE - 1) LOSA_STAMP(2);         // ring filled once without waiting
             meta[stage] = vj;
             stage_round[stage] = round;
             const uint32_t fb = full0 + 8 * stage, dst = stage0 + stage * STAGE;
@@ -412,6 +459,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       }
       sg = __shfl_sync(0xffffffffu, sg, nb - 1);
     }
+    if (lane == 0) LOSA_STAMP(3);                    // all copies issued
     return;
   }
 
@@ -420,6 +468,9 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   const int g8 = lane >> 2, q4 = lane & 3;
   const float scale2 = p.sm_scale * kLog2e;
   int sg = sg0, item = lo;
+#ifdef LOSA_TRACE
+  long long trace_wait = 0, trace_busy = 0;
+#endif
   while (item < hi) {
     const int seg_end = min(hi, pre[sg + 1]);
     const int npg = seg_end - item;
@@ -465,8 +516,16 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       const int it = item + j - lo, stage = it % NSTAGE, round = it / NSTAGE;
       // A parity wait is only meaningful once the stage is in this item's pass over the ring:
       // this warp may get here while the stage's previous page is still in flight.
+#ifdef LOSA_TRACE
+      const long long tw0 = clock64();
+#endif
       const bool ready = wait_round(stage_round + stage, round, abort_flag, p.status) &&
                          mbar_wait(full0 + 8 * stage, round & 1, abort_flag, p.status);
+#ifdef LOSA_TRACE
+      const long long tw1 = clock64();
+      trace_wait += tw1 - tw0;
+#endif
+      if (tid == 0 && it == 0) LOSA_STAMP(4);        // first page landed
       if (ready && has_rows) {
         const int valid = meta[stage];
         const uint32_t kt = stage0 + stage * STAGE, vt = kt + KBYTES;
@@ -480,21 +539,30 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           __syncwarp();
         }
-        // ---- S = Q K^T
+        // ---- S = Q K^T.  The K fragments of k-step ks+1 are requested before the MMAs of k-step
+        // ks are issued, so shared-memory latency hides behind tensor-core work.
         float sacc[NT][4];
 #pragma unroll
         for (int n = 0; n < NT; ++n) { sacc[n][0] = sacc[n][1] = sacc[n][2] = sacc[n][3] = 0.f; }
+        const int mi = lane >> 3, l7 = lane & 7;
         {
-          const int mi = lane >> 3;
+          // row of the K tile this lane addresses for n-tile pair np is np*16 + krow; its chunk for
+          // k-step ks is ks*2 + (mi & 1)
+          const int krow = (mi >> 1) * 8 + l7;
+          uint32_t kb[2][NT / 2][4];
+#pragma unroll
+          for (int np = 0; np < NT / 2; ++np) ldsm_x4(kt + tile_off<GP>(np * 16 + krow, (mi & 1)), kb[0][np]);
 #pragma unroll
           for (int ks = 0; ks < KS; ++ks) {
+            if (ks + 1 < KS) {
+#pragma unroll
+              for (int np = 0; np < NT / 2; ++np)
+                ldsm_x4(kt + tile_off<GP>(np * 16 + krow, (ks + 1) * 2 + (mi & 1)), kb[(ks + 1) & 1][np]);
+            }
 #pragma unroll
             for (int np = 0; np < NT / 2; ++np) {
-              uint32_t b[4];
-              const int t = (np * 2 + (mi >> 1)) * 8 + (lane & 7);
-              ldsm_x4(kt + tile_off<GP>(t, ks * 2 + (mi & 1)), b);
-              mma_bf16(sacc[2 * np], qf[ks], b[0], b[1]);
-              mma_bf16(sacc[2 * np + 1], qf[ks], b[2], b[3]);
+              mma_bf16(sacc[2 * np], qf[ks], kb[ks & 1][np][0], kb[ks & 1][np][1]);
+              mma_bf16(sacc[2 * np + 1], qf[ks], kb[ks & 1][np][2], kb[ks & 1][np][3]);
             }
           }
         }
@@ -531,28 +599,38 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         }
         l0 = l0 * c0 + s0;
         l1 = l1 * c1 + s1;
+        if (__any_sync(0xffffffffu, c0 != 1.f || c1 != 1.f)) {      // rescale only when some row maximum moved
 #pragma unroll
-        for (int n = 0; n < ND; ++n) { oacc[n][0] *= c0; oacc[n][1] *= c0; oacc[n][2] *= c1; oacc[n][3] *= c1; }
-        // ---- O += P V
+          for (int n = 0; n < ND; ++n) { oacc[n][0] *= c0; oacc[n][1] *= c0; oacc[n][2] *= c1; oacc[n][3] *= c1; }
+        }
+        // ---- O += P V, V fragments fetched two MMA pairs ahead
         {
-          const int mi = lane >> 3;
+          constexpr int NV = (GP / 16) * (ND / 2);       // ldmatrix.x4.trans loads per page
+          const int vrow = (mi & 1) * 8 + l7;
+          uint32_t vb[3][4];
+          auto vload = [&](int i, uint32_t (&dst)[4]) {
+            const int k2 = i / (ND / 2), np = i % (ND / 2);
+            ldsm_x4_trans(vt + tile_off<GP>(k2 * 16 + vrow, np * 2 + (mi >> 1)), dst);
+          };
+          vload(0, vb[0]);
+          if (NV > 1) vload(1, vb[1]);
 #pragma unroll
-          for (int k2 = 0; k2 < GP / 16; ++k2) {
-#pragma unroll
-            for (int np = 0; np < ND / 2; ++np) {
-              uint32_t b[4];
-              const int t = k2 * 16 + (mi & 1) * 8 + (lane & 7);
-              ldsm_x4_trans(vt + tile_off<GP>(t, np * 2 + (mi >> 1)), b);
-              mma_bf16(oacc[2 * np], pa[k2], b[0], b[1]);
-              mma_bf16(oacc[2 * np + 1], pa[k2], b[2], b[3]);
-            }
+          for (int i = 0; i < NV; ++i) {
+            if (i + 2 < NV) vload(i + 2, vb[(i + 2) % 3]);
+            const int k2 = i / (ND / 2), np = i % (ND / 2);
+            mma_bf16(oacc[2 * np], pa[k2], vb[i % 3][0], vb[i % 3][1]);
+            mma_bf16(oacc[2 * np + 1], pa[k2], vb[i % 3][2], vb[i % 3][3]);
           }
         }
       }
       __syncwarp();
+#ifdef LOSA_TRACE
+      trace_busy += clock64() - tw1;
+#endif
       if (ready && lane == 0) mbar_arrive(empty0 + 8 * stage, static_cast<uint32_t>(ns));
     }
 
+    if (tid == 0 && seg_end == hi) LOSA_STAMP(5);    // warp 0 done with its pages
     // ---- merge the page slots of each row tile through shared memory (tree), slot 0 keeps it
     float* scr = reinterpret_cast<float*>(qs_gen);
     for (int stride = ns >> 1; stride >= 1; stride >>= 1) {
@@ -616,6 +694,10 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     ++sg;
     while (item < hi && pre[sg + 1] <= item) ++sg;
   }
+  if (tid == 0) LOSA_STAMP(6);
+#ifdef LOSA_TRACE
+  if (lane == 0 && p.trace) { p.trace[p.n_ctas * 8 + (blockIdx.x * 8 + warp) * 2] = trace_wait; p.trace[p.n_ctas * 8 + (blockIdx.x * 8 + warp) * 2 + 1] = trace_busy; }
+#endif
 }
 
 // ===================================================================== host side
@@ -715,6 +797,11 @@ int32_t dispatch_page(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
 
 }  // namespace
 
+#ifdef LOSA_TRACE
+unsigned long long* g_trace = nullptr;
+extern "C" void losa_debug_set_trace(void* p) { g_trace = static_cast<unsigned long long*>(p); }
+#endif
+
 int32_t launch_sparse_prefix_attn(losa_ctx* c, const void* q, const losa_kv_t* kv,
                                   const int32_t* active_idx, const int32_t* n_active,
                                   const int32_t* union_pages, const int32_t* union_count,
@@ -751,6 +838,9 @@ int32_t launch_sparse_prefix_attn(losa_ctx* c, const void* q, const losa_kv_t* k
   ap.n_seg = c->lay.n_segments;
   ap.n_ctas = c->lay.n_ctas;
   ap.sm_scale = sh.sm_scale;
+#ifdef LOSA_TRACE
+  ap.trace = g_trace;
+#endif
   return sh.head_dim == 128 ? dispatch_page<128>(c, ap, st) : dispatch_page<64>(c, ap, st);
 }
 
