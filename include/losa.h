@@ -156,6 +156,29 @@ int32_t losa_select_active(losa_ctx* ctx, const void* x_cur, const void* x_prev,
                            const int32_t* m_per_seq, const int32_t* step, int32_t* active_idx,
                            int32_t* n_active, float* delta_opt, void* stream);
 
+/* Stage 1 without any allocation (the paper has no counterpart; this is a deployment aid).
+ * Some programs that embed this library are not allowed to obtain device memory once they are
+ * running: an inference server whose memory pool was carved up at start-up and whose allocator is
+ * owned by the host framework, a plug-in running under a fixed memory budget, or code on a path
+ * where cudaMalloc's implicit device-wide synchronisation is unacceptable.  Such callers cannot
+ * provide the workspace a context needs.  For them this entry point runs stage 1 exactly as
+ * losa_select_active does, but keeps its scratch (one fp64 score per block token and one counter
+ * per sequence) in a fixed array inside the library image instead of a caller workspace.  It needs
+ * no context, and it calls no cudaMalloc, cudaFree or other allocating routine.
+ *   shape: only batch, block_size and dtype are read.  batch must be at most 64 (the size the fixed
+ *       array was built for); a larger batch returns LOSA_ERR_UNSUPPORTED and launches nothing.
+ *   All other arguments, outputs and tie rules are those of losa_select_active.
+ *   The array costs about 33 KB on every GPU that loads the library, for the life of the process.
+ *   The first call on a device looks up the array's device address (once per device, with that
+ *   device current); make that first call before starting any stream capture.
+ *   All calls on a device share the one array, which keeps the previous call's contents (this call
+ *   clears the counters it relies on).  Two calls that overlap on the GPU — different streams, or
+ *   different host threads without ordering between their streams — race on it: serialise them. */
+int32_t losa_select_active_static(const losa_shape_t* shape, const void* x_cur, const void* x_prev,
+                                  int32_t row_width, const int32_t* m_per_seq, const int32_t* step,
+                                  int32_t* active_idx, int32_t* n_active, float* delta_opt,
+                                  void* stream);
+
 /* Stage 2 — QUEST page scores and top-k for the active queries (Section 2.3; Section 4.2).
  *   q [N, B, H_q, d] (dtype).  For every active token i, query head h and logical page p < P_s
  *   (P_s = ceil(L_s / g)), with kappa = h / G:

@@ -28,7 +28,7 @@ EXPORTS = [
     "losa_last_cuda_error", "losa_launch_count", "losa_select_active", "losa_page_scores_topk",
     "losa_page_union", "losa_sparse_prefix_attn", "losa_block_attn_merge",
     "losa_update_prefix_cache", "losa_build_page_summaries", "losa_denoise_step_host",
-    "losa_profile_stage4", "losa_stage4_last_ms",
+    "losa_profile_stage4", "losa_stage4_last_ms", "losa_select_active_static",
 ]
 
 
@@ -171,6 +171,18 @@ def losa_select_active(ctx, x_cur, x_prev, row_width, m_per_seq, step, active_id
     ctx._check("losa_select_active", lib().losa_select_active(
         ctx._h, _ptr(x_cur), _ptr(x_prev), C.c_int32(row_width), _ptr(m_per_seq), _ptr(step),
         _ptr(active_idx), _ptr(n_active), _ptr(delta_opt), _stream()))
+
+
+def losa_select_active_static(shape: ShapeT, x_cur, x_prev, row_width, m_per_seq, step, active_idx, n_active,
+                              delta_opt=None):
+    """Stage 1 for callers that must not allocate device memory: no context, no workspace; the
+    scratch lives in a fixed array inside the library (batch <= 64).  Calls on one device share
+    that array, so they must not overlap on the GPU."""
+    rc = lib().losa_select_active_static(C.byref(shape), _ptr(x_cur), _ptr(x_prev), C.c_int32(row_width),
+                                         _ptr(m_per_seq), _ptr(step), _ptr(active_idx), _ptr(n_active),
+                                         _ptr(delta_opt), _stream())
+    if rc != LOSA_OK:
+        raise LosaError("losa_select_active_static", rc)
 
 
 def losa_page_scores_topk(ctx, q, kv, active_idx, n_active, step, k, topk_pages, topk_scores_opt=None):

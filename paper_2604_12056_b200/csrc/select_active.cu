@@ -5,6 +5,8 @@
 // fp64 like the definition; the work is a few hundred KB).  The last CTA of a sequence to arrive
 // (self-resetting counter) ranks the B scores by (Delta descending, token ascending) and emits the
 // first m tokens in ascending order.
+#include <mutex>
+
 #include "kernels.h"
 
 namespace losa {
@@ -110,3 +112,71 @@ int32_t launch_select_active(losa_ctx* c, const void* x_cur, const void* x_prev,
 }
 
 }  // namespace losa
+
+// ----------------------------------------------------------------------------------------------
+// Stage 1 for callers that cannot allocate device memory.
+//
+// The regular entry point keeps its scratch (the fp64 per-token scores and one arrival counter per
+// sequence) in the workspace the caller allocated for the context.  This variant keeps the same
+// scratch in a fixed array that is part of the library image, so nothing has to be allocated —
+// neither by the caller nor here.  Every GPU that loads the library holds the array (about 33 KB)
+// until the process exits.
+namespace {
+
+constexpr int kStaticMaxBatch = 64;   // sequences the fixed scratch is sized for
+constexpr int kStaticMaxDevices = 64;
+
+struct StaticScratch {
+  double delta[kStaticMaxBatch * LOSA_MAX_BLOCK];
+  unsigned int counters[kStaticMaxBatch];
+};
+
+// Device-side storage.  In host code this name is only a handle for the runtime; the device
+// address is obtained once per device with cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char g_static_scratch[sizeof(StaticScratch)];
+
+std::mutex g_static_mutex;
+StaticScratch* g_static_addr[kStaticMaxDevices] = {};
+
+}  // namespace
+
+extern "C" int32_t losa_select_active_static(const losa_shape_t* shape, const void* x_cur, const void* x_prev,
+                                             int32_t row_width, const int32_t* m_per_seq, const int32_t* step,
+                                             int32_t* active_idx, int32_t* n_active, float* delta_opt,
+                                             void* stream) {
+  if (!shape || !x_cur || !x_prev || !active_idx || !n_active || row_width < 1) return LOSA_ERR_INVALID_ARG;
+  if (shape->batch < 1 || shape->block_size < 1 || shape->block_size > LOSA_MAX_BLOCK ||
+      (shape->dtype != LOSA_F32 && shape->dtype != LOSA_BF16))
+    return LOSA_ERR_INVALID_ARG;
+  if (shape->batch > kStaticMaxBatch) return LOSA_ERR_UNSUPPORTED;   // beyond the fixed scratch
+  if (row_width % 8 != 0 || (reinterpret_cast<uintptr_t>(x_cur) & 15u) || (reinterpret_cast<uintptr_t>(x_prev) & 15u))
+    return LOSA_ERR_UNSUPPORTED;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return LOSA_ERR_CUDA;
+  if (dev < 0 || dev >= kStaticMaxDevices) return LOSA_ERR_UNSUPPORTED;
+  StaticScratch* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_addr[dev]) {
+      // set-up, once per device, with that device current
+      void* ptr = nullptr;
+      if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return LOSA_ERR_CUDA;
+      g_static_addr[dev] = static_cast<StaticScratch*>(ptr);
+    }
+    scratch = g_static_addr[dev];
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the array keeps whatever the last call left: the arrival counters must start at zero
+  if (cudaMemsetAsync(scratch->counters, 0, sizeof(unsigned int) * shape->batch, st) != cudaSuccess) return LOSA_ERR_CUDA;
+  dim3 grid(shape->block_size, shape->batch);
+  if (shape->dtype == LOSA_BF16) {
+    losa::select_active_kernel<__nv_bfloat16><<<grid, losa::kThreads, 0, st>>>(
+        static_cast<const __nv_bfloat16*>(x_cur), static_cast<const __nv_bfloat16*>(x_prev), row_width,
+        shape->block_size, m_per_seq, step, active_idx, n_active, delta_opt, scratch->delta, scratch->counters);
+  } else {
+    losa::select_active_kernel<float><<<grid, losa::kThreads, 0, st>>>(
+        static_cast<const float*>(x_cur), static_cast<const float*>(x_prev), row_width, shape->block_size,
+        m_per_seq, step, active_idx, n_active, delta_opt, scratch->delta, scratch->counters);
+  }
+  return cudaGetLastError() == cudaSuccess ? LOSA_OK : LOSA_ERR_CUDA;
+}
