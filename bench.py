@@ -8,8 +8,9 @@ denoising step.  Steps cycle through whole denoising blocks of the workload (ste
 the dense first step, the others are LoSA steps).  Prints ONE JSON line.
 
 Timing: the layer-step is captured once in a CUDA graph and replayed; each step is bracketed by
-CUDA events on the launching stream; between steps the L2 is flushed by writing a 256 MiB buffer
-outside the timed region.  The time of K steps is the sum of the K event intervals; with several
+CUDA events on the launching stream; between steps, outside the timed region, the L2 is flushed by
+writing a 256 MiB buffer and then reading a second one (the read pass makes the cache write its
+dirty lines back, so that write-back traffic of the flush itself does not land in the timed step).  The time of K steps is the sum of the K event intervals; with several
 GPUs every rank runs its own replica of the workload (weak scaling, no data-path collective) and
 the maximum over ranks is reported.
 """
@@ -239,7 +240,15 @@ def run_ours(args, cfg):
                  for i in host_steps]
     q_s, k_s, v_s = (torch.empty_like(t) for t in dev_steps[0][:3])
     m_s = torch.empty_like(dev_steps[0][3])
-    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    flush_w = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    flush_r = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.float32, device=dev)   # fp32: sum() reads it in place
+
+    class _Flush:
+        """Evicts the L2 (write > L2, then read > L2 so that no dirty lines are left behind)."""
+        def fill_(self, v):
+            flush_w.fill_(v)
+            flush_r.sum()
+    flush = _Flush()
 
     def load(i):
         q, k, v, m = dev_steps[i]
@@ -301,7 +310,7 @@ def run_ours(args, cfg):
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": workload_name(cfg), "sequences_per_gpu": cfg.batch,
                    "launch": "CUDA graph replay of the six stage calls",
-                   "l2": "flushed between steps (256 MiB write outside the timed region)"},
+                   "l2": "flushed between steps, outside the timed region: 256 MiB write, then 256 MiB read so no dirty lines remain"},
         "clocks": clocks, "gpu_launches": launches_per_step * args.steps,
         "step_us": {"losa_step_median": float(np.median(sparse_ms)) * 1e3 if sparse_ms else None,
                     "dense_first_step_median": float(np.median(dense_ms)) * 1e3 if dense_ms else None},

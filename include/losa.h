@@ -183,9 +183,12 @@ int32_t losa_select_active_static(const losa_shape_t* shape, const void* x_cur, 
  *   q [N, B, H_q, d] (dtype).  For every active token i, query head h and logical page p < P_s
  *   (P_s = ceil(L_s / g)), with kappa = h / G:
  *       U(p) = sum_j max(q_j * kmin[p,kappa,j], q_j * kmax[p,kappa,j])
- *   in fp32 in a fixed order: products rounded to nearest; the 8 terms of each run of 8
- *   consecutive j added left to right; the d/8 run sums combined by the butterfly
- *   c[i] <- c[i] + c[i xor off], off = d/16 .. 1; finally + 0.0f.
+ *            = sum_j (max(q_j, 0) * kmax[p,kappa,j] + min(q_j, 0) * kmin[p,kappa,j])     (kmin <= kmax)
+ *   evaluated in fp32 in a fixed order, because it decides integer page ids: for each run of 8
+ *   consecutive j an accumulator starts at +0 and takes, j ascending, first
+ *   acc = fma(max(q_j,0), kmax_j, acc), then acc = fma(min(q_j,0), kmin_j, acc) (fused, round to
+ *   nearest); the d/8 run sums are combined by the butterfly c[i] <- c[i] + c[i xor off],
+ *   off = d/16 .. 1; finally + 0.0f.
  *   topk_pages [N, B, H_q, k] int32 out: the min(k, P_s) pages with the largest U, ordered by
  *       (U descending, page ascending), then -1.  Rows of stable tokens, and of sequences whose
  *       step[s] == 0 (their union is "all pages" anyway), are not written.

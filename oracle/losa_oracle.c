@@ -126,8 +126,11 @@ void oracle_select_active(const oracle_shape_t* sh, const void* x_cur, const voi
  * q_j kmax_j) — the tightest bound those summaries allow.  The 1/sqrt(d) factor is omitted: it
  * does not change the ranking. */
 
-/* fp32, fixed order: products rounded to nearest; each run of 8 consecutive j added left to
- * right; the d/8 run sums combined by c[i] <- c[i] + c[i xor off], off = d/16 .. 1; then + 0.0f. */
+/* fp32 in the order the library's interface fixes (the paper fixes none).  Since kmin <= kmax,
+ * max(q kmin, q kmax) = max(q,0) kmax + min(q,0) kmin, one of the two terms being zero.  Each run
+ * of 8 consecutive j: acc = +0, then for j ascending acc = fma(max(q_j,0), kmax_j, acc) followed by
+ * acc = fma(min(q_j,0), kmin_j, acc); the d/8 run sums are combined by c[i] <- c[i] + c[i xor off],
+ * off = d/16 .. 1; then + 0.0f.  fmaf is the correctly rounded fused operation. */
 static float page_bound_f32(const float* q, const float* lo, const float* hi, int d) {
   float c[64], n[64];
   const int nc = d / 8;
@@ -135,10 +138,10 @@ static float page_bound_f32(const float* q, const float* lo, const float* hi, in
     float acc = 0.0f;
     for (int jj = 0; jj < 8; ++jj) {
       const int j = r * 8 + jj;
-      const float a = q[j] * lo[j];
-      const float b = q[j] * hi[j];
-      const float t = (a > b) ? a : b;
-      acc = (jj == 0) ? t : acc + t;
+      const float qp = (q[j] > 0.0f) ? q[j] : 0.0f;
+      const float qn = (q[j] < 0.0f) ? q[j] : 0.0f;
+      acc = fmaf(qp, hi[j], acc);
+      acc = fmaf(qn, lo[j], acc);
     }
     c[r] = acc;
   }

@@ -4,13 +4,13 @@
 //   page_scores_kernel : each CTA reads the min/max keys of 64 pages of one (sequence, KV head)
 //                        once and scores them against every active query of that KV head.  A page
 //                        is handled by d/8 lanes: one 16-byte vector of kmin and kmax per lane,
-//                        eight products per lane added left to right, then an xor-butterfly over
-//                        the lanes — exactly the summation order the interface fixes, so the fp32
-//                        result is reproducible bit for bit.
-//   topk_kernel        : one CTA per (sequence, active token, head) sorts 64-bit keys
-//                        (order-preserving score bits, inverted page id) with a shared-memory
-//                        bitonic network; the first k keys are the answer in the required order
-//                        (score descending, page ascending), with no tie handling left to do.
+//                        a chain of 16 fused multiply-adds per lane (q+ kmax, q- kmin), then an
+//                        xor-butterfly over the lanes — exactly the order the interface fixes, so
+//                        the fp32 result is reproducible bit for bit.
+//   topk_select_kernel : one warp per (sequence, active token, head); threshold search over
+//                        64-bit keys (order-preserving score bits, inverted page id), see below.
+//   topk_kernel        : budgets above 512 pages: one CTA per query sorts all keys with a
+//                        shared-memory bitonic network.
 //   union_kernel       : one CTA per (sequence, KV head) ORs the selected ids into a bitmap and
 //                        emits the set bits in ascending order with a popcount scan.
 #include "kernels.h"
@@ -40,7 +40,11 @@ page_scores_kernel(const T* __restrict__ q, const T* __restrict__ kmin, const T*
   const int G = Hq / Hkv, rows = na * G;
   if (rows == 0) return;
 
-  __shared__ __align__(16) T qs[kRowTile * D];
+  // positive and negative parts of the staged queries, fp32: U = sum q+ kmax + q- kmin.  A row is
+  // stored as two halves [half][lane chunk][4 floats] so that the d/8 lanes of a page read
+  // consecutive 16-byte words (no bank conflicts): element j = 8*c + e sits at (e/4)*(D/2) + 4*c + e%4.
+  __shared__ __align__(16) float qpos[kRowTile * D];
+  __shared__ __align__(16) float qneg[kRowTile * D];
   __shared__ float sc[kRowTile][kPagesPerCta + 1];
   const int tid = threadIdx.x;
   const int grp = tid / LPP, sub = tid % LPP;
@@ -48,15 +52,19 @@ page_scores_kernel(const T* __restrict__ q, const T* __restrict__ kmin, const T*
 
   for (int r0 = 0; r0 < rows; r0 += kRowTile) {
     const int nr = min(kRowTile, rows - r0);
-    // stage the queries of this row tile (16-byte chunks)
-    constexpr int CH = 16 / sizeof(T);   // elements per 16 bytes
-    for (int idx = tid; idx < nr * (D / CH); idx += kThreads) {
-      const int r = idx / (D / CH), ch = idx % (D / CH);
+    for (int idx = tid; idx < nr * (D / 8); idx += kThreads) {
+      const int r = idx / (D / 8), ch = idx % (D / 8);
       const int row = r0 + r, a = row / G, gi = row % G;
       int tok = active_idx[s * B + a];
       if (tok < 0 || tok >= B) { set_status(status, LOSA_ERR_BOUNDS); tok = 0; }
-      const T* src = q + ((static_cast<size_t>(s) * B + tok) * Hq + kh * G + gi) * D + ch * CH;
-      *reinterpret_cast<uint4*>(&qs[r * D + ch * CH]) = *reinterpret_cast<const uint4*>(src);
+      float v[8];
+      load8(q + ((static_cast<size_t>(s) * B + tok) * Hq + kh * G + gi) * D + ch * 8, v);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int at = r * D + (e >> 2) * (D / 2) + ch * 4 + (e & 3);
+        qpos[at] = fmaxf(v[e], 0.f);
+        qneg[at] = fminf(v[e], 0.f);
+      }
     }
     __syncthreads();
     // the trip count is the same for every lane: the butterfly below needs whole warps
@@ -71,13 +79,19 @@ page_scores_kernel(const T* __restrict__ q, const T* __restrict__ kmin, const T*
         load8(kmin + so, lo);
         load8(kmax + so, hi);
       }
+#pragma unroll 2
       for (int r = 0; r < nr; ++r) {
-        float qv[8];
-        load8(&qs[r * D + sub * 8], qv);
-        float acc = fmaxf(__fmul_rn(qv[0], lo[0]), __fmul_rn(qv[0], hi[0]));
+        float qp[8], qn[8];
+        *reinterpret_cast<float4*>(&qp[0]) = *reinterpret_cast<const float4*>(&qpos[r * D + sub * 4]);
+        *reinterpret_cast<float4*>(&qp[4]) = *reinterpret_cast<const float4*>(&qpos[r * D + D / 2 + sub * 4]);
+        *reinterpret_cast<float4*>(&qn[0]) = *reinterpret_cast<const float4*>(&qneg[r * D + sub * 4]);
+        *reinterpret_cast<float4*>(&qn[4]) = *reinterpret_cast<const float4*>(&qneg[r * D + D / 2 + sub * 4]);
+        float acc = 0.f;
 #pragma unroll
-        for (int j = 1; j < 8; ++j)
-          acc = __fadd_rn(acc, fmaxf(__fmul_rn(qv[j], lo[j]), __fmul_rn(qv[j], hi[j])));
+        for (int j = 0; j < 8; ++j) {
+          acc = __fmaf_rn(qp[j], hi[j], acc);
+          acc = __fmaf_rn(qn[j], lo[j], acc);
+        }
 #pragma unroll
         for (int off = LPP / 2; off >= 1; off >>= 1)
           acc = __fadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
@@ -169,63 +183,68 @@ __device__ __forceinline__ unsigned long long make_key(uint32_t ob, int p) {
          static_cast<unsigned long long>(0xffffffffu - static_cast<uint32_t>(p));
 }
 
-__global__ void __launch_bounds__(kSelWarps * 32)
-topk_select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ kv_len,
-                   const int32_t* __restrict__ active_idx, const int32_t* __restrict__ n_active,
-                   const int32_t* __restrict__ step, int32_t* __restrict__ topk_pages,
-                   float* __restrict__ topk_scores, int N, int B, int Hq, int g, int k, int score_stride,
-                   int32_t* __restrict__ status) {
-  __shared__ unsigned long long s_cand[kSelWarps][kSelCap];
-  __shared__ int s_hist[kSelWarps][kSelBins];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int qid = blockIdx.x * kSelWarps + warp;
-  const int h = qid % Hq, a = (qid / Hq) % B, s = qid / (Hq * B);
-  if (s >= N) return;
-  if (step && step[s] == 0) return;
-  int na = n_active[s];
-  na = na > B ? B : na;
-  if (a >= na) return;
-  const int tok = active_idx[s * B + a];
-  if (tok < 0 || tok >= B) { if (lane == 0) set_status(status, LOSA_ERR_BOUNDS); return; }
-  const int P = pages_of(kv_len[s], g);
-  const int kk = min(k, P);
-  const float* row = scores + ((static_cast<size_t>(s) * B + a) * Hq + h) * score_stride;
-  unsigned long long* cand = s_cand[warp];
-  int* hist = s_hist[warp];
-  const unsigned below = (1u << lane) - 1u;
-
-  uint32_t lo = 0xffffffffu, hi = 0u;
-  for (int p = lane; p < P; p += 32) {
-    const uint32_t ob = order_bits(row[p]);
-    lo = min(lo, ob);
-    hi = max(hi, ob);
+// Visits the warp's keys in page order, 32 per round: f(ob, p, in_range) is called by every lane in
+// every round (so f may use warp-wide votes); in_range says whether p < P.  With CACHED the order
+// bits of the P <= 1024 scores sit in registers (one global pass for the whole selection).
+template <bool CACHED, typename F>
+__device__ __forceinline__ void for_each_key(const uint32_t (&cache)[32], const float* __restrict__ row, int P,
+                                             int lane, F&& f) {
+  if (CACHED) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      if (32 * i >= P) break;
+      const int p = lane + 32 * i;
+      f(cache[i], p, p < P);
+    }
+  } else {
+    for (int base = 0; base < P; base += 32) {
+      const int p = base + lane;
+      f(p < P ? order_bits(row[p]) : 0u, p, p < P);
+    }
   }
+}
+
+template <bool CACHED>
+__device__ __forceinline__ void topk_select_body(const float* __restrict__ row, int P, int kk, int k,
+                                                 unsigned long long* cand, int* hist, int32_t* out_pages,
+                                                 float* out_scores, int lane) {
+  const unsigned below = (1u << lane) - 1u;
+  uint32_t cache[32];
+  if (CACHED) {
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+      const int p = lane + 32 * i;
+      cache[i] = p < P ? order_bits(row[p]) : 0u;
+    }
+  }
+  uint32_t lo = 0xffffffffu, hi = 0u;
+  for_each_key<CACHED>(cache, row, P, lane, [&](uint32_t ob, int, bool in) {
+    if (in) { lo = min(lo, ob); hi = max(hi, ob); }
+  });
   lo = __reduce_min_sync(0xffffffffu, lo);
   hi = __reduce_max_sync(0xffffffffu, hi);
   int need = kk, ncand = 0;
   while (need > 0) {
     if (lo == hi) {
       // every remaining candidate has the same score: lowest pages first, in page order
-      for (int base = 0; base < P && need > 0; base += 32) {
-        const int p = base + lane;
-        const bool hit = p < P && order_bits(row[p]) == lo;
+      for_each_key<CACHED>(cache, row, P, lane, [&](uint32_t ob, int p, bool in) {
+        const bool hit = in && ob == lo && need > 0;
         const unsigned bal = __ballot_sync(0xffffffffu, hit);
         const int rank = __popc(bal & below);
         if (hit && rank < need) cand[ncand + rank] = make_key(lo, p);
         const int taken = min(need, __popc(bal));
         ncand += taken;
         need -= taken;
-      }
+      });
       break;
     }
     const int width = 32 - __clz(hi - lo);           // bits needed for hi - lo  (>= 1)
     const int shift = width > 8 ? width - 8 : 0;      // (ob - lo) >> shift is in [0, 255]
     for (int b = lane; b < kSelBins; b += 32) hist[b] = 0;
     __syncwarp();
-    for (int p = lane; p < P; p += 32) {
-      const uint32_t ob = order_bits(row[p]);
-      if (ob >= lo && ob <= hi) atomicAdd(&hist[(ob - lo) >> shift], 1);
-    }
+    for_each_key<CACHED>(cache, row, P, lane, [&](uint32_t ob, int, bool in) {
+      if (in && ob >= lo && ob <= hi) atomicAdd(&hist[(ob - lo) >> shift], 1);
+    });
     __syncwarp();
     // lane owns bins [8*lane, 8*lane+8); suffix sums over lanes locate the threshold bin
     int c[8], tot = 0;
@@ -254,21 +273,16 @@ topk_select_kernel(const float* __restrict__ scores, const int32_t* __restrict__
     cnt_thr = __shfl_sync(0xffffffffu, cnt_thr, src);
     const bool finish = ncand + cnt_above + cnt_thr <= kSelCap;
     // take the keys above the threshold bin (and, when finishing, the threshold bin itself)
-    for (int base = 0; base < P; base += 32) {
-      const int p = base + lane;
+    for_each_key<CACHED>(cache, row, P, lane, [&](uint32_t ob, int p, bool in) {
       bool take = false;
-      uint32_t ob = 0;
-      if (p < P) {
-        ob = order_bits(row[p]);
-        if (ob >= lo && ob <= hi) {
-          const int bin = static_cast<int>((ob - lo) >> shift);
-          take = bin > bstar || (finish && bin == bstar);
-        }
+      if (in && ob >= lo && ob <= hi) {
+        const int bin = static_cast<int>((ob - lo) >> shift);
+        take = bin > bstar || (finish && bin == bstar);
       }
       const unsigned bal = __ballot_sync(0xffffffffu, take);
       if (take) cand[ncand + __popc(bal & below)] = make_key(ob, p);
       ncand += __popc(bal);
-    }
+    });
     if (finish) break;
     need -= cnt_above;
     const uint32_t nlo = lo + (static_cast<uint32_t>(bstar) << shift);
@@ -292,16 +306,45 @@ topk_select_kernel(const float* __restrict__ scores, const int32_t* __restrict__
       __syncwarp();
     }
   }
-  const size_t o = ((static_cast<size_t>(s) * B + tok) * Hq + h) * k;
   for (int j = lane; j < k; j += 32) {
     if (j < kk) {
       const unsigned long long key = cand[j];
-      topk_pages[o + j] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(key));
-      if (topk_scores) topk_scores[o + j] = unorder_bits(static_cast<uint32_t>(key >> 32));
+      out_pages[j] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(key));
+      if (out_scores) out_scores[j] = unorder_bits(static_cast<uint32_t>(key >> 32));
     } else {
-      topk_pages[o + j] = -1;
+      out_pages[j] = -1;
     }
   }
+}
+
+__global__ void __launch_bounds__(kSelWarps * 32)
+topk_select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ kv_len,
+                   const int32_t* __restrict__ active_idx, const int32_t* __restrict__ n_active,
+                   const int32_t* __restrict__ step, int32_t* __restrict__ topk_pages,
+                   float* __restrict__ topk_scores, int N, int B, int Hq, int g, int k, int score_stride,
+                   int32_t* __restrict__ status) {
+  __shared__ unsigned long long s_cand[kSelWarps][kSelCap];
+  __shared__ int s_hist[kSelWarps][kSelBins];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int qid = blockIdx.x * kSelWarps + warp;
+  const int h = qid % Hq, a = (qid / Hq) % B, s = qid / (Hq * B);
+  if (s >= N) return;
+  if (step && step[s] == 0) return;
+  int na = n_active[s];
+  na = na > B ? B : na;
+  if (a >= na) return;
+  const int tok = active_idx[s * B + a];
+  if (tok < 0 || tok >= B) { if (lane == 0) set_status(status, LOSA_ERR_BOUNDS); return; }
+  const int P = pages_of(kv_len[s], g);
+  const int kk = min(k, P);
+  const float* row = scores + ((static_cast<size_t>(s) * B + a) * Hq + h) * score_stride;
+  const size_t o = ((static_cast<size_t>(s) * B + tok) * Hq + h) * k;
+  if (P <= 1024)
+    topk_select_body<true>(row, P, kk, k, s_cand[warp], s_hist[warp], topk_pages + o,
+                           topk_scores ? topk_scores + o : nullptr, lane);
+  else
+    topk_select_body<false>(row, P, kk, k, s_cand[warp], s_hist[warp], topk_pages + o,
+                            topk_scores ? topk_scores + o : nullptr, lane);
 }
 
 __global__ void __launch_bounds__(kThreads)

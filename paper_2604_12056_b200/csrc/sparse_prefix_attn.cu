@@ -8,13 +8,15 @@
 // segment by log-sum-exp — the same merge Section 2.2 uses between prefix and block — and writes
 // (o_p, L_p) of the ACTIVE tokens only, which is what keeps the reuse rule exact for the others.
 //
-// bf16 kernel: one producer warp resolves union position -> logical page -> physical page 32
-//   items ahead and streams each page's K and V slice into a ring of shared-memory stages with
+// bf16 kernel: four producer warps resolve union position -> logical page -> physical page two
+//   batches ahead and stream each page's K and V slice into a ring of shared-memory stages with
 //   TMA tensor copies (128-byte swizzle, completion on an mbarrier); eight consumer warps run
 //   Q K^T and P V on the tensor cores (bf16 m16n8k16, fp32 accumulate) straight from the swizzled
 //   tiles with ldmatrix, with an online softmax in registers.  Query rows are the GQA-grouped
 //   (active token, head) pairs of the KV head: 16-row tiles; with few rows the eight warps take
 //   different pages of the ring, with many rows they take different row tiles of the same page.
+//   Consumer warps never synchronise with each other: each keeps its own (m, l, o), reads its own
+//   query fragments from global memory and writes its own 16-row record per (CTA, segment) piece.
 // fp32 kernel: CUDA cores, fp32 FMA (bf16 tensor cores cannot meet the 1e-5 fp32 tolerance).
 //
 // Every wait on an mbarrier is bounded; when a bound runs out the CTA records LOSA_ERR_TIMEOUT,
@@ -43,7 +45,7 @@ struct AttnParams {
   float* o_p;
   float* lse_p;
   int32_t* status;
-  int B, Hq, Hkv, G, Pmax, n_phys, n_rg, n_seg, n_ctas;
+  int N, B, Hq, Hkv, G, Pmax, n_phys, n_rg, n_seg, n_ctas;
   float sm_scale;
 #ifdef LOSA_TRACE
   unsigned long long* trace;   // [n_ctas][8] timestamps, development builds only
@@ -61,8 +63,18 @@ __device__ __forceinline__ unsigned long long gtime() {
 #define LOSA_STAMP(slot) do { } while (0)
 #endif
 
-__device__ __forceinline__ float* partial_base(float* partials, int slot, int D) {
-  return partials + static_cast<size_t>(slot) * kRowsPerGroup * (D + 2);
+// Partial results.  A slot (CTA b, segment seg -> b + seg) holds eight records of one 16-row tile
+// each: m[16], l[16], o[16][D] (un-normalised, relative to m).  The tensor-core kernel writes one
+// record per consumer warp; the fp32 kernel writes record t for rows 16t .. 16t+15.
+constexpr int kTileRows = 16;
+__device__ __forceinline__ float* record_base(float* partials, int slot, int w, int D) {
+  return partials + (static_cast<size_t>(slot) * 8 + w) * kTileRows * (D + 2);
+}
+// How the eight consumer warps split a segment with `rows` query rows: nrtp row tiles (padded to a
+// power of two) times ns = 8 / nrtp page slots.
+__device__ __forceinline__ int row_tiles_padded(int rows) {
+  const int nrt = (rows + kTileRows - 1) / kTileRows;
+  return nrt <= 1 ? 1 : (nrt <= 2 ? 2 : (nrt <= 4 ? 4 : 8));
 }
 
 __device__ __forceinline__ int clamp_active(int na, int B) { return na < 0 ? 0 : (na > B ? B : na); }
@@ -175,9 +187,15 @@ __global__ void __launch_bounds__(256, 1) attn_simt_kernel(AttnParams p) {
       }
     }
     __syncthreads();
-    float* part = partial_base(p.partials, blockIdx.x + sg, D);
-    for (int r = tid; r < rows; r += 256) { part[r] = Ms[r]; part[kRowsPerGroup + r] = Ls[r]; }
-    for (int idx = tid; idx < rows * D; idx += 256) part[2 * kRowsPerGroup + idx] = Os[idx];
+    for (int r = tid; r < rows; r += 256) {
+      float* rec = record_base(p.partials, blockIdx.x + sg, r / kTileRows, D);
+      rec[r % kTileRows] = Ms[r];
+      rec[kTileRows + r % kTileRows] = Ls[r];
+    }
+    for (int idx = tid; idx < rows * D; idx += 256) {
+      const int r = idx / D;
+      record_base(p.partials, blockIdx.x + sg, r / kTileRows, D)[2 * kTileRows + (r % kTileRows) * D + idx % D] = Os[idx];
+    }
     item = seg_end;
     ++sg;
     while (item < hi && pre[sg + 1] <= item) ++sg;
@@ -186,10 +204,12 @@ __global__ void __launch_bounds__(256, 1) attn_simt_kernel(AttnParams p) {
 
 // ===================================================================== combine kernel
 // grid (n_seg, 16): warp = one query row of the segment's row group.  The CTAs whose item range
-// meets the segment are consecutive; lanes take one piece each for the row maxima and sums, then
-// the warp walks the pieces with every load of a group of four issued together.  LOG2 says
-// whether the partial maxima are in base-2 units (tensor-core kernel) or natural units (fp32).
-template <int D, bool LOG2>
+// meets the segment are consecutive; each of them left up to `ns` records for the row's tile (one
+// per page slot).  Lanes take one (piece, slot) pair each for the row maxima and sums, then the
+// warp walks the pairs with the loads of four records issued together.  LOG2: partial maxima in
+// base-2 units (tensor-core kernel) or natural units (fp32 kernel, which writes one record per
+// row tile: SIMT).
+template <int D, bool LOG2, bool SIMT>
 __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
   __shared__ int pre[kMaxSegments + 1];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -206,6 +226,8 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
   const size_t orow = (static_cast<size_t>(s) * p.B + tok) * p.Hq + kh * p.G + gi;
   const int start = pre[sg], end = pre[sg + 1];
   const long long T_all = pre[p.n_seg];
+  const int nrtp = SIMT ? 8 : row_tiles_padded(rows), ns = 8 / nrtp;
+  const int tile = r / kTileRows, rr = r % kTileRows;
   constexpr int C = D / 32;
   float acc[C];
 #pragma unroll
@@ -216,38 +238,38 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
     while (b0 + 1 < p.n_ctas && cta_lo(T_all, b0 + 1, p.n_ctas) <= start) ++b0;
     int b1 = static_cast<int>((static_cast<long long>(end - 1) * p.n_ctas) / T_all);   // last CTA that can meet it
     while (b1 + 1 < p.n_ctas && cta_lo(T_all, b1 + 1, p.n_ctas) < end) ++b1;
-    // pass 1: the row maximum over the pieces
-    for (int base = b0; base <= b1; base += 32) {
-      const int b = base + lane;
-      float mj = -INFINITY;
-      if (b <= b1) {
-        const long long lo = cta_lo(T_all, b, p.n_ctas), hi = cta_lo(T_all, b + 1, p.n_ctas);
-        if (lo < end && hi > start && hi > lo) mj = partial_base(p.partials, b + sg, D)[r];
-      }
-      M = fmaxf(M, warp_max(mj));
+    const int n_pairs = (b1 - b0 + 1) * ns;
+    // record of pair x (piece x / ns, page slot x % ns), or null when that warp had no page
+    auto record_of = [&](int x) -> const float* {
+      if (x >= n_pairs) return nullptr;
+      const int b = b0 + x / ns, sl = x % ns;
+      const long long lo = max(cta_lo(T_all, b, p.n_ctas), static_cast<long long>(start));
+      const long long hi = min(cta_lo(T_all, b + 1, p.n_ctas), static_cast<long long>(end));
+      if (hi - lo <= sl) return nullptr;              // fewer pages in the piece than this slot index
+      return record_base(p.partials, b + sg, tile + nrtp * sl, D);
+    };
+    for (int base = 0; base < n_pairs; base += 32) {
+      const float* rec = record_of(base + lane);
+      M = fmaxf(M, warp_max(rec ? rec[rr] : -INFINITY));
     }
-    // pass 2: weights, sum and output
-    for (int base = b0; base <= b1; base += 32) {
-      const int b = base + lane;
+    for (int base = 0; base < n_pairs; base += 32) {
+      const float* rec = record_of(base + lane);
       float wj = 0.f, lj = 0.f;
-      if (b <= b1) {
-        const long long lo = cta_lo(T_all, b, p.n_ctas), hi = cta_lo(T_all, b + 1, p.n_ctas);
-        if (lo < end && hi > start && hi > lo) {
-          const float* part = partial_base(p.partials, b + sg, D);
-          const float mj = part[r];
-          wj = (mj == -INFINITY) ? 0.f : (LOG2 ? exp2f(mj - M) : expf(mj - M));
-          lj = part[kRowsPerGroup + r];
-        }
+      if (rec) {
+        const float mj = rec[rr];
+        wj = (mj == -INFINITY) ? 0.f : (LOG2 ? exp2f(mj - M) : expf(mj - M));
+        lj = rec[kTileRows + rr];
       }
       Lsum += warp_sum(lj * wj);
-      const int n = min(32, b1 - base + 1);
+      const int n = min(32, n_pairs - base);
       for (int i0 = 0; i0 < n; i0 += 4) {
         float w[4], v[4][C];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
           const int i = i0 + u;
           w[u] = (i < n) ? __shfl_sync(0xffffffffu, wj, i & 31) : 0.f;
-          const float* src = partial_base(p.partials, base + i + sg, D) + 2 * kRowsPerGroup + r * D + lane;
+          const unsigned long long addr = __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(rec), i & 31);
+          const float* src = reinterpret_cast<const float*>(addr) + 2 * kTileRows + rr * D + lane;
 #pragma unroll
           for (int c = 0; c < C; ++c) v[u][c] = (w[u] != 0.f) ? src[32 * c] : 0.f;
         }
@@ -267,20 +289,21 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
 
 // ===================================================================== bf16 TMA + tensor-core kernel
 constexpr int kConsumerWarps = 8;
-constexpr int kMmaThreads = (kConsumerWarps + 1) * 32;
+constexpr int kProducerWarps = 4;    // registers are allocated per 4 warps: 9 warps would cost the same as 12
+constexpr int kMmaThreads = (kConsumerWarps + kProducerWarps) * 32;
 constexpr long long kWaitCycles = 2000000000ll;   // ~1 s: bound of every mbarrier wait
 constexpr int kSmemBudget = 232448;                // 227 KB opt-in limit per CTA
 
-template <int D> constexpr int q_stride_bytes() { return D * 2 + 16; }
-template <int D> constexpr int q_region_bytes() { return kRowsPerGroup * q_stride_bytes<D>(); }
 template <int D, int GP> constexpr int stage_bytes() { return 2 * GP * D * 2; }
-constexpr int kTailBytes = 512 + (kMaxSegments + 1) * 4;   // barriers, per-stage meta, flags, prefix
+constexpr int kStageIdx = 1024;     // active_idx entries (N * B) cached in shared memory when they fit
+constexpr int kStageSeq = 64;       // ... together with n_active and kv_len of up to this many sequences
+constexpr int kTailBytes = 512 + (kMaxSegments + 1) * 4 + 4 + kStageIdx * 4 + 2 * kStageSeq * 4;   // barriers, meta, prefix, index cache
 template <int D, int GP> constexpr int n_stages() {
-  const int n = (kSmemBudget - 1024 - q_region_bytes<D>() - kTailBytes) / stage_bytes<D, GP>();
+  const int n = (kSmemBudget - 1024 - kTailBytes) / stage_bytes<D, GP>();
   return n > 16 ? 16 : n;
 }
 template <int D, int GP> constexpr int mma_smem_bytes() {
-  return 1024 + n_stages<D, GP>() * stage_bytes<D, GP>() + q_region_bytes<D>() + kTailBytes;
+  return 1024 + n_stages<D, GP>() * stage_bytes<D, GP>() + kTailBytes;
 }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* ptr) {
@@ -326,6 +349,7 @@ __device__ __forceinline__ bool wait_round(volatile int* tag, int round, volatil
   if (*tag == round) return true;
   const long long t0 = clock64();
   while (*tag != round) {
+    __nanosleep(64);                 // the producers share this SM's issue slots: do not spin hot
     if (*abort_flag) return false;
     if (clock64() - t0 > kWaitCycles) {
       *abort_flag = 1;
@@ -340,6 +364,17 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
   asm volatile(
       "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+// Loads whose issue point must stay where it is written (they are prefetches): volatile asm.
+__device__ __forceinline__ int ld_nc_s32(const int32_t* ptr) {
+  int v;
+  asm volatile("ld.global.nc.s32 %0, [%1];" : "=r"(v) : "l"(ptr));
+  return v;
+}
+__device__ __forceinline__ uint32_t ld_nc_u32(const uint32_t* ptr) {
+  uint32_t v;
+  asm volatile("ld.global.nc.b32 %0, [%1];" : "=r"(v) : "l"(ptr));
+  return v;
 }
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
   asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -359,7 +394,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
-__device__ __forceinline__ void consumer_bar() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 
 // Byte offset of 16-byte chunk `chunk` (0 .. D/8-1) of token row `t` inside a K or V tile that TMA
 // wrote as D/64 boxes of [GP rows][64 bf16] with the 128-byte swizzle.
@@ -377,7 +411,6 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   constexpr int NT = GP / 8;        // score n-tiles per page
   constexpr int KS = D / 16;        // k-steps of Q K^T
   constexpr int ND = D / 8;         // output n-tiles
-  constexpr int QSTR = q_stride_bytes<D>();
   constexpr int OREGS = ND * 4;
 
   extern __shared__ uint8_t smem_raw[];
@@ -385,15 +418,17 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   const uint32_t base = (raw + 1023u) & ~1023u;          // swizzled tiles need 1024-byte alignment
   uint8_t* gen = smem_raw + (base - raw);                 // generic pointer to the same place
   const uint32_t stage0 = base;
-  const uint32_t qs = base + NSTAGE * STAGE;
-  uint8_t* qs_gen = gen + NSTAGE * STAGE;
-  uint8_t* tail = qs_gen + q_region_bytes<D>();
-  const uint32_t full0 = qs + q_region_bytes<D>();       // full[NSTAGE], then empty[NSTAGE]
+  uint8_t* tail = gen + NSTAGE * STAGE;
+  const uint32_t full0 = base + NSTAGE * STAGE;          // full[NSTAGE], then empty[NSTAGE]
   const uint32_t empty0 = full0 + 8 * NSTAGE;
   volatile int* meta = reinterpret_cast<volatile int*>(tail + 16 * NSTAGE);        // valid tokens per stage
   volatile int* stage_round = meta + NSTAGE;   // which pass over the ring the stage's current page belongs to
   volatile int* abort_flag = stage_round + NSTAGE;
   int* pre = reinterpret_cast<int*>(tail + 512);
+  int* tok_s = pre + kMaxSegments + 2;          // [N][B] active_idx, when staged
+  int* na_s = tok_s + kStageIdx;                // [N] clamped n_active
+  int* len_s = na_s + kStageSeq;                // [N] kv_len
+  const bool staged = p.N * p.B <= kStageIdx && p.N <= kStageSeq;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) LOSA_STAMP(0);
@@ -407,7 +442,17 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 0) segment_prefix(pre, p.n_seg, p.n_rg, p.Hkv, p.G, p.n_active, p.union_count, p.B, lane);
+  if (warp == 0) {
+    segment_prefix(pre, p.n_seg, p.n_rg, p.Hkv, p.G, p.n_active, p.union_count, p.B, lane);
+  } else if (staged) {
+    // The small index arrays are read now, while the memory system is idle: once the page stream
+    // saturates it, every dependent global load costs microseconds of queueing.
+    for (int i = tid - 32; i < p.N * p.B; i += kMmaThreads - 32) tok_s[i] = p.active_idx[i];
+    for (int i = tid - 32; i < p.N; i += kMmaThreads - 32) {
+      na_s[i] = clamp_active(p.n_active[i], p.B);
+      len_s[i] = p.kv_len[i];
+    }
+  }
   __syncthreads();
   const long long T_all = pre[p.n_seg];
   const int lo = static_cast<int>(cta_lo(T_all, blockIdx.x, p.n_ctas));
@@ -416,33 +461,70 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   int sg0 = 0;
   while (pre[sg0 + 1] <= lo) ++sg0;
   if (tid == 0) LOSA_STAMP(1);
+  auto n_active_of = [&](int s) { return staged ? na_s[s] : clamp_active(p.n_active[s], p.B); };
+  auto kv_len_of = [&](int s) { return staged ? len_s[s] : p.kv_len[s]; };
+  auto token_of = [&](int s, int a) { return staged ? tok_s[s * p.B + a] : p.active_idx[s * p.B + a]; };
 
-  if (warp == kConsumerWarps) {
+  if (warp >= kConsumerWarps) {
     // ------------------------------------------------------------------ producer warp
-    int sg = sg0;
-    for (int b0 = lo; b0 < hi; b0 += 32) {
-      const int i = b0 + lane;
-      int phys = 0, kh = 0, valid = 0;
+    // Issuing a page (four tensor copies plus barrier traffic) costs one thread ~0.3 us, more than
+    // the 0.37 us the HBM needs to deliver it, so kProducerWarps warps share the work: producer w
+    // takes the CTA's items w, w + kProducerWarps, ...  Lane j of a batch of 32 such items resolves
+    // item -> logical page -> physical page.  The two loads depend on each other, so they run as a
+    // pipeline over batches: while the copies of batch k are issued, the physical pages of batch
+    // k+1 and the logical pages of batch k+2 are in flight.
+    const int pw = warp - kConsumerWarps;
+    constexpr int STEP = 32 * kProducerWarps;       // items covered by one batch of every producer
+    int cursor = sg0;                               // segment cursor of the first pipeline stage
+    int page_a = -1, sk_a = 0;                      // batch k+1: logical page (loaded) and its (sequence, KV head)
+    int phys_b = 0, kh_b = 0, valid_b = 0;          // batch k  : ready to issue
+    auto stage_a = [&](int i, int& page, int& sk) {
+      page = -1; sk = 0;
       if (i < hi) {
-        while (pre[sg + 1] <= i) ++sg;
-        const int u = i - pre[sg], sk = sg / p.n_rg, s = sk / p.Hkv;
-        kh = sk % p.Hkv;
-        const int page = p.union_pages[static_cast<size_t>(sk) * p.Pmax + u];
-        bool ok = page >= 0 && page < p.Pmax;
-        phys = ok ? p.page_table[static_cast<size_t>(s) * p.Pmax + page] : 0;
-        ok = ok && phys >= 0 && phys < p.n_phys;
-        valid = ok ? min(GP, p.kv_len[s] - page * GP) : 0;
-        if (!ok || valid <= 0) { set_status(p.status, LOSA_ERR_BOUNDS); phys = 0; valid = 0; }
+        while (pre[cursor + 1] <= i) ++cursor;
+        sk = cursor / p.n_rg;
+        page = ld_nc_s32(p.union_pages + static_cast<size_t>(sk) * p.Pmax + (i - pre[cursor]));
       }
-      const int nb = min(32, hi - b0);
+    };
+    auto stage_b = [&](int i, int page, int sk, int& phys, int& kh, int& valid) {
+      phys = 0; kh = 0; valid = 0;
+      if (i < hi) {
+        const int s = sk / p.Hkv;
+        kh = sk % p.Hkv;
+        const bool ok = page >= 0 && page < p.Pmax;
+        phys = ok ? ld_nc_s32(p.page_table + static_cast<size_t>(s) * p.Pmax + page) : -1;
+        valid = ok ? min(GP, kv_len_of(s) - page * GP) : 0;
+      }
+    };
+    const int mine = lo + pw + kProducerWarps * lane;        // this lane's item in the first batch
+    stage_a(mine, page_a, sk_a);
+    stage_b(mine, page_a, sk_a, phys_b, kh_b, valid_b);
+    stage_a(mine + STEP, page_a, sk_a);
+    for (int b0 = lo; b0 + pw < hi; b0 += STEP) {
+      int page_n, sk_n, phys_n, kh_n, valid_n;
+      const int i_lane = b0 + pw + kProducerWarps * lane;
+      stage_a(i_lane + 2 * STEP, page_n, sk_n);
+      stage_b(i_lane + STEP, page_a, sk_a, phys_n, kh_n, valid_n);
+      if (i_lane < hi && (phys_b < 0 || phys_b >= p.n_phys || valid_b <= 0)) {
+        set_status(p.status, LOSA_ERR_BOUNDS);
+        phys_b = 0;
+        valid_b = 0;
+      }
+      const int nb = min(32, (hi - b0 - pw + kProducerWarps - 1) / kProducerWarps);
       for (int j = 0; j < nb; ++j) {
-        const int ph = __shfl_sync(0xffffffffu, phys, j);
-        const int khj = __shfl_sync(0xffffffffu, kh, j);
-        const int vj = __shfl_sync(0xffffffffu, valid, j);
+        const int ph = __shfl_sync(0xffffffffu, phys_b, j);
+        const int khj = __shfl_sync(0xffffffffu, kh_b, j);
+        const int vj = __shfl_sync(0xffffffffu, valid_b, j);
         if (lane == 0) {
-          const int it = b0 + j - lo, stage = it % NSTAGE, round = it / NSTAGE;
-          const bool go = mbar_wait(empty0 + 8 * stage, (round & 1) ^ 1, abort_flag, p.status);
+          const int it = b0 + pw + kProducerWarps * j - lo, stage = it % NSTAGE, round = it / NSTAGE;
+          // Another producer fills this stage in the previous pass over the ring; until it has
+          // done so (tag == round - 1) the parity wait below would look at the wrong phase.
+          const bool go = (round == 0 || wait_round(stage_round + stage, round - 1, abort_flag, p.status)) &&
+                          mbar_wait(empty0 + 8 * stage, (round & 1) ^ 1, abort_flag, p.status);
           if (go) {
+#ifdef LOSA_TRACE
+            if (p.trace && it < 80) p.trace[p.n_ctas * 34 + (blockIdx.x * 80 + it) * 2] = gtime();
+#endif
             if (it == 0) LOSA_STAMP(7);                  // about to issue the first copy
             if (it == NSTAGE - 1) LOSA_STAMP(2);         // ring filled once without waiting
             meta[stage] = vj;
@@ -457,13 +539,17 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
           }
         }
       }
-      sg = __shfl_sync(0xffffffffu, sg, nb - 1);
+      page_a = page_n; sk_a = sk_n;
+      phys_b = phys_n; kh_b = kh_n; valid_b = valid_n;
     }
-    if (lane == 0) LOSA_STAMP(3);                    // all copies issued
+    if (lane == 0 && pw == 0) LOSA_STAMP(3);         // producer 0 has issued all its copies
     return;
   }
 
   // -------------------------------------------------------------------- consumer warps
+  // Each warp is on its own: it reads its query fragments straight from global memory, keeps its own
+  // running (m, l, o) and leaves its own 16-row record per piece; no barrier ties the warps of a
+  // CTA together, so a change of segment stalls one warp for one memory latency, nothing else.
   const __nv_bfloat16* q = static_cast<const __nv_bfloat16*>(p.q);
   const int g8 = lane >> 2, q4 = lane & 3;
   const float scale2 = p.sm_scale * kLog2e;
@@ -471,44 +557,82 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #ifdef LOSA_TRACE
   long long trace_wait = 0, trace_busy = 0;
 #endif
-  while (item < hi) {
-    const int seg_end = min(hi, pre[sg + 1]);
-    const int npg = seg_end - item;
-    const int rg = sg % p.n_rg, sk = sg / p.n_rg, s = sk / p.Hkv, kh = sk % p.Hkv;
-    const int rows = rows_in_group(clamp_active(p.n_active[s], p.B), p.G, rg);
-    const int nrt = (rows + 15) >> 4;
-    const int nrtp = nrt <= 1 ? 1 : (nrt <= 2 ? 2 : (nrt <= 4 ? 4 : 8));
-    const int ns = kConsumerWarps / nrtp;
-    const int rt = warp % nrtp, slot = warp / nrtp;
-    const bool has_rows = rt < nrt;
-
-    // ---- gather the query rows of this row group (16-byte chunks, padded row stride)
-    consumer_bar();
-    for (int idx = tid; idx < nrtp * 16 * (D / 8); idx += kConsumerWarps * 32) {
-      const int r = idx / (D / 8), ch = idx % (D / 8);
-      uint4 v = make_uint4(0u, 0u, 0u, 0u);
-      if (r < rows) {
-        const int row = rg * kRowsPerGroup + r, a = row / p.G, gi = row % p.G;
-        int tok = p.active_idx[s * p.B + a];
-        if (tok < 0 || tok >= p.B) { set_status(p.status, LOSA_ERR_BOUNDS); tok = 0; }
-        v = *reinterpret_cast<const uint4*>(q + ((static_cast<size_t>(s) * p.B + tok) * p.Hq + kh * p.G + gi) * D + ch * 8);
-      }
-      *reinterpret_cast<uint4*>(qs_gen + r * QSTR + ch * 16) = v;
-    }
-    consumer_bar();
-    uint32_t qf[KS][4];
-    {
-      const int mi = lane >> 3, r = rt * 16 + (mi & 1) * 8 + (lane & 7);
+  // How this warp takes part in the piece of segment `g` that starts at item `first`.
+  struct Piece { int seg_end, npg, rows, nrt, nrtp, ns, rt, slot, s, kh, rg; bool has_rows, works; };
+  auto piece_of = [&](int g, int first) {
+    Piece c;
+    c.seg_end = min(hi, pre[g + 1]);
+    c.npg = c.seg_end - first;
+    c.rg = g % p.n_rg;
+    const int sk = g / p.n_rg;
+    c.s = sk / p.Hkv;
+    c.kh = sk % p.Hkv;
+    c.rows = rows_in_group(n_active_of(c.s), p.G, c.rg);
+    c.nrt = (c.rows + kTileRows - 1) / kTileRows;
+    c.nrtp = row_tiles_padded(c.rows);
+    c.ns = kConsumerWarps / c.nrtp;
+    c.rt = warp % c.nrtp;
+    c.slot = warp / c.nrtp;
+    c.has_rows = c.rt < c.nrt;
+    c.works = c.has_rows && c.slot < c.npg;
+    return c;
+  };
+  // Row pointers of this lane's two rows (rt*16 + g8, +8) of a piece, null for padding rows.
+  auto row_ptrs = [&](const Piece& c, const uint32_t* (&rowp)[2]) {
 #pragma unroll
-      for (int ks = 0; ks < KS; ++ks) ldsm_x4(qs + r * QSTR + (ks * 2 + (mi >> 1)) * 16, qf[ks]);
+    for (int hrow = 0; hrow < 2; ++hrow) {
+      const int r = c.rt * kTileRows + g8 + 8 * hrow;
+      rowp[hrow] = nullptr;
+      if (c.works && r < c.rows) {
+        const int row = c.rg * kRowsPerGroup + r, a = row / p.G, gi = row % p.G;
+        int tok = token_of(c.s, a);
+        if (tok < 0 || tok >= p.B) { set_status(p.status, LOSA_ERR_BOUNDS); tok = 0; }
+        rowp[hrow] = reinterpret_cast<const uint32_t*>(q + ((static_cast<size_t>(c.s) * p.B + tok) * p.Hq + c.kh * p.G + gi) * D);
+      }
     }
-    consumer_bar();   // the Q region now doubles as scratch for the cross-warp merge
+  };
+  // Pulls the query rows of a later piece into L2 (no registers held).
+  auto prefetch_q = [&](const Piece& c) {
+    const uint32_t* rowp[2];
+    row_ptrs(c, rowp);
+#pragma unroll
+    for (int hrow = 0; hrow < 2; ++hrow)
+      if (rowp[hrow] && q4 < (D * 2 + 127) / 128)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const char*>(rowp[hrow]) + q4 * 128));
+  };
+  // A fragments: 4-byte loads of two adjacent bf16, zero for padding rows.
+  auto load_q = [&](const Piece& c, uint32_t (&dst)[KS][4]) {
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) { dst[ks][0] = dst[ks][1] = dst[ks][2] = dst[ks][3] = 0u; }
+    const uint32_t* rowp[2];
+    row_ptrs(c, rowp);
+#pragma unroll
+    for (int ks = 0; ks < KS; ++ks) {
+      const int w0 = ks * 8 + q4;                     // 32-bit word index of columns ks*16 + q4*2
+      if (rowp[0]) { dst[ks][0] = ld_nc_u32(rowp[0] + w0); dst[ks][2] = ld_nc_u32(rowp[0] + w0 + 4); }
+      if (rowp[1]) { dst[ks][1] = ld_nc_u32(rowp[1] + w0); dst[ks][3] = ld_nc_u32(rowp[1] + w0 + 4); }
+    }
+  };
+  Piece cur = piece_of(sg, item);
+  uint32_t qf[KS][4];
+  load_q(cur, qf);
+  while (item < hi) {
+    const int seg_end = cur.seg_end, npg = cur.npg, ns = cur.ns, slot = cur.slot;
+    const bool has_rows = cur.has_rows, works = cur.works;
+    // The next piece's query rows are pulled into L2 now and loaded after this piece's pages: a
+    // miss then would cost microseconds, because the page stream keeps the memory queues full.
+    int sg_next = sg + 1;
+    while (seg_end < hi && pre[sg_next + 1] <= seg_end) ++sg_next;
+    Piece nxt = cur;
+    if (seg_end < hi) {
+      nxt = piece_of(sg_next, seg_end);
+      prefetch_q(nxt);
+    }
 
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
     float oacc[ND][4];
 #pragma unroll
     for (int n = 0; n < ND; ++n) { oacc[n][0] = oacc[n][1] = oacc[n][2] = oacc[n][3] = 0.f; }
-
     // Page j of the piece belongs to the warps of page slot j % ns (one warp per row tile).  Only
     // they wait for it and release it, each with weight ns, so that a stage always collects
     // kConsumerWarps arrivals and is refilled as soon as ITS readers are done with it.
@@ -524,6 +648,7 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #ifdef LOSA_TRACE
       const long long tw1 = clock64();
       trace_wait += tw1 - tw0;
+      if (lane == 0 && p.trace && it < 80) p.trace[p.n_ctas * 34 + (blockIdx.x * 80 + it) * 2 + 1] = gtime();
 #endif
       if (tid == 0 && it == 0) LOSA_STAMP(4);        // first page landed
       if (ready && has_rows) {
@@ -631,72 +756,40 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     }
 
     if (tid == 0 && seg_end == hi) LOSA_STAMP(5);    // warp 0 done with its pages
-    // ---- merge the page slots of each row tile through shared memory (tree), slot 0 keeps it
-    float* scr = reinterpret_cast<float*>(qs_gen);
-    for (int stride = ns >> 1; stride >= 1; stride >>= 1) {
-      const int nw = stride * nrtp;                 // writers this round
-      if (slot >= stride && slot < 2 * stride) {
-        const int w = (slot - stride) * nrtp + rt;
-        float* dst = scr + w * 32 + lane;
-        dst[0 * nw * 32] = m0; dst[1 * nw * 32] = m1; dst[2 * nw * 32] = l0; dst[3 * nw * 32] = l1;
-#pragma unroll
-        for (int n = 0; n < ND; ++n)
-#pragma unroll
-          for (int e = 0; e < 4; ++e) dst[(4 + n * 4 + e) * nw * 32] = oacc[n][e];
-      }
-      consumer_bar();
-      if (slot < stride) {
-        const int w = slot * nrtp + rt;
-        const float* src = scr + w * 32 + lane;
-        const float pm0 = src[0 * nw * 32], pm1 = src[1 * nw * 32];
-        const float pl0 = src[2 * nw * 32], pl1 = src[3 * nw * 32];
-        const float mn0 = fmaxf(m0, pm0), mn1 = fmaxf(m1, pm1);
-        const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0, ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
-        const float a0 = exp2f(m0 - ms0), b0 = exp2f(pm0 - ms0);
-        const float a1 = exp2f(m1 - ms1), b1 = exp2f(pm1 - ms1);
-        m0 = mn0; m1 = mn1;
-        l0 = l0 * a0 + pl0 * b0;
-        l1 = l1 * a1 + pl1 * b1;
-#pragma unroll
-        for (int n = 0; n < ND; ++n) {
-          oacc[n][0] = oacc[n][0] * a0 + src[(4 + n * 4 + 0) * nw * 32] * b0;
-          oacc[n][1] = oacc[n][1] * a0 + src[(4 + n * 4 + 1) * nw * 32] * b0;
-          oacc[n][2] = oacc[n][2] * a1 + src[(4 + n * 4 + 2) * nw * 32] * b1;
-          oacc[n][3] = oacc[n][3] * a1 + src[(4 + n * 4 + 3) * nw * 32] * b1;
-        }
-      }
-      consumer_bar();
-    }
-    static_assert((4 + OREGS) * 4 * 32 * 4 <= q_region_bytes<D>(), "merge scratch must fit the Q region");
-
-    // ---- un-normalised partial of this (CTA, segment) piece
-    if (slot == 0 && has_rows) {
+#ifdef LOSA_TRACE
+    const long long ts0 = clock64();
+#endif
+    // ---- this warp's un-normalised record for the piece
+    if (works) {
       l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
       l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
       l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
       l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
-      float* part = partial_base(p.partials, blockIdx.x + sg, D);
-      const int r0 = rt * 16 + g8, r1 = r0 + 8;
-      if (r0 < rows) {
-        if (q4 == 0) { part[r0] = m0; part[kRowsPerGroup + r0] = l0; }
-#pragma unroll
-        for (int n = 0; n < ND; ++n)
-          *reinterpret_cast<float2*>(part + 2 * kRowsPerGroup + r0 * D + n * 8 + q4 * 2) = make_float2(oacc[n][0], oacc[n][1]);
+      float* rec = record_base(p.partials, blockIdx.x + sg, warp, D);
+      if (q4 == 0) {
+        rec[g8] = m0; rec[g8 + 8] = m1;
+        rec[kTileRows + g8] = l0; rec[kTileRows + g8 + 8] = l1;
       }
-      if (r1 < rows) {
-        if (q4 == 0) { part[r1] = m1; part[kRowsPerGroup + r1] = l1; }
 #pragma unroll
-        for (int n = 0; n < ND; ++n)
-          *reinterpret_cast<float2*>(part + 2 * kRowsPerGroup + r1 * D + n * 8 + q4 * 2) = make_float2(oacc[n][2], oacc[n][3]);
+      for (int n = 0; n < ND; ++n) {
+        *reinterpret_cast<float2*>(rec + 2 * kTileRows + g8 * D + n * 8 + q4 * 2) = make_float2(oacc[n][0], oacc[n][1]);
+        *reinterpret_cast<float2*>(rec + 2 * kTileRows + (g8 + 8) * D + n * 8 + q4 * 2) = make_float2(oacc[n][2], oacc[n][3]);
       }
     }
     item = seg_end;
-    ++sg;
-    while (item < hi && pre[sg + 1] <= item) ++sg;
+    sg = sg_next;
+    if (item < hi) {
+      cur = nxt;
+      load_q(cur, qf);
+#ifdef LOSA_TRACE
+      if (lane == 0 && p.trace) p.trace[p.n_ctas * 26 + blockIdx.x * 8 + warp] = (clock64() - ts0) + ((long long)(qf[0][0] & 1) << 40);
+#endif
+    }
   }
   if (tid == 0) LOSA_STAMP(6);
 #ifdef LOSA_TRACE
   if (lane == 0 && p.trace) { p.trace[p.n_ctas * 8 + (blockIdx.x * 8 + warp) * 2] = trace_wait; p.trace[p.n_ctas * 8 + (blockIdx.x * 8 + warp) * 2 + 1] = trace_busy; }
+  if (tid == 0 && p.trace) { unsigned smid; asm volatile("mov.u32 %0, %%smid;" : "=r"(smid)); p.trace[p.n_ctas * 24 + blockIdx.x * 2] = smid; p.trace[p.n_ctas * 24 + blockIdx.x * 2 + 1] = sg - sg0; }
 #endif
 }
 
@@ -767,7 +860,7 @@ int32_t launch_mma(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
   if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_end, st));
   int32_t rc = after_launch(c);
   if (rc != LOSA_OK) return rc;
-  attn_combine_kernel<D, true><<<dim3(ap.n_seg, kRowsPerGroup / 8), 256, 0, st>>>(ap);
+  attn_combine_kernel<D, true, false><<<dim3(ap.n_seg, kRowsPerGroup / 8), 256, 0, st>>>(ap);
   return after_launch(c);
 }
 
@@ -781,7 +874,7 @@ int32_t launch_simt(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
   if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_end, st));
   int32_t rc = after_launch(c);
   if (rc != LOSA_OK) return rc;
-  attn_combine_kernel<D, false><<<dim3(ap.n_seg, kRowsPerGroup / 8), 256, 0, st>>>(ap);
+  attn_combine_kernel<D, false, true><<<dim3(ap.n_seg, kRowsPerGroup / 8), 256, 0, st>>>(ap);
   return after_launch(c);
 }
 
@@ -828,6 +921,7 @@ int32_t launch_sparse_prefix_attn(losa_ctx* c, const void* q, const losa_kv_t* k
   ap.o_p = state->o_p;
   ap.lse_p = state->lse_p;
   ap.status = status_ptr(c);
+  ap.N = sh.batch;
   ap.B = sh.block_size;
   ap.Hq = sh.n_q_heads;
   ap.Hkv = sh.n_kv_heads;

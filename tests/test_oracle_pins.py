@@ -200,14 +200,28 @@ def test_fixed_order_fp32_score_matches_its_specification():
     orc.build_page_summaries(pb.sh, pb.kv)
     u32, _ = orc.page_scores_one(pb.sh, pb.q, pb.kv, 0, 0, 1)
     q = pb.q[0, 0, 1].astype(np.float32)
+    from fractions import Fraction
+
+    def round_f32(x: Fraction) -> np.float32:
+        """Exact rational -> nearest float32, ties to even (no double rounding)."""
+        f = np.float32(float(x))                      # float(Fraction) is correctly rounded to fp64
+        cands = {f, np.nextafter(f, np.float32(np.inf)), np.nextafter(f, np.float32(-np.inf))}
+        best = min(cands, key=lambda c: (abs(Fraction(float(c)) - x), int(np.float32(c).view(np.uint32)) & 1))
+        return np.float32(best)
+
+    def fma32(a, b, c):
+        return round_f32(Fraction(float(a)) * Fraction(float(b)) + Fraction(float(c)))
+
     for p in range(16):
         ph = pb.page_table[0, p]
-        t = np.maximum(q * pb.kmin[ph, 0], q * pb.kmax[ph, 0]).astype(np.float32)
+        lo, hi = pb.kmin[ph, 0], pb.kmax[ph, 0]
         c = np.zeros(8, np.float32)
         for r in range(8):
-            acc = t[8 * r]
-            for jj in range(1, 8):
-                acc = np.float32(acc + t[8 * r + jj])
+            acc = np.float32(0.0)
+            for jj in range(8):
+                j = 8 * r + jj
+                acc = fma32(max(q[j], np.float32(0)), hi[j], acc)
+                acc = fma32(min(q[j], np.float32(0)), lo[j], acc)
             c[r] = acc
         for off in (4, 2, 1):
             c = np.array([np.float32(c[i] + c[i ^ off]) for i in range(8)], np.float32)
