@@ -4,7 +4,7 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload c3]
 
 One "step" is one layer-step: stages 1-6 of include/losa.h for one attention layer and one
-denoising step.  Steps cycle through whole denoising blocks of the workload (step 0 of a block is
+denoising step, issued through the whole-step entry point losa_denoise_step.  Steps cycle through whole denoising blocks of the workload (step 0 of a block is
 the dense first step, the others are LoSA steps).  Prints ONE JSON line.
 
 Timing: the layer-step is captured once in a CUDA graph and replayed; each step is bracketed by
@@ -256,15 +256,16 @@ def run_ours(args, cfg):
         if i % T == 0:
             layer.step.zero_()          # a new block starts: no valid cache
 
-    # eager warm-up of every kernel (tensor maps, attributes), then capture the layer-step
+    # eager warm-up of every kernel (tensor maps, attributes, second stream), then capture the
+    # whole-step call
     load(0)
-    layer.run_step(q_s, k_s, v_s, m_s)
+    layer.run_step_fused(q_s, k_s, v_s, m_s)
     torch.cuda.synchronize()
     assert layer.ctx.poll_status() == 0
     n0 = layer.ctx.launch_count()
     graph = torch.cuda.CUDAGraph()
     with torch.cuda.graph(graph):
-        layer.run_step(q_s, k_s, v_s, m_s)
+        layer.run_step_fused(q_s, k_s, v_s, m_s)
     launches_per_step = layer.ctx.launch_count() - n0
 
     def timed_pass(first, count, record_pages=None):
@@ -309,7 +310,7 @@ def run_ours(args, cfg):
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": workload_name(cfg), "sequences_per_gpu": cfg.batch,
-                   "launch": "CUDA graph replay of the six stage calls",
+                   "launch": "CUDA graph replay of losa_denoise_step (stages 1-6 in one call)",
                    "l2": "flushed between steps, outside the timed region: 256 MiB write, then 256 MiB read so no dirty lines remain"},
         "clocks": clocks, "gpu_launches": launches_per_step * args.steps,
         "step_us": {"losa_step_median": float(np.median(sparse_ms)) * 1e3 if sparse_ms else None,
@@ -330,7 +331,7 @@ def run_ours(args, cfg):
     for i in range(first, min(total, first + max(args.steps, T))):
         load(i)
         flush.fill_(i & 0xff)
-        layer.run_step(q_s, k_s, v_s, m_s)
+        layer.run_step_fused(q_s, k_s, v_s, m_s)
         k_ms.append(layer.ctx.stage4_last_ms())
         k_bytes.append(stage4_bytes(cfg, to_host(layer.union_pages), to_host(layer.union_count),
                                     to_host(layer.n_active), to_host(layer.kv_len)))

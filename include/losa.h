@@ -243,18 +243,33 @@ int32_t losa_update_prefix_cache(losa_ctx* ctx, losa_kv_t* kv, losa_state_t* sta
  * logical page p < P_s over its valid tokens. */
 int32_t losa_build_page_summaries(losa_ctx* ctx, losa_kv_t* kv, void* stream);
 
-/* One whole layer-step from HOST buffers: copies q, k_blk, v_blk [as above, dtype] from host
- * memory to device staging buffers supplied by the caller (d_q, d_k_blk, d_v_blk, d_out and the
- * index buffers below), runs stages 1-6 in order on `stream`, and copies `out` back to the host
- * buffer h_out.  Does not synchronise.  All h_* pointers are HOST pointers (pinned for true
- * asynchrony); everything else is device memory owned by the caller.
- *   m_per_seq as in stage 1; k as in stage 2. */
+/* Device buffers a whole-step call needs besides its inputs and outputs (caller-owned). */
 typedef struct {
-  void *d_q, *d_k_blk, *d_v_blk, *d_out;
+  void *d_q, *d_k_blk, *d_v_blk, *d_out;  /* staging of the host variant; unused by losa_denoise_step */
   int32_t *active_idx, *n_active;      /* [N,B], [N]                     */
   int32_t *topk_pages;                 /* [N,B,H_q,k]                    */
   int32_t *union_pages, *union_count;  /* [N,H_kv,P_max], [N,H_kv]       */
 } losa_step_buffers_t;
+
+/* One whole layer-step (the method-overview workflow of Section 4, stages 1-6 with
+ * finalize_block = 0) in one call, with the same results as the six calls in order: the index
+ * buffers of `buf` receive what stages 1-3 produce, state->o_p / lse_p what stage 4 produces,
+ * out / lse_out_opt what stage 5 produces; q_prev and step are updated as by stage 6.
+ * Being one call, it may schedule freely inside: the in-block attention of stage 5 (which needs
+ * nothing from stages 1-4) runs on a second stream owned by the context and is joined before a
+ * final merge kernel that also keeps the queries.  All work is ordered after prior work on
+ * `stream` and complete when `stream` reaches the end of the call's work; the call can be captured
+ * in a CUDA graph after one un-captured call on the context (which creates the second stream). */
+int32_t losa_denoise_step(losa_ctx* ctx, const void* q, const void* k_blk, const void* v_blk, void* out,
+                          float* lse_out_opt, losa_kv_t* kv, losa_state_t* state,
+                          const losa_step_buffers_t* buf, const int32_t* m_per_seq, int32_t k,
+                          void* stream);
+
+/* The same whole layer-step from HOST buffers: copies q, k_blk, v_blk [dtype] from host memory to
+ * the device staging buffers d_q, d_k_blk, d_v_blk of `buf`, runs losa_denoise_step on them with
+ * d_out as output, and copies d_out back to the host buffer h_out.  Does not synchronise.  All
+ * h_* pointers are HOST pointers (pinned for true asynchrony); everything else is device memory
+ * owned by the caller.  m_per_seq as in stage 1; k as in stage 2. */
 int32_t losa_denoise_step_host(losa_ctx* ctx, const void* h_q, const void* h_k_blk,
                                const void* h_v_blk, void* h_out, losa_kv_t* kv, losa_state_t* state,
                                const losa_step_buffers_t* buf, const int32_t* m_per_seq, int32_t k,

@@ -29,6 +29,7 @@ EXPORTS = [
     "losa_page_union", "losa_sparse_prefix_attn", "losa_block_attn_merge",
     "losa_update_prefix_cache", "losa_build_page_summaries", "losa_denoise_step_host",
     "losa_profile_stage4", "losa_stage4_last_ms", "losa_select_active_static",
+    "losa_denoise_step",
 ]
 
 
@@ -216,6 +217,12 @@ def losa_update_prefix_cache(ctx, kv, state, q, k_blk, v_blk, finalize_block):
 
 def losa_build_page_summaries(ctx, kv):
     ctx._check("losa_build_page_summaries", lib().losa_build_page_summaries(ctx._h, C.byref(kv), _stream()))
+
+
+def losa_denoise_step(ctx, q, k_blk, v_blk, out, lse_out_opt, kv, state, buf, m_per_seq, k):
+    ctx._check("losa_denoise_step", lib().losa_denoise_step(
+        ctx._h, _ptr(q), _ptr(k_blk), _ptr(v_blk), _ptr(out), _ptr(lse_out_opt), C.byref(kv), C.byref(state),
+        C.byref(buf), _ptr(m_per_seq), C.c_int32(k), _stream()))
 
 
 def losa_denoise_step_host(ctx, h_q, h_k_blk, h_v_blk, h_out, kv, state, buf, m_per_seq, k):

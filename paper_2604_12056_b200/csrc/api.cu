@@ -42,6 +42,9 @@ int32_t make_layout(const losa_shape_t* sh, int n_ctas, WorkspaceLayout* L) {
   off = align_up(off + sizeof(float) * static_cast<size_t>(sh->batch) * sh->block_size * sh->n_q_heads * L->score_stride, 256);
   L->partials = off;
   off = align_up(off + sizeof(float) * static_cast<size_t>(L->n_slots) * kRowsPerGroup * (sh->head_dim + 2), 256);
+  const size_t rows = static_cast<size_t>(sh->batch) * sh->block_size * sh->n_q_heads;
+  L->block_o = off;   off = align_up(off + sizeof(float) * rows * sh->head_dim, 256);
+  L->block_lse = off; off = align_up(off + sizeof(float) * rows, 256);
   L->total = off;
   return LOSA_OK;
 }
@@ -121,6 +124,9 @@ int32_t losa_destroy(losa_ctx* ctx) {
   if (!ctx) return LOSA_ERR_INVALID_ARG;
   if (ctx->ev_begin) cudaEventDestroy(ctx->ev_begin);
   if (ctx->ev_end) cudaEventDestroy(ctx->ev_end);
+  if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+  if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+  if (ctx->side_stream) cudaStreamDestroy(ctx->side_stream);
   delete ctx;
   return LOSA_OK;
 }
@@ -219,6 +225,43 @@ int32_t losa_build_page_summaries(losa_ctx* ctx, losa_kv_t* kv, void* stream) {
   return launch_build_page_summaries(ctx, kv, as_stream(stream));
 }
 
+int32_t losa_denoise_step(losa_ctx* ctx, const void* q, const void* k_blk, const void* v_blk, void* out,
+                          float* lse_out_opt, losa_kv_t* kv, losa_state_t* state, const losa_step_buffers_t* buf,
+                          const int32_t* m_per_seq, int32_t k, void* stream) {
+  if (!ctx || !q || !k_blk || !v_blk || !out || !buf || !state || !state->step || !state->q_prev || !state->o_p ||
+      !state->lse_p || k < 1)
+    return LOSA_ERR_INVALID_ARG;
+  if (!buf->active_idx || !buf->n_active || !buf->topk_pages || !buf->union_pages || !buf->union_count)
+    return LOSA_ERR_INVALID_ARG;
+  int32_t rc = check_kv(ctx, kv, true);
+  if (rc != LOSA_OK) return rc;
+  if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out) || !aligned16(state->q_prev) ||
+      !aligned16(state->o_p))
+    return LOSA_ERR_UNSUPPORTED;
+  if (!ctx->side_stream) {
+    LOSA_CUDA_TRY(ctx, cudaStreamCreateWithFlags(&ctx->side_stream, cudaStreamNonBlocking));
+    LOSA_CUDA_TRY(ctx, cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming));
+    LOSA_CUDA_TRY(ctx, cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming));
+  }
+  cudaStream_t st = as_stream(stream);
+  const losa_shape_t& sh = ctx->shape;
+  // fork: the in-block attention needs nothing from stages 1-4
+  LOSA_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_fork, st));
+  LOSA_CUDA_TRY(ctx, cudaStreamWaitEvent(ctx->side_stream, ctx->ev_fork, 0));
+  rc = launch_block_attn(ctx, q, k_blk, v_blk, ctx->side_stream);
+  if (rc != LOSA_OK) return rc;
+  LOSA_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_join, ctx->side_stream));
+  rc = launch_select_active(ctx, q, state->q_prev, sh.n_q_heads * sh.head_dim, m_per_seq, state->step,
+                            buf->active_idx, buf->n_active, nullptr, st);
+  if (rc == LOSA_OK) rc = launch_page_scores_topk(ctx, q, kv, buf->active_idx, buf->n_active, state->step, k, buf->topk_pages, nullptr, st);
+  if (rc == LOSA_OK) rc = launch_page_union(ctx, buf->topk_pages, buf->active_idx, buf->n_active, k, kv->kv_len, state->step, buf->union_pages, buf->union_count, st);
+  if (rc == LOSA_OK) rc = launch_sparse_prefix_attn(ctx, q, kv, buf->active_idx, buf->n_active, buf->union_pages, buf->union_count, state, st);
+  if (rc != LOSA_OK) return rc;
+  // join, then merge + commit in one pass over the rows
+  LOSA_CUDA_TRY(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0));
+  return launch_merge_commit(ctx, q, state, out, lse_out_opt, st);
+}
+
 int32_t losa_denoise_step_host(losa_ctx* ctx, const void* h_q, const void* h_k_blk, const void* h_v_blk,
                                void* h_out, losa_kv_t* kv, losa_state_t* state, const losa_step_buffers_t* buf,
                                const int32_t* m_per_seq, int32_t k, void* stream) {
@@ -237,13 +280,7 @@ int32_t losa_denoise_step_host(losa_ctx* ctx, const void* h_q, const void* h_k_b
   LOSA_CUDA_TRY(ctx, cudaMemcpyAsync(buf->d_q, h_q, qb, cudaMemcpyHostToDevice, st));
   LOSA_CUDA_TRY(ctx, cudaMemcpyAsync(buf->d_k_blk, h_k_blk, kb, cudaMemcpyHostToDevice, st));
   LOSA_CUDA_TRY(ctx, cudaMemcpyAsync(buf->d_v_blk, h_v_blk, kb, cudaMemcpyHostToDevice, st));
-  rc = losa_select_active(ctx, buf->d_q, state->q_prev, sh.n_q_heads * sh.head_dim, m_per_seq, state->step,
-                          buf->active_idx, buf->n_active, nullptr, stream);
-  if (rc == LOSA_OK) rc = losa_page_scores_topk(ctx, buf->d_q, kv, buf->active_idx, buf->n_active, state->step, k, buf->topk_pages, nullptr, stream);
-  if (rc == LOSA_OK) rc = losa_page_union(ctx, buf->topk_pages, buf->active_idx, buf->n_active, k, kv->kv_len, state->step, buf->union_pages, buf->union_count, stream);
-  if (rc == LOSA_OK) rc = losa_sparse_prefix_attn(ctx, buf->d_q, kv, buf->active_idx, buf->n_active, buf->union_pages, buf->union_count, state, stream);
-  if (rc == LOSA_OK) rc = losa_block_attn_merge(ctx, buf->d_q, buf->d_k_blk, buf->d_v_blk, state, buf->d_out, nullptr, stream);
-  if (rc == LOSA_OK) rc = losa_update_prefix_cache(ctx, kv, state, buf->d_q, buf->d_k_blk, buf->d_v_blk, 0, stream);
+  rc = losa_denoise_step(ctx, buf->d_q, buf->d_k_blk, buf->d_v_blk, buf->d_out, nullptr, kv, state, buf, m_per_seq, k, stream);
   if (rc != LOSA_OK) return rc;
   LOSA_CUDA_TRY(ctx, cudaMemcpyAsync(h_out, buf->d_out, qb, cudaMemcpyDeviceToHost, st));
   return LOSA_OK;

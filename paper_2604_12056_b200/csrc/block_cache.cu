@@ -17,12 +17,14 @@ constexpr int kTokTile = 2;
 // the kernel pays one memory latency, not one per operand.  Scores: lane = block key, columns
 // visited in a rotated order so that the 32 lanes hit 32 banks, four independent partial sums;
 // P V: lane = output column.
-template <typename T, int D>
+// MERGE = false (whole-step path): only the in-block part, normalised o_b to `ob_out` and L_b to
+// `lse_out`; the prefix statistics are not touched, so this can run beside stages 1-4.
+template <typename T, int D, bool MERGE>
 __global__ void __launch_bounds__(kThreads)
 block_attn_merge_kernel(const T* __restrict__ q, const T* __restrict__ k_blk, const T* __restrict__ v_blk,
                         const float* __restrict__ o_p, const float* __restrict__ lse_p,
-                        T* __restrict__ out, float* __restrict__ lse_out, int B, int Hq, int Hkv,
-                        float sm_scale) {
+                        T* __restrict__ out, float* __restrict__ lse_out, float* __restrict__ ob_out,
+                        int B, int Hq, int Hkv, float sm_scale) {
   extern __shared__ __align__(16) float smem[];
   float* Ks = smem;                 // [B][D]
   float* Vs = Ks + B * D;           // [B][D]
@@ -42,9 +44,9 @@ block_attn_merge_kernel(const T* __restrict__ q, const T* __restrict__ k_blk, co
 #pragma unroll
     for (int c = 0; c < C; ++c) {
       qv[c] = to_f32(q[row * D + lane + 32 * c]);
-      opv[c] = o_p[row * D + lane + 32 * c];
+      opv[c] = MERGE ? o_p[row * D + lane + 32 * c] : 0.f;
     }
-    Lp = lse_p[row];
+    Lp = MERGE ? lse_p[row] : 0.f;
   };
   if (have) fetch();
   for (int idx = tid * 8; idx < B * D; idx += kThreads * 8) {
@@ -99,19 +101,61 @@ block_attn_merge_kernel(const T* __restrict__ q, const T* __restrict__ k_blk, co
 #pragma unroll
       for (int c = 0; c < C; ++c) ob[c] = fmaf(pt, Vs[t * D + lane + 32 * c], ob[c]);
     }
-    const float M2 = fmaxf(Lp, Lb);
-    const float L = M2 + logf(expf(Lp - M2) + expf(Lb - M2));
-    const float wp = expf(Lp - L), wb = expf(Lb - L) / sum;
+    if (MERGE) {
+      const float M2 = fmaxf(Lp, Lb);
+      const float L = M2 + logf(expf(Lp - M2) + expf(Lb - M2));
+      const float wp = expf(Lp - L), wb = expf(Lb - L) / sum;
 #pragma unroll
-    for (int c = 0; c < C; ++c) {
-      const float v = (wp > 0.f ? wp * opv[c] : 0.f) + wb * ob[c];
-      out[row * D + lane + 32 * c] = from_f32<T>(v);
+      for (int c = 0; c < C; ++c) {
+        const float v = (wp > 0.f ? wp * opv[c] : 0.f) + wb * ob[c];
+        out[row * D + lane + 32 * c] = from_f32<T>(v);
+      }
+      if (lse_out && lane == 0) lse_out[row] = L;
+    } else {
+      const float inv = 1.f / sum;
+#pragma unroll
+      for (int c = 0; c < C; ++c) ob_out[row * D + lane + 32 * c] = ob[c] * inv;
+      if (lane == 0) lse_out[row] = Lb;
     }
-    if (lse_out && lane == 0) lse_out[row] = L;
     r += kThreads / 32;
     have = r < ntok * G;
     if (have) fetch();
   }
+}
+
+// Whole-step path, last kernel: one warp per (token, head) row merges the prefix statistics with
+// the in-block part (Section 2.2 / 4.3), writes the output, and keeps the row's query for the next
+// step's Eq. 1; block 0 also bumps the step counters.
+template <typename T, int D>
+__global__ void __launch_bounds__(kThreads)
+merge_commit_kernel(const T* __restrict__ q, T* __restrict__ q_prev, const float* __restrict__ o_p,
+                    const float* __restrict__ lse_p, const float* __restrict__ o_b,
+                    const float* __restrict__ lse_b, T* __restrict__ out, float* __restrict__ lse_out,
+                    int32_t* __restrict__ step, int N, size_t n_rows) {
+  const int lane = threadIdx.x & 31;
+  const size_t row = static_cast<size_t>(blockIdx.x) * (kThreads / 32) + (threadIdx.x >> 5);
+  if (blockIdx.x == 0)
+    for (int s = threadIdx.x; s < N; s += kThreads) step[s] += 1;
+  if (row >= n_rows) return;
+  constexpr int C = D / 32;
+  float a[C], b[C];
+  T qv[C];
+#pragma unroll
+  for (int c = 0; c < C; ++c) {
+    a[c] = o_p[row * D + lane + 32 * c];
+    b[c] = o_b[row * D + lane + 32 * c];
+    qv[c] = q[row * D + lane + 32 * c];
+  }
+  const float Lp = lse_p[row], Lb = lse_b[row];
+  const float M = fmaxf(Lp, Lb);
+  const float L = M + logf(expf(Lp - M) + expf(Lb - M));
+  const float wp = expf(Lp - L), wb = expf(Lb - L);
+#pragma unroll
+  for (int c = 0; c < C; ++c) {
+    out[row * D + lane + 32 * c] = from_f32<T>((wp > 0.f ? wp * a[c] : 0.f) + wb * b[c]);
+    q_prev[row * D + lane + 32 * c] = qv[c];
+  }
+  if (lse_out && lane == 0) lse_out[row] = L;
 }
 
 template <typename T>
@@ -200,17 +244,31 @@ __global__ void finalize_counters_kernel(int32_t* __restrict__ kv_len, int32_t* 
   if (s < N) { kv_len[s] += B; step[s] = 0; }
 }
 
-template <typename T, int D>
+template <typename T, int D, bool MERGE>
 int32_t launch_merge_t(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk,
-                       const losa_state_t* state, void* out, float* lse_out, cudaStream_t st) {
+                       const losa_state_t* state, void* out, float* lse_out, float* ob_out, cudaStream_t st) {
   const losa_shape_t& sh = c->shape;
   const size_t smem = (static_cast<size_t>(2) * sh.block_size * D + (kThreads / 32) * D) * sizeof(float);
   if (smem > 48 * 1024)
-    LOSA_CUDA_TRY(c, cudaFuncSetAttribute(block_attn_merge_kernel<T, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    LOSA_CUDA_TRY(c, cudaFuncSetAttribute(block_attn_merge_kernel<T, D, MERGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   dim3 grid((sh.block_size + kTokTile - 1) / kTokTile, sh.n_kv_heads, sh.batch);
-  block_attn_merge_kernel<T, D><<<grid, kThreads, smem, st>>>(
-      static_cast<const T*>(q), static_cast<const T*>(k_blk), static_cast<const T*>(v_blk), state->o_p,
-      state->lse_p, static_cast<T*>(out), lse_out, sh.block_size, sh.n_q_heads, sh.n_kv_heads, sh.sm_scale);
+  block_attn_merge_kernel<T, D, MERGE><<<grid, kThreads, smem, st>>>(
+      static_cast<const T*>(q), static_cast<const T*>(k_blk), static_cast<const T*>(v_blk),
+      state ? state->o_p : nullptr, state ? state->lse_p : nullptr, static_cast<T*>(out), lse_out, ob_out,
+      sh.block_size, sh.n_q_heads, sh.n_kv_heads, sh.sm_scale);
+  return after_launch(c);
+}
+
+template <typename T, int D>
+int32_t launch_merge_commit_t(losa_ctx* c, const void* q, losa_state_t* state, void* out, float* lse_out,
+                              cudaStream_t st) {
+  const losa_shape_t& sh = c->shape;
+  const size_t n_rows = static_cast<size_t>(sh.batch) * sh.block_size * sh.n_q_heads;
+  const int blocks = static_cast<int>((n_rows + kThreads / 32 - 1) / (kThreads / 32));
+  merge_commit_kernel<T, D><<<blocks, kThreads, 0, st>>>(
+      static_cast<const T*>(q), static_cast<T*>(state->q_prev), state->o_p, state->lse_p,
+      reinterpret_cast<const float*>(c->ws + c->lay.block_o), reinterpret_cast<const float*>(c->ws + c->lay.block_lse),
+      static_cast<T*>(out), lse_out, state->step, sh.batch, n_rows);
   return after_launch(c);
 }
 
@@ -254,10 +312,29 @@ int32_t launch_summaries_t(losa_ctx* c, losa_kv_t* kv, cudaStream_t st) {
 int32_t launch_block_attn_merge(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk,
                                 const losa_state_t* state, void* out, float* lse_out_opt, cudaStream_t st) {
   const bool bf = c->shape.dtype == LOSA_BF16;
-  if (bf && c->shape.head_dim == 128) return launch_merge_t<__nv_bfloat16, 128>(c, q, k_blk, v_blk, state, out, lse_out_opt, st);
-  if (bf) return launch_merge_t<__nv_bfloat16, 64>(c, q, k_blk, v_blk, state, out, lse_out_opt, st);
-  if (c->shape.head_dim == 128) return launch_merge_t<float, 128>(c, q, k_blk, v_blk, state, out, lse_out_opt, st);
-  return launch_merge_t<float, 64>(c, q, k_blk, v_blk, state, out, lse_out_opt, st);
+  if (bf && c->shape.head_dim == 128) return launch_merge_t<__nv_bfloat16, 128, true>(c, q, k_blk, v_blk, state, out, lse_out_opt, nullptr, st);
+  if (bf) return launch_merge_t<__nv_bfloat16, 64, true>(c, q, k_blk, v_blk, state, out, lse_out_opt, nullptr, st);
+  if (c->shape.head_dim == 128) return launch_merge_t<float, 128, true>(c, q, k_blk, v_blk, state, out, lse_out_opt, nullptr, st);
+  return launch_merge_t<float, 64, true>(c, q, k_blk, v_blk, state, out, lse_out_opt, nullptr, st);
+}
+
+int32_t launch_block_attn(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk, cudaStream_t st) {
+  const bool bf = c->shape.dtype == LOSA_BF16;
+  float* ob = reinterpret_cast<float*>(c->ws + c->lay.block_o);
+  float* lb = reinterpret_cast<float*>(c->ws + c->lay.block_lse);
+  if (bf && c->shape.head_dim == 128) return launch_merge_t<__nv_bfloat16, 128, false>(c, q, k_blk, v_blk, nullptr, nullptr, lb, ob, st);
+  if (bf) return launch_merge_t<__nv_bfloat16, 64, false>(c, q, k_blk, v_blk, nullptr, nullptr, lb, ob, st);
+  if (c->shape.head_dim == 128) return launch_merge_t<float, 128, false>(c, q, k_blk, v_blk, nullptr, nullptr, lb, ob, st);
+  return launch_merge_t<float, 64, false>(c, q, k_blk, v_blk, nullptr, nullptr, lb, ob, st);
+}
+
+int32_t launch_merge_commit(losa_ctx* c, const void* q, losa_state_t* state, void* out, float* lse_out_opt,
+                            cudaStream_t st) {
+  const bool bf = c->shape.dtype == LOSA_BF16;
+  if (bf && c->shape.head_dim == 128) return launch_merge_commit_t<__nv_bfloat16, 128>(c, q, state, out, lse_out_opt, st);
+  if (bf) return launch_merge_commit_t<__nv_bfloat16, 64>(c, q, state, out, lse_out_opt, st);
+  if (c->shape.head_dim == 128) return launch_merge_commit_t<float, 128>(c, q, state, out, lse_out_opt, st);
+  return launch_merge_commit_t<float, 64>(c, q, state, out, lse_out_opt, st);
 }
 
 int32_t launch_update_prefix_cache(losa_ctx* c, losa_kv_t* kv, losa_state_t* state, const void* q,

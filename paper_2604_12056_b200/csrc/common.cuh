@@ -23,6 +23,8 @@ struct WorkspaceLayout {
   size_t delta;      // double[N*B]
   size_t scores;     // float[N*B*H_q*score_stride]
   size_t partials;   // float[n_slots * kRowsPerGroup * (d + 2)]
+  size_t block_o;    // float[N*B*H_q*d]  : in-block attention output of the whole-step path
+  size_t block_lse;  // float[N*B*H_q]    : its log-normaliser
   size_t total;
   int32_t score_stride;  // P_max rounded up to 64
   int32_t n_slots;       // n_ctas + n_segments
@@ -50,6 +52,9 @@ struct losa_ctx {
   int64_t tmap_strides[3];
   int32_t tmap_n_phys;
   void* encode_fn;  // cuTensorMapEncodeTiled, resolved through the runtime
+  // second stream and fork/join events of the whole-step path (created on first use)
+  cudaStream_t side_stream;
+  cudaEvent_t ev_fork, ev_join;
   // optional timing of the stage-4 main kernel
   int32_t profile;
   cudaEvent_t ev_begin, ev_end;

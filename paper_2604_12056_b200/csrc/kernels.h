@@ -28,6 +28,12 @@ int32_t launch_block_attn_merge(losa_ctx* c, const void* q, const void* k_blk, c
                                 const losa_state_t* state, void* out, float* lse_out_opt,
                                 cudaStream_t st);
 
+// Whole-step path: in-block attention alone (o_b, L_b into the workspace), then merge with the
+// prefix statistics, write the output, keep the queries and bump the step counters.
+int32_t launch_block_attn(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk, cudaStream_t st);
+int32_t launch_merge_commit(losa_ctx* c, const void* q, losa_state_t* state, void* out, float* lse_out_opt,
+                            cudaStream_t st);
+
 int32_t launch_update_prefix_cache(losa_ctx* c, losa_kv_t* kv, losa_state_t* state, const void* q,
                                    const void* k_blk, const void* v_blk, int32_t finalize_block,
                                    cudaStream_t st);

@@ -7,7 +7,7 @@
 //                        a chain of 16 fused multiply-adds per lane (q+ kmax, q- kmin), then an
 //                        xor-butterfly over the lanes — exactly the order the interface fixes, so
 //                        the fp32 result is reproducible bit for bit.
-//   topk_select_kernel : one warp per (sequence, active token, head); threshold search over
+//   topk_select_kernel : one 128-thread CTA per (sequence, active token, head); threshold search over
 //                        64-bit keys (order-preserving score bits, inverted page id), see below.
 //   topk_kernel        : budgets above 512 pages: one CTA per query sorts all keys with a
 //                        shared-memory bitonic network.
@@ -67,35 +67,57 @@ page_scores_kernel(const T* __restrict__ q, const T* __restrict__ kmin, const T*
       }
     }
     __syncthreads();
-    // the trip count is the same for every lane: the butterfly below needs whole warps
-    for (int pbase = 0; pbase < np; pbase += GROUPS) {
-      const int pl = pbase + grp;
-      const bool ok = pl < np;
-      float lo[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, hi[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-      if (ok) {
-        int phys = page_table[static_cast<size_t>(s) * Pmax + p0 + pl];
-        if (phys < 0 || phys >= n_phys) { set_status(status, LOSA_ERR_BOUNDS); phys = 0; }
-        const size_t so = (static_cast<size_t>(phys) * Hkv + kh) * D + sub * 8;
-        load8(kmin + so, lo);
-        load8(kmax + so, hi);
+    // All summary loads of this CTA's pages are issued before any arithmetic (two dependent
+    // latencies in total instead of two per page).  The trip counts are the same for every lane:
+    // the butterfly below needs whole warps.
+    constexpr int ITER = kPagesPerCta / GROUPS;
+    float lo[ITER][8], hi[ITER][8];
+    int phys[ITER];
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+      const int pl = it * GROUPS + grp;
+      phys[it] = pl < np ? page_table[static_cast<size_t>(s) * Pmax + p0 + pl] : -1;
+    }
+#pragma unroll
+    for (int it = 0; it < ITER; ++it) {
+      const int pl = it * GROUPS + grp;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) { lo[it][e] = 0.f; hi[it][e] = 0.f; }
+      if (pl < np) {
+        int ph = phys[it];
+        if (ph < 0 || ph >= n_phys) { set_status(status, LOSA_ERR_BOUNDS); ph = 0; }
+        const size_t so = (static_cast<size_t>(ph) * Hkv + kh) * D + sub * 8;
+        load8(kmin + so, lo[it]);
+        load8(kmax + so, hi[it]);
       }
-#pragma unroll 2
-      for (int r = 0; r < nr; ++r) {
-        float qp[8], qn[8];
-        *reinterpret_cast<float4*>(&qp[0]) = *reinterpret_cast<const float4*>(&qpos[r * D + sub * 4]);
-        *reinterpret_cast<float4*>(&qp[4]) = *reinterpret_cast<const float4*>(&qpos[r * D + D / 2 + sub * 4]);
-        *reinterpret_cast<float4*>(&qn[0]) = *reinterpret_cast<const float4*>(&qneg[r * D + sub * 4]);
-        *reinterpret_cast<float4*>(&qn[4]) = *reinterpret_cast<const float4*>(&qneg[r * D + D / 2 + sub * 4]);
-        float acc = 0.f;
+    }
+    // one query load feeds the chains of all ITER pages held in registers
+    for (int r = 0; r < nr; ++r) {
+      float qp[8], qn[8];
+      *reinterpret_cast<float4*>(&qp[0]) = *reinterpret_cast<const float4*>(&qpos[r * D + sub * 4]);
+      *reinterpret_cast<float4*>(&qp[4]) = *reinterpret_cast<const float4*>(&qpos[r * D + D / 2 + sub * 4]);
+      *reinterpret_cast<float4*>(&qn[0]) = *reinterpret_cast<const float4*>(&qneg[r * D + sub * 4]);
+      *reinterpret_cast<float4*>(&qn[4]) = *reinterpret_cast<const float4*>(&qneg[r * D + D / 2 + sub * 4]);
+      float acc[ITER];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          acc = __fmaf_rn(qp[j], hi[j], acc);
-          acc = __fmaf_rn(qn[j], lo[j], acc);
+      for (int it = 0; it < ITER; ++it) acc[it] = 0.f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+#pragma unroll
+        for (int it = 0; it < ITER; ++it) {
+          acc[it] = __fmaf_rn(qp[j], hi[it][j], acc[it]);
+          acc[it] = __fmaf_rn(qn[j], lo[it][j], acc[it]);
         }
+      }
 #pragma unroll
-        for (int off = LPP / 2; off >= 1; off >>= 1)
-          acc = __fadd_rn(acc, __shfl_xor_sync(0xffffffffu, acc, off));
-        if (ok && sub == 0) sc[r][pl] = __fadd_rn(acc, 0.0f);
+      for (int off = LPP / 2; off >= 1; off >>= 1) {
+#pragma unroll
+        for (int it = 0; it < ITER; ++it) acc[it] = __fadd_rn(acc[it], __shfl_xor_sync(0xffffffffu, acc[it], off));
+      }
+#pragma unroll
+      for (int it = 0; it < ITER; ++it) {
+        const int pl = it * GROUPS + grp;
+        if (pl < np && sub == 0) sc[r][pl] = __fadd_rn(acc[it], 0.0f);
       }
     }
     __syncthreads();
@@ -167,14 +189,13 @@ topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ kv_len
   }
 }
 
-// ---- top-k by threshold search: one warp per query, O(P) work --------------------------------
+// ---- top-k by threshold search: one small CTA per query, O(P) work ---------------------------
 // Keys are (order-preserving score bits, inverted page id), all distinct, so "the k largest keys"
-// is the required answer with ties already broken.  The warp histograms the score bits of the
+// is the required answer with ties already broken.  The CTA histograms the score bits of the
 // still-undecided range into 256 equal-width bins, finds the bin holding the k-th largest, takes
 // every key above that bin, and either finishes by sorting "taken + threshold bin" (a few dozen
 // keys) or narrows the range to the threshold bin and repeats.  A range of one value means the
 // remaining candidates tie on the score: the lowest page ids win, taken in page order.
-constexpr int kSelWarps = 4;
 constexpr int kSelCap = 512;     // candidate keys a warp can sort; also the largest k of this path
 constexpr int kSelBins = 256;
 
@@ -183,105 +204,112 @@ __device__ __forceinline__ unsigned long long make_key(uint32_t ob, int p) {
          static_cast<unsigned long long>(0xffffffffu - static_cast<uint32_t>(p));
 }
 
-// Visits the warp's keys in page order, 32 per round: f(ob, p, in_range) is called by every lane in
-// every round (so f may use warp-wide votes); in_range says whether p < P.  With CACHED the order
-// bits of the P <= 1024 scores sit in registers (one global pass for the whole selection).
+// One CTA of kSelThreads per query.  Thread t owns keys p = t + kSelThreads * i; with CACHED
+// (P <= kSelThreads * kSelPerThread) their order bits stay in registers for the whole selection.
+constexpr int kSelThreads = 128;
+constexpr int kSelPerThread = 8;
+
 template <bool CACHED, typename F>
-__device__ __forceinline__ void for_each_key(const uint32_t (&cache)[32], const float* __restrict__ row, int P,
-                                             int lane, F&& f) {
+__device__ __forceinline__ void for_each_key(const uint32_t (&cache)[kSelPerThread], const float* __restrict__ row,
+                                             int P, int tid, F&& f) {
   if (CACHED) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      if (32 * i >= P) break;
-      const int p = lane + 32 * i;
-      f(cache[i], p, p < P);
+    for (int i = 0; i < kSelPerThread; ++i) {
+      const int p = tid + kSelThreads * i;
+      if (p < P) f(cache[i], p);
     }
   } else {
-    for (int base = 0; base < P; base += 32) {
-      const int p = base + lane;
-      f(p < P ? order_bits(row[p]) : 0u, p, p < P);
-    }
+    for (int p = tid; p < P; p += kSelThreads) f(order_bits(row[p]), p);
   }
 }
 
 template <bool CACHED>
 __device__ __forceinline__ void topk_select_body(const float* __restrict__ row, int P, int kk, int k,
-                                                 unsigned long long* cand, int* hist, int32_t* out_pages,
-                                                 float* out_scores, int lane) {
-  const unsigned below = (1u << lane) - 1u;
-  uint32_t cache[32];
+                                                 int32_t* out_pages, float* out_scores) {
+  __shared__ unsigned long long cand[kSelCap];
+  __shared__ int hist[kSelBins];
+  __shared__ uint32_t s_red[2][kSelThreads / 32];
+  __shared__ int s_ncand, s_bstar, s_above, s_thr;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  uint32_t cache[kSelPerThread];
   if (CACHED) {
 #pragma unroll
-    for (int i = 0; i < 32; ++i) {
-      const int p = lane + 32 * i;
+    for (int i = 0; i < kSelPerThread; ++i) {
+      const int p = tid + kSelThreads * i;
       cache[i] = p < P ? order_bits(row[p]) : 0u;
     }
   }
   uint32_t lo = 0xffffffffu, hi = 0u;
-  for_each_key<CACHED>(cache, row, P, lane, [&](uint32_t ob, int, bool in) {
-    if (in) { lo = min(lo, ob); hi = max(hi, ob); }
-  });
+  for_each_key<CACHED>(cache, row, P, tid, [&](uint32_t ob, int) { lo = min(lo, ob); hi = max(hi, ob); });
   lo = __reduce_min_sync(0xffffffffu, lo);
   hi = __reduce_max_sync(0xffffffffu, hi);
-  int need = kk, ncand = 0;
+  if (lane == 0) { s_red[0][warp] = lo; s_red[1][warp] = hi; }
+  if (tid == 0) s_ncand = 0;
+  __syncthreads();
+#pragma unroll
+  for (int w = 0; w < kSelThreads / 32; ++w) { lo = min(lo, s_red[0][w]); hi = max(hi, s_red[1][w]); }
+  int need = kk;
   while (need > 0) {
     if (lo == hi) {
-      // every remaining candidate has the same score: lowest pages first, in page order
-      for_each_key<CACHED>(cache, row, P, lane, [&](uint32_t ob, int p, bool in) {
-        const bool hit = in && ob == lo && need > 0;
-        const unsigned bal = __ballot_sync(0xffffffffu, hit);
-        const int rank = __popc(bal & below);
-        if (hit && rank < need) cand[ncand + rank] = make_key(lo, p);
-        const int taken = min(need, __popc(bal));
-        ncand += taken;
-        need -= taken;
-      });
+      // every remaining candidate has the same score: lowest pages first, in page order (rare;
+      // one warp walks the pages so that the order is kept)
+      if (warp == 0) {
+        int ncand = s_ncand;
+        const unsigned below = (1u << lane) - 1u;
+        for (int base = 0; base < P && need > 0; base += 32) {
+          const int p = base + lane;
+          const bool hit = p < P && order_bits(row[p]) == lo;
+          const unsigned bal = __ballot_sync(0xffffffffu, hit);
+          const int rank = __popc(bal & below);
+          if (hit && rank < need) cand[ncand + rank] = make_key(lo, p);
+          const int taken = min(need, __popc(bal));
+          ncand += taken;
+          need -= taken;
+        }
+        if (lane == 0) s_ncand = ncand;
+      }
       break;
     }
     const int width = 32 - __clz(hi - lo);           // bits needed for hi - lo  (>= 1)
     const int shift = width > 8 ? width - 8 : 0;      // (ob - lo) >> shift is in [0, 255]
-    for (int b = lane; b < kSelBins; b += 32) hist[b] = 0;
-    __syncwarp();
-    for_each_key<CACHED>(cache, row, P, lane, [&](uint32_t ob, int, bool in) {
-      if (in && ob >= lo && ob <= hi) atomicAdd(&hist[(ob - lo) >> shift], 1);
+    for (int b = tid; b < kSelBins; b += kSelThreads) hist[b] = 0;
+    __syncthreads();
+    for_each_key<CACHED>(cache, row, P, tid, [&](uint32_t ob, int) {
+      if (ob >= lo && ob <= hi) atomicAdd(&hist[(ob - lo) >> shift], 1);
     });
-    __syncwarp();
-    // lane owns bins [8*lane, 8*lane+8); suffix sums over lanes locate the threshold bin
-    int c[8], tot = 0;
+    __syncthreads();
+    if (warp == 0) {
+      // lane owns bins [8*lane, 8*lane+8); suffix sums over lanes locate the threshold bin
+      int c[8], tot = 0;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) { c[e] = hist[8 * lane + e]; tot += c[e]; }
-    int suf = tot;                                     // inclusive suffix: lanes >= this one
+      for (int e = 0; e < 8; ++e) { c[e] = hist[8 * lane + e]; tot += c[e]; }
+      int suf = tot;                                   // inclusive suffix: lanes >= this one
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int t = __shfl_down_sync(0xffffffffu, suf, o);
-      if (lane + o < 32) suf += t;
-    }
-    const int above_lanes = suf - tot;
-    const bool owner = above_lanes < need && need <= suf;
-    int bstar = 0, cnt_above = 0, cnt_thr = 0;
-    if (owner) {
-      int run = above_lanes;
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_down_sync(0xffffffffu, suf, o);
+        if (lane + o < 32) suf += t;
+      }
+      const int above_lanes = suf - tot;
+      if (above_lanes < need && need <= suf) {
+        int run = above_lanes;
 #pragma unroll
-      for (int e = 7; e >= 0; --e) {
-        if (run < need && need <= run + c[e]) { bstar = 8 * lane + e; cnt_above = run; cnt_thr = c[e]; }
-        run += c[e];
+        for (int e = 7; e >= 0; --e) {
+          if (run < need && need <= run + c[e]) { s_bstar = 8 * lane + e; s_above = run; s_thr = c[e]; }
+          run += c[e];
+        }
       }
     }
-    const int src = __ffs(__ballot_sync(0xffffffffu, owner)) - 1;
-    bstar = __shfl_sync(0xffffffffu, bstar, src);
-    cnt_above = __shfl_sync(0xffffffffu, cnt_above, src);
-    cnt_thr = __shfl_sync(0xffffffffu, cnt_thr, src);
-    const bool finish = ncand + cnt_above + cnt_thr <= kSelCap;
-    // take the keys above the threshold bin (and, when finishing, the threshold bin itself)
-    for_each_key<CACHED>(cache, row, P, lane, [&](uint32_t ob, int p, bool in) {
-      bool take = false;
-      if (in && ob >= lo && ob <= hi) {
+    __syncthreads();
+    const int bstar = s_bstar, cnt_above = s_above, cnt_thr = s_thr;
+    const bool finish = s_ncand + cnt_above + cnt_thr <= kSelCap;
+    __syncthreads();                                   // everyone has read s_ncand before it moves
+    // take the keys above the threshold bin (and, when finishing, the threshold bin itself); the
+    // order inside cand does not matter: it is sorted below
+    for_each_key<CACHED>(cache, row, P, tid, [&](uint32_t ob, int p) {
+      if (ob >= lo && ob <= hi) {
         const int bin = static_cast<int>((ob - lo) >> shift);
-        take = bin > bstar || (finish && bin == bstar);
+        if (bin > bstar || (finish && bin == bstar)) cand[atomicAdd(&s_ncand, 1)] = make_key(ob, p);
       }
-      const unsigned bal = __ballot_sync(0xffffffffu, take);
-      if (take) cand[ncand + __popc(bal & below)] = make_key(ob, p);
-      ncand += __popc(bal);
     });
     if (finish) break;
     need -= cnt_above;
@@ -289,24 +317,27 @@ __device__ __forceinline__ void topk_select_body(const float* __restrict__ row, 
     const unsigned long long top = static_cast<unsigned long long>(nlo) + ((1ull << shift) - 1ull);
     hi = top < hi ? static_cast<uint32_t>(top) : hi;
     lo = nlo;
+    __syncthreads();
   }
+  __syncthreads();
   // sort the candidates (descending) and emit the first kk
+  const int ncand = s_ncand;
   int n2 = 2;
   while (n2 < ncand) n2 <<= 1;
-  for (int i = ncand + lane; i < n2; i += 32) cand[i] = 0ull;
-  __syncwarp();
+  for (int i = ncand + tid; i < n2; i += kSelThreads) cand[i] = 0ull;
+  __syncthreads();
   for (int k2 = 2; k2 <= n2; k2 <<= 1) {
     for (int j = k2 >> 1; j > 0; j >>= 1) {
-      for (int t = lane; t < (n2 >> 1); t += 32) {
+      for (int t = tid; t < (n2 >> 1); t += kSelThreads) {
         const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
         const int x = i | j;
         const unsigned long long ka = cand[i], kb = cand[x];
         if ((ka < kb) == ((i & k2) == 0)) { cand[i] = kb; cand[x] = ka; }
       }
-      __syncwarp();
+      __syncthreads();
     }
   }
-  for (int j = lane; j < k; j += 32) {
+  for (int j = tid; j < k; j += kSelThreads) {
     if (j < kk) {
       const unsigned long long key = cand[j];
       out_pages[j] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(key));
@@ -317,34 +348,29 @@ __device__ __forceinline__ void topk_select_body(const float* __restrict__ row, 
   }
 }
 
-__global__ void __launch_bounds__(kSelWarps * 32)
+__global__ void __launch_bounds__(kSelThreads)
 topk_select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ kv_len,
                    const int32_t* __restrict__ active_idx, const int32_t* __restrict__ n_active,
                    const int32_t* __restrict__ step, int32_t* __restrict__ topk_pages,
                    float* __restrict__ topk_scores, int N, int B, int Hq, int g, int k, int score_stride,
                    int32_t* __restrict__ status) {
-  __shared__ unsigned long long s_cand[kSelWarps][kSelCap];
-  __shared__ int s_hist[kSelWarps][kSelBins];
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int qid = blockIdx.x * kSelWarps + warp;
-  const int h = qid % Hq, a = (qid / Hq) % B, s = qid / (Hq * B);
-  if (s >= N) return;
+  // queries of the same active slot are adjacent, so the CTAs that have work are the first ones
+  const int qid = blockIdx.x;
+  const int h = qid % Hq, s = (qid / Hq) % N, a = qid / (Hq * N);
   if (step && step[s] == 0) return;
   int na = n_active[s];
   na = na > B ? B : na;
   if (a >= na) return;
   const int tok = active_idx[s * B + a];
-  if (tok < 0 || tok >= B) { if (lane == 0) set_status(status, LOSA_ERR_BOUNDS); return; }
+  if (tok < 0 || tok >= B) { if (threadIdx.x == 0) set_status(status, LOSA_ERR_BOUNDS); return; }
   const int P = pages_of(kv_len[s], g);
   const int kk = min(k, P);
   const float* row = scores + ((static_cast<size_t>(s) * B + a) * Hq + h) * score_stride;
   const size_t o = ((static_cast<size_t>(s) * B + tok) * Hq + h) * k;
-  if (P <= 1024)
-    topk_select_body<true>(row, P, kk, k, s_cand[warp], s_hist[warp], topk_pages + o,
-                           topk_scores ? topk_scores + o : nullptr, lane);
+  if (P <= kSelThreads * kSelPerThread)
+    topk_select_body<true>(row, P, kk, k, topk_pages + o, topk_scores ? topk_scores + o : nullptr);
   else
-    topk_select_body<false>(row, P, kk, k, s_cand[warp], s_hist[warp], topk_pages + o,
-                            topk_scores ? topk_scores + o : nullptr, lane);
+    topk_select_body<false>(row, P, kk, k, topk_pages + o, topk_scores ? topk_scores + o : nullptr);
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -460,7 +486,7 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
   const float* sc = reinterpret_cast<const float*>(c->ws + c->lay.scores);
   if (k <= kSelCap) {
     const int queries = sh.batch * sh.block_size * sh.n_q_heads;
-    topk_select_kernel<<<(queries + kSelWarps - 1) / kSelWarps, kSelWarps * 32, 0, st>>>(
+    topk_select_kernel<<<queries, kSelThreads, 0, st>>>(
         sc, kv->kv_len, active_idx, n_active, step, topk_pages, topk_scores_opt, sh.batch, sh.block_size,
         sh.n_q_heads, sh.page_size, k, c->lay.score_stride, status_ptr(c));
     return after_launch(c);

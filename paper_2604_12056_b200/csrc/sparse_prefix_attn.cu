@@ -262,10 +262,11 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
       }
       Lsum += warp_sum(lj * wj);
       const int n = min(32, n_pairs - base);
-      for (int i0 = 0; i0 < n; i0 += 4) {
-        float w[4], v[4][C];
+      constexpr int U = 8;                            // records whose loads are in flight together
+      for (int i0 = 0; i0 < n; i0 += U) {
+        float w[U], v[U][C];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < U; ++u) {
           const int i = i0 + u;
           w[u] = (i < n) ? __shfl_sync(0xffffffffu, wj, i & 31) : 0.f;
           const unsigned long long addr = __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(rec), i & 31);
@@ -274,7 +275,7 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
           for (int c = 0; c < C; ++c) v[u][c] = (w[u] != 0.f) ? src[32 * c] : 0.f;
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u)
+        for (int u = 0; u < U; ++u)
 #pragma unroll
           for (int c = 0; c < C; ++c) acc[c] = fmaf(v[u][c], w[u], acc[c]);
       }

@@ -93,6 +93,17 @@ class LosaLayer:
         B.losa_block_attn_merge(c, q, k_blk, v_blk, self.state, self.out, self.lse_out)
         B.losa_update_prefix_cache(c, self.kv, self.state, q, k_blk, v_blk, False)
 
+    def run_step_fused(self, q, k_blk, v_blk, m_per_seq):
+        """The same layer-step through the single whole-step entry point (losa_denoise_step)."""
+        if self.mode != "losa":
+            raise ValueError("the whole-step call implements the method itself; baselines use run_step")
+        if not hasattr(self, "_step_buf"):
+            self._step_buf = B.StepBuffersT(0, 0, 0, 0, self.active_idx.data_ptr(), self.n_active.data_ptr(),
+                                            self.topk_pages.data_ptr(), self.union_pages.data_ptr(),
+                                            self.union_count.data_ptr())
+        B.losa_denoise_step(self.ctx, q, k_blk, v_blk, self.out, self.lse_out, self.kv, self.state,
+                            self._step_buf, m_per_seq, self.cfg.topk)
+
     def finalize_block(self, k_blk, v_blk):
         B.losa_update_prefix_cache(self.ctx, self.kv, self.state, None, k_blk, v_blk, True)
 

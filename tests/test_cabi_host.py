@@ -81,7 +81,7 @@ def test_null_arguments_are_rejected_without_a_device(lib):
     for fn, nargs in (("losa_select_active", 10), ("losa_page_scores_topk", 10), ("losa_page_union", 10),
                       ("losa_sparse_prefix_attn", 9), ("losa_block_attn_merge", 8),
                       ("losa_update_prefix_cache", 8), ("losa_build_page_summaries", 3),
-                      ("losa_denoise_step_host", 11)):
+                      ("losa_denoise_step_host", 11), ("losa_denoise_step", 12)):
         args = [None] * nargs
         if fn in ("losa_select_active",):
             args[3] = C.c_int32(64)
