@@ -338,6 +338,10 @@ def run_ours(args, cfg):
         kinds.append("dense" if i % T == 0 else "losa")
     layer.ctx.profile_stage4(False)
 
+    # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of this kernel, from the
+    # ncu capture summarised in profiles/attn_mma_kernel_c3.txt (same command, workload c3 only)
+    ncu_traffic = {"losa": 162.49e6 + 5.42e6, "dense": 438.54e6 + 6.88e6} if cfg.name == "c3" and args.active_frac is None else None
+
     def roof(sel):
         b = sum(x for x, k in zip(k_bytes, kinds) if k in sel)
         t = sum(x for x, k in zip(k_ms, kinds) if k in sel)
@@ -347,7 +351,8 @@ def run_ours(args, cfg):
         ach = b / (t * 1e-3) / 1e9
         return {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
                 "frac_of_8TBps_nominal": ach / 8000.0, "launches": n, "bytes_per_launch": b / n,
-                "us_per_launch": t / n * 1e3, "traffic": None,
+                "us_per_launch": t / n * 1e3,
+                "traffic": (sum(ncu_traffic[k] for k in kinds if k in sel) / n) if ncu_traffic else None,
                 "peak_source": "measured (MEASURED_PEAKS.json hbm_gbs)" if peaks else "fallback 6650 GB/s"}
     result["roofline"] = roof(("losa", "dense")) or {}
     result["roofline"]["kernel"] = "stage-4 main kernel (paged prefix attention), every launch of whole blocks"
