@@ -209,25 +209,21 @@ def run_reference(args, cfg):
 # ------------------------------------------------------------------------------- GPU arm
 def run_ours(args, cfg):
     import torch
-    import torch.distributed as dist
     from paper_2604_12056_b200 import binding as B
     from paper_2604_12056_b200 import build as build_mod
+    from paper_2604_12056_b200 import dist as D
     from paper_2604_12056_b200.layer import LosaLayer, to_device, to_host
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    local = D.env_rank()[2]
     torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    dev = torch.device("cuda", local)
+    rank, world, local = D.init("nccl", dev)
     if not os.path.exists(B.LIB_PATH):
         if local == 0:
             build_mod.build()
-        if world > 1:
-            dist.barrier()
-    dev = torch.device("cuda", local)
+        D.barrier()
 
-    w = wl.Workload(cfg, replica=rank)
+    w = wl.Workload(cfg, replica=D.replica_of(rank))
     layer = LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len, "losa", dev)
     T = cfg.steps
     total = args.warmup + args.steps
@@ -284,23 +280,17 @@ def run_ours(args, cfg):
         return [a.elapsed_time(b) for a, b in evs]
 
     timed_pass(0, args.warmup)
-    if world > 1:
-        dist.barrier()
+    D.barrier()
     torch.cuda.synchronize()
     sampler = ClockSampler(local)
     sampler.start()
     pages = []
     ms = timed_pass(args.warmup, args.steps, pages)
     torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
+    D.barrier()
     clocks = sampler.stop()
     assert layer.ctx.poll_status() == 0
-    total_ms = float(sum(ms))
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = D.max_over_ranks(float(sum(ms)), dev)
     ms_per_step = total_ms / args.steps
     sparse_ms = [x for x, (t, _) in zip(ms, pages) if t != 0]
     dense_ms = [x for x, (t, _) in zip(ms, pages) if t == 0]
@@ -388,11 +378,7 @@ def run_ours(args, cfg):
         if i >= args.warmup:
             e2e_ms.append(max(a.elapsed_time(b), 0.0))
     assert layer.ctx.poll_status() == 0
-    e2e_total = float(sum(host_t[args.warmup:])) * 1e3          # host wall clock of the K calls incl. sync
-    if world > 1:
-        t = torch.tensor([e2e_total], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_total = float(t.item())
+    e2e_total = D.max_over_ranks(float(sum(host_t[args.warmup:])) * 1e3, dev)   # host wall clock of the K calls incl. sync
     es = 2 if cfg.dtype == "bf16" else 4
     result["e2e"] = {"value": e2e_total / args.steps * 1e3, "unit": UNIT,
                      "h2d_bytes_per_step": N * Bk * (Hq + 2 * Hkv) * d * es,
@@ -405,9 +391,7 @@ def run_ours(args, cfg):
         extras(args, cfg, w, layer, host_steps, dev_steps, load, flush, (q_s, k_s, v_s, m_s), result, pages)
     if rank == 0:
         print(json.dumps(result))
-    if world > 1:
-        dist.barrier()
-        dist.destroy_process_group()
+    D.shutdown()
 
 
 def extras(args, cfg, w, layer, host_steps, dev_steps, load, flush, static, result, pages):

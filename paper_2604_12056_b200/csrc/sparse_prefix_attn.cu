@@ -391,6 +391,12 @@ __device__ __forceinline__ void mma_bf16(float (&c)[4], const uint32_t (&a)[4], 
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+// 2^x, one MUFU instruction (ex2.approx: 2 ulp; -inf -> 0); the bf16 rounding of P dwarfs its error
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -692,32 +698,36 @@ attn_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             }
           }
         }
-        // ---- online softmax (base-2 units), rows g8 and g8 + 8 of the tile
+        // ---- online softmax (base-2 units), rows g8 and g8 + 8 of the tile.  Raw scores stay in
+        // sacc; the scale is folded into the exponent: p = 2^(s * scale2 - m).
+        if (valid < GP) {                                // only a sequence's last page can be partial
+#pragma unroll
+          for (int n = 0; n < NT; ++n)
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+              if (n * 8 + q4 * 2 + (e & 1) >= valid) sacc[n][e] = -INFINITY;
+        }
         float mx0 = -INFINITY, mx1 = -INFINITY;
 #pragma unroll
         for (int n = 0; n < NT; ++n) {
-#pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const int col = n * 8 + q4 * 2 + (e & 1);
-            const float v = (col < valid) ? sacc[n][e] * scale2 : -INFINITY;
-            sacc[n][e] = v;
-            if (e < 2) mx0 = fmaxf(mx0, v); else mx1 = fmaxf(mx1, v);
-          }
+          mx0 = fmaxf(mx0, fmaxf(sacc[n][0], sacc[n][1]));
+          mx1 = fmaxf(mx1, fmaxf(sacc[n][2], sacc[n][3]));
         }
         mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
         mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
         mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
         mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
-        const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+        // scale2 > 0, so the maximum of the scaled scores is the scaled maximum
+        const float mn0 = fmaxf(m0, mx0 * scale2), mn1 = fmaxf(m1, mx1 * scale2);
         const float ms0 = (mn0 == -INFINITY) ? 0.f : mn0, ms1 = (mn1 == -INFINITY) ? 0.f : mn1;
-        const float c0 = exp2f(m0 - ms0), c1 = exp2f(m1 - ms1);
+        const float c0 = ex2(m0 - ms0), c1 = ex2(m1 - ms1);
         m0 = mn0; m1 = mn1;
         float s0 = 0.f, s1 = 0.f;
         uint32_t pa[GP / 16][4];
 #pragma unroll
         for (int n = 0; n < NT; ++n) {
-          const float e0 = exp2f(sacc[n][0] - ms0), e1 = exp2f(sacc[n][1] - ms0);
-          const float e2 = exp2f(sacc[n][2] - ms1), e3 = exp2f(sacc[n][3] - ms1);
+          const float e0 = ex2(fmaf(sacc[n][0], scale2, -ms0)), e1 = ex2(fmaf(sacc[n][1], scale2, -ms0));
+          const float e2 = ex2(fmaf(sacc[n][2], scale2, -ms1)), e3 = ex2(fmaf(sacc[n][3], scale2, -ms1));
           s0 += e0 + e1;
           s1 += e2 + e3;
           pa[n >> 1][(n & 1) * 2] = pack_bf16(e0, e1);
