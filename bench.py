@@ -35,15 +35,18 @@ from paper_2604_12056_b200 import workloads as wl  # noqa: E402
 METRIC = "denoise-step attention us/layer"
 UNIT = "us/layer-step"
 L2_FLUSH_BYTES = 256 << 20
+# ncu DRAM traffic per stage-4 launch (read + write bytes), by workload; see profiles/
+NCU_TRAFFIC = {"c3": {"losa": 162.49e6 + 5.42e6, "dense": 438.54e6 + 6.88e6}}
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=64)
-    ap.add_argument("--warmup", type=int, default=8)
+    ap.add_argument("--steps", type=int, default=0, help="timed layer-steps (default: 4 blocks of all layers)")
+    ap.add_argument("--warmup", type=int, default=0, help="untimed layer-steps (default: 1 block of all layers)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c3", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--layers", type=int, default=0, help="attention layers (default: 36 for c5, else 1)")
     ap.add_argument("--active-frac", type=float, default=None, help="override the active fraction")
     ap.add_argument("--no-extras", action="store_true", help="skip baselines, stage breakdown, cpu baseline")
     return ap.parse_args()
@@ -51,19 +54,20 @@ def parse_args():
 
 def make_config(args):
     cfg = wl.config(args.workload)
-    if args.workload == "c5":
-        cfg = wl.config("c5", n_blocks=1)     # one layer of the loop; blocks restart on the same prefix
     if args.active_frac is not None:
         cfg = wl.config(args.workload, m_active=wl.active_count(args.active_frac, cfg.block_size),
                         n_blocks=cfg.n_blocks, beta_active=False)
     return cfg
 
 
-def workload_name(cfg):
+def workload_name(cfg, layers=1):
     lens = "/".join(f"{L // 1024}K" for L in cfg.kv_lens)
-    return (f"{cfg.name}: batch {cfg.batch}, prefix {lens} tokens, pages of {cfg.page_size}, "
+    if len(set(cfg.kv_lens)) == 1:
+        lens = f"{cfg.kv_lens[0] // 1024}K"
+    act = "Beta(2,18)*B active tokens/step" if cfg.beta_active else f"{cfg.m_active} active tokens/step"
+    return (f"{cfg.name}: {layers} layer(s), batch {cfg.batch}, prefix {lens} tokens, pages of {cfg.page_size}, "
             f"{cfg.n_q_heads}/{cfg.n_kv_heads} heads x {cfg.head_dim}, block {cfg.block_size}, "
-            f"{cfg.steps} steps/block, {cfg.m_active} active tokens/step, top-{cfg.topk} pages, {cfg.dtype}")
+            f"{cfg.steps} steps/block, {act}, top-{cfg.topk} pages, {cfg.dtype}")
 
 
 # ------------------------------------------------------------------------------- clocks sampling
@@ -199,7 +203,7 @@ def run_reference(args, cfg):
         "impl": "reference", "metric": METRIC, "value": us, "unit": UNIT, "n_gpus": args.gpus,
         "steps": len(timed), "warmup": n_warm, "ms_per_step": us / 1e3,
         "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": workload_name(cfg)},
+        "config": {"workload": workload_name(cfg, 36 if cfg.name == "c5" else 1) + " (the oracle is timed on layer 0)"},
         "cpu_baseline": {"value": us, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": us, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -207,12 +211,60 @@ def run_reference(args, cfg):
 
 
 # ------------------------------------------------------------------------------- GPU arm
-def run_ours(args, cfg):
+class LayerRun:
+    """One attention layer of the workload on the device: its own seeded pool, LoSA cache, static
+    input buffers and two CUDA graphs (the whole-step call; block finalisation)."""
+
+    def __init__(self, cfg, rank, layer, dev):
+        import torch
+        from paper_2604_12056_b200.layer import LosaLayer
+        self.torch, self.cfg = torch, cfg
+        self.w = wl.DeviceWorkload(cfg, replica=rank, layer=layer, device=dev)
+        self.layer = LosaLayer(cfg, self.w.k_pages, self.w.v_pages, self.w.page_table, self.w.kv_len, "losa", dev)
+        self.inputs = {}                       # block -> list of DeviceStepInputs (current and previous block)
+        self.next_block = 0
+        first = self.block_inputs(0)[0]
+        self.q_s, self.k_s, self.v_s, self.m_s = (torch.empty_like(t) for t in (first.q, first.k_blk, first.v_blk, first.m_per_seq))
+        self.graph = self.graph_fin = None
+
+    def block_inputs(self, b):
+        """Inputs of block b (generated in block order; every layer draws the same active counts)."""
+        assert b >= self.next_block - 2, "blocks are generated in order; only the last two are kept"
+        while self.next_block <= b:
+            nb = self.next_block
+            self.inputs[nb] = [self.w.start_block()] + [self.w.next_step() for _ in range(self.cfg.steps - 1)]
+            self.next_block = nb + 1
+            for old in [k for k in self.inputs if k < nb - 1]:
+                del self.inputs[old]
+        return self.inputs[b]
+
+    def load(self, b, t):
+        i = self.block_inputs(b)[t]
+        self.q_s.copy_(i.q); self.k_s.copy_(i.k_blk); self.v_s.copy_(i.v_blk); self.m_s.copy_(i.m_per_seq)
+
+    def capture(self):
+        torch = self.torch
+        self.load(0, 0)
+        self.layer.run_step_fused(self.q_s, self.k_s, self.v_s, self.m_s)      # un-captured first call
+        torch.cuda.synchronize()
+        self.layer.step.zero_()
+        n0 = self.layer.ctx.launch_count()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            self.layer.run_step_fused(self.q_s, self.k_s, self.v_s, self.m_s)
+        n1 = self.layer.ctx.launch_count()
+        self.graph_fin = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph_fin):
+            self.layer.finalize_block(self.k_s, self.v_s)
+        return n1 - n0, self.layer.ctx.launch_count() - n1
+
+
+def run_ours(args, cfg0):
     import torch
     from paper_2604_12056_b200 import binding as B
     from paper_2604_12056_b200 import build as build_mod
     from paper_2604_12056_b200 import dist as D
-    from paper_2604_12056_b200.layer import LosaLayer, to_device, to_host
+    from paper_2604_12056_b200.layer import to_host
 
     local = D.env_rank()[2]
     torch.cuda.set_device(local)
@@ -223,73 +275,68 @@ def run_ours(args, cfg):
             build_mod.build()
         D.barrier()
 
-    w = wl.Workload(cfg, replica=D.replica_of(rank))
-    layer = LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len, "losa", dev)
-    T = cfg.steps
-    total = args.warmup + args.steps
-    n_blocks = (total + T - 1) // T
-    host_steps = []
-    for _ in range(n_blocks):
-        host_steps += w.block_steps()
-    host_steps = host_steps[:total]
-    dev_steps = [(to_device(i.q, dev), to_device(i.k_blk, dev), to_device(i.v_blk, dev), to_device(i.m_per_seq, dev))
-                 for i in host_steps]
-    q_s, k_s, v_s = (torch.empty_like(t) for t in dev_steps[0][:3])
-    m_s = torch.empty_like(dev_steps[0][3])
+    L = args.layers if args.layers else (36 if cfg0.name == "c5" else 1)
+    T = cfg0.steps
+    per_block = T * L
+    n_prof = min(args.steps, per_block)                       # eager pass with events around the stage-4 kernel
+    n_e2e = min(args.steps, per_block)                        # host-buffer pass
+    def blocks_for(n):
+        return (n + per_block - 1) // per_block
+    total_blocks = blocks_for(args.warmup + args.steps) + blocks_for(n_prof) + blocks_for(n_e2e) + 2
+    cfg = wl.config(cfg0.name, n_blocks=total_blocks, m_active=cfg0.m_active, beta_active=cfg0.beta_active)
+    runs = [LayerRun(cfg, D.replica_of(rank), l, dev) for l in range(L)]
+    launches_step = launches_fin = 0
+    for r in runs:
+        launches_step, launches_fin = r.capture()
     flush_w = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
     flush_r = torch.zeros(L2_FLUSH_BYTES // 4, dtype=torch.float32, device=dev)   # fp32: sum() reads it in place
+    use_flush = L == 1            # with several layers, consecutive steps read different ~1 GiB pools
 
-    class _Flush:
+    def flush(v):
         """Evicts the L2 (write > L2, then read > L2 so that no dirty lines are left behind)."""
-        def fill_(self, v):
-            flush_w.fill_(v)
+        if use_flush:
+            flush_w.fill_(v & 0xff)
             flush_r.sum()
-    flush = _Flush()
 
-    def load(i):
-        q, k, v, m = dev_steps[i]
-        q_s.copy_(q); k_s.copy_(k); v_s.copy_(v); m_s.copy_(m)
-        if i % T == 0:
-            layer.step.zero_()          # a new block starts: no valid cache
+    def where(i):
+        return i // per_block, (i % per_block) // L, i % L     # block, denoising step, layer
 
-    # eager warm-up of every kernel (tensor maps, attributes, second stream), then capture the
-    # whole-step call
-    load(0)
-    layer.run_step_fused(q_s, k_s, v_s, m_s)
-    torch.cuda.synchronize()
-    assert layer.ctx.poll_status() == 0
-    n0 = layer.ctx.launch_count()
-    graph = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(graph):
-        layer.run_step_fused(q_s, k_s, v_s, m_s)
-    launches_per_step = layer.ctx.launch_count() - n0
+    state = {"launches": 0}
 
-    def timed_pass(first, count, record_pages=None):
+    def graph_pass(first, count, record=None):
+        """Layer-steps first .. first+count-1 in order, one CUDA-event pair per layer-step."""
         evs = []
         for i in range(first, first + count):
-            load(i)
-            flush.fill_(i & 0xff)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            graph.replay()
-            b.record()
-            evs.append((a, b))
-            if record_pages is not None:
-                record_pages.append((i % T, pages_read(to_host(layer.union_count))))
+            b, t, l = where(i)
+            r = runs[l]
+            r.load(b, t)
+            flush(i)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            r.graph.replay()
+            if t == T - 1:
+                r.graph_fin.replay()                           # the block is finalised: append K_b, V_b
+            e1.record()
+            evs.append((e0, e1))
+            state["launches"] += launches_step + (launches_fin if t == T - 1 else 0)
+            if record is not None:
+                record.append((t, pages_read(to_host(r.layer.union_count))))
         torch.cuda.synchronize()
         return [a.elapsed_time(b) for a, b in evs]
 
-    timed_pass(0, args.warmup)
+    graph_pass(0, args.warmup)
     D.barrier()
     torch.cuda.synchronize()
     sampler = ClockSampler(local)
     sampler.start()
     pages = []
-    ms = timed_pass(args.warmup, args.steps, pages)
+    state["launches"] = 0
+    ms = graph_pass(args.warmup, args.steps, pages)
     torch.cuda.synchronize()
     D.barrier()
     clocks = sampler.stop()
-    assert layer.ctx.poll_status() == 0
+    for r in runs:
+        assert r.layer.ctx.poll_status() == 0
     total_ms = D.max_over_ranks(float(sum(ms)), dev)
     ms_per_step = total_ms / args.steps
     sparse_ms = [x for x, (t, _) in zip(ms, pages) if t != 0]
@@ -299,38 +346,49 @@ def run_ours(args, cfg):
         "metric": METRIC, "value": ms_per_step * 1e3, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-        "config": {"workload": workload_name(cfg), "sequences_per_gpu": cfg.batch,
+        "config": {"workload": workload_name(cfg0, L), "sequences_per_gpu": cfg.batch, "layers": L,
+                   "step": "one layer-step = stages 1-6 for one layer and one denoising step; steps run in model order "
+                           "(block, denoising step, layer); the last step of a block also appends the block to the cache",
                    "launch": "CUDA graph replay of losa_denoise_step (stages 1-6 in one call)",
-                   "l2": "flushed between steps, outside the timed region: 256 MiB write, then 256 MiB read so no dirty lines remain"},
-        "clocks": clocks, "gpu_launches": launches_per_step * args.steps,
+                   "l2": ("flushed between steps, outside the timed region: 256 MiB write, then 256 MiB read so no dirty "
+                          "lines remain") if use_flush else
+                         ("inputs larger than L2: consecutive layer-steps read different per-layer KV pools "
+                          f"({runs[0].w.k_pages.numel() * 4 / 2**20:.0f} MiB each), no flush")},
+        "clocks": clocks, "gpu_launches": state["launches"],
         "step_us": {"losa_step_median": float(np.median(sparse_ms)) * 1e3 if sparse_ms else None,
                     "dense_first_step_median": float(np.median(dense_ms)) * 1e3 if dense_ms else None},
     }
 
-    # ---- dominant kernel (stage-4 main kernel), eager launches of the same steps, events around it
+    # ---- dominant kernel (stage-4 main kernel): eager launches of the following layer-steps, events
+    # recorded by the library immediately around that kernel
     peaks = {}
     try:
         peaks = json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))
     except Exception:
         pass
     peak = float(peaks.get("hbm_gbs", 6650.0))
-    layer.ctx.profile_stage4(True)
+    first = blocks_for(args.warmup + args.steps) * per_block           # continue at the next block boundary
     k_bytes, k_ms, kinds = [], [], []
-    first = args.warmup - (args.warmup % T)       # start at a block boundary
-    first = first if first + args.steps <= total else 0
-    for i in range(first, min(total, first + max(args.steps, T))):
-        load(i)
-        flush.fill_(i & 0xff)
-        layer.run_step_fused(q_s, k_s, v_s, m_s)
-        k_ms.append(layer.ctx.stage4_last_ms())
-        k_bytes.append(stage4_bytes(cfg, to_host(layer.union_pages), to_host(layer.union_count),
-                                    to_host(layer.n_active), to_host(layer.kv_len)))
-        kinds.append("dense" if i % T == 0 else "losa")
-    layer.ctx.profile_stage4(False)
-
+    for r in runs:
+        r.layer.step.zero_()                                           # a new block starts for every layer
+        r.layer.ctx.profile_stage4(True)
+    for i in range(first, first + n_prof):
+        b, t, l = where(i)
+        r = runs[l]
+        r.load(b, t)
+        flush(i)
+        r.layer.run_step_fused(r.q_s, r.k_s, r.v_s, r.m_s)
+        k_ms.append(r.layer.ctx.stage4_last_ms())
+        k_bytes.append(stage4_bytes(cfg, to_host(r.layer.union_pages), to_host(r.layer.union_count),
+                                    to_host(r.layer.n_active), to_host(r.layer.kv_len)))
+        kinds.append("dense" if t == 0 else "losa")
+        if t == T - 1:
+            r.layer.finalize_block(r.k_s, r.v_s)
+    for r in runs:
+        r.layer.ctx.profile_stage4(False)
     # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of this kernel, from the
-    # ncu capture summarised in profiles/attn_mma_kernel_c3.txt (same command, workload c3 only)
-    ncu_traffic = {"losa": 162.49e6 + 5.42e6, "dense": 438.54e6 + 6.88e6} if cfg.name == "c3" and args.active_frac is None else None
+    # ncu captures summarised under profiles/ (same command, that workload only)
+    ncu_traffic = NCU_TRAFFIC.get(cfg0.name) if args.active_frac is None else None
 
     def roof(sel):
         b = sum(x for x, k in zip(k_bytes, kinds) if k in sel)
@@ -349,66 +407,69 @@ def run_ours(args, cfg):
     result["roofline_losa_steps"] = roof(("losa",))
     result["roofline_dense_first_step"] = roof(("dense",))
 
-    # ---- end to end through the host-buffer entry point
+    # ---- end to end through the host-buffer entry point (eager, pinned host inputs, output read back)
     k = cfg.topk
     N, Bk, Hq, Hkv, d = cfg.batch, cfg.block_size, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
-    td = B.torch_dtype(layer.dtype)
+    td = B.torch_dtype(runs[0].layer.dtype)
     pin = lambda shape: torch.empty(shape, dtype=td).pin_memory()
     h_q, h_k, h_v, h_o = pin((N, Bk, Hq, d)), pin((N, Bk, Hkv, d)), pin((N, Bk, Hkv, d)), pin((N, Bk, Hq, d))
-    d_q, d_k, d_v = torch.empty_like(q_s), torch.empty_like(k_s), torch.empty_like(v_s)
-    buf = B.StepBuffersT(d_q.data_ptr(), d_k.data_ptr(), d_v.data_ptr(), layer.out.data_ptr(),
-                         layer.active_idx.data_ptr(), layer.n_active.data_ptr(), layer.topk_pages.data_ptr(),
-                         layer.union_pages.data_ptr(), layer.union_count.data_ptr())
-    e2e_ms = []
+    d_q, d_k, d_v = (torch.empty_like(t) for t in (runs[0].q_s, runs[0].k_s, runs[0].v_s))
+    first = (blocks_for(args.warmup + args.steps) + blocks_for(n_prof)) * per_block
+    for r in runs:
+        r.layer.step.zero_()
     host_t = []
-    for i in range(total):
-        q, kk, vv, m = dev_steps[i]
-        h_q.copy_(q.cpu()); h_k.copy_(kk.cpu()); h_v.copy_(vv.cpu()); m_s.copy_(m)
-        if i % T == 0:
-            layer.step.zero_()
-        flush.fill_(i & 0xff)
+    for i in range(first, first + n_e2e):
+        b, t, l = where(i)
+        r = runs[l]
+        lay = r.layer
+        inp = r.block_inputs(b)[t]
+        h_q.copy_(inp.q.cpu()); h_k.copy_(inp.k_blk.cpu()); h_v.copy_(inp.v_blk.cpu()); r.m_s.copy_(inp.m_per_seq)
+        buf = B.StepBuffersT(d_q.data_ptr(), d_k.data_ptr(), d_v.data_ptr(), lay.out.data_ptr(),
+                             lay.active_idx.data_ptr(), lay.n_active.data_ptr(), lay.topk_pages.data_ptr(),
+                             lay.union_pages.data_ptr(), lay.union_count.data_ptr())
+        flush(i)
         torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         t0 = time.perf_counter()
-        a.record()
-        B.losa_denoise_step_host(layer.ctx, h_q, h_k, h_v, h_o, layer.kv, layer.state, buf, m_s, k)
-        b.record()
-        b.synchronize()
+        B.losa_denoise_step_host(lay.ctx, h_q, h_k, h_v, h_o, lay.kv, lay.state, buf, r.m_s, k)
+        if t == T - 1:
+            lay.finalize_block(d_k, d_v)
+        torch.cuda.synchronize()
         host_t.append(time.perf_counter() - t0)
-        if i >= args.warmup:
-            e2e_ms.append(max(a.elapsed_time(b), 0.0))
-    assert layer.ctx.poll_status() == 0
-    e2e_total = D.max_over_ranks(float(sum(host_t[args.warmup:])) * 1e3, dev)   # host wall clock of the K calls incl. sync
+    for r in runs:
+        assert r.layer.ctx.poll_status() == 0
+    e2e_total = D.max_over_ranks(float(sum(host_t)) * 1e3, dev)
     es = 2 if cfg.dtype == "bf16" else 4
-    result["e2e"] = {"value": e2e_total / args.steps * 1e3, "unit": UNIT,
+    result["e2e"] = {"value": e2e_total / n_e2e * 1e3, "unit": UNIT, "steps": n_e2e,
                      "h2d_bytes_per_step": N * Bk * (Hq + 2 * Hkv) * d * es,
                      "d2h_bytes_per_step": N * Bk * Hq * d * es,
-                     "device_span_us": float(np.mean(e2e_ms)) * 1e3,
                      "how": "losa_denoise_step_host on pinned host q/k_blk/v_blk -> host out, eager launches, "
                             "host wall clock per call including the final synchronise"}
 
     if rank == 0 and not args.no_extras:
-        extras(args, cfg, w, layer, host_steps, dev_steps, load, flush, (q_s, k_s, v_s, m_s), result, pages)
+        extras(args, cfg, runs[0], flush, result, pages, (blocks_for(args.warmup + args.steps) + blocks_for(n_prof) + blocks_for(n_e2e)))
     if rank == 0:
         print(json.dumps(result))
     D.shutdown()
 
 
-def extras(args, cfg, w, layer, host_steps, dev_steps, load, flush, static, result, pages):
-    """Stage breakdown, the two comparison policies on the same inputs, pages read, oracle timing."""
+def extras(args, cfg, run, flush, result, pages, block0):
+    """Layer 0 only: stage breakdown, the two comparison policies on the same inputs, pages read,
+    oracle timing.  Uses the two blocks after `block0`; no block is finalised here."""
     import torch
     from paper_2604_12056_b200 import binding as B
     from paper_2604_12056_b200.layer import LosaLayer, to_host
-    q_s, k_s, v_s, m_s = static
-    T = cfg.steps
+    layer, T = run.layer, cfg.steps
+    q_s, k_s, v_s, m_s = run.q_s, run.k_s, run.v_s, run.m_s
     c = layer.ctx
+    seq = [(block0 + j // T, j % T) for j in range(2 * T)]
 
-    # per-stage device time of LoSA steps (eager, one synchronise before each call)
     names = ["select_active", "page_scores_topk", "page_union", "sparse_prefix_attn", "block_attn_merge",
              "update_prefix_cache"]
     acc = {n: [] for n in names}
-    for i in range(min(len(dev_steps), 2 * T)):
-        load(i)
+    for i, (b, t) in enumerate(seq):
+        run.load(b, t)
+        if t == 0:
+            layer.step.zero_()
         st = layer.stage_step_arg()
         calls = [
             lambda: B.losa_select_active(c, q_s, layer.q_prev, q_s.numel() // (cfg.batch * cfg.block_size), m_s, st,
@@ -422,59 +483,51 @@ def extras(args, cfg, w, layer, host_steps, dev_steps, load, flush, static, resu
             lambda: B.losa_block_attn_merge(c, q_s, k_s, v_s, layer.state, layer.out, layer.lse_out),
             lambda: B.losa_update_prefix_cache(c, layer.kv, layer.state, q_s, k_s, v_s, False),
         ]
-        flush.fill_(i & 0xff)
+        flush(i)
         for n, f in zip(names, calls):
             torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(); f(); b.record(); b.synchronize()
-            if i % T:
-                acc[n].append(a.elapsed_time(b) * 1e3)
-    result["stage_us_losa_step"] = {n: float(np.median(v)) for n, v in acc.items() if v}
+            a, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); f(); b2.record(); b2.synchronize()
+            if t:
+                acc[n].append(a.elapsed_time(b2) * 1e3)
+    result["stage_us_losa_step_eager_calls"] = {n: float(np.median(v)) for n, v in acc.items() if v}
 
-    # pages read per step (sum over sequences and KV heads of the union size)
-    dense_pages = int(sum((int(L) + cfg.page_size - 1) // cfg.page_size for L in cfg.kv_lens) * cfg.n_kv_heads)
+    dense_pages = int(sum((int(L) + cfg.page_size - 1) // cfg.page_size for L in to_host(layer.kv_len)) * cfg.n_kv_heads)
     losa_pages = [p for t, p in pages if t != 0]
-    result["pages_read_per_step"] = {"losa": float(np.mean(losa_pages)) if losa_pages else None, "dense": dense_pages}
+    result["pages_read_per_step"] = {"losa": float(np.mean(losa_pages)) if losa_pages else None, "dense": dense_pages,
+                                     "note": "sum over sequences and KV heads of the (page, KV head) slices listed, per layer-step"}
 
-    # naive per-query sparse attention and dense prefix attention, same inputs, same calls
-    for mode in ("naive", "dense"):
-        other = LosaLayer(cfg, None, None, None, layer.kv_len, mode, q_s.device, share_pool_with=layer)
+    result["baselines_us_per_step_eager"] = {}
+    for mode in ("naive", "dense", "losa"):
+        other = layer if mode == "losa" else LosaLayer(cfg, None, None, None, layer.kv_len, mode, q_s.device, share_pool_with=layer)
         ms, pg = [], []
-        for i in range(min(len(dev_steps), 2 * T)):
-            q, k, v, m = dev_steps[i]
-            q_s.copy_(q); k_s.copy_(k); v_s.copy_(v); m_s.copy_(m)
-            if i % T == 0:
+        for i, (b, t) in enumerate(seq):
+            run.load(b, t)
+            if t == 0:
                 other.step.zero_()
-            flush.fill_(i & 0xff)
+            flush(i)
             torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(); other.run_step(q_s, k_s, v_s, m_s); b.record(); b.synchronize()
-            if i % T:
-                ms.append(a.elapsed_time(b) * 1e3)
+            a, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); other.run_step(q_s, k_s, v_s, m_s); b2.record(); b2.synchronize()
+            if t:
+                ms.append(a.elapsed_time(b2) * 1e3)
                 pg.append(pages_read(to_host(other.union_count)))
-        result.setdefault("baselines_us_per_step_eager", {})[mode] = float(np.median(ms)) if ms else None
-        result["pages_read_per_step"][mode if mode == "naive" else "dense_measured"] = float(np.mean(pg)) if pg else None
-        other.ctx.close()
-    # LoSA eager for a like-for-like comparison with the two eager baselines above
-    ms = []
-    for i in range(min(len(dev_steps), 2 * T)):
-        load(i)
-        flush.fill_(i & 0xff)
-        torch.cuda.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record(); layer.run_step(q_s, k_s, v_s, m_s); b.record(); b.synchronize()
-        if i % T:
-            ms.append(a.elapsed_time(b) * 1e3)
-    result["baselines_us_per_step_eager"]["losa"] = float(np.median(ms)) if ms else None
+        result["baselines_us_per_step_eager"][mode] = float(np.median(ms)) if ms else None
+        if mode != "losa":
+            result["pages_read_per_step"][mode if mode == "naive" else "dense_measured"] = float(np.mean(pg)) if pg else None
+            other.ctx.close()
 
     # the oracle on this machine's host cores (a reported baseline, not a target)
     try:
         from oracle import oracle as orc
         orc.build()
-        per_step, t_dense, t_sparse, cores = oracle_block_time(cfg, w, host_steps[:T])
+        host_w = run.w.host_copy()
+        host_w.kv_len = to_host(layer.kv_len).astype(np.int32)
+        host_steps = [x.host_copy() for x in run.block_inputs(block0)]
+        per_step, t_dense, t_sparse, cores = oracle_block_time(cfg, host_w, host_steps)
         result["cpu_baseline"] = {
             "value": per_step * 1e6, "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": (f"one full LoSA layer-step ({t_sparse:.2f} s) and a dense first step whose prefix attention ran "
+            "sample": (f"layer 0: one full LoSA layer-step ({t_sparse:.2f} s) and a dense first step whose prefix attention ran "
                        f"on 2 of {cfg.block_size} block tokens and was scaled x{cfg.block_size // 2} ({t_dense:.2f} s), "
                        f"averaged over a block of {T} steps")}
     except Exception as ex:  # pragma: no cover
@@ -484,9 +537,15 @@ def extras(args, cfg, w, layer, host_steps, dev_steps, load, flush, static, resu
 
 def main():
     args = parse_args()
+    cfg = make_config(args)
+    layers = args.layers if args.layers else (36 if cfg.name == "c5" else 1)
+    per_block = cfg.steps * layers
+    if args.steps <= 0:
+        args.steps = 4 * per_block if args.impl == "ours" else 3
+    if args.warmup <= 0:
+        args.warmup = per_block if args.impl == "ours" else 3
     if args.warmup < 3:
         args.warmup = 3
-    cfg = make_config(args)
     if args.impl == "reference":
         run_reference(args, cfg)
     else:

@@ -299,3 +299,175 @@ class Workload:
     # -- bookkeeping ------------------------------------------------------------------------------
     def pool_bytes(self) -> int:
         return self.k_pages.nbytes + self.v_pages.nbytes
+
+
+# ---------------------------------------------------------------- device-side generation (torch)
+class DeviceWorkload:
+    """The same recipe as `Workload`, drawn with torch on a CUDA device.
+
+    Used where host generation would take minutes (the 36-layer configuration: about 1 GiB of K/V
+    per layer).  Tensors live on the device (bf16 / fp32 / int32); `host_copy()` returns numpy
+    arrays in the formats `Workload` uses, so that a CPU checker can be fed the same bytes.  The
+    number of active tokens per step is drawn on the host from a seed that does not depend on the
+    layer, so all layers of a model share it."""
+
+    def __init__(self, cfg: Config, replica: int = 0, layer: int = 0, device="cuda"):
+        import torch
+        self.torch = torch
+        self.cfg, self.replica, self.layer, self.device = cfg, replica, layer, device
+        self.gen = torch.Generator(device=device)
+        self.gen.manual_seed(seed_for(cfg, replica, layer))
+        self.m_rng = np.random.Generator(np.random.PCG64(seed_for(cfg, replica, 0) + 7))
+        self.dt = torch.bfloat16 if cfg.dtype == "bf16" else torch.float32
+        N, Hkv, g, d = cfg.batch, cfg.n_kv_heads, cfg.page_size, cfg.head_dim
+        Pmax = cfg.max_pages_per_seq
+        self.n_phys = N * Pmax
+        self.page_table = torch.randperm(self.n_phys, generator=self.gen, device=device).to(torch.int32).reshape(N, Pmax).contiguous()
+        self.kv_len = torch.tensor(cfg.kv_lens, dtype=torch.int32, device=device)
+        self.k_pages = torch.zeros((self.n_phys, Hkv, g, d), dtype=self.dt, device=device)
+        self.v_pages = torch.zeros((self.n_phys, Hkv, g, d), dtype=self.dt, device=device)
+        self.page_means, self.common_dir = [], []
+        for s in range(N):
+            self._fill_prefix(s)
+        self._cur = None
+
+    def _randn(self, *shape):
+        return self.torch.randn(*shape, generator=self.gen, device=self.device, dtype=self.torch.float32)
+
+    def _unit(self, x):
+        return x / x.norm(dim=-1, keepdim=True)
+
+    def _fill_prefix(self, s):
+        torch, c = self.torch, self.cfg
+        Hkv, g, d = c.n_kv_heads, c.page_size, c.head_dim
+        L = int(c.kv_lens[s])
+        P = (L + g - 1) // g
+        if P == 0:
+            self.page_means.append(torch.zeros((0, Hkv, d), device=self.device))
+            self.common_dir.append(self._unit(self._randn(Hkv, d)))
+            return
+        rt_d = float(np.sqrt(d))
+        if c.clustered:
+            u = self._unit(self._randn(P, Hkv, d))
+            pick = torch.randint(0, P, (Hkv, 16), generator=self.gen, device=self.device)
+            cdir = self._unit(torch.stack([u[pick[h], h].sum(0) for h in range(Hkv)]))
+            if c.heavy_frac > 0:
+                nh = int(round(c.heavy_frac * P))
+                heavy = torch.randperm(P, generator=self.gen, device=self.device)[:nh]
+                o = self._randn(nh, Hkv, d)
+                o = self._unit(o - (o * cdir[None]).sum(-1, keepdim=True) * cdir[None])
+                u[heavy] = 0.8 * cdir[None] + 0.6 * o
+            self.page_means.append(u)
+            self.common_dir.append(cdir)
+        phys = self.page_table[s, :P].long()
+        chunk = max(1, (1 << 26) // (Hkv * g * d))
+        for p0 in range(0, P, chunk):
+            p1 = min(P, p0 + chunk)
+            noise = self._randn(p1 - p0, Hkv, g, d)
+            if c.clustered:
+                kk = rt_d * self.page_means[s][p0:p1, :, None, :] + 0.5 * noise
+                vv = self._randn(p1 - p0, Hkv, g, d)
+            else:
+                kk = noise / rt_d
+                vv = self._randn(p1 - p0, Hkv, g, d) / rt_d
+            if p1 == P and L % g:
+                kk[-1, :, L % g:, :] = float("nan")
+                vv[-1, :, L % g:, :] = float("nan")
+            self.k_pages[phys[p0:p1]] = kk.to(self.dt)
+            self.v_pages[phys[p0:p1]] = vv.to(self.dt)
+
+    def _draw_q_rows(self, s, n):
+        torch, c = self.torch, self.cfg
+        Hq, d, G = c.n_q_heads, c.head_dim, c.group
+        if not c.clustered or self.page_means[s].shape[0] == 0:
+            return self._randn(n, Hq, d) / float(np.sqrt(d))
+        u = self.page_means[s]
+        P = u.shape[0]
+        pick = torch.randint(0, P, (n, Hq, 8), generator=self.gen, device=self.device)
+        kh = (torch.arange(Hq, device=self.device) // G)
+        t = u[pick, kh[None, :, None]].sum(2)
+        if P < 8:
+            t = self._unit(t) + 0.5 * self._unit(self._randn(n, Hq, d))
+        t = self._unit(t)
+        cd = self.common_dir[s][kh][None]
+        mix = c.rho * cd + float(np.sqrt(1 - c.rho ** 2)) * t
+        return float(c.tau * np.sqrt(d)) * self._unit(mix)
+
+    def _draw_kv_rows(self, s, n):
+        c = self.cfg
+        Hkv, d = c.n_kv_heads, c.head_dim
+        if c.clustered:
+            k = float(np.sqrt(d)) * self._blk_mean[s][None] + 0.5 * self._randn(n, Hkv, d)
+            v = self._randn(n, Hkv, d)
+        else:
+            k = self._randn(n, Hkv, d) / float(np.sqrt(d))
+            v = self._randn(n, Hkv, d) / float(np.sqrt(d))
+        return k, v
+
+    def start_block(self):
+        torch, c = self.torch, self.cfg
+        N, B = c.batch, c.block_size
+        self._blk_mean = [self._unit(self._randn(c.n_kv_heads, c.head_dim)) for _ in range(N)]
+        q = torch.stack([self._draw_q_rows(s, B) for s in range(N)])
+        kv = [self._draw_kv_rows(s, B) for s in range(N)]
+        k = torch.stack([a for a, _ in kv])
+        v = torch.stack([b for _, b in kv])
+        self._cur = tuple(x.to(self.dt).float() for x in (q, k, v))
+        return self._pack([np.arange(B)] * N, np.full(N, B, np.int32))
+
+    def draw_m(self) -> int:
+        c = self.cfg
+        if c.beta_active:
+            return int(min(c.block_size, max(1, int(np.floor(self.m_rng.beta(2.0, 18.0) * c.block_size + 0.5)))))
+        return c.m_active
+
+    def next_step(self, m: Optional[int] = None):
+        torch, c = self.torch, self.cfg
+        N, B = c.batch, c.block_size
+        if m is None:
+            m = self.draw_m()
+        q, k, v = (x.clone() for x in self._cur)
+        planted = []
+        for s in range(N):
+            perm = torch.randperm(B, generator=self.gen, device=self.device)
+            act = perm[:m].sort().values
+            noisy = perm[m:]
+            q[s, act] = self._draw_q_rows(s, m)
+            kk, vv = self._draw_kv_rows(s, m)
+            k[s, act], v[s, act] = kk, vv
+            q[s, noisy] += 1e-3 * self._randn(noisy.numel(), *q.shape[2:])
+            k[s, noisy] += 1e-3 * self._randn(noisy.numel(), *k.shape[2:])
+            v[s, noisy] += 1e-3 * self._randn(noisy.numel(), *v.shape[2:])
+            planted.append(act.cpu().numpy())
+        self._cur = tuple(x.to(self.dt).float() for x in (q, k, v))
+        return self._pack(planted, np.full(N, m, np.int32))
+
+    def _pack(self, planted, m_per_seq):
+        q, k, v = (x.to(self.dt).contiguous() for x in self._cur)
+        return DeviceStepInputs(q, k, v, planted, self.torch.from_numpy(m_per_seq).to(self.device))
+
+    def host_copy(self):
+        """numpy view of the pool for a CPU checker (bf16 as uint16 bit patterns)."""
+        import types
+        def np_of(t):
+            t = t.detach().cpu()
+            return t.view(self.torch.int16).numpy().view(np.uint16) if t.dtype == self.torch.bfloat16 else t.numpy()
+        return types.SimpleNamespace(cfg=self.cfg, k_pages=np_of(self.k_pages), v_pages=np_of(self.v_pages),
+                                     page_table=np_of(self.page_table), kv_len=np_of(self.kv_len), n_phys=self.n_phys)
+
+
+@dataclass
+class DeviceStepInputs:
+    q: object
+    k_blk: object
+    v_blk: object
+    planted: List[np.ndarray]
+    m_per_seq: object
+
+    def host_copy(self) -> StepInputs:
+        import torch
+        def np_of(t):
+            t = t.detach().cpu()
+            return t.view(torch.int16).numpy().view(np.uint16) if t.dtype == torch.bfloat16 else t.numpy()
+        return StepInputs(np_of(self.q), np_of(self.k_blk), np_of(self.v_blk), None, self.planted,
+                          [-1] * len(self.planted), np_of(self.m_per_seq).astype(np.int32))

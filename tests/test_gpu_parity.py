@@ -266,3 +266,63 @@ def test_whole_step_call_in_a_cuda_graph_full_size():
     compare(s1, ref, cfg, "c3 whole-step call, graph replay")
     assert (s1["step"] == 2).all()
 
+
+
+def test_full_size_c5_layer_in_the_benchmark_configuration():
+    """One layer of the benchmark's default workload (batch 8 x 32K prefix, Beta(2,18) active
+    counts, top-64 pages), generated on the device like the benchmark does, through the whole-step
+    call replayed from a CUDA graph, followed by the block finalisation.  The LoSA step is compared
+    with the oracle in full; the dense step and the appended block on samples."""
+    import torch
+    from oracle import oracle as orc
+    from paper_2604_12056_b200.layer import LosaLayer
+    cfg = wl.config("c5", n_blocks=2)
+    dw = wl.DeviceWorkload(cfg, replica=0, layer=17)
+    g = LosaLayer(cfg, dw.k_pages, dw.v_pages, dw.page_table, dw.kv_len)
+    d0, d1 = dw.start_block(), dw.next_step()
+    q, kb, vb, m = d0.q.clone(), d0.k_blk.clone(), d0.v_blk.clone(), d0.m_per_seq.clone()
+    g.run_step_fused(q, kb, vb, m)                       # step 0 (dense), un-captured
+    torch.cuda.synchronize()
+    s0 = g.snapshot()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        g.run_step_fused(q, kb, vb, m)
+    for dst, src in ((q, d1.q), (kb, d1.k_blk), (vb, d1.v_blk), (m, d1.m_per_seq)):
+        dst.copy_(src)
+    graph.replay()
+    torch.cuda.synchronize()
+    s1 = g.snapshot()
+    assert g.ctx.poll_status() == 0
+    o = OracleLayer(dw.host_copy())
+    h0, h1 = d0.host_copy(), d1.host_copy()
+    N, B = cfg.batch, cfg.block_size
+    # dense step: two sampled tokens per sequence, one by one on the CPU
+    sample = np.array([3, 28], np.int32)
+    act_s = np.full((N, B), -1, np.int32)
+    act_s[:, :2] = sample
+    up = np.full((N, cfg.n_kv_heads, cfg.max_pages_per_seq), -1, np.int32)
+    up[:, :, :1024] = np.arange(1024, dtype=np.int32)
+    uc = np.full((N, cfg.n_kv_heads), 1024, np.int32)
+    o.o_p[:] = s0["o_p"]
+    o.lse_p[:] = s0["lse_p"]
+    orc.sparse_prefix_attn(o.sh, h0.q, o.kv, act_s, np.full(N, 2, np.int32), up, uc, o.o_p, o.lse_p)
+    assert_close(s0["o_p"][:, sample], o.o_p[:, sample], cfg.dtype, "c5 dense step, sampled o_p")
+    assert_lse_close(s0["lse_p"][:, sample], o.lse_p[:, sample], "c5 dense step, sampled lse_p")
+    # LoSA step in full
+    o.q_prev[:] = h0.q
+    o.step[:] = 1
+    ref = o.run_step(h1)
+    m1 = int(h1.m_per_seq[0])
+    for s in range(N):
+        assert ref["act"][s, :m1].tolist() == sorted(h1.planted[s].tolist())
+    s1["delta"] = ref["delta"]
+    compare(s1, ref, cfg, "c5 layer, LoSA step from a graph")
+    # block finalisation: lengths, and the appended tokens of one sequence / KV head
+    g.finalize_block(kb, vb)
+    torch.cuda.synchronize()
+    s2 = g.snapshot()
+    assert (s2["kv_len"] == 32768 + 32).all() and (s2["step"] == 0).all()
+    from paper_2604_12056_b200.layer import to_host
+    phys = int(to_host(g.page_table)[5, 1024])
+    np.testing.assert_array_equal(to_host(g.k_pages[phys, 3]), to_host(kb[5, :, 3]))
+    np.testing.assert_array_equal(to_host(g.kmax[phys, 3]), to_host(kb[5, :, 3]).max(0))
