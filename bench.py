@@ -35,8 +35,12 @@ from paper_2604_12056_b200 import workloads as wl  # noqa: E402
 METRIC = "denoise-step attention us/layer"
 UNIT = "us/layer-step"
 L2_FLUSH_BYTES = 256 << 20
-# ncu DRAM traffic per stage-4 launch (read + write bytes), by workload; see profiles/
-NCU_TRAFFIC = {"c3": {"losa": 162.49e6 + 5.42e6, "dense": 438.54e6 + 6.88e6}}
+# DRAM traffic of the stage-4 main kernel per listed (page, KV head) slice, from the ncu capture in
+# profiles/attn_mma_kernel_c3.txt (dram__bytes_read.sum + dram__bytes_write.sum over the slices of that
+# launch: 167.91 MB / 9,916 slices on a LoSA step, 445.42 MB / 26,624 on a dense step; 16,384 of
+# these bytes are the slice's K and V).  Traffic grows in proportion to the slices, so a launch's
+# traffic is reported as slices x this figure (pages of 32 tokens, head dim 128, bf16 only).
+NCU_BYTES_PER_SLICE = {"losa": 167.91e6 / 9916, "dense": 445.42e6 / 26624}
 
 
 def parse_args():
@@ -368,7 +372,7 @@ def run_ours(args, cfg0):
         pass
     peak = float(peaks.get("hbm_gbs", 6650.0))
     first = blocks_for(args.warmup + args.steps) * per_block           # continue at the next block boundary
-    k_bytes, k_ms, kinds = [], [], []
+    k_bytes, k_ms, kinds, k_slices = [], [], [], []
     for r in runs:
         r.layer.step.zero_()                                           # a new block starts for every layer
         r.layer.ctx.profile_stage4(True)
@@ -382,13 +386,12 @@ def run_ours(args, cfg0):
         k_bytes.append(stage4_bytes(cfg, to_host(r.layer.union_pages), to_host(r.layer.union_count),
                                     to_host(r.layer.n_active), to_host(r.layer.kv_len)))
         kinds.append("dense" if t == 0 else "losa")
+        k_slices.append(pages_read(to_host(r.layer.union_count)))
         if t == T - 1:
             r.layer.finalize_block(r.k_s, r.v_s)
     for r in runs:
         r.layer.ctx.profile_stage4(False)
-    # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) per launch of this kernel, from the
-    # ncu captures summarised under profiles/ (same command, that workload only)
-    ncu_traffic = NCU_TRAFFIC.get(cfg0.name) if args.active_frac is None else None
+    scalable = cfg.page_size == 32 and cfg.head_dim == 128 and cfg.dtype == "bf16"
 
     def roof(sel):
         b = sum(x for x, k in zip(k_bytes, kinds) if k in sel)
@@ -400,7 +403,7 @@ def run_ours(args, cfg0):
         return {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
                 "frac_of_8TBps_nominal": ach / 8000.0, "launches": n, "bytes_per_launch": b / n,
                 "us_per_launch": t / n * 1e3,
-                "traffic": (sum(ncu_traffic[k] for k in kinds if k in sel) / n) if ncu_traffic else None,
+                "traffic": (sum(NCU_BYTES_PER_SLICE[k] * sl for k, sl in zip(kinds, k_slices) if k in sel) / n) if scalable else None,
                 "peak_source": "measured (MEASURED_PEAKS.json hbm_gbs)" if peaks else "fallback 6650 GB/s"}
     result["roofline"] = roof(("losa", "dense")) or {}
     result["roofline"]["kernel"] = "stage-4 main kernel (paged prefix attention), every launch of whole blocks"
