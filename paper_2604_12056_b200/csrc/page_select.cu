@@ -22,6 +22,34 @@ constexpr int kThreads = 256;
 constexpr int kPagesPerCta = 64;
 constexpr int kRowTile = 32;
 
+// Eight consecutive elements as loaded, converted to fp32 later: lets several dependent-free loads
+// be in flight before any of them is used.
+template <typename T> struct Raw8;
+template <> struct Raw8<__nv_bfloat16> {
+  uint4 u;
+  __device__ __forceinline__ void load(const __nv_bfloat16* p) { u = *reinterpret_cast<const uint4*>(p); }
+  __device__ __forceinline__ void zero() { u = make_uint4(0u, 0u, 0u, 0u); }
+  __device__ __forceinline__ void unpack(float (&v)[8]) const {
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      v[2 * i] = __uint_as_float(w[i] << 16);
+      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+    }
+  }
+};
+template <> struct Raw8<float> {
+  float4 a, b;
+  __device__ __forceinline__ void load(const float* p) {
+    a = *reinterpret_cast<const float4*>(p);
+    b = *reinterpret_cast<const float4*>(p + 4);
+  }
+  __device__ __forceinline__ void zero() { a = make_float4(0.f, 0.f, 0.f, 0.f); b = a; }
+  __device__ __forceinline__ void unpack(float (&v)[8]) const {
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+  }
+};
+
 template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 page_scores_kernel(const T* __restrict__ q, const T* __restrict__ kmin, const T* __restrict__ kmax,
@@ -45,88 +73,149 @@ page_scores_kernel(const T* __restrict__ q, const T* __restrict__ kmin, const T*
   // consecutive 16-byte words (no bank conflicts): element j = 8*c + e sits at (e/4)*(D/2) + 4*c + e%4.
   __shared__ __align__(16) float qpos[kRowTile * D];
   __shared__ __align__(16) float qneg[kRowTile * D];
-  __shared__ float sc[kRowTile][kPagesPerCta + 1];
   const int tid = threadIdx.x;
   const int grp = tid / LPP, sub = tid % LPP;
   const int np = min(kPagesPerCta, P - p0);
 
+  // Three dependent round trips to memory per CTA: (1) the scalars above, (2) this lane's physical
+  // page ids and the block positions of the query rows it will stage, (3) its share of the pages'
+  // kmin / kmax (kept in registers for every query row) and the query rows themselves.  Everything
+  // of a trip is requested before anything of it is used.
+  constexpr int ITER = kPagesPerCta / GROUPS;
+  constexpr int STG = (kRowTile * (D / 8) + kThreads - 1) / kThreads;   // staging items per thread and row tile
+  const int nr_first = min(kRowTile, rows);
+  int phys[ITER], tok0[STG];
+#pragma unroll
+  for (int it = 0; it < ITER; ++it) {
+    const int pl = grp * ITER + it;
+    phys[it] = pl < np ? page_table[static_cast<size_t>(s) * Pmax + p0 + pl] : -1;
+  }
+#pragma unroll
+  for (int i = 0; i < STG; ++i) {
+    const int idx = tid + i * kThreads;
+    tok0[i] = idx < nr_first * (D / 8) ? active_idx[s * B + (idx / (D / 8)) / G] : 0;
+  }
+  Raw8<T> klo[ITER], khi[ITER], q0[STG];
+#pragma unroll
+  for (int it = 0; it < ITER; ++it) {
+    klo[it].zero();
+    khi[it].zero();
+    if (grp * ITER + it < np) {
+      int ph = phys[it];
+      if (ph < 0 || ph >= n_phys) { set_status(status, LOSA_ERR_BOUNDS); ph = 0; }
+      const size_t so = (static_cast<size_t>(ph) * Hkv + kh) * D + sub * 8;
+      klo[it].load(kmin + so);
+      khi[it].load(kmax + so);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < STG; ++i) {
+    const int idx = tid + i * kThreads;
+    q0[i].zero();
+    if (idx < nr_first * (D / 8)) {
+      const int r = idx / (D / 8), ch = idx % (D / 8), gi = r % G;
+      int tok = tok0[i];
+      if (tok < 0 || tok >= B) { set_status(status, LOSA_ERR_BOUNDS); tok = 0; }
+      q0[i].load(q + ((static_cast<size_t>(s) * B + tok) * Hq + kh * G + gi) * D + ch * 8);
+    }
+  }
+  auto stage = [&](int r, int ch, const float (&v)[8]) {
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+      const int at = r * D + (e >> 2) * (D / 2) + ch * 4 + (e & 3);
+      qpos[at] = fmaxf(v[e], 0.f);
+      qneg[at] = fminf(v[e], 0.f);
+    }
+  };
+  float lo[ITER][8], hi[ITER][8];
   for (int r0 = 0; r0 < rows; r0 += kRowTile) {
     const int nr = min(kRowTile, rows - r0);
-    for (int idx = tid; idx < nr * (D / 8); idx += kThreads) {
-      const int r = idx / (D / 8), ch = idx % (D / 8);
-      const int row = r0 + r, a = row / G, gi = row % G;
-      int tok = active_idx[s * B + a];
-      if (tok < 0 || tok >= B) { set_status(status, LOSA_ERR_BOUNDS); tok = 0; }
-      float v[8];
-      load8(q + ((static_cast<size_t>(s) * B + tok) * Hq + kh * G + gi) * D + ch * 8, v);
+    if (r0 == 0) {
 #pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const int at = r * D + (e >> 2) * (D / 2) + ch * 4 + (e & 3);
-        qpos[at] = fmaxf(v[e], 0.f);
-        qneg[at] = fminf(v[e], 0.f);
-      }
-    }
-    __syncthreads();
-    // All summary loads of this CTA's pages are issued before any arithmetic (two dependent
-    // latencies in total instead of two per page).  The trip counts are the same for every lane:
-    // the butterfly below needs whole warps.
-    constexpr int ITER = kPagesPerCta / GROUPS;
-    float lo[ITER][8], hi[ITER][8];
-    int phys[ITER];
-#pragma unroll
-    for (int it = 0; it < ITER; ++it) {
-      const int pl = it * GROUPS + grp;
-      phys[it] = pl < np ? page_table[static_cast<size_t>(s) * Pmax + p0 + pl] : -1;
-    }
-#pragma unroll
-    for (int it = 0; it < ITER; ++it) {
-      const int pl = it * GROUPS + grp;
-#pragma unroll
-      for (int e = 0; e < 8; ++e) { lo[it][e] = 0.f; hi[it][e] = 0.f; }
-      if (pl < np) {
-        int ph = phys[it];
-        if (ph < 0 || ph >= n_phys) { set_status(status, LOSA_ERR_BOUNDS); ph = 0; }
-        const size_t so = (static_cast<size_t>(ph) * Hkv + kh) * D + sub * 8;
-        load8(kmin + so, lo[it]);
-        load8(kmax + so, hi[it]);
-      }
-    }
-    // one query load feeds the chains of all ITER pages held in registers
-    for (int r = 0; r < nr; ++r) {
-      float qp[8], qn[8];
-      *reinterpret_cast<float4*>(&qp[0]) = *reinterpret_cast<const float4*>(&qpos[r * D + sub * 4]);
-      *reinterpret_cast<float4*>(&qp[4]) = *reinterpret_cast<const float4*>(&qpos[r * D + D / 2 + sub * 4]);
-      *reinterpret_cast<float4*>(&qn[0]) = *reinterpret_cast<const float4*>(&qneg[r * D + sub * 4]);
-      *reinterpret_cast<float4*>(&qn[4]) = *reinterpret_cast<const float4*>(&qneg[r * D + D / 2 + sub * 4]);
-      float acc[ITER];
-#pragma unroll
-      for (int it = 0; it < ITER; ++it) acc[it] = 0.f;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-#pragma unroll
-        for (int it = 0; it < ITER; ++it) {
-          acc[it] = __fmaf_rn(qp[j], hi[it][j], acc[it]);
-          acc[it] = __fmaf_rn(qn[j], lo[it][j], acc[it]);
+      for (int i = 0; i < STG; ++i) {
+        const int idx = tid + i * kThreads;
+        if (idx < nr * (D / 8)) {
+          float v[8];
+          q0[i].unpack(v);
+          stage(idx / (D / 8), idx % (D / 8), v);
         }
       }
 #pragma unroll
-      for (int off = LPP / 2; off >= 1; off >>= 1) {
-#pragma unroll
-        for (int it = 0; it < ITER; ++it) acc[it] = __fadd_rn(acc[it], __shfl_xor_sync(0xffffffffu, acc[it], off));
-      }
-#pragma unroll
       for (int it = 0; it < ITER; ++it) {
-        const int pl = it * GROUPS + grp;
-        if (pl < np && sub == 0) sc[r][pl] = __fadd_rn(acc[it], 0.0f);
+        klo[it].unpack(lo[it]);
+        khi[it].unpack(hi[it]);
+      }
+    } else {
+      for (int idx = tid; idx < nr * (D / 8); idx += kThreads) {
+        const int r = idx / (D / 8), ch = idx % (D / 8);
+        const int row = r0 + r, a = row / G, gi = row % G;
+        int tok = active_idx[s * B + a];
+        if (tok < 0 || tok >= B) { set_status(status, LOSA_ERR_BOUNDS); tok = 0; }
+        float v[8];
+        load8(q + ((static_cast<size_t>(s) * B + tok) * Hq + kh * G + gi) * D + ch * 8, v);
+        stage(r, ch, v);
       }
     }
     __syncthreads();
-    for (int idx = tid; idx < nr * kPagesPerCta; idx += kThreads) {
-      const int r = idx / kPagesPerCta, pl = idx % kPagesPerCta;
-      if (pl < np) {
-        const int row = r0 + r, a = row / G, gi = row % G;
-        scores[((static_cast<size_t>(s) * B + a) * Hq + kh * G + gi) * score_stride + p0 + pl] = sc[r][pl];
+    // Two query rows at a time: one load of a row's run feeds the chains of the ITER pages held in
+    // registers.  A lane then has NV = 2 * ITER run sums, one per (page, row) pair; every pair needs
+    // the butterfly c[i] += c[i ^ off] (off = LPP/2 .. 1) over the LPP lanes of its group.  Taken as
+    // a reduce-scatter it costs NV shuffles per lane instead of NV * log2(LPP): at each level the
+    // lane keeps the half of its values chosen by its own bit `off` and sends the other half; the
+    // additions, and their order, are those of the plain butterfly (fp32 addition commutes), so the
+    // result is the same bit for bit.  Lanes 2i and 2i+1 end with pair i = (page it = i / 2, row i % 2).
+    constexpr int NV = 2 * ITER;
+    static_assert(NV == LPP / 2, "one result per pair of lanes");
+    int a = r0 / G, gi = r0 % G;          // row r0 + r = (active token a, head gi of the KV head), gi fastest
+    for (int r = 0; r < nr; r += 2) {
+      float v[NV];
+#pragma unroll
+      for (int rr = 0; rr < 2; ++rr) {
+        const int rs = min(r + rr, nr - 1);         // an odd tail computes its last row twice and stores it once
+        float qp[8], qn[8];
+        *reinterpret_cast<float4*>(&qp[0]) = *reinterpret_cast<const float4*>(&qpos[rs * D + sub * 4]);
+        *reinterpret_cast<float4*>(&qp[4]) = *reinterpret_cast<const float4*>(&qpos[rs * D + D / 2 + sub * 4]);
+        *reinterpret_cast<float4*>(&qn[0]) = *reinterpret_cast<const float4*>(&qneg[rs * D + sub * 4]);
+        *reinterpret_cast<float4*>(&qn[4]) = *reinterpret_cast<const float4*>(&qneg[rs * D + D / 2 + sub * 4]);
+        float acc[ITER];
+#pragma unroll
+        for (int it = 0; it < ITER; ++it) acc[it] = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+#pragma unroll
+          for (int it = 0; it < ITER; ++it) {
+            acc[it] = __fmaf_rn(qp[j], hi[it][j], acc[it]);
+            acc[it] = __fmaf_rn(qn[j], lo[it][j], acc[it]);
+          }
+        }
+#pragma unroll
+        for (int it = 0; it < ITER; ++it) v[it * 2 + rr] = acc[it];
       }
+      {
+        int n = NV;
+#pragma unroll
+        for (int off = LPP / 2; off >= 2; off >>= 1) {
+          n >>= 1;
+          const bool up = (sub & off) != 0;
+#pragma unroll
+          for (int k = 0; k < NV / 2; ++k) {
+            if (k < n) {
+              const float send = up ? v[k] : v[k + n];
+              const float keep = up ? v[k + n] : v[k];
+              v[k] = __fadd_rn(keep, __shfl_xor_sync(0xffffffffu, send, off));
+            }
+          }
+        }
+        v[0] = __fadd_rn(v[0], __shfl_xor_sync(0xffffffffu, v[0], 1));
+      }
+      const int i = sub >> 1, it = i >> 1, rr = i & 1, pl = grp * ITER + it;
+      if ((sub & 1) == 0 && pl < np && r + rr < nr) {
+        int a2 = a, g2 = gi + rr;
+        if (g2 >= G) { g2 -= G; ++a2; }
+        scores[((static_cast<size_t>(s) * B + a2) * Hq + kh * G + g2) * score_stride + p0 + pl] = __fadd_rn(v[0], 0.0f);
+      }
+      gi += 2;
+      while (gi >= G) { gi -= G; ++a; }
     }
     __syncthreads();
   }
