@@ -25,6 +25,7 @@ block_attn_merge_kernel(const T* __restrict__ q, const T* __restrict__ k_blk, co
                         const float* __restrict__ o_p, const float* __restrict__ lse_p,
                         T* __restrict__ out, float* __restrict__ lse_out, float* __restrict__ ob_out,
                         int B, int Hq, int Hkv, float sm_scale) {
+  grid_dep_wait();
   extern __shared__ __align__(16) float smem[];
   float* Ks = smem;                 // [B][D]
   float* Vs = Ks + B * D;           // [B][D]
@@ -132,6 +133,7 @@ merge_commit_kernel(const T* __restrict__ q, T* __restrict__ q_prev, const float
                     const float* __restrict__ lse_p, const float* __restrict__ o_b,
                     const float* __restrict__ lse_b, T* __restrict__ out, float* __restrict__ lse_out,
                     int32_t* __restrict__ step, int N, size_t n_rows) {
+  grid_dep_wait();
   const int lane = threadIdx.x & 31;
   const size_t row = static_cast<size_t>(blockIdx.x) * (kThreads / 32) + (threadIdx.x >> 5);
   if (blockIdx.x == 0)
@@ -162,6 +164,7 @@ template <typename T>
 __global__ void __launch_bounds__(kThreads)
 commit_step_kernel(const uint4* __restrict__ q, uint4* __restrict__ q_prev, size_t n_vec,
                    int32_t* __restrict__ step, int N) {
+  grid_dep_wait();
   for (size_t i = blockIdx.x * static_cast<size_t>(kThreads) + threadIdx.x; i < n_vec;
        i += static_cast<size_t>(gridDim.x) * kThreads)
     q_prev[i] = q[i];
@@ -196,6 +199,7 @@ __global__ void build_summaries_kernel(const T* __restrict__ k_pages, T* __restr
                                        const int32_t* __restrict__ kv_len, int64_t stride_page,
                                        int64_t stride_head, int64_t stride_tok, int Hkv, int D, int g,
                                        int Pmax, int n_phys, int32_t* __restrict__ status) {
+  grid_dep_wait();
   const int p = blockIdx.x, kh = blockIdx.y, s = blockIdx.z, j = threadIdx.x;
   const int len = kv_len[s];
   const int valid = min(g, len - p * g);
@@ -218,6 +222,7 @@ __global__ void append_block_kernel(T* __restrict__ k_pages, T* __restrict__ v_p
                                     const int32_t* __restrict__ kv_len, int64_t stride_page,
                                     int64_t stride_head, int64_t stride_tok, int B, int Hkv, int D,
                                     int g, int Pmax, int n_phys, int32_t* __restrict__ status) {
+  grid_dep_wait();
   const int kh = blockIdx.y, s = blockIdx.z, j = threadIdx.x;
   const int L0 = kv_len[s];
   const int p = L0 / g + blockIdx.x;
@@ -240,6 +245,7 @@ __global__ void append_block_kernel(T* __restrict__ k_pages, T* __restrict__ v_p
 }
 
 __global__ void finalize_counters_kernel(int32_t* __restrict__ kv_len, int32_t* __restrict__ step, int N, int B) {
+  grid_dep_wait();
   const int s = threadIdx.x;
   if (s < N) { kv_len[s] += B; step[s] = 0; }
 }
@@ -252,7 +258,7 @@ int32_t launch_merge_t(losa_ctx* c, const void* q, const void* k_blk, const void
   if (smem > 48 * 1024)
     LOSA_CUDA_TRY(c, cudaFuncSetAttribute(block_attn_merge_kernel<T, D, MERGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   dim3 grid((sh.block_size + kTokTile - 1) / kTokTile, sh.n_kv_heads, sh.batch);
-  block_attn_merge_kernel<T, D, MERGE><<<grid, kThreads, smem, st>>>(
+  launch_k(block_attn_merge_kernel<T, D, MERGE>, grid, kThreads, smem, st, 
       static_cast<const T*>(q), static_cast<const T*>(k_blk), static_cast<const T*>(v_blk),
       state ? state->o_p : nullptr, state ? state->lse_p : nullptr, static_cast<T*>(out), lse_out, ob_out,
       sh.block_size, sh.n_q_heads, sh.n_kv_heads, sh.sm_scale);
@@ -265,7 +271,7 @@ int32_t launch_merge_commit_t(losa_ctx* c, const void* q, losa_state_t* state, v
   const losa_shape_t& sh = c->shape;
   const size_t n_rows = static_cast<size_t>(sh.batch) * sh.block_size * sh.n_q_heads;
   const int blocks = static_cast<int>((n_rows + kThreads / 32 - 1) / (kThreads / 32));
-  merge_commit_kernel<T, D><<<blocks, kThreads, 0, st>>>(
+  launch_k(merge_commit_kernel<T, D>, blocks, kThreads, 0, st, 
       static_cast<const T*>(q), static_cast<T*>(state->q_prev), state->o_p, state->lse_p,
       reinterpret_cast<const float*>(c->ws + c->lay.block_o), reinterpret_cast<const float*>(c->ws + c->lay.block_lse),
       static_cast<T*>(out), lse_out, state->step, sh.batch, n_rows);
@@ -279,19 +285,19 @@ int32_t launch_update_t(losa_ctx* c, losa_kv_t* kv, losa_state_t* state, const v
   if (!finalize_block) {
     const size_t n_vec = static_cast<size_t>(sh.batch) * sh.block_size * sh.n_q_heads * sh.head_dim * sizeof(T) / 16;
     const int blocks = static_cast<int>(std::min<size_t>((n_vec + kThreads - 1) / kThreads, static_cast<size_t>(c->n_sms) * 4));
-    commit_step_kernel<T><<<std::max(blocks, 1), kThreads, 0, st>>>(
+    launch_k(commit_step_kernel<T>, std::max(blocks, 1), kThreads, 0, st, 
         static_cast<const uint4*>(q), static_cast<uint4*>(state->q_prev), n_vec, state->step, sh.batch);
     return after_launch(c);
   }
   dim3 grid((sh.block_size + sh.page_size - 1) / sh.page_size + 1, sh.n_kv_heads, sh.batch);
-  append_block_kernel<T><<<grid, sh.head_dim, 0, st>>>(
+  launch_k(append_block_kernel<T>, grid, sh.head_dim, 0, st, 
       static_cast<T*>(kv->k_pages), static_cast<T*>(kv->v_pages), static_cast<T*>(kv->kmin),
       static_cast<T*>(kv->kmax), static_cast<const T*>(k_blk), static_cast<const T*>(v_blk),
       kv->page_table, kv->kv_len, kv->stride_page, kv->stride_head, kv->stride_tok, sh.block_size,
       sh.n_kv_heads, sh.head_dim, sh.page_size, sh.max_pages_per_seq, kv->n_phys_pages, status_ptr(c));
   int32_t rc = after_launch(c);
   if (rc != LOSA_OK) return rc;
-  finalize_counters_kernel<<<1, std::max(32, sh.batch), 0, st>>>(kv->kv_len, state->step, sh.batch, sh.block_size);
+  launch_k(finalize_counters_kernel, 1, std::max(32, sh.batch), 0, st, kv->kv_len, state->step, sh.batch, sh.block_size);
   return after_launch(c);
 }
 
@@ -300,7 +306,7 @@ int32_t launch_summaries_t(losa_ctx* c, losa_kv_t* kv, cudaStream_t st) {
   const losa_shape_t& sh = c->shape;
   if (sh.max_pages_per_seq == 0) return LOSA_OK;
   dim3 grid(sh.max_pages_per_seq, sh.n_kv_heads, sh.batch);
-  build_summaries_kernel<T><<<grid, sh.head_dim, 0, st>>>(
+  launch_k(build_summaries_kernel<T>, grid, sh.head_dim, 0, st, 
       static_cast<const T*>(kv->k_pages), static_cast<T*>(kv->kmin), static_cast<T*>(kv->kmax),
       kv->page_table, kv->kv_len, kv->stride_page, kv->stride_head, kv->stride_tok, sh.n_kv_heads,
       sh.head_dim, sh.page_size, sh.max_pages_per_seq, kv->n_phys_pages, status_ptr(c));

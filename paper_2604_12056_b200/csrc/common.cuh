@@ -85,6 +85,26 @@ inline int32_t after_launch(losa_ctx* c, int n = 1) {
 // ----------------------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
 
+// Every kernel of the library is launched with programmatic stream serialisation: its CTAs may be
+// scheduled while the previous kernel of the stream is still draining, and it calls grid_dep_wait()
+// before its first access to global memory, which returns once that kernel has completed and its
+// writes are visible.  Launch latency and the tail of one kernel overlap the start of the next.
+template <typename... KArgs, typename... Args>
+inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);   // the error, if any, is read by after_launch()
+}
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void set_status(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }
 
 __device__ __forceinline__ float to_f32(float x) { return x; }

@@ -57,6 +57,7 @@ page_scores_kernel(const T* __restrict__ q, const T* __restrict__ kmin, const T*
                    const int32_t* __restrict__ active_idx, const int32_t* __restrict__ n_active,
                    const int32_t* __restrict__ step, float* __restrict__ scores, int B, int Hq, int Hkv,
                    int g, int Pmax, int n_phys, int score_stride, int32_t* __restrict__ status) {
+  grid_dep_wait();
   constexpr int LPP = D / 8;            // lanes per page
   constexpr int GROUPS = kThreads / LPP;
   const int s = blockIdx.z, kh = blockIdx.y, p0 = blockIdx.x * kPagesPerCta;
@@ -235,6 +236,7 @@ topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ kv_len
             const int32_t* __restrict__ step, int32_t* __restrict__ topk_pages,
             float* __restrict__ topk_scores, int B, int Hq, int g, int k, int score_stride,
             int32_t* __restrict__ status) {
+  grid_dep_wait();
   extern __shared__ __align__(16) unsigned long long keys[];
   const int h = blockIdx.x, a = blockIdx.y, s = blockIdx.z;
   if (step && step[s] == 0) return;
@@ -443,6 +445,7 @@ topk_select_kernel(const float* __restrict__ scores, const int32_t* __restrict__
                    const int32_t* __restrict__ step, int32_t* __restrict__ topk_pages,
                    float* __restrict__ topk_scores, int N, int B, int Hq, int g, int k, int score_stride,
                    int32_t* __restrict__ status) {
+  grid_dep_wait();
   // queries of the same active slot are adjacent, so the CTAs that have work are the first ones
   const int qid = blockIdx.x;
   const int h = qid % Hq, s = (qid / Hq) % N, a = qid / (Hq * N);
@@ -468,6 +471,7 @@ union_kernel(const int32_t* __restrict__ topk_pages, const int32_t* __restrict__
              const int32_t* __restrict__ step, int32_t* __restrict__ union_pages,
              int32_t* __restrict__ union_count, int B, int Hq, int Hkv, int g, int k, int Pmax,
              int32_t* __restrict__ status) {
+  grid_dep_wait();
   extern __shared__ uint32_t bitmap[];
   __shared__ int s_warp[kThreads / 32];
   const int kh = blockIdx.x, s = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -537,7 +541,7 @@ void launch_scores(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_
                    const int32_t* n_active, const int32_t* step, cudaStream_t st) {
   const losa_shape_t& sh = c->shape;
   dim3 grid((sh.max_pages_per_seq + kPagesPerCta - 1) / kPagesPerCta, sh.n_kv_heads, sh.batch);
-  page_scores_kernel<T, D><<<grid, kThreads, 0, st>>>(
+  launch_k(page_scores_kernel<T, D>, grid, kThreads, 0, st, 
       static_cast<const T*>(q), static_cast<const T*>(kv->kmin), static_cast<const T*>(kv->kmax),
       kv->page_table, kv->kv_len, active_idx, n_active, step,
       reinterpret_cast<float*>(c->ws + c->lay.scores), sh.block_size, sh.n_q_heads, sh.n_kv_heads,
@@ -575,7 +579,7 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
   const float* sc = reinterpret_cast<const float*>(c->ws + c->lay.scores);
   if (k <= kSelCap) {
     const int queries = sh.batch * sh.block_size * sh.n_q_heads;
-    topk_select_kernel<<<queries, kSelThreads, 0, st>>>(
+    launch_k(topk_select_kernel, queries, kSelThreads, 0, st, 
         sc, kv->kv_len, active_idx, n_active, step, topk_pages, topk_scores_opt, sh.batch, sh.block_size,
         sh.n_q_heads, sh.page_size, k, c->lay.score_stride, status_ptr(c));
     return after_launch(c);
@@ -585,7 +589,7 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
   if (smem > 48 * 1024)
     LOSA_CUDA_TRY(c, cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   dim3 grid(sh.n_q_heads, sh.block_size, sh.batch);
-  topk_kernel<<<grid, kThreads, smem, st>>>(sc, kv->kv_len, active_idx, n_active, step, topk_pages,
+  launch_k(topk_kernel, grid, kThreads, smem, st, sc, kv->kv_len, active_idx, n_active, step, topk_pages,
                                             topk_scores_opt, sh.block_size, sh.n_q_heads, sh.page_size,
                                             k, c->lay.score_stride, status_ptr(c));
   return after_launch(c);
@@ -598,7 +602,7 @@ int32_t launch_page_union(losa_ctx* c, const int32_t* topk_pages, const int32_t*
   const losa_shape_t& sh = c->shape;
   const size_t smem = static_cast<size_t>((sh.max_pages_per_seq + 31) / 32 + 1) * sizeof(uint32_t);
   dim3 grid(sh.n_kv_heads, sh.batch);
-  union_kernel<<<grid, kThreads, smem, st>>>(topk_pages, active_idx, n_active, kv_len, step, union_pages,
+  launch_k(union_kernel, grid, kThreads, smem, st, topk_pages, active_idx, n_active, kv_len, step, union_pages,
                                              union_count, sh.block_size, sh.n_q_heads, sh.n_kv_heads,
                                              sh.page_size, k, sh.max_pages_per_seq, status_ptr(c));
   return after_launch(c);

@@ -21,6 +21,7 @@ select_active_kernel(const T* __restrict__ x_cur, const T* __restrict__ x_prev, 
                      int32_t* __restrict__ active_idx, int32_t* __restrict__ n_active,
                      float* __restrict__ delta_opt, double* __restrict__ delta_ws,
                      unsigned int* __restrict__ counters) {
+  grid_dep_wait();
   const int i = blockIdx.x, s = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const size_t row = (static_cast<size_t>(s) * B + i) * row_width;
@@ -100,11 +101,11 @@ int32_t launch_select_active(losa_ctx* c, const void* x_cur, const void* x_prev,
   double* dws = reinterpret_cast<double*>(c->ws + c->lay.delta);
   unsigned int* ctr = reinterpret_cast<unsigned int*>(c->ws + c->lay.counters);
   if (sh.dtype == LOSA_BF16) {
-    select_active_kernel<__nv_bfloat16><<<grid, kThreads, 0, st>>>(
+    launch_k(select_active_kernel<__nv_bfloat16>, grid, kThreads, 0, st, 
         static_cast<const __nv_bfloat16*>(x_cur), static_cast<const __nv_bfloat16*>(x_prev), row_width,
         sh.block_size, m_per_seq, step, active_idx, n_active, delta_opt, dws, ctr);
   } else {
-    select_active_kernel<float><<<grid, kThreads, 0, st>>>(
+    launch_k(select_active_kernel<float>, grid, kThreads, 0, st, 
         static_cast<const float*>(x_cur), static_cast<const float*>(x_prev), row_width, sh.block_size,
         m_per_seq, step, active_idx, n_active, delta_opt, dws, ctr);
   }
@@ -170,11 +171,11 @@ extern "C" int32_t losa_select_active_static(const losa_shape_t* shape, const vo
   if (cudaMemsetAsync(scratch->counters, 0, sizeof(unsigned int) * shape->batch, st) != cudaSuccess) return LOSA_ERR_CUDA;
   dim3 grid(shape->block_size, shape->batch);
   if (shape->dtype == LOSA_BF16) {
-    losa::select_active_kernel<__nv_bfloat16><<<grid, losa::kThreads, 0, st>>>(
+    losa::launch_k(losa::select_active_kernel<__nv_bfloat16>, grid, losa::kThreads, 0, st, 
         static_cast<const __nv_bfloat16*>(x_cur), static_cast<const __nv_bfloat16*>(x_prev), row_width,
         shape->block_size, m_per_seq, step, active_idx, n_active, delta_opt, scratch->delta, scratch->counters);
   } else {
-    losa::select_active_kernel<float><<<grid, losa::kThreads, 0, st>>>(
+    losa::launch_k(losa::select_active_kernel<float>, grid, losa::kThreads, 0, st, 
         static_cast<const float*>(x_cur), static_cast<const float*>(x_prev), row_width, shape->block_size,
         m_per_seq, step, active_idx, n_active, delta_opt, scratch->delta, scratch->counters);
   }

@@ -70,6 +70,7 @@ __device__ __forceinline__ int clamp_active(int na, int B) { return na < 0 ? 0 :
 // ===================================================================== fp32 / CUDA-core kernel
 template <typename T, int D, int GP>
 __global__ void __launch_bounds__(256, 1) attn_simt_kernel(AttnParams p) {
+  grid_dep_wait();
   extern __shared__ __align__(16) float sm[];
   float* Ks = sm;                         // [GP][D]
   float* Vs = Ks + GP * D;                // [GP][D]
@@ -198,6 +199,7 @@ __global__ void __launch_bounds__(256, 1) attn_simt_kernel(AttnParams p) {
 // natural units (fp32 kernel).
 template <int D, bool LOG2>
 __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
+  grid_dep_wait();
   __shared__ int pre[kMaxSegments + 1];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sg = blockIdx.x, r = blockIdx.y * 8 + warp;
@@ -406,11 +408,11 @@ int32_t launch_tc5(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
   memcpy(&mk, c->tmap_k, sizeof(mk));
   memcpy(&mv, c->tmap_v, sizeof(mv));
   if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_begin, st));
-  attn_tc5_kernel<D, GP><<<ap.n_ctas, kTc5Threads, smem, st>>>(mk, mv, ap);
+  launch_k(attn_tc5_kernel<D, GP>, ap.n_ctas, kTc5Threads, smem, st, mk, mv, ap);
   if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_end, st));
   int32_t rc = after_launch(c);
   if (rc != LOSA_OK) return rc;
-  attn_combine_kernel<D, true><<<dim3(ap.n_seg, kRowsPerGroup / 8), 256, 0, st>>>(ap);
+  launch_k(attn_combine_kernel<D, true>, dim3(ap.n_seg, kRowsPerGroup / 8), 256, 0, st, ap);
   return after_launch(c);
 }
 
@@ -420,11 +422,11 @@ int32_t launch_simt(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
                       (ap.n_seg + 1) * sizeof(int);
   LOSA_CUDA_TRY(c, cudaFuncSetAttribute(attn_simt_kernel<T, D, GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_begin, st));
-  attn_simt_kernel<T, D, GP><<<ap.n_ctas, 256, smem, st>>>(ap);
+  launch_k(attn_simt_kernel<T, D, GP>, ap.n_ctas, 256, smem, st, ap);
   if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_end, st));
   int32_t rc = after_launch(c);
   if (rc != LOSA_OK) return rc;
-  attn_combine_kernel<D, false><<<dim3(ap.n_seg, kRowsPerGroup / 8), 256, 0, st>>>(ap);
+  launch_k(attn_combine_kernel<D, false>, dim3(ap.n_seg, kRowsPerGroup / 8), 256, 0, st, ap);
   return after_launch(c);
 }
 
