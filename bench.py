@@ -36,11 +36,13 @@ METRIC = "denoise-step attention us/layer"
 UNIT = "us/layer-step"
 L2_FLUSH_BYTES = 256 << 20
 # DRAM traffic of the stage-4 main kernel per listed (page, KV head) slice, from the ncu capture in
-# profiles/attn_mma_kernel_c3.txt (dram__bytes_read.sum + dram__bytes_write.sum over the slices of that
-# launch: 167.91 MB / 9,916 slices on a LoSA step, 445.42 MB / 26,624 on a dense step; 16,384 of
-# these bytes are the slice's K and V).  Traffic grows in proportion to the slices, so a launch's
-# traffic is reported as slices x this figure (pages of 32 tokens, head dim 128, bf16 only).
-NCU_BYTES_PER_SLICE = {"losa": 167.91e6 / 9916, "dense": 445.42e6 / 26624}
+# profiles/attn_tc5_kernel_c5.txt: the dense launch there moved dram__bytes_read.sum +
+# dram__bytes_write.sum = 1,087.26 MB for its 65,984 slices (16,384 of the 16,478 bytes per slice are
+# the slice's K and V).  Traffic grows in proportion to the slices, so a launch's traffic is reported
+# as slices x this figure; LoSA launches add the partial records they write (3.7-4.8 MB of DRAM
+# writes in the three LoSA launches of that capture).  Pages of 32 tokens, head dim 128, bf16 only.
+NCU_BYTES_PER_SLICE = {"losa": 1087.26e6 / 65984, "dense": 1087.26e6 / 65984}
+NCU_FIXED_BYTES = {"losa": 4.8e6, "dense": 0.0}
 
 
 def parse_args():
@@ -403,7 +405,7 @@ def run_ours(args, cfg0):
         return {"bound": "hbm", "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
                 "frac_of_8TBps_nominal": ach / 8000.0, "launches": n, "bytes_per_launch": b / n,
                 "us_per_launch": t / n * 1e3,
-                "traffic": (sum(NCU_BYTES_PER_SLICE[k] * sl for k, sl in zip(kinds, k_slices) if k in sel) / n) if scalable else None,
+                "traffic": (sum(NCU_BYTES_PER_SLICE[k] * sl + NCU_FIXED_BYTES[k] for k, sl in zip(kinds, k_slices) if k in sel) / n) if scalable else None,
                 "peak_source": "measured (MEASURED_PEAKS.json hbm_gbs)" if peaks else "fallback 6650 GB/s"}
     result["roofline"] = roof(("losa", "dense")) or {}
     result["roofline"]["kernel"] = "stage-4 main kernel (paged prefix attention), every launch of whole blocks"
