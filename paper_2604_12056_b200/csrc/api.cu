@@ -239,7 +239,10 @@ int32_t losa_denoise_step(losa_ctx* ctx, const void* q, const void* k_blk, const
       !aligned16(state->o_p))
     return LOSA_ERR_UNSUPPORTED;
   if (!ctx->side_stream) {
-    LOSA_CUDA_TRY(ctx, cudaStreamCreateWithFlags(&ctx->side_stream, cudaStreamNonBlocking));
+    // lowest priority: when CTAs of both streams are pending, those of stages 1-4 go first
+    int prio_lo = 0, prio_hi = 0;
+    LOSA_CUDA_TRY(ctx, cudaDeviceGetStreamPriorityRange(&prio_lo, &prio_hi));
+    LOSA_CUDA_TRY(ctx, cudaStreamCreateWithPriority(&ctx->side_stream, cudaStreamNonBlocking, prio_lo));
     LOSA_CUDA_TRY(ctx, cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming));
     LOSA_CUDA_TRY(ctx, cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming));
   }

@@ -9,118 +9,146 @@ namespace losa {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kTokTile = 2;
+constexpr int kTokTile = 4;        // block tokens per CTA of the in-block attention
+constexpr int kBaThreads = 128;
+constexpr int kBaRows = 4;         // query rows a warp works on together
 
-// One CTA per (pair of block tokens, KV head, sequence): K_b, V_b of the KV head staged in shared
-// memory as fp32; one warp per query row (the G heads of the two tokens).  Everything a row needs
-// from global memory (its query, cached L_p and o_p) is requested before the arithmetic starts, so
-// the kernel pays one memory latency, not one per operand.  Scores: lane = block key, columns
-// visited in a rotated order so that the 32 lanes hit 32 banks, four independent partial sums;
-// P V: lane = output column.
+// One CTA per (four block tokens, KV head, sequence): K_b, V_b of the KV head and the CTA's query
+// rows staged in shared memory as fp32.  A warp takes four query rows at a time (with G = 4 the
+// heads of one token), so every K_b / V_b element read from shared memory feeds four multiply-adds:
+// the kernel is bound by shared-memory reads, and this is what keeps it short enough to hide beside
+// stages 1-3.  Scores: lane = block key (rows of K_b padded by four floats: conflict-free 16-byte
+// reads), the four query rows read as broadcasts; P V: lane = output column, probabilities by shuffle.
 // MERGE = false (whole-step path): only the in-block part, normalised o_b to `ob_out` and L_b to
 // `lse_out`; the prefix statistics are not touched, so this can run beside stages 1-4.
 template <typename T, int D, bool MERGE>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kBaThreads)
 block_attn_merge_kernel(const T* __restrict__ q, const T* __restrict__ k_blk, const T* __restrict__ v_blk,
                         const float* __restrict__ o_p, const float* __restrict__ lse_p,
                         T* __restrict__ out, float* __restrict__ lse_out, float* __restrict__ ob_out,
                         int B, int Hq, int Hkv, float sm_scale) {
   grid_dep_wait();
+  constexpr int KS = D + 4;         // padded row of K_b
+  constexpr int C = D / 32;
+  constexpr int U = 2;              // block keys per lane (B <= 64)
   extern __shared__ __align__(16) float smem[];
-  float* Ks = smem;                 // [B][D]
-  float* Vs = Ks + B * D;           // [B][D]
-  float* Qs = Vs + B * D;           // [warps][D]
+  float* Ks = smem;                 // [B][D + 4]
+  float* Vs = Ks + B * KS;          // [B][D]
+  float* Qs = Vs + B * D;           // [kTokTile * G][D]
   const int t0 = blockIdx.x * kTokTile, kh = blockIdx.y, s = blockIdx.z;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = Hq / Hkv;
-  const int ntok = min(kTokTile, B - t0);
-  constexpr int C = D / 32;
-  // this warp's first row: issue its loads before staging K_b / V_b
-  int r = warp;
-  bool have = r < ntok * G;
-  size_t row = 0;
-  float qv[C], opv[C], Lp = 0.f;
-  auto fetch = [&]() {
-    row = (static_cast<size_t>(s) * B + t0 + r / G) * Hq + kh * G + r % G;
-#pragma unroll
-    for (int c = 0; c < C; ++c) {
-      qv[c] = to_f32(q[row * D + lane + 32 * c]);
-      opv[c] = MERGE ? o_p[row * D + lane + 32 * c] : 0.f;
-    }
-    Lp = MERGE ? lse_p[row] : 0.f;
-  };
-  if (have) fetch();
-  for (int idx = tid * 8; idx < B * D; idx += kThreads * 8) {
+  const int nrow = min(kTokTile, B - t0) * G;
+  auto row_of = [&](int r) { return (static_cast<size_t>(s) * B + t0 + r / G) * Hq + kh * G + r % G; };
+  for (int idx = tid * 8; idx < nrow * D; idx += kBaThreads * 8) {
+    float a[8];
+    load8(q + row_of(idx / D) * D + idx % D, a);
+    *reinterpret_cast<float4*>(Qs + idx) = make_float4(a[0], a[1], a[2], a[3]);
+    *reinterpret_cast<float4*>(Qs + idx + 4) = make_float4(a[4], a[5], a[6], a[7]);
+  }
+  for (int idx = tid * 8; idx < B * D; idx += kBaThreads * 8) {
     const int t = idx / D, j = idx % D;
     const size_t src = ((static_cast<size_t>(s) * B + t) * Hkv + kh) * D + j;
     float a[8], b[8];
     load8(k_blk + src, a);
     load8(v_blk + src, b);
-    *reinterpret_cast<float4*>(Ks + idx) = make_float4(a[0], a[1], a[2], a[3]);
-    *reinterpret_cast<float4*>(Ks + idx + 4) = make_float4(a[4], a[5], a[6], a[7]);
+    *reinterpret_cast<float4*>(Ks + t * KS + j) = make_float4(a[0], a[1], a[2], a[3]);
+    *reinterpret_cast<float4*>(Ks + t * KS + j + 4) = make_float4(a[4], a[5], a[6], a[7]);
     *reinterpret_cast<float4*>(Vs + idx) = make_float4(b[0], b[1], b[2], b[3]);
     *reinterpret_cast<float4*>(Vs + idx + 4) = make_float4(b[4], b[5], b[6], b[7]);
   }
   __syncthreads();
-  float* qw = Qs + warp * D;
-  while (have) {
-    __syncwarp();
+  for (int r0 = warp * kBaRows; r0 < nrow; r0 += (kBaThreads / 32) * kBaRows) {
+    const int nr = min(kBaRows, nrow - r0);
+    // prefix statistics of the rows (MERGE): requested now, used after the arithmetic
+    float opv[kBaRows][C], Lp[kBaRows];
 #pragma unroll
-    for (int c = 0; c < C; ++c) qw[lane + 32 * c] = qv[c];
-    __syncwarp();
-    float sc[2];
+    for (int r = 0; r < kBaRows; ++r) {
+      const size_t row = row_of(r0 + min(r, nr - 1));
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
-      const int t = lane + 32 * u;
-      float d0 = 0.f, d1 = 0.f, d2 = 0.f, d3 = 0.f;
-      if (t < B) {
-        const float* kr = Ks + t * D;
+      for (int c = 0; c < C; ++c) opv[r][c] = MERGE ? o_p[row * D + lane + 32 * c] : 0.f;
+      Lp[r] = MERGE ? lse_p[row] : 0.f;
+    }
+    // ---- scores: lane = block key (two keys per lane when B > 32)
+    float sc[U][kBaRows];
+#pragma unroll
+    for (int u = 0; u < U; ++u)
+#pragma unroll
+      for (int r = 0; r < kBaRows; ++r) sc[u][r] = 0.f;
+    const float* qr = Qs + r0 * D;
 #pragma unroll 4
-        for (int j = 0; j < D; j += 4) {
-          const int j0 = (j + lane) & (D - 1), j1 = (j + 1 + lane) & (D - 1);
-          const int j2 = (j + 2 + lane) & (D - 1), j3 = (j + 3 + lane) & (D - 1);
-          d0 = fmaf(qw[j0], kr[j0], d0);
-          d1 = fmaf(qw[j1], kr[j1], d1);
-          d2 = fmaf(qw[j2], kr[j2], d2);
-          d3 = fmaf(qw[j3], kr[j3], d3);
+    for (int j = 0; j < D; j += 4) {
+      float4 kv[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int t = lane + 32 * u;
+        kv[u] = (t < B) ? *reinterpret_cast<const float4*>(Ks + t * KS + j) : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+#pragma unroll
+      for (int r = 0; r < kBaRows; ++r) {
+        const float4 qv = *reinterpret_cast<const float4*>(qr + min(r, nr - 1) * D + j);
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+          sc[u][r] = fmaf(qv.w, kv[u].w, fmaf(qv.z, kv[u].z, fmaf(qv.y, kv[u].y, fmaf(qv.x, kv[u].x, sc[u][r]))));
+      }
+    }
+    // ---- softmax over the block keys, per row
+    float p[U][kBaRows], sum[kBaRows], Lb[kBaRows];
+#pragma unroll
+    for (int r = 0; r < kBaRows; ++r) {
+      float mx = -INFINITY;
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        sc[u][r] = (lane + 32 * u < B) ? sc[u][r] * sm_scale : -INFINITY;
+        mx = fmaxf(mx, sc[u][r]);
+      }
+      const float M = warp_max(mx);
+      float ps = 0.f;
+#pragma unroll
+      for (int u = 0; u < U; ++u) { p[u][r] = expf(sc[u][r] - M); ps += p[u][r]; }
+      sum[r] = warp_sum(ps);
+      Lb[r] = M + logf(sum[r]);
+    }
+    // ---- P V: lane = output column
+    float ob[kBaRows][C];
+#pragma unroll
+    for (int r = 0; r < kBaRows; ++r)
+#pragma unroll
+      for (int c = 0; c < C; ++c) ob[r][c] = 0.f;
+#pragma unroll 2
+    for (int t = 0; t < B; ++t) {
+      float v[C];
+#pragma unroll
+      for (int c = 0; c < C; ++c) v[c] = Vs[t * D + lane + 32 * c];
+#pragma unroll
+      for (int r = 0; r < kBaRows; ++r) {
+        const float pt = __shfl_sync(0xffffffffu, t < 32 ? p[0][r] : p[1][r], t & 31);
+#pragma unroll
+        for (int c = 0; c < C; ++c) ob[r][c] = fmaf(pt, v[c], ob[r][c]);
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < kBaRows; ++r) {
+      if (r < nr) {
+        const size_t row = row_of(r0 + r);
+        if (MERGE) {
+          const float M2 = fmaxf(Lp[r], Lb[r]);
+          const float L = M2 + logf(expf(Lp[r] - M2) + expf(Lb[r] - M2));
+          const float wp = expf(Lp[r] - L), wb = expf(Lb[r] - L) / sum[r];
+#pragma unroll
+          for (int c = 0; c < C; ++c) {
+            const float v = (wp > 0.f ? wp * opv[r][c] : 0.f) + wb * ob[r][c];
+            out[row * D + lane + 32 * c] = from_f32<T>(v);
+          }
+          if (lse_out && lane == 0) lse_out[row] = L;
+        } else {
+          const float inv = 1.f / sum[r];
+#pragma unroll
+          for (int c = 0; c < C; ++c) ob_out[row * D + lane + 32 * c] = ob[r][c] * inv;
+          if (lane == 0) lse_out[row] = Lb[r];
         }
       }
-      sc[u] = (t < B) ? ((d0 + d1) + (d2 + d3)) * sm_scale : -INFINITY;
     }
-    const float M = warp_max(fmaxf(sc[0], sc[1]));
-    float p[2];
-    p[0] = expf(sc[0] - M);
-    p[1] = expf(sc[1] - M);
-    const float sum = warp_sum(p[0] + p[1]);
-    const float Lb = M + logf(sum);
-    float ob[C];
-#pragma unroll
-    for (int c = 0; c < C; ++c) ob[c] = 0.f;
-#pragma unroll 4
-    for (int t = 0; t < B; ++t) {
-      const float pt = __shfl_sync(0xffffffffu, t < 32 ? p[0] : p[1], t & 31);
-#pragma unroll
-      for (int c = 0; c < C; ++c) ob[c] = fmaf(pt, Vs[t * D + lane + 32 * c], ob[c]);
-    }
-    if (MERGE) {
-      const float M2 = fmaxf(Lp, Lb);
-      const float L = M2 + logf(expf(Lp - M2) + expf(Lb - M2));
-      const float wp = expf(Lp - L), wb = expf(Lb - L) / sum;
-#pragma unroll
-      for (int c = 0; c < C; ++c) {
-        const float v = (wp > 0.f ? wp * opv[c] : 0.f) + wb * ob[c];
-        out[row * D + lane + 32 * c] = from_f32<T>(v);
-      }
-      if (lse_out && lane == 0) lse_out[row] = L;
-    } else {
-      const float inv = 1.f / sum;
-#pragma unroll
-      for (int c = 0; c < C; ++c) ob_out[row * D + lane + 32 * c] = ob[c] * inv;
-      if (lane == 0) lse_out[row] = Lb;
-    }
-    r += kThreads / 32;
-    have = r < ntok * G;
-    if (have) fetch();
   }
 }
 
@@ -254,11 +282,12 @@ template <typename T, int D, bool MERGE>
 int32_t launch_merge_t(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk,
                        const losa_state_t* state, void* out, float* lse_out, float* ob_out, cudaStream_t st) {
   const losa_shape_t& sh = c->shape;
-  const size_t smem = (static_cast<size_t>(2) * sh.block_size * D + (kThreads / 32) * D) * sizeof(float);
+  const int G = sh.n_q_heads / sh.n_kv_heads;
+  const size_t smem = (static_cast<size_t>(sh.block_size) * (2 * D + 4) + static_cast<size_t>(kTokTile) * G * D) * sizeof(float);
   if (smem > 48 * 1024)
     LOSA_CUDA_TRY(c, cudaFuncSetAttribute(block_attn_merge_kernel<T, D, MERGE>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   dim3 grid((sh.block_size + kTokTile - 1) / kTokTile, sh.n_kv_heads, sh.batch);
-  launch_k(block_attn_merge_kernel<T, D, MERGE>, grid, kThreads, smem, st, 
+  launch_k(block_attn_merge_kernel<T, D, MERGE>, grid, kBaThreads, smem, st, 
       static_cast<const T*>(q), static_cast<const T*>(k_blk), static_cast<const T*>(v_blk),
       state ? state->o_p : nullptr, state ? state->lse_p : nullptr, static_cast<T*>(out), lse_out, ob_out,
       sh.block_size, sh.n_q_heads, sh.n_kv_heads, sh.sm_scale);

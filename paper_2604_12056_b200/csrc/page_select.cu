@@ -3,10 +3,11 @@
 //
 //   page_scores_kernel : each CTA reads the min/max keys of 64 pages of one (sequence, KV head)
 //                        once and scores them against every active query of that KV head.  A page
-//                        is handled by d/8 lanes: one 16-byte vector of kmin and kmax per lane,
-//                        a chain of 16 fused multiply-adds per lane (q+ kmax, q- kmin), then an
-//                        xor-butterfly over the lanes — exactly the order the interface fixes, so
-//                        the fp32 result is reproducible bit for bit.
+//                        is handled by d/8 lanes: one 16-byte vector of kmin and kmax per lane
+//                        (four pages per lane), a chain of 16 fused multiply-adds per lane and
+//                        page (q+ kmax, q- kmin), then the butterfly over the lanes as a
+//                        reduce-scatter over two query rows at a time: exactly the additions and
+//                        the order the interface fixes, so the fp32 result is reproducible bit for bit.
 //   topk_select_kernel : one 128-thread CTA per (sequence, active token, head); threshold search over
 //                        64-bit keys (order-preserving score bits, inverted page id), see below.
 //   topk_kernel        : budgets above 512 pages: one CTA per query sorts all keys with a
