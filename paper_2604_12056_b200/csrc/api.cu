@@ -37,6 +37,7 @@ int32_t make_layout(const losa_shape_t* sh, int n_ctas, WorkspaceLayout* L) {
   size_t off = 0;
   L->status = off;   off = align_up(off + 16, 256);
   L->counters = off; off = align_up(off + sizeof(uint32_t) * sh->batch, 256);
+  L->seg_prefix = off; off = align_up(off + sizeof(int32_t) * (kMaxSegments + 1), 256);
   L->delta = off;    off = align_up(off + sizeof(double) * sh->batch * sh->block_size, 256);
   L->scores = off;
   off = align_up(off + sizeof(float) * static_cast<size_t>(sh->batch) * sh->block_size * sh->n_q_heads * L->score_stride, 256);

@@ -37,6 +37,7 @@ struct AttnParams {
   const int32_t* union_pages;
   const int32_t* union_count;
   float* partials;
+  int32_t* seg_prefix;  // workspace copy of the segment prefix (written by the bf16 main kernel, read by its combine kernel)
   float* o_p;
   float* lse_p;
   int32_t* status;
@@ -197,7 +198,7 @@ __global__ void __launch_bounds__(256, 1) attn_simt_kernel(AttnParams p) {
 // take one piece each for the row maxima and sums, then the warp walks the pieces with the loads of
 // eight records issued together.  LOG2: partial maxima in base-2 units (tensor-core kernel) or
 // natural units (fp32 kernel).
-template <int D, bool LOG2>
+template <int D, bool LOG2, bool PRE>
 __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
   grid_dep_wait();
   __shared__ int pre[kMaxSegments + 1];
@@ -206,7 +207,11 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
   const int rg = sg % p.n_rg, sk = sg / p.n_rg, s = sk / p.Hkv, kh = sk % p.Hkv;
   const int rows = rows_in_group(clamp_active(p.n_active[s], p.B), p.G, rg);
   if (blockIdx.y * 8 >= rows) return;                 // whole CTA idle: skip the prefix as well
-  if (warp == 0) segment_prefix(pre, p.n_seg, p.n_rg, p.Hkv, p.G, p.n_active, p.union_count, p.B, lane);
+  if (PRE) {                                          // the main kernel left the prefix in the workspace
+    if (tid == 0) { pre[sg] = p.seg_prefix[sg]; pre[sg + 1] = p.seg_prefix[sg + 1]; pre[p.n_seg] = p.seg_prefix[p.n_seg]; }
+  } else if (warp == 0) {
+    segment_prefix(pre, p.n_seg, p.n_rg, p.Hkv, p.G, p.n_active, p.union_count, p.B, lane);
+  }
   __syncthreads();
   if (r >= rows) return;
   const int row = rg * kRowsPerGroup + r, a = row / p.G, gi = row % p.G;
@@ -412,7 +417,7 @@ int32_t launch_tc5(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
   if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_end, st));
   int32_t rc = after_launch(c);
   if (rc != LOSA_OK) return rc;
-  launch_k(attn_combine_kernel<D, true>, dim3(ap.n_seg, kRowsPerGroup / 8), 256, 0, st, ap);
+  launch_k(attn_combine_kernel<D, true, true>, dim3(ap.n_seg, kRowsPerGroup / 8), 256, 0, st, ap);
   return after_launch(c);
 }
 
@@ -426,7 +431,7 @@ int32_t launch_simt(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
   if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_end, st));
   int32_t rc = after_launch(c);
   if (rc != LOSA_OK) return rc;
-  launch_k(attn_combine_kernel<D, false>, dim3(ap.n_seg, kRowsPerGroup / 8), 256, 0, st, ap);
+  launch_k(attn_combine_kernel<D, false, false>, dim3(ap.n_seg, kRowsPerGroup / 8), 256, 0, st, ap);
   return after_launch(c);
 }
 
@@ -470,6 +475,7 @@ int32_t launch_sparse_prefix_attn(losa_ctx* c, const void* q, const losa_kv_t* k
   ap.union_pages = union_pages;
   ap.union_count = union_count;
   ap.partials = reinterpret_cast<float*>(c->ws + c->lay.partials);
+  ap.seg_prefix = reinterpret_cast<int32_t*>(c->ws + c->lay.seg_prefix);
   ap.o_p = state->o_p;
   ap.lse_p = state->lse_p;
   ap.status = status_ptr(c);

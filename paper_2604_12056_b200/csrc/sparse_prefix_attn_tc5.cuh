@@ -190,6 +190,8 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     }
   }
   __syncthreads();
+  if (blockIdx.x == 0)                             // the combine kernel reads the prefix instead of recomputing it
+    for (int i = tid; i <= p.n_seg; i += kTc5Threads) p.seg_prefix[i] = pre[i];
   const long long T_all = pre[p.n_seg];
   const int lo = static_cast<int>(cta_lo(T_all, blockIdx.x, p.n_ctas));
   const int hi = static_cast<int>(cta_lo(T_all, blockIdx.x + 1, p.n_ctas));

@@ -123,6 +123,16 @@ def test_ragged_batch_partial_pages_and_empty_prefix(g, d, hq, hkv, dtype):
     run_blocks(cfg, modes=("losa", "naive"))
 
 
+@pytest.mark.parametrize("g,d", [(16, 64), (16, 128), (32, 64), (64, 64)])
+def test_page_groups_of_the_tensor_core_kernel(g, d):
+    # the bf16 stage-4 kernel takes pages in groups of 128 tokens: several whole groups, a last group
+    # with fewer pages (also one that ends inside a 32-column chunk), a partial last page with NaN
+    # behind it, every page listed (dense mode) and few listed (LoSA)
+    cfg = wl.config("c2", n_q_heads=8, n_kv_heads=2, head_dim=d, page_size=g, kv_lens=(21 * g + 5, 9 * g, 128 + g),
+                    block_size=16, steps=3, topk=6, m_active=3)
+    run_blocks(cfg, modes=("losa", "dense"))
+
+
 @pytest.mark.parametrize("m", [0, 1, 16])
 def test_active_count_extremes(m):
     cfg = wl.config("c2", kv_lens=(700, 333), block_size=16, steps=3, topk=4, m_active=max(m, 1))
