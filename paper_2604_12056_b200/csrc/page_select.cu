@@ -14,6 +14,8 @@
 //                        shared-memory bitonic network.
 //   union_kernel       : one CTA per (sequence, KV head) ORs the selected ids into a bitmap and
 //                        emits the set bits in ascending order with a popcount scan.
+#include <algorithm>
+
 #include "kernels.h"
 
 namespace losa {
@@ -300,6 +302,7 @@ __device__ __forceinline__ unsigned long long make_key(uint32_t ob, int p) {
 // (P <= kSelThreads * kSelPerThread) their order bits stay in registers for the whole selection.
 constexpr int kSelThreads = 128;
 constexpr int kSelPerThread = 8;
+constexpr int kSelSlots = 8;        // CTAs per (sequence, head): active slots are dealt out round-robin
 
 template <bool CACHED, typename F>
 __device__ __forceinline__ void for_each_key(const uint32_t (&cache)[kSelPerThread], const float* __restrict__ row,
@@ -447,23 +450,26 @@ topk_select_kernel(const float* __restrict__ scores, const int32_t* __restrict__
                    float* __restrict__ topk_scores, int N, int B, int Hq, int g, int k, int score_stride,
                    int32_t* __restrict__ status) {
   grid_dep_wait();
-  // queries of the same active slot are adjacent, so the CTAs that have work are the first ones
+  // A CTA serves the active slots a = j, j + kSelSlots, ... of one (sequence, head): launching a CTA
+  // costs about as much as an idle CTA's whole life, and most of the B slots are idle on most steps.
   const int qid = blockIdx.x;
-  const int h = qid % Hq, s = (qid / Hq) % N, a = qid / (Hq * N);
+  const int h = qid % Hq, s = (qid / Hq) % N, j = qid / (Hq * N);
   if (step && step[s] == 0) return;
   int na = n_active[s];
   na = na > B ? B : na;
-  if (a >= na) return;
-  const int tok = active_idx[s * B + a];
-  if (tok < 0 || tok >= B) { if (threadIdx.x == 0) set_status(status, LOSA_ERR_BOUNDS); return; }
   const int P = pages_of(kv_len[s], g);
   const int kk = min(k, P);
-  const float* row = scores + ((static_cast<size_t>(s) * B + a) * Hq + h) * score_stride;
-  const size_t o = ((static_cast<size_t>(s) * B + tok) * Hq + h) * k;
-  if (P <= kSelThreads * kSelPerThread)
-    topk_select_body<true>(row, P, kk, k, topk_pages + o, topk_scores ? topk_scores + o : nullptr);
-  else
-    topk_select_body<false>(row, P, kk, k, topk_pages + o, topk_scores ? topk_scores + o : nullptr);
+  for (int a = j; a < na; a += kSelSlots) {
+    const int tok = active_idx[s * B + a];
+    if (tok < 0 || tok >= B) { if (threadIdx.x == 0) set_status(status, LOSA_ERR_BOUNDS); continue; }
+    const float* row = scores + ((static_cast<size_t>(s) * B + a) * Hq + h) * score_stride;
+    const size_t o = ((static_cast<size_t>(s) * B + tok) * Hq + h) * k;
+    if (P <= kSelThreads * kSelPerThread)
+      topk_select_body<true>(row, P, kk, k, topk_pages + o, topk_scores ? topk_scores + o : nullptr);
+    else
+      topk_select_body<false>(row, P, kk, k, topk_pages + o, topk_scores ? topk_scores + o : nullptr);
+    __syncthreads();                                 // the shared state is reused by the next slot
+  }
 }
 
 __global__ void __launch_bounds__(kThreads)
@@ -579,7 +585,7 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
 
   const float* sc = reinterpret_cast<const float*>(c->ws + c->lay.scores);
   if (k <= kSelCap) {
-    const int queries = sh.batch * sh.block_size * sh.n_q_heads;
+    const int queries = sh.batch * std::min<int>(sh.block_size, kSelSlots) * sh.n_q_heads;
     launch_k(topk_select_kernel, queries, kSelThreads, 0, st, 
         sc, kv->kv_len, active_idx, n_active, step, topk_pages, topk_scores_opt, sh.batch, sh.block_size,
         sh.n_q_heads, sh.page_size, k, c->lay.score_stride, status_ptr(c));

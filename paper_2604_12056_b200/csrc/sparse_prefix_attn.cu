@@ -193,7 +193,7 @@ __global__ void __launch_bounds__(256, 1) attn_simt_kernel(AttnParams p) {
 }
 
 // ===================================================================== combine kernel
-// grid (n_seg, 16): warp = one query row of the segment's row group.  The CTAs whose item range
+// grid (n_seg, 8): warp = one query row of the segment's row group at a time.  The CTAs whose item range
 // meets the segment are consecutive; each of them left one record for the row's 16-row tile.  Lanes
 // take one piece each for the row maxima and sums, then the warp walks the pieces with the loads of
 // eight records issued together.  LOG2: partial maxima in base-2 units (tensor-core kernel) or
@@ -203,7 +203,7 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
   grid_dep_wait();
   __shared__ int pre[kMaxSegments + 1];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int sg = blockIdx.x, r = blockIdx.y * 8 + warp;
+  const int sg = blockIdx.x;
   const int rg = sg % p.n_rg, sk = sg / p.n_rg, s = sk / p.Hkv, kh = sk % p.Hkv;
   const int rows = rows_in_group(clamp_active(p.n_active[s], p.B), p.G, rg);
   if (blockIdx.y * 8 >= rows) return;                 // whole CTA idle: skip the prefix as well
@@ -213,10 +213,10 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
     segment_prefix(pre, p.n_seg, p.n_rg, p.Hkv, p.G, p.n_active, p.union_count, p.B, lane);
   }
   __syncthreads();
-  if (r >= rows) return;
+  for (int r = blockIdx.y * 8 + warp; r < rows; r += gridDim.y * 8) {   // few CTAs per segment: most row blocks are empty on most steps
   const int row = rg * kRowsPerGroup + r, a = row / p.G, gi = row % p.G;
   const int tok = p.active_idx[s * p.B + a];
-  if (tok < 0 || tok >= p.B) { set_status(p.status, LOSA_ERR_BOUNDS); return; }
+  if (tok < 0 || tok >= p.B) { set_status(p.status, LOSA_ERR_BOUNDS); continue; }
   const size_t orow = (static_cast<size_t>(s) * p.B + tok) * p.Hq + kh * p.G + gi;
   const int start = pre[sg], end = pre[sg + 1];
   const long long T_all = pre[p.n_seg];
@@ -279,6 +279,7 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
 #pragma unroll
   for (int c = 0; c < C; ++c) p.o_p[orow * D + lane + 32 * c] = acc[c] * inv;
   if (lane == 0) p.lse_p[orow] = empty ? -INFINITY : (LOG2 ? (M + log2f(Lsum)) * kLn2 : M + logf(Lsum));
+  }
 }
 
 // ===================================================================== bf16 TMA + tensor-core kernel: shared pieces
@@ -417,7 +418,7 @@ int32_t launch_tc5(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
   if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_end, st));
   int32_t rc = after_launch(c);
   if (rc != LOSA_OK) return rc;
-  launch_k(attn_combine_kernel<D, true, true>, dim3(ap.n_seg, kRowsPerGroup / 8), 256, 0, st, ap);
+  launch_k(attn_combine_kernel<D, true, true>, dim3(ap.n_seg, 8), 256, 0, st, ap);
   return after_launch(c);
 }
 
@@ -431,7 +432,7 @@ int32_t launch_simt(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
   if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_end, st));
   int32_t rc = after_launch(c);
   if (rc != LOSA_OK) return rc;
-  launch_k(attn_combine_kernel<D, false, false>, dim3(ap.n_seg, kRowsPerGroup / 8), 256, 0, st, ap);
+  launch_k(attn_combine_kernel<D, false, false>, dim3(ap.n_seg, 8), 256, 0, st, ap);
   return after_launch(c);
 }
 
