@@ -259,10 +259,11 @@ int32_t losa_denoise_step(losa_ctx* ctx, const void* q, const void* k_blk, const
                             buf->active_idx, buf->n_active, nullptr, st);
   if (rc == LOSA_OK) rc = launch_page_scores_topk(ctx, q, kv, buf->active_idx, buf->n_active, state->step, k, buf->topk_pages, nullptr, st);
   if (rc == LOSA_OK) rc = launch_page_union(ctx, buf->topk_pages, buf->active_idx, buf->n_active, k, kv->kv_len, state->step, buf->union_pages, buf->union_count, st);
-  if (rc == LOSA_OK) rc = launch_sparse_prefix_attn(ctx, q, kv, buf->active_idx, buf->n_active, buf->union_pages, buf->union_count, state, st);
+  if (rc == LOSA_OK) rc = launch_sparse_prefix_attn(ctx, q, kv, buf->active_idx, buf->n_active, buf->union_pages, buf->union_count, state, st, true);
   if (rc != LOSA_OK) return rc;
-  // join, then merge + commit in one pass over the rows
+  // join, then one pass over the rows: (merge of the partial records,) merge with the block part, commit
   LOSA_CUDA_TRY(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0));
+  if (finish_fuses_combine(ctx)) return launch_attn_finish(ctx, q, buf->active_idx, buf->n_active, state, out, lse_out_opt, st);
   return launch_merge_commit(ctx, q, state, out, lse_out_opt, st);
 }
 

@@ -22,7 +22,13 @@ int32_t launch_page_union(losa_ctx* c, const int32_t* topk_pages, const int32_t*
 int32_t launch_sparse_prefix_attn(losa_ctx* c, const void* q, const losa_kv_t* kv,
                                   const int32_t* active_idx, const int32_t* n_active,
                                   const int32_t* union_pages, const int32_t* union_count,
-                                  losa_state_t* state, cudaStream_t st);
+                                  losa_state_t* state, cudaStream_t st, bool defer_combine = false);
+// Whole-step path: with defer_combine the bf16 main kernel leaves its partial records unmerged and
+// launch_attn_finish merges them, merges with the in-block part, writes the output, keeps the
+// queries and bumps the step (one kernel instead of combine + merge_commit).
+bool finish_fuses_combine(const losa_ctx* c);
+int32_t launch_attn_finish(losa_ctx* c, const void* q, const int32_t* active_idx, const int32_t* n_active,
+                           losa_state_t* state, void* out, float* lse_out_opt, cudaStream_t st);
 
 int32_t launch_block_attn_merge(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk,
                                 const losa_state_t* state, void* out, float* lse_out_opt,

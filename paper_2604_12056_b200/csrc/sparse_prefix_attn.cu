@@ -198,6 +198,66 @@ __global__ void __launch_bounds__(256, 1) attn_simt_kernel(AttnParams p) {
 // take one piece each for the row maxima and sums, then the warp walks the pieces with the loads of
 // eight records issued together.  LOG2: partial maxima in base-2 units (tensor-core kernel) or
 // natural units (fp32 kernel).
+// Merge of the partial records of row r of segment sg by one warp: returns the un-normalised
+// output columns lane + 32 c in acc, the reference maximum M and the sum of weights Lsum.
+template <int D, bool LOG2>
+__device__ __forceinline__ void merge_records(const AttnParams& p, int sg, int r, int start, int end, long long T_all,
+                                              int lane, float (&acc)[D / 32], float& M, float& Lsum) {
+  constexpr int C = D / 32;
+  const int tile = r / kTileRows, rr = r % kTileRows;
+#pragma unroll
+  for (int c = 0; c < C; ++c) acc[c] = 0.f;
+  M = -INFINITY;
+  Lsum = 0.f;
+  if (end <= start) return;
+  int b0 = static_cast<int>((static_cast<long long>(start) * p.n_ctas) / T_all);
+  while (b0 + 1 < p.n_ctas && cta_lo(T_all, b0 + 1, p.n_ctas) <= start) ++b0;
+  int b1 = static_cast<int>((static_cast<long long>(end - 1) * p.n_ctas) / T_all);   // last CTA that can meet it
+  while (b1 + 1 < p.n_ctas && cta_lo(T_all, b1 + 1, p.n_ctas) < end) ++b1;
+  const int n_pairs = b1 - b0 + 1;
+  // record of piece x, or null when CTA b0 + x has no page of this segment
+  auto record_of = [&](int x) -> const float* {
+    if (x >= n_pairs) return nullptr;
+    const int b = b0 + x;
+    const long long lo = max(cta_lo(T_all, b, p.n_ctas), static_cast<long long>(start));
+    const long long hi = min(cta_lo(T_all, b + 1, p.n_ctas), static_cast<long long>(end));
+    if (hi <= lo) return nullptr;
+    return record_base(p.partials, b + sg, tile, D);
+  };
+  for (int base = 0; base < n_pairs; base += 32) {
+    const float* rec = record_of(base + lane);
+    M = fmaxf(M, warp_max(rec ? rec[rr] : -INFINITY));
+  }
+  for (int base = 0; base < n_pairs; base += 32) {
+    const float* rec = record_of(base + lane);
+    float wj = 0.f, lj = 0.f;
+    if (rec) {
+      const float mj = rec[rr];
+      wj = (mj == -INFINITY) ? 0.f : (LOG2 ? exp2f(mj - M) : expf(mj - M));
+      lj = rec[kTileRows + rr];
+    }
+    Lsum += warp_sum(lj * wj);
+    const int n = min(32, n_pairs - base);
+    constexpr int U = 8;                            // records whose loads are in flight together
+    for (int i0 = 0; i0 < n; i0 += U) {
+      float w[U], v[U][C];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int i = i0 + u;
+        w[u] = (i < n) ? __shfl_sync(0xffffffffu, wj, i & 31) : 0.f;
+        const unsigned long long addr = __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(rec), i & 31);
+        const float* src = reinterpret_cast<const float*>(addr) + 2 * kTileRows + rr * D + lane;
+#pragma unroll
+        for (int c = 0; c < C; ++c) v[u][c] = (w[u] != 0.f) ? src[32 * c] : 0.f;
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u)
+#pragma unroll
+        for (int c = 0; c < C; ++c) acc[c] = fmaf(v[u][c], w[u], acc[c]);
+    }
+  }
+}
+
 template <int D, bool LOG2, bool PRE>
 __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
   grid_dep_wait();
@@ -213,73 +273,99 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
     segment_prefix(pre, p.n_seg, p.n_rg, p.Hkv, p.G, p.n_active, p.union_count, p.B, lane);
   }
   __syncthreads();
-  for (int r = blockIdx.y * 8 + warp; r < rows; r += gridDim.y * 8) {   // few CTAs per segment: most row blocks are empty on most steps
-  const int row = rg * kRowsPerGroup + r, a = row / p.G, gi = row % p.G;
-  const int tok = p.active_idx[s * p.B + a];
-  if (tok < 0 || tok >= p.B) { set_status(p.status, LOSA_ERR_BOUNDS); continue; }
-  const size_t orow = (static_cast<size_t>(s) * p.B + tok) * p.Hq + kh * p.G + gi;
-  const int start = pre[sg], end = pre[sg + 1];
-  const long long T_all = pre[p.n_seg];
-  const int tile = r / kTileRows, rr = r % kTileRows;
   constexpr int C = D / 32;
-  float acc[C];
+  for (int r = blockIdx.y * 8 + warp; r < rows; r += gridDim.y * 8) {   // few CTAs per segment: most row blocks are empty on most steps
+    const int row = rg * kRowsPerGroup + r, a = row / p.G, gi = row % p.G;
+    const int tok = p.active_idx[s * p.B + a];
+    if (tok < 0 || tok >= p.B) { set_status(p.status, LOSA_ERR_BOUNDS); continue; }
+    const size_t orow = (static_cast<size_t>(s) * p.B + tok) * p.Hq + kh * p.G + gi;
+    float acc[C], M, Lsum;
+    merge_records<D, LOG2>(p, sg, r, pre[sg], pre[sg + 1], pre[p.n_seg], lane, acc, M, Lsum);
+    const bool empty = !(Lsum > 0.f);
+    const float inv = empty ? 0.f : 1.f / Lsum;
 #pragma unroll
-  for (int c = 0; c < C; ++c) acc[c] = 0.f;
-  float M = -INFINITY, Lsum = 0.f;
-  if (end > start) {
-    int b0 = static_cast<int>((static_cast<long long>(start) * p.n_ctas) / T_all);
-    while (b0 + 1 < p.n_ctas && cta_lo(T_all, b0 + 1, p.n_ctas) <= start) ++b0;
-    int b1 = static_cast<int>((static_cast<long long>(end - 1) * p.n_ctas) / T_all);   // last CTA that can meet it
-    while (b1 + 1 < p.n_ctas && cta_lo(T_all, b1 + 1, p.n_ctas) < end) ++b1;
-    const int n_pairs = b1 - b0 + 1;
-    // record of piece x, or null when CTA b0 + x has no page of this segment
-    auto record_of = [&](int x) -> const float* {
-      if (x >= n_pairs) return nullptr;
-      const int b = b0 + x;
-      const long long lo = max(cta_lo(T_all, b, p.n_ctas), static_cast<long long>(start));
-      const long long hi = min(cta_lo(T_all, b + 1, p.n_ctas), static_cast<long long>(end));
-      if (hi <= lo) return nullptr;
-      return record_base(p.partials, b + sg, tile, D);
-    };
-    for (int base = 0; base < n_pairs; base += 32) {
-      const float* rec = record_of(base + lane);
-      M = fmaxf(M, warp_max(rec ? rec[rr] : -INFINITY));
-    }
-    for (int base = 0; base < n_pairs; base += 32) {
-      const float* rec = record_of(base + lane);
-      float wj = 0.f, lj = 0.f;
-      if (rec) {
-        const float mj = rec[rr];
-        wj = (mj == -INFINITY) ? 0.f : (LOG2 ? exp2f(mj - M) : expf(mj - M));
-        lj = rec[kTileRows + rr];
-      }
-      Lsum += warp_sum(lj * wj);
-      const int n = min(32, n_pairs - base);
-      constexpr int U = 8;                            // records whose loads are in flight together
-      for (int i0 = 0; i0 < n; i0 += U) {
-        float w[U], v[U][C];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-          const int i = i0 + u;
-          w[u] = (i < n) ? __shfl_sync(0xffffffffu, wj, i & 31) : 0.f;
-          const unsigned long long addr = __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(rec), i & 31);
-          const float* src = reinterpret_cast<const float*>(addr) + 2 * kTileRows + rr * D + lane;
-#pragma unroll
-          for (int c = 0; c < C; ++c) v[u][c] = (w[u] != 0.f) ? src[32 * c] : 0.f;
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u)
-#pragma unroll
-          for (int c = 0; c < C; ++c) acc[c] = fmaf(v[u][c], w[u], acc[c]);
-      }
-    }
+    for (int c = 0; c < C; ++c) p.o_p[orow * D + lane + 32 * c] = acc[c] * inv;
+    if (lane == 0) p.lse_p[orow] = empty ? -INFINITY : (LOG2 ? (M + log2f(Lsum)) * kLn2 : M + logf(Lsum));
   }
-  const bool empty = !(Lsum > 0.f);
-  const float inv = empty ? 0.f : 1.f / Lsum;
+}
+
+// Whole-step path, last kernel (bf16 main kernel): one warp per (sequence, block token, head) row.
+// An active row merges its partial records (as the combine kernel does) and stores the new prefix
+// statistics; a stable row reads its cached ones (reuse rule, Section 4.2).  Either way the row is
+// then merged with the in-block part by log-sum-exp (Section 2.2 / 4.3), the output is written and
+// the row's query kept for the next step's Eq. 1; block 0 also bumps the step counters.
+struct FinishParams {
+  const void* q;
+  void* q_prev;
+  const float* o_b;
+  const float* lse_b;
+  void* out;
+  float* lse_out;
+  int32_t* step;
+  size_t n_rows;
+};
+
+template <typename T, int D>
+__global__ void __launch_bounds__(256) attn_finish_kernel(AttnParams p, FinishParams f) {
+  grid_dep_wait();
+  constexpr int C = D / 32;
+  const int lane = threadIdx.x & 31;
+  const size_t row = static_cast<size_t>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+  if (blockIdx.x == 0)
+    for (int s = threadIdx.x; s < p.N; s += 256) f.step[s] += 1;
+  if (row >= f.n_rows) return;
+  const int hq = static_cast<int>(row % p.Hq), tok = static_cast<int>((row / p.Hq) % p.B);
+  const int s = static_cast<int>(row / (static_cast<size_t>(p.Hq) * p.B));
+  const int kh = hq / p.G, gi = hq % p.G;
+  // operands that do not depend on the row being active: requested first
+  const T* q = static_cast<const T*>(f.q);
+  float b[C];
+  T qv[C];
 #pragma unroll
-  for (int c = 0; c < C; ++c) p.o_p[orow * D + lane + 32 * c] = acc[c] * inv;
-  if (lane == 0) p.lse_p[orow] = empty ? -INFINITY : (LOG2 ? (M + log2f(Lsum)) * kLn2 : M + logf(Lsum));
+  for (int c = 0; c < C; ++c) {
+    b[c] = f.o_b[row * D + lane + 32 * c];
+    qv[c] = q[row * D + lane + 32 * c];
   }
+  const float Lb = f.lse_b[row];
+  // the row's slot in the active list, if any (the list has at most B <= 64 entries)
+  const int na = clamp_active(p.n_active[s], p.B);
+  int slot = -1;
+  for (int base = 0; base < na && slot < 0; base += 32) {
+    const int i = base + lane;
+    const unsigned hit = __ballot_sync(0xffffffffu, i < na && p.active_idx[s * p.B + i] == tok);
+    if (hit) slot = base + __ffs(hit) - 1;
+  }
+  float a[C], Lp;
+  if (slot >= 0) {
+    const int rowk = slot * p.G + gi, rg = rowk / kRowsPerGroup, r = rowk % kRowsPerGroup;
+    const int sg = (s * p.Hkv + kh) * p.n_rg + rg;
+    float acc[C], M, Lsum;
+    merge_records<D, true>(p, sg, r, p.seg_prefix[sg], p.seg_prefix[sg + 1], p.seg_prefix[p.n_seg], lane, acc, M, Lsum);
+    const bool empty = !(Lsum > 0.f);
+    const float inv = empty ? 0.f : 1.f / Lsum;
+    Lp = empty ? -INFINITY : (M + log2f(Lsum)) * kLn2;
+#pragma unroll
+    for (int c = 0; c < C; ++c) {
+      a[c] = acc[c] * inv;
+      p.o_p[row * D + lane + 32 * c] = a[c];
+    }
+    if (lane == 0) p.lse_p[row] = Lp;
+  } else {
+#pragma unroll
+    for (int c = 0; c < C; ++c) a[c] = p.o_p[row * D + lane + 32 * c];
+    Lp = p.lse_p[row];
+  }
+  const float Mx = fmaxf(Lp, Lb);
+  const float L = Mx + logf(expf(Lp - Mx) + expf(Lb - Mx));
+  const float wp = expf(Lp - L), wb = expf(Lb - L);
+  T* out = static_cast<T*>(f.out);
+  T* q_prev = static_cast<T*>(f.q_prev);
+#pragma unroll
+  for (int c = 0; c < C; ++c) {
+    out[row * D + lane + 32 * c] = from_f32<T>((wp > 0.f ? wp * a[c] : 0.f) + wb * b[c]);
+    q_prev[row * D + lane + 32 * c] = qv[c];
+  }
+  if (f.lse_out && lane == 0) f.lse_out[row] = L;
 }
 
 // ===================================================================== bf16 TMA + tensor-core kernel: shared pieces
@@ -403,7 +489,7 @@ int32_t ensure_tensor_maps(losa_ctx* c, const losa_kv_t* kv) {
 }
 
 template <int D, int GP>
-int32_t launch_tc5(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
+int32_t launch_tc5(losa_ctx* c, const AttnParams& ap, cudaStream_t st, bool with_combine) {
   constexpr int smem = tc5_smem_bytes<D>();
   static int attr_device = -1;
   if (attr_device != c->device) {
@@ -417,7 +503,7 @@ int32_t launch_tc5(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
   launch_k(attn_tc5_kernel<D, GP>, ap.n_ctas, kTc5Threads, smem, st, mk, mv, ap);
   if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_end, st));
   int32_t rc = after_launch(c);
-  if (rc != LOSA_OK) return rc;
+  if (rc != LOSA_OK || !with_combine) return rc;
   launch_k(attn_combine_kernel<D, true, true>, dim3(ap.n_seg, 8), 256, 0, st, ap);
   return after_launch(c);
 }
@@ -437,12 +523,12 @@ int32_t launch_simt(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
 }
 
 template <int D>
-int32_t dispatch_page(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
+int32_t dispatch_page(losa_ctx* c, const AttnParams& ap, cudaStream_t st, bool with_combine) {
   const bool bf = c->shape.dtype == LOSA_BF16;
   switch (c->shape.page_size) {
-    case 16: return bf ? launch_tc5<D, 16>(c, ap, st) : launch_simt<float, D, 16>(c, ap, st);
-    case 32: return bf ? launch_tc5<D, 32>(c, ap, st) : launch_simt<float, D, 32>(c, ap, st);
-    default: return bf ? launch_tc5<D, 64>(c, ap, st) : launch_simt<float, D, 64>(c, ap, st);
+    case 16: return bf ? launch_tc5<D, 16>(c, ap, st, with_combine) : launch_simt<float, D, 16>(c, ap, st);
+    case 32: return bf ? launch_tc5<D, 32>(c, ap, st, with_combine) : launch_simt<float, D, 32>(c, ap, st);
+    default: return bf ? launch_tc5<D, 64>(c, ap, st, with_combine) : launch_simt<float, D, 64>(c, ap, st);
   }
 }
 
@@ -456,7 +542,7 @@ extern "C" void losa_debug_set_trace(void* p) { g_trace = static_cast<unsigned l
 int32_t launch_sparse_prefix_attn(losa_ctx* c, const void* q, const losa_kv_t* kv,
                                   const int32_t* active_idx, const int32_t* n_active,
                                   const int32_t* union_pages, const int32_t* union_count,
-                                  losa_state_t* state, cudaStream_t st) {
+                                  losa_state_t* state, cudaStream_t st, bool defer_combine) {
   const losa_shape_t& sh = c->shape;
   if (sh.dtype == LOSA_BF16) {
     int32_t rc = ensure_tensor_maps(c, kv);
@@ -494,7 +580,44 @@ int32_t launch_sparse_prefix_attn(losa_ctx* c, const void* q, const losa_kv_t* k
 #ifdef LOSA_TRACE
   ap.trace = g_trace;
 #endif
-  return sh.head_dim == 128 ? dispatch_page<128>(c, ap, st) : dispatch_page<64>(c, ap, st);
+  const bool with_combine = !(defer_combine && finish_fuses_combine(c));
+  return sh.head_dim == 128 ? dispatch_page<128>(c, ap, st, with_combine) : dispatch_page<64>(c, ap, st, with_combine);
+}
+
+bool finish_fuses_combine(const losa_ctx* c) { return c->shape.dtype == LOSA_BF16; }
+
+int32_t launch_attn_finish(losa_ctx* c, const void* q, const int32_t* active_idx, const int32_t* n_active,
+                           losa_state_t* state, void* out, float* lse_out_opt, cudaStream_t st) {
+  const losa_shape_t& sh = c->shape;
+  AttnParams ap = {};
+  ap.active_idx = active_idx;
+  ap.n_active = n_active;
+  ap.partials = reinterpret_cast<float*>(c->ws + c->lay.partials);
+  ap.seg_prefix = reinterpret_cast<int32_t*>(c->ws + c->lay.seg_prefix);
+  ap.o_p = state->o_p;
+  ap.lse_p = state->lse_p;
+  ap.status = status_ptr(c);
+  ap.N = sh.batch;
+  ap.B = sh.block_size;
+  ap.Hq = sh.n_q_heads;
+  ap.Hkv = sh.n_kv_heads;
+  ap.G = sh.n_q_heads / sh.n_kv_heads;
+  ap.n_rg = c->lay.n_row_groups;
+  ap.n_seg = c->lay.n_segments;
+  ap.n_ctas = c->lay.n_ctas;
+  FinishParams fp;
+  fp.q = q;
+  fp.q_prev = state->q_prev;
+  fp.o_b = reinterpret_cast<const float*>(c->ws + c->lay.block_o);
+  fp.lse_b = reinterpret_cast<const float*>(c->ws + c->lay.block_lse);
+  fp.out = out;
+  fp.lse_out = lse_out_opt;
+  fp.step = state->step;
+  fp.n_rows = static_cast<size_t>(sh.batch) * sh.block_size * sh.n_q_heads;
+  const int blocks = static_cast<int>((fp.n_rows + 7) / 8);
+  if (sh.head_dim == 128) launch_k(attn_finish_kernel<__nv_bfloat16, 128>, blocks, 256, 0, st, ap, fp);
+  else launch_k(attn_finish_kernel<__nv_bfloat16, 64>, blocks, 256, 0, st, ap, fp);
+  return after_launch(c);
 }
 
 }  // namespace losa
