@@ -179,6 +179,10 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  if (warp == 0) {                                 // tensor memory: taken while the previous kernel drains
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
   grid_dep_wait();                                 // nothing above touches global memory
   if (warp == 0) {
     segment_prefix(pre, p.n_seg, p.n_rg, p.Hkv, p.G, p.n_active, p.union_count, p.B, lane);
@@ -189,21 +193,19 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       len_s[i] = p.kv_len[i];
     }
   }
+  tc5_fence_before();
   __syncthreads();
+  tc5_fence_after();
+  const uint32_t tmem = *tmem_slot;
   if (blockIdx.x == 0)                             // the combine kernel reads the prefix instead of recomputing it
     for (int i = tid; i <= p.n_seg; i += kTc5Threads) p.seg_prefix[i] = pre[i];
   const long long T_all = pre[p.n_seg];
   const int lo = static_cast<int>(cta_lo(T_all, blockIdx.x, p.n_ctas));
   const int hi = static_cast<int>(cta_lo(T_all, blockIdx.x + 1, p.n_ctas));
-  if (lo >= hi) return;                           // before any tensor memory is allocated
-  if (warp == 0) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "n"(TMEM_COLS) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  if (lo >= hi) {                                  // nothing to do: give the tensor memory back
+    if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(TMEM_COLS) : "memory");
+    return;
   }
-  tc5_fence_before();
-  __syncthreads();
-  tc5_fence_after();
-  const uint32_t tmem = *tmem_slot;
   int sg0 = 0;
   while (pre[sg0 + 1] <= lo) ++sg0;
   auto n_active_of = [&](int s) { return staged ? na_s[s] : clamp_active(p.n_active[s], p.B); };
