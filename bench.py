@@ -51,7 +51,8 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=0, help="timed layer-steps (default: 4 blocks of all layers)")
     ap.add_argument("--warmup", type=int, default=0, help="untimed layer-steps (default: 1 block of all layers)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5"])
+    ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5", "p1", "p2"])
+    ap.add_argument("--topk", type=int, default=0, help="override the page budget per query (pages)")
     ap.add_argument("--layers", type=int, default=0, help="attention layers (default: 36 for c5, else 1)")
     ap.add_argument("--active-frac", type=float, default=None, help="override the active fraction")
     ap.add_argument("--no-extras", action="store_true", help="skip baselines, stage breakdown, cpu baseline")
@@ -60,9 +61,11 @@ def parse_args():
 
 def make_config(args):
     cfg = wl.config(args.workload)
+    if args.topk > 0:
+        cfg = wl.config(args.workload, topk=args.topk)
     if args.active_frac is not None:
         cfg = wl.config(args.workload, m_active=wl.active_count(args.active_frac, cfg.block_size),
-                        n_blocks=cfg.n_blocks, beta_active=False)
+                        n_blocks=cfg.n_blocks, beta_active=False, topk=cfg.topk)
     return cfg
 
 
@@ -289,7 +292,7 @@ def run_ours(args, cfg0):
     def blocks_for(n):
         return (n + per_block - 1) // per_block
     total_blocks = blocks_for(args.warmup + args.steps) + blocks_for(n_prof) + blocks_for(n_e2e) + 2
-    cfg = wl.config(cfg0.name, n_blocks=total_blocks, m_active=cfg0.m_active, beta_active=cfg0.beta_active)
+    cfg = wl.config(cfg0.name, n_blocks=total_blocks, m_active=cfg0.m_active, beta_active=cfg0.beta_active, topk=cfg0.topk)
     runs = [LayerRun(cfg, D.replica_of(rank), l, dev) for l in range(L)]
     launches_step = launches_fin = 0
     for r in runs:

@@ -95,7 +95,7 @@ def active_count(frac: float, block: int) -> int:
 
 
 def config(name: str, **kw) -> Config:
-    """The five benchmark configurations (c1 .. c5) and reduced variants for tests."""
+    """The five benchmark configurations (c1 .. c5), the paper-shaped p1 / p2, and reduced variants for tests."""
     qwen = dict(n_q_heads=32, n_kv_heads=8, head_dim=128)
     table = {
         # tiny fp32 single layer: 64 pages of 16, block 16, 4 steps, 4 planted tokens, k = 8
@@ -115,6 +115,12 @@ def config(name: str, **kw) -> Config:
         "c5": Config("c5", 5, page_size=32, kv_lens=(32768,) * 8, block_size=32, steps=8, topk=64,
                      m_active=active_count(0.10, 32), dtype="bf16", clustered=True, n_blocks=4,
                      beta_active=True, **qwen),
+        # the shapes of the paper's latency study (Section 5.4), batch 1, five active tokens per step,
+        # budget 512 tokens = 16 pages by default: p1 = 64K context / block 16, p2 = 32K context / block 32
+        "p1": Config("p1", 6, page_size=32, kv_lens=(65536,), block_size=16, steps=8, topk=16,
+                     m_active=5, dtype="bf16", clustered=True, **qwen),
+        "p2": Config("p2", 7, page_size=32, kv_lens=(32768,), block_size=32, steps=8, topk=16,
+                     m_active=5, dtype="bf16", clustered=True, **qwen),
     }
     return replace(table[name], **kw)
 

@@ -133,6 +133,12 @@ def test_page_groups_of_the_tensor_core_kernel(g, d):
     run_blocks(cfg, modes=("losa", "dense"))
 
 
+@pytest.mark.parametrize("name", ["p1", "p2"])
+def test_paper_shaped_workloads_reduced(name):
+    # the shapes of the paper's latency study (batch 1, five active tokens, budget 16 pages), shorter prefix
+    run_blocks(wl.config(name, kv_lens=(4096 + 77,), steps=4), modes=("losa", "naive", "dense"))
+
+
 @pytest.mark.parametrize("m", [0, 1, 16])
 def test_active_count_extremes(m):
     cfg = wl.config("c2", kv_lens=(700, 333), block_size=16, steps=3, topk=4, m_active=max(m, 1))
