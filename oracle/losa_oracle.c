@@ -121,6 +121,60 @@ void oracle_select_active(const oracle_shape_t* sh, const void* x_cur, const voi
   free(dl);
 }
 
+/* ---------- threshold variant of the pruning rule (appendix, locality heat maps with tau = 0.5) ----------
+ * Tokens are ranked as above; the active set is the shortest leading part of the ranking whose
+ * Delta values add up to at least tau times the sum over the block ("the boundary where the
+ * cumulative normalised MSE reaches 50% of the total").  Both sums run over the ranking in order.
+ * A block whose Delta are all zero has no active token.  m_cap (optional) bounds the count from
+ * above; step == 0 makes every token active. */
+void oracle_select_active_tau(const oracle_shape_t* sh, const void* x_cur, const void* x_prev,
+                              int32_t row_width, double tau, const int32_t* m_cap, const int32_t* step,
+                              int32_t* active_idx, int32_t* n_active, double* delta) {
+  const int B = sh->block_size;
+  double* dl = (double*)malloc(sizeof(double) * (size_t)B);
+  double* sorted = (double*)malloc(sizeof(double) * (size_t)B);
+  int* rank = (int*)malloc(sizeof(int) * (size_t)B);
+  for (int s = 0; s < sh->batch; ++s) {
+    for (int i = 0; i < B; ++i) {
+      const int64_t row = ((int64_t)s * B + i) * row_width;
+      double acc = 0.0;
+      for (int c = 0; c < row_width; ++c) {
+        double df = ld(x_cur, sh->dtype, row + c) - ld(x_prev, sh->dtype, row + c);
+        acc += df * df;
+      }
+      dl[i] = acc / (double)row_width;
+      if (delta) delta[(int64_t)s * B + i] = dl[i];
+    }
+    for (int i = 0; i < B; ++i) {
+      int r = 0;
+      for (int j = 0; j < B; ++j)
+        if (dl[j] > dl[i] || (dl[j] == dl[i] && j < i)) ++r;
+      rank[i] = r;
+      sorted[r] = dl[i];
+    }
+    int m;
+    if (step && step[s] == 0) {
+      m = B;
+    } else {
+      double total = 0.0;
+      for (int r = 0; r < B; ++r) total += sorted[r];
+      const double thr = tau * total;
+      double cum = 0.0;
+      m = 0;
+      while (m < B && cum < thr) cum += sorted[m++];
+      if (m_cap && m_cap[s] >= 0 && m_cap[s] < m) m = m_cap[s];
+    }
+    int cnt = 0;
+    for (int i = 0; i < B; ++i)
+      if (rank[i] < m) active_idx[(int64_t)s * B + cnt++] = i;
+    n_active[s] = cnt;
+    for (int i = cnt; i < B; ++i) active_idx[(int64_t)s * B + i] = -1;
+  }
+  free(dl);
+  free(sorted);
+  free(rank);
+}
+
 /* ---------- Section 2.3: query-dependent upper bound of the attention score per page ----------
  * For a page with element-wise key bounds kmin <= k <= kmax, q.k <= sum_j max(q_j kmin_j,
  * q_j kmax_j) — the tightest bound those summaries allow.  The 1/sqrt(d) factor is omitted: it

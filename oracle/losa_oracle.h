@@ -43,6 +43,12 @@ void oracle_select_active(const oracle_shape_t* sh, const void* x_cur, const voi
                           int32_t row_width, const int32_t* m_per_seq, const int32_t* step,
                           int32_t* active_idx, int32_t* n_active, double* delta);
 
+/* Threshold variant (appendix figures, tau = 0.5): the shortest leading part of the ranking whose
+ * Delta add up to at least tau times the block's total; m_cap (optional, per sequence) bounds it. */
+void oracle_select_active_tau(const oracle_shape_t* sh, const void* x_cur, const void* x_prev,
+                              int32_t row_width, double tau, const int32_t* m_cap, const int32_t* step,
+                              int32_t* active_idx, int32_t* n_active, double* delta);
+
 /* Section 2.3 page upper bound for one (sequence, token, head): fp32 in the interface's fixed
  * order (u32, may be NULL) and plain fp64 (u64, may be NULL); P_s entries each. */
 void oracle_page_scores_one(const oracle_shape_t* sh, const void* q, const oracle_kv_t* kv,

@@ -134,6 +134,23 @@ def select_active(sh: Shape, x_cur, x_prev, m_per_seq=None, step=None):
     return act, na, delta
 
 
+def select_active_tau(sh: Shape, x_cur, x_prev, tau: float, m_cap=None, step=None):
+    """Threshold variant of the pruning rule.  Returns (active_idx, n_active, delta) as select_active."""
+    N, B = sh.batch, sh.block_size
+    x_cur = _chk(x_cur, sh.elem, "x_cur")
+    x_prev = _chk(x_prev, sh.elem, "x_prev")
+    w = x_cur.size // (N * B)
+    act = np.full((N, B), -7, np.int32)
+    na = np.zeros(N, np.int32)
+    delta = np.zeros((N, B), np.float64)
+    m = None if m_cap is None else _chk(np.ascontiguousarray(m_cap, np.int32), np.int32, "m_cap")
+    st = None if step is None else _chk(np.ascontiguousarray(step, np.int32), np.int32, "step")
+    s = sh.c()
+    lib().oracle_select_active_tau(C.byref(s), _p(x_cur), _p(x_prev), C.c_int32(w), C.c_double(tau), _p(m), _p(st),
+                                   _p(act), _p(na), _p(delta))
+    return act, na, delta
+
+
 def page_scores_one(sh: Shape, q, kv: KV, s_idx: int, tok: int, head: int):
     """Returns (u32 [P_s] float32 in the fixed order, u64 [P_s] float64)."""
     P = (int(kv.kv_len[s_idx]) + sh.page_size - 1) // sh.page_size

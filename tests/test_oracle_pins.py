@@ -286,6 +286,48 @@ def test_locality_score_and_ranking(dtype):
     assert nan_.tolist() == [7, 7]
 
 
+# --- I7b: threshold variant of the pruning rule (appendix heat maps, tau = 0.5) --------------------
+def test_threshold_pruning_rule():
+    # a worked example with exact arithmetic: one changed element per token gives Delta_i = c_i^2 / w
+    pb = Problem(12, N=2, Hq=4, Hkv=2, d=16, B=6, g=4, kv_lens=(8, 8), dtype="f32")
+    sh, w = pb.sh, 16
+    x0 = np.zeros((2, 6, w), np.float32)
+    x1 = x0.copy()
+    amps = np.array([1.0, 4.0, 2.0, 0.0, 2.0, 1.0], np.float32)          # squares 1 16 4 0 4 1: total 26
+    x1[0, np.arange(6), 0] = amps
+    x1[1] = 0.0                                                          # nothing changed: no active token
+    one = np.ones(2, np.int32)
+    act, na, delta = orc.select_active_tau(sh, x1, x0, 0.5, None, one)
+    np.testing.assert_array_equal(delta[0] * w, amps.astype(np.float64) ** 2)
+    assert na.tolist() == [1, 0] and act[0, 0] == 1                      # 16 >= 13
+    act, na, _ = orc.select_active_tau(sh, x1, x0, 16.0 / 26.0 + 1e-9, None, one)
+    assert na[0] == 2 and act[0, :2].tolist() == [1, 2]                  # tie 4 = 4: the lower index first
+    act, na, _ = orc.select_active_tau(sh, x1, x0, 24.0 / 26.0, None, one)
+    assert na[0] == 3 and act[0, :3].tolist() == [1, 2, 4]               # 16 + 4 + 4 = 24 reaches 24 exactly
+    act, na, _ = orc.select_active_tau(sh, x1, x0, 1.0, None, one)
+    assert na[0] == 5 and act[0, :5].tolist() == [0, 1, 2, 4, 5]         # the unchanged token is never needed
+    act, na, _ = orc.select_active_tau(sh, x1, x0, 1.0, np.array([2, 2], np.int32), one)
+    assert na.tolist() == [2, 0] and act[0, :2].tolist() == [1, 2]       # capped
+    act, na, _ = orc.select_active_tau(sh, x1, x0, 0.5, None, np.zeros(2, np.int32))
+    assert na.tolist() == [6, 6]                                         # first step of a block: everything
+    # against numpy on random data: sort, cumulative sum, first index reaching tau * total
+    rng = np.random.default_rng(5)
+    pb2 = Problem(13, N=3, Hq=4, Hkv=2, d=16, B=16, g=4, kv_lens=(8, 8, 8), dtype="bf16")
+    y0 = pb2.rand_elem((3, 16, 24))
+    y1 = y0.copy()
+    for s_ in range(3):
+        for t in rng.choice(16, size=5, replace=False):
+            y1[s_, t] = pb2.rand_elem((24,), scale=float(rng.uniform(0.2, 3.0)))
+    for tau in (0.25, 0.5, 0.9):
+        act, na, delta = orc.select_active_tau(pb2.sh, y1, y0, tau, None, np.ones(3, np.int32))
+        for s_ in range(3):
+            order = np.argsort(-delta[s_], kind="stable")
+            cum = np.cumsum(delta[s_][order])
+            m = int(np.searchsorted(cum, tau * cum[-1], side="left")) + 1
+            assert abs(cum[m - 1] - tau * cum[-1]) > 1e-9 * cum[-1]      # the case is not a near-tie
+            assert na[s_] == m and act[s_, :m].tolist() == sorted(order[:m].tolist())
+
+
 # --- I8: results do not depend on where pages live physically --------------------------------------
 def test_physical_page_permutation_invariance():
     a = Problem(12, N=2, Hq=4, Hkv=2, d=16, B=4, g=4, kv_lens=(27, 14), shuffle=True)
