@@ -156,6 +156,19 @@ int32_t losa_select_active(losa_ctx* ctx, const void* x_cur, const void* x_prev,
                            const int32_t* m_per_seq, const int32_t* step, int32_t* active_idx,
                            int32_t* n_active, float* delta_opt, void* stream);
 
+/* Stage 1, threshold variant (appendix: the locality heat maps select tokens "where cumulative
+ * normalised MSE reaches 50% of the layer total", tau = 0.5).  Delta and the ranking are those of
+ * losa_select_active; the active set is the shortest leading part of the ranking whose Delta add up
+ * to at least tau times the sum of Delta over the block (both sums taken over the ranking in order,
+ * in fp64).  A block whose queries did not change at all has no active token.
+ *   tau in (0, 1] (host value); anything else returns LOSA_ERR_INVALID_ARG.
+ *   m_cap_opt [N] int32 or NULL: an upper bound on the count per sequence (negative = none).
+ *   step[s] == 0 makes every token of sequence s active, as in losa_select_active.
+ *   All other arguments and outputs are those of losa_select_active. */
+int32_t losa_select_active_tau(losa_ctx* ctx, const void* x_cur, const void* x_prev, int32_t row_width,
+                               double tau, const int32_t* m_cap_opt, const int32_t* step, int32_t* active_idx,
+                               int32_t* n_active, float* delta_opt, void* stream);
+
 /* Stage 1 without any allocation (the paper has no counterpart; this is a deployment aid).
  * Some programs that embed this library are not allowed to obtain device memory once they are
  * running: an inference server whose memory pool was carved up at start-up and whose allocator is

@@ -29,7 +29,7 @@ EXPORTS = [
     "losa_page_union", "losa_sparse_prefix_attn", "losa_block_attn_merge",
     "losa_update_prefix_cache", "losa_build_page_summaries", "losa_denoise_step_host",
     "losa_profile_stage4", "losa_stage4_last_ms", "losa_select_active_static",
-    "losa_denoise_step",
+    "losa_denoise_step", "losa_select_active_tau",
 ]
 
 
@@ -171,6 +171,13 @@ class Context:
 def losa_select_active(ctx, x_cur, x_prev, row_width, m_per_seq, step, active_idx, n_active, delta_opt=None):
     ctx._check("losa_select_active", lib().losa_select_active(
         ctx._h, _ptr(x_cur), _ptr(x_prev), C.c_int32(row_width), _ptr(m_per_seq), _ptr(step),
+        _ptr(active_idx), _ptr(n_active), _ptr(delta_opt), _stream()))
+
+
+def losa_select_active_tau(ctx, x_cur, x_prev, row_width, tau, m_cap_opt, step, active_idx, n_active, delta_opt=None):
+    """Stage 1, threshold variant: tokens are kept until their Delta reach tau of the block's total."""
+    ctx._check("losa_select_active_tau", lib().losa_select_active_tau(
+        ctx._h, _ptr(x_cur), _ptr(x_prev), C.c_int32(row_width), C.c_double(tau), _ptr(m_cap_opt), _ptr(step),
         _ptr(active_idx), _ptr(n_active), _ptr(delta_opt), _stream()))
 
 

@@ -169,6 +169,15 @@ int32_t losa_select_active(losa_ctx* ctx, const void* x_cur, const void* x_prev,
   return launch_select_active(ctx, x_cur, x_prev, row_width, m_per_seq, step, active_idx, n_active, delta_opt, as_stream(stream));
 }
 
+int32_t losa_select_active_tau(losa_ctx* ctx, const void* x_cur, const void* x_prev, int32_t row_width,
+                               double tau, const int32_t* m_cap_opt, const int32_t* step, int32_t* active_idx,
+                               int32_t* n_active, float* delta_opt, void* stream) {
+  if (!ctx || !x_cur || !x_prev || !active_idx || !n_active || row_width < 1 || !(tau > 0.0) || tau > 1.0)
+    return LOSA_ERR_INVALID_ARG;
+  if (row_width % 8 != 0 || !aligned16(x_cur) || !aligned16(x_prev)) return LOSA_ERR_UNSUPPORTED;
+  return launch_select_active(ctx, x_cur, x_prev, row_width, m_cap_opt, step, active_idx, n_active, delta_opt, as_stream(stream), tau);
+}
+
 int32_t losa_page_scores_topk(losa_ctx* ctx, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
                               const int32_t* n_active, const int32_t* step, int32_t k, int32_t* topk_pages,
                               float* topk_scores_opt, void* stream) {

@@ -7,7 +7,7 @@ namespace losa {
 
 int32_t launch_select_active(losa_ctx* c, const void* x_cur, const void* x_prev, int32_t row_width,
                              const int32_t* m_per_seq, const int32_t* step, int32_t* active_idx,
-                             int32_t* n_active, float* delta_opt, cudaStream_t st);
+                             int32_t* n_active, float* delta_opt, cudaStream_t st, double tau = 0.0);
 
 int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
                                 const int32_t* active_idx, const int32_t* n_active,

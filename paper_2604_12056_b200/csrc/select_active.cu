@@ -20,7 +20,7 @@ select_active_kernel(const T* __restrict__ x_cur, const T* __restrict__ x_prev, 
                      const int32_t* __restrict__ m_per_seq, const int32_t* __restrict__ step,
                      int32_t* __restrict__ active_idx, int32_t* __restrict__ n_active,
                      float* __restrict__ delta_opt, double* __restrict__ delta_ws,
-                     unsigned int* __restrict__ counters) {
+                     unsigned int* __restrict__ counters, double tau) {
   grid_dep_wait();
   const int i = blockIdx.x, s = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -63,23 +63,45 @@ select_active_kernel(const T* __restrict__ x_cur, const T* __restrict__ x_prev, 
   if (warp != 0) return;
 
   int m = m_per_seq ? m_per_seq[s] : -1;
-  if (m < 0 || m > B || (step && step[s] == 0)) m = B;
-  // token t = lane (+32): active when fewer than m tokens precede it in the ranking
-  bool act[2];
+  const bool first_step = step && step[s] == 0;
+  if (m < 0 || m > B || first_step) m = B;
+  // token t = lane (+32): rank under (Delta descending, token ascending)
+  int rank[2] = {B, B};
 #pragma unroll
   for (int half = 0; half < 2; ++half) {
     const int t = lane + 32 * half;
-    act[half] = false;
     if (t < B) {
       const double dt = s_delta[t];
-      int rank = 0;
+      int r = 0;
       for (int j = 0; j < B; ++j) {
         const double dj = s_delta[j];
-        rank += (dj > dt || (dj == dt && j < t)) ? 1 : 0;
+        r += (dj > dt || (dj == dt && j < t)) ? 1 : 0;
       }
-      act[half] = rank < m;
+      rank[half] = r;
     }
   }
+  if (tau > 0.0 && !first_step) {
+    // threshold variant: the shortest leading part of the ranking whose Delta add up to at least
+    // tau times the block's total; both sums run over the ranking in order, in fp64, by one lane
+    __shared__ double s_sorted[LOSA_MAX_BLOCK];
+#pragma unroll
+    for (int half = 0; half < 2; ++half)
+      if (lane + 32 * half < B) s_sorted[rank[half]] = s_delta[lane + 32 * half];
+    __syncwarp();
+    int mt = 0;
+    if (lane == 0) {
+      double total = 0.0;
+      for (int r = 0; r < B; ++r) total += s_sorted[r];
+      const double thr = tau * total;
+      double cum = 0.0;
+      while (mt < B && cum < thr) cum += s_sorted[mt++];
+    }
+    mt = __shfl_sync(0xffffffffu, mt, 0);
+    m = min(m, mt);                                   // m_per_seq, when given, is an upper bound here
+  }
+  bool act[2];
+#pragma unroll
+  for (int half = 0; half < 2; ++half) act[half] = rank[half] < m;
   const unsigned b0 = __ballot_sync(0xffffffffu, act[0]);
   const unsigned b1 = __ballot_sync(0xffffffffu, act[1]);
   const unsigned below = (1u << lane) - 1u;
@@ -95,7 +117,7 @@ select_active_kernel(const T* __restrict__ x_cur, const T* __restrict__ x_prev, 
 
 int32_t launch_select_active(losa_ctx* c, const void* x_cur, const void* x_prev, int32_t row_width,
                              const int32_t* m_per_seq, const int32_t* step, int32_t* active_idx,
-                             int32_t* n_active, float* delta_opt, cudaStream_t st) {
+                             int32_t* n_active, float* delta_opt, cudaStream_t st, double tau) {
   const losa_shape_t& sh = c->shape;
   dim3 grid(sh.block_size, sh.batch);
   double* dws = reinterpret_cast<double*>(c->ws + c->lay.delta);
@@ -103,11 +125,11 @@ int32_t launch_select_active(losa_ctx* c, const void* x_cur, const void* x_prev,
   if (sh.dtype == LOSA_BF16) {
     launch_k(select_active_kernel<__nv_bfloat16>, grid, kThreads, 0, st, 
         static_cast<const __nv_bfloat16*>(x_cur), static_cast<const __nv_bfloat16*>(x_prev), row_width,
-        sh.block_size, m_per_seq, step, active_idx, n_active, delta_opt, dws, ctr);
+        sh.block_size, m_per_seq, step, active_idx, n_active, delta_opt, dws, ctr, tau);
   } else {
     launch_k(select_active_kernel<float>, grid, kThreads, 0, st, 
         static_cast<const float*>(x_cur), static_cast<const float*>(x_prev), row_width, sh.block_size,
-        m_per_seq, step, active_idx, n_active, delta_opt, dws, ctr);
+        m_per_seq, step, active_idx, n_active, delta_opt, dws, ctr, tau);
   }
   return after_launch(c);
 }
@@ -173,11 +195,11 @@ extern "C" int32_t losa_select_active_static(const losa_shape_t* shape, const vo
   if (shape->dtype == LOSA_BF16) {
     losa::launch_k(losa::select_active_kernel<__nv_bfloat16>, grid, losa::kThreads, 0, st, 
         static_cast<const __nv_bfloat16*>(x_cur), static_cast<const __nv_bfloat16*>(x_prev), row_width,
-        shape->block_size, m_per_seq, step, active_idx, n_active, delta_opt, scratch->delta, scratch->counters);
+        shape->block_size, m_per_seq, step, active_idx, n_active, delta_opt, scratch->delta, scratch->counters, 0.0);
   } else {
     losa::launch_k(losa::select_active_kernel<float>, grid, losa::kThreads, 0, st, 
         static_cast<const float*>(x_cur), static_cast<const float*>(x_prev), row_width, shape->block_size,
-        m_per_seq, step, active_idx, n_active, delta_opt, scratch->delta, scratch->counters);
+        m_per_seq, step, active_idx, n_active, delta_opt, scratch->delta, scratch->counters, 0.0);
   }
   return cudaGetLastError() == cudaSuccess ? LOSA_OK : LOSA_ERR_CUDA;
 }

@@ -33,8 +33,9 @@ class LosaLayer:
     """
 
     def __init__(self, cfg, k_pages, v_pages, page_table, kv_len, mode="losa", device="cuda",
-                 share_pool_with: "LosaLayer | None" = None):
+                 share_pool_with: "LosaLayer | None" = None, tau: float = 0.0):
         self.cfg, self.mode, self.device = cfg, mode, device
+        self.tau = tau            # > 0: stage 1 keeps tokens until their Delta reach tau of the block's total
         N, Bk, Hq, Hkv, d = cfg.batch, cfg.block_size, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
         self.dtype = B.LOSA_BF16 if cfg.dtype == "bf16" else B.LOSA_F32
         td = B.torch_dtype(self.dtype)
@@ -83,7 +84,10 @@ class LosaLayer:
         m = None if self.mode == "naive" else m_per_seq
         xc, xp = (q, self.q_prev) if x_sel is None else x_sel
         row_width = xc.numel() // (cfg.batch * cfg.block_size)
-        B.losa_select_active(c, xc, xp, row_width, m, st, self.active_idx, self.n_active, self.delta)
+        if self.tau > 0.0 and self.mode == "losa":
+            B.losa_select_active_tau(c, xc, xp, row_width, self.tau, None, st, self.active_idx, self.n_active, self.delta)
+        else:
+            B.losa_select_active(c, xc, xp, row_width, m, st, self.active_idx, self.n_active, self.delta)
         B.losa_page_scores_topk(c, q, self.kv, self.active_idx, self.n_active, st, cfg.topk, self.topk_pages,
                                 self.topk_scores if want_scores else None)
         B.losa_page_union(c, self.topk_pages, self.active_idx, self.n_active, cfg.topk, self.kv_len, st,

@@ -104,7 +104,8 @@ class OracleLayer:
     attention applied to the whole block, Section 5.1 baselines); "dense": step counter pinned to
     0, i.e. dense prefix attention every step."""
 
-    def __init__(self, w, mode="losa"):
+    def __init__(self, w, mode="losa", tau=0.0):
+        self.tau = tau
         cfg = w.cfg
         self.w, self.cfg, self.mode = w, cfg, mode
         self.sh = oracle_shape_of(cfg)
@@ -130,7 +131,10 @@ class OracleLayer:
         step = np.zeros_like(self.step) if self.mode == "dense" else self.step
         m = None if self.mode == "naive" else inp.m_per_seq
         xc, xp = (inp.q, self.q_prev) if x_sel is None else x_sel
-        act, na, delta = orc.select_active(sh, xc, xp, m, step)
+        if self.tau > 0.0 and self.mode == "losa":
+            act, na, delta = orc.select_active_tau(sh, xc, xp, self.tau, None, step)
+        else:
+            act, na, delta = orc.select_active(sh, xc, xp, m, step)
         orc.page_scores_topk(sh, inp.q, self.kv, act, na, cfg.topk, step, topk_pages=self.topk)
         up, uc = orc.page_union(sh, self.topk, act, na, cfg.topk, self.kv_len, step)
         orc.sparse_prefix_attn(sh, inp.q, self.kv, act, na, up, uc, self.o_p, self.lse_p)
@@ -152,3 +156,17 @@ def delta_gap_ok(delta_row, m, rel=1e-3):
         return True
     a, b = d[m - 1], d[m]
     return a == b or (a - b) > rel * max(abs(a), abs(b))
+
+
+def tau_gap_ok(delta_row, m, tau, rel=1e-9):
+    """The threshold rule's decision is clear of rounding: the cumulative Delta of the first m ranked
+    tokens exceeds tau * total by a margin, and that of the first m - 1 stays below it by one."""
+    d = np.sort(np.asarray(delta_row, np.float64))[::-1]
+    total = d.sum()
+    if total == 0.0:
+        return m == 0
+    cum = np.cumsum(d)
+    thr = tau * total
+    hi_ok = m == d.size or m == 0 or cum[m - 1] - thr > rel * total or cum[m - 1] == thr
+    lo_ok = m <= 1 or thr - cum[m - 2] > rel * total
+    return bool(hi_ok and lo_ok)

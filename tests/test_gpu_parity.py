@@ -7,7 +7,7 @@ outputs within the stated tolerances: fp32 mode |a-b| <= 1e-5 * max(|b|, max|b_r
 import numpy as np
 import pytest
 
-from helpers import OracleLayer, delta_gap_ok
+from helpers import OracleLayer, delta_gap_ok, tau_gap_ok
 from paper_2604_12056_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -31,25 +31,28 @@ def assert_lse_close(got, want, what):
     assert (np.abs(got[~inf] - want[~inf]) <= 1e-3).all(), f"{what}: worst {np.abs(got[~inf] - want[~inf]).max():.3e}"
 
 
-def compare(snap, ref, cfg, what):
+def compare(snap, ref, cfg, what, tau=0.0):
     for key in ("act", "na", "topk", "up", "uc"):
         assert (snap[key] == ref[key]).all(), f"{what}: {key} differs"
     np.testing.assert_allclose(snap["delta"], ref["delta"], rtol=1e-5, atol=1e-12, err_msg=what)
     for s in range(cfg.batch):
         m = int(ref["na"][s])
-        assert delta_gap_ok(ref["delta"][s], m), f"{what}: selection-ambiguous Delta in sequence {s}"
+        if tau > 0.0 and m < cfg.block_size:
+            assert tau_gap_ok(ref["delta"][s], m, tau), f"{what}: threshold-ambiguous Delta in sequence {s}"
+        else:
+            assert delta_gap_ok(ref["delta"][s], m), f"{what}: selection-ambiguous Delta in sequence {s}"
     assert_close(snap["o_p"], ref["o_p"], cfg.dtype, what + " o_p")
     assert_lse_close(snap["lse_p"], ref["lse_p"], what + " lse_p")
     assert_close(snap["out"], ref["out"], cfg.dtype, what + " out")
     assert_lse_close(snap["lse"], ref["lse"], what + " lse")
 
 
-def run_blocks(cfg, modes=("losa",), m=None, n_blocks=1, pad_nan=True, want_scores=True, fused=False):
+def run_blocks(cfg, modes=("losa",), m=None, n_blocks=1, pad_nan=True, want_scores=True, fused=False, tau=0.0):
     """Runs n_blocks blocks through GPU and oracle in lock-step, comparing after every step."""
     from paper_2604_12056_b200.layer import LosaLayer, to_device
     w = wl.Workload(cfg, pad_nan=pad_nan)
-    gpu = {md: LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len, md) for md in modes}
-    ora = {md: OracleLayer(w, md) for md in modes}
+    gpu = {md: LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len, md, tau=tau) for md in modes}
+    ora = {md: OracleLayer(w, md, tau=tau) for md in modes}
     for md in modes:     # page summaries: exact min / max on both sides
         from paper_2604_12056_b200.layer import to_host
         P = [(int(L) + cfg.page_size - 1) // cfg.page_size for L in w.kv_len]
@@ -74,7 +77,7 @@ def run_blocks(cfg, modes=("losa",), m=None, n_blocks=1, pad_nan=True, want_scor
                 ref = ora[md].run_step(inp, finalize=last)
                 if fused:
                     snap["delta"] = ref["delta"]          # the whole-step call does not export Delta
-                compare(snap, ref, cfg, f"{cfg.name}/{md} block {b} step {t}")
+                compare(snap, ref, cfg, f"{cfg.name}/{md} block {b} step {t}", tau if md == "losa" else 0.0)
                 if want_scores and not fused and md == "losa" and t > 0:
                     sel = ref["topk"] >= 0
                     rows = np.zeros_like(sel)
@@ -131,6 +134,14 @@ def test_page_groups_of_the_tensor_core_kernel(g, d):
     cfg = wl.config("c2", n_q_heads=8, n_kv_heads=2, head_dim=d, page_size=g, kv_lens=(21 * g + 5, 9 * g, 128 + g),
                     block_size=16, steps=3, topk=6, m_active=3)
     run_blocks(cfg, modes=("losa", "dense"))
+
+
+@pytest.mark.parametrize("tau", [0.3, 0.5, 0.9])
+def test_threshold_pruning_rule_whole_blocks(tau):
+    # stage 1 keeps tokens until their Delta reach tau of the block's total; everything downstream
+    # follows the active set it produces (bf16 and fp32, two sequences)
+    run_blocks(wl.config("c2", kv_lens=(1500, 700), steps=4, block_size=16, topk=6), tau=tau)
+    run_blocks(wl.config("c1", kv_lens=(300, 180), steps=3), tau=tau)
 
 
 @pytest.mark.parametrize("name", ["p1", "p2"])
