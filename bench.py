@@ -7,10 +7,15 @@ One "step" is one layer-step: stages 1-6 of include/losa.h for one attention lay
 denoising step, issued through the whole-step entry point losa_denoise_step.  Steps cycle through whole denoising blocks of the workload (step 0 of a block is
 the dense first step, the others are LoSA steps).  Prints ONE JSON line.
 
-Timing: the layer-step is captured once in a CUDA graph and replayed; each step is bracketed by
-CUDA events on the launching stream; between steps, outside the timed region, the L2 is flushed by
-writing a 256 MiB buffer and then reading a second one (the read pass makes the cache write its
-dirty lines back, so that write-back traffic of the flush itself does not land in the timed step).  The time of K steps is the sum of the K event intervals; with several
+Timing: with one layer, the layer-step is captured once in a CUDA graph and replayed; each step is
+bracketed by CUDA events on the launching stream; between steps, outside the timed region, the L2
+is flushed by writing a 256 MiB buffer and then reading a second one (the read pass makes the cache
+write its dirty lines back, so that write-back traffic of the flush itself does not land in the
+timed step).  With several layers (the default), one denoising step of the whole model - the
+layers' steps in order, each on its own ~1 GiB KV pool, so nothing a step reads is left in L2 - is
+one CUDA graph; one event pair brackets each replay and a layer-step counts as 1/layers of it (when
+K and W are not multiples of the layer count, one graph per layer-step is replayed instead).
+The time of K steps is the sum of the event intervals; with several
 GPUs every rank runs its own replica of the workload (weak scaling, no data-path collective) and
 the maximum over ranks is reported.
 """
@@ -312,7 +317,55 @@ def run_ours(args, cfg0):
 
     state = {"launches": 0}
 
+    # With several layers, one denoising step of the whole model (all layers in order) is one CUDA
+    # graph, as a serving engine would capture it; the last step of a block also finalises each
+    # layer's block.  Timed per model step and reported per layer-step.
+    model_graphs = None
+    if L > 1:
+        model_graphs = []
+        for with_fin in (False, True):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for r in runs:
+                    r.layer.run_step_fused(r.q_s, r.k_s, r.v_s, r.m_s)
+                    if with_fin:
+                        r.layer.finalize_block(r.k_s, r.v_s)
+            model_graphs.append(g)
+        for r in runs:
+            r.layer.step.zero_()
+
+    def model_pass(first, count, record=None):
+        """Whole model steps (L layer-steps each) first .. first+count-1, one event pair per model step."""
+        evs, ts = [], []
+        log = torch.zeros((max(count, 1),), dtype=torch.int64, device=dev) if record is not None else None
+        for i0 in range(first, first + count, L):
+            b, t, _ = where(i0)
+            for r in runs:
+                r.load(b, t)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            model_graphs[1 if t == T - 1 else 0].replay()
+            e1.record()
+            evs.append((e0, e1))
+            state["launches"] += L * (launches_step + (launches_fin if t == T - 1 else 0))
+            for l, r in enumerate(runs):
+                if log is not None:
+                    log[i0 - first + l] = r.layer.union_count.sum()
+                ts.append(t)
+        torch.cuda.synchronize()
+        if record is not None:
+            record.extend(zip(ts, (int(x) for x in log.cpu().tolist())))
+        out = []
+        for a, b2 in evs:
+            out.extend([a.elapsed_time(b2) / L] * L)
+        return out
+
     def graph_pass(first, count, record=None):
+        if model_graphs is not None and first % L == 0 and count % L == 0:
+            return model_pass(first, count, record)
+        return layer_pass(first, count, record)
+
+    def layer_pass(first, count, record=None):
         """Layer-steps first .. first+count-1 in order, one CUDA-event pair per layer-step.  Nothing
         is read back inside the loop (the union sizes go to a device log), so the host runs ahead
         and the steps execute back to back as they would in a model."""
@@ -365,7 +418,9 @@ def run_ours(args, cfg0):
         "config": {"workload": workload_name(cfg0, L), "sequences_per_gpu": cfg.batch, "layers": L,
                    "step": "one layer-step = stages 1-6 for one layer and one denoising step; steps run in model order "
                            "(block, denoising step, layer); the last step of a block also appends the block to the cache",
-                   "launch": "CUDA graph replay of losa_denoise_step (stages 1-6 in one call)",
+                   "launch": ("CUDA graph replay of one denoising step of all layers (losa_denoise_step per layer, in order), "
+                              "timed per model step" if (L > 1 and args.warmup % L == 0 and args.steps % L == 0) else
+                              "CUDA graph replay of losa_denoise_step (stages 1-6 in one call), one graph per layer-step"),
                    "l2": ("flushed between steps, outside the timed region: 256 MiB write, then 256 MiB read so no dirty "
                           "lines remain") if use_flush else
                          ("inputs larger than L2: consecutive layer-steps read different per-layer KV pools "
