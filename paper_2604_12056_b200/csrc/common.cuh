@@ -105,6 +105,11 @@ inline void launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t sme
   (void)cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);   // the error, if any, is read by after_launch()
 }
 __device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel of the stream be scheduled now instead of when this grid has drained: its
+// CTAs take free resources, run their prologue and stop at their own grid_dep_wait() until this
+// grid has completed and its writes are visible.  Only for kernels whose whole grid is resident at
+// once and whose successor has a prologue worth hiding.
+__device__ __forceinline__ void grid_dep_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ void set_status(int32_t* status, int32_t code) { atomicCAS(status, 0, code); }
 

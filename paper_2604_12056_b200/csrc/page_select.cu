@@ -449,6 +449,7 @@ topk_select_kernel(const float* __restrict__ scores, const int32_t* __restrict__
                    const int32_t* __restrict__ step, int32_t* __restrict__ topk_pages,
                    float* __restrict__ topk_scores, int N, int B, int Hq, int g, int k, int score_stride,
                    int32_t* __restrict__ status) {
+  grid_dep_trigger();
   grid_dep_wait();
   // A CTA serves the active slots a = j, j + kSelSlots, ... of one (sequence, head): launching a CTA
   // costs about as much as an idle CTA's whole life, and most of the B slots are idle on most steps.
@@ -478,6 +479,7 @@ union_kernel(const int32_t* __restrict__ topk_pages, const int32_t* __restrict__
              const int32_t* __restrict__ step, int32_t* __restrict__ union_pages,
              int32_t* __restrict__ union_count, int B, int Hq, int Hkv, int g, int k, int Pmax,
              int32_t* __restrict__ status) {
+  grid_dep_trigger();                              // the stage-4 kernel sets up its barriers and tensor memory meanwhile
   grid_dep_wait();
   extern __shared__ uint32_t bitmap[];
   __shared__ int s_warp[kThreads / 32];

@@ -21,6 +21,7 @@ select_active_kernel(const T* __restrict__ x_cur, const T* __restrict__ x_prev, 
                      int32_t* __restrict__ active_idx, int32_t* __restrict__ n_active,
                      float* __restrict__ delta_opt, double* __restrict__ delta_ws,
                      unsigned int* __restrict__ counters, double tau) {
+  grid_dep_trigger();
   grid_dep_wait();
   const int i = blockIdx.x, s = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;

@@ -307,6 +307,7 @@ struct FinishParams {
 
 template <typename T, int D>
 __global__ void __launch_bounds__(256) attn_finish_kernel(AttnParams p, FinishParams f) {
+  grid_dep_trigger();
   grid_dep_wait();
   constexpr int C = D / 32;
   const int lane = threadIdx.x & 31;
