@@ -489,8 +489,8 @@ def run_ours(args, cfg0):
         r.layer.step.zero_()
     es = 2 if cfg.dtype == "bf16" else 4
     if L > 1:
-        # Consecutive layer-steps belong to different layers and are independent, so they alternate
-        # between two streams: the host->device copies of one step overlap the kernels of the other
+        # Consecutive layer-steps belong to different layers and are independent, so they rotate over
+        # a few streams: the host->device and device->host copies of some steps overlap the kernels of another
         # (steps of one layer stay on one stream, in order).  Every step still copies its own inputs
         # from pinned host memory and its output back; the host buffers of all steps are filled
         # before the clock starts, the clock stops after the last output has arrived.
@@ -500,14 +500,15 @@ def run_ours(args, cfg0):
             inp = runs[l].block_inputs(b)[t]
             steps.append((l, t, pin((N, Bk, Hq, d)).copy_(inp.q), pin((N, Bk, Hkv, d)).copy_(inp.k_blk),
                           pin((N, Bk, Hkv, d)).copy_(inp.v_blk), inp.m_per_seq.clone()))
-        streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+        n_str = next(n for n in (4, 3, 2, 1) if L % n == 0)     # a layer's steps stay on one stream
+        streams = [torch.cuda.Stream() for _ in range(n_str)]
         stage = [tuple(torch.empty_like(x) for x in (runs[0].q_s, runs[0].k_s, runs[0].v_s)) for _ in streams]
         h_out = [pin((N, Bk, Hq, d)) for _ in streams]
         torch.cuda.synchronize()
         D.barrier()
         t0 = time.perf_counter()
         for l, t, hq, hk, hv, m in steps:
-            lay, j = runs[l].layer, l % 2
+            lay, j = runs[l].layer, l % n_str
             dq, dk, dv = stage[j]
             buf = B.StepBuffersT(dq.data_ptr(), dk.data_ptr(), dv.data_ptr(), lay.out.data_ptr(),
                                  lay.active_idx.data_ptr(), lay.n_active.data_ptr(), lay.topk_pages.data_ptr(),
@@ -519,7 +520,7 @@ def run_ours(args, cfg0):
         torch.cuda.synchronize()
         host_t = [time.perf_counter() - t0]
         how = ("losa_denoise_step_host on pinned host q/k_blk/v_blk -> host out, eager launches; consecutive "
-               "layer-steps (different layers) alternate between two streams so that copies overlap kernels; "
+               f"layer-steps (different layers) rotate over {n_str} streams so that copies overlap kernels; "
                "host wall clock over all steps up to the last output's arrival")
     else:
         host_t = []
