@@ -274,6 +274,47 @@ void oracle_page_scores_topk(const oracle_shape_t* sh, const void* q, const orac
   }
 }
 
+/* ---------- Selector variant: one list per (token, KV head) ---------------------------------
+ * Section 2.3 calls the method independent of the selector.  With grouped-query attention the G
+ * heads of a KV head read the same pages, so this variant scores a page once per KV head: the
+ * pooled score is the largest of the G heads' upper bounds (each in the interface's fixed fp32
+ * order), the k best pages by (pooled score descending, page ascending) are chosen, and every
+ * head of the group receives that list.  With G = 1 it is oracle_page_scores_topk. */
+void oracle_page_scores_topk_pooled(const oracle_shape_t* sh, const void* q, const oracle_kv_t* kv,
+                                    const int32_t* active_idx, const int32_t* n_active,
+                                    const int32_t* step, int32_t k, int32_t* topk_pages,
+                                    float* topk_scores) {
+  const int B = sh->block_size, Hq = sh->n_q_heads, Hkv = sh->n_kv_heads, G = Hq / Hkv;
+  for (int s = 0; s < sh->batch; ++s) {
+    if (step && step[s] == 0) continue;
+    const int P = pages_of(kv->kv_len[s], sh->page_size);
+    const int work = n_active[s] * Hkv;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int w = 0; w < work; ++w) {
+      const int tok = active_idx[(int64_t)s * B + w / Hkv], kh = w % Hkv;
+      float* u = (float*)malloc(sizeof(float) * (size_t)(P > 0 ? P : 1));
+      scored_t* sc = (scored_t*)malloc(sizeof(scored_t) * (size_t)(P > 0 ? P : 1));
+      for (int gi = 0; gi < G; ++gi) {
+        oracle_page_scores_one(sh, q, kv, s, tok, kh * G + gi, u, NULL);
+        for (int p = 0; p < P; ++p) {
+          if (gi == 0 || u[p] > sc[p].u) sc[p].u = u[p];
+          sc[p].p = p;
+        }
+      }
+      qsort(sc, (size_t)P, sizeof(scored_t), cmp_scored);
+      for (int gi = 0; gi < G; ++gi) {
+        const int64_t o = (((int64_t)s * B + tok) * Hq + kh * G + gi) * k;
+        for (int j = 0; j < k; ++j) {
+          topk_pages[o + j] = (j < P) ? sc[j].p : -1;
+          if (topk_scores && j < P) topk_scores[o + j] = sc[j].u;
+        }
+      }
+      free(u);
+      free(sc);
+    }
+  }
+}
+
 /* ---------- Section 4.2 / 4.4: I = union over active tokens (and the G heads of a KV head) ---- */
 void oracle_page_union(const oracle_shape_t* sh, const int32_t* topk_pages,
                        const int32_t* active_idx, const int32_t* n_active, int32_t k,

@@ -13,8 +13,9 @@
  * Pins (tests/test_oracle_*.py): brute-force dense softmax attention when every token is active
  * and every page selected; LSE merge vs softmax over the concatenation; bit-exact reuse for stable
  * tokens; page-score upper-bound property and its reduction to exact top-k keys at page size 1;
- * union-size inequalities; invariance under physical page permutation.  No function here is
- * "parity unpinned".
+ * union-size inequalities; invariance under physical page permutation; the threshold rule and the
+ * pooled selector each by a worked example with exact arithmetic and a numpy re-derivation.  No
+ * function here is "parity unpinned".
  */
 #ifndef LOSA_ORACLE_H_
 #define LOSA_ORACLE_H_
@@ -59,6 +60,15 @@ void oracle_page_scores_topk(const oracle_shape_t* sh, const void* q, const orac
                              const int32_t* active_idx, const int32_t* n_active,
                              const int32_t* step, int32_t k, int32_t* topk_pages,
                              float* topk_scores);
+
+/* Selector variant for grouped-query attention: a page's pooled score is the largest of the upper
+ * bounds of the G heads of its KV head; one top-k list per (token, KV head), stored for every head
+ * of the group (same layout as above).  Not in the paper, which leaves the selector open
+ * (Section 2.3). */
+void oracle_page_scores_topk_pooled(const oracle_shape_t* sh, const void* q, const oracle_kv_t* kv,
+                                    const int32_t* active_idx, const int32_t* n_active,
+                                    const int32_t* step, int32_t k, int32_t* topk_pages,
+                                    float* topk_scores);
 
 /* Section 4.2 / 4.4: union per (sequence, KV head). */
 void oracle_page_union(const oracle_shape_t* sh, const int32_t* topk_pages,

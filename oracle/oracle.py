@@ -180,6 +180,24 @@ def page_scores_topk(sh: Shape, q, kv: KV, active_idx, n_active, k: int, step=No
     return topk_pages, topk_scores
 
 
+def page_scores_topk_pooled(sh: Shape, q, kv: KV, active_idx, n_active, k: int, step=None,
+                            topk_pages=None, topk_scores=None):
+    """Selector variant: one list per (token, KV head) from the largest of the G heads' bounds,
+    stored for every head of the group.  Same outputs as page_scores_topk."""
+    N, B, H = sh.batch, sh.block_size, sh.n_q_heads
+    if topk_pages is None:
+        topk_pages = np.full((N, B, H, k), -9, np.int32)
+    if topk_scores is None:
+        topk_scores = np.full((N, B, H, k), np.nan, np.float32)
+    st = None if step is None else np.ascontiguousarray(step, np.int32)
+    s, kk = sh.c(), kv.c()
+    lib().oracle_page_scores_topk_pooled(C.byref(s), _p(_chk(q, sh.elem, "q")), C.byref(kk),
+                                         _p(_chk(active_idx, np.int32, "active_idx")),
+                                         _p(_chk(n_active, np.int32, "n_active")), _p(st), C.c_int32(k),
+                                         _p(topk_pages), _p(topk_scores))
+    return topk_pages, topk_scores
+
+
 def page_union(sh: Shape, topk_pages, active_idx, n_active, k: int, kv_len, step=None):
     """Returns (union_pages [N,H_kv,P_max] int32, union_count [N,H_kv] int32)."""
     N, Hkv, P = sh.batch, sh.n_kv_heads, sh.max_pages_per_seq

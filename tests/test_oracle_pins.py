@@ -228,6 +228,75 @@ def test_fixed_order_fp32_score_matches_its_specification():
         assert np.float32(c[0] + np.float32(0.0)).tobytes() == u32[p].tobytes()
 
 
+# --- selector variant: one list per (token, KV head), pooled over the G heads (Section 2.3 leaves the selector open)
+def test_pooled_selector_worked_example():
+    # pages of one token, two heads sharing one KV head; q0 = e0, q1 = e1, keys (a_p, b_p, 0, ...):
+    # head 0 scores a_p, head 1 scores b_p, the pooled score is max(a_p, b_p) - all exact in fp32
+    pb = Problem(21, N=1, Hq=2, Hkv=1, d=16, B=1, g=1, kv_lens=(6,), extra_pages=0, shuffle=True)
+    keys = [(3, 0), (1, 5), (2, 2), (5, 1), (0, 4), (4, 4)]
+    pb.q[:] = 0
+    pb.q[0, 0, 0, 0] = 1.0
+    pb.q[0, 0, 1, 1] = 1.0
+    for p, (a, b) in enumerate(keys):
+        row = np.zeros(16, np.float32)
+        row[0], row[1] = a, b
+        pb.k_pages[pb.page_table[0, p], 0, 0] = row
+    orc.build_page_summaries(pb.sh, pb.kv)
+    act, na = np.array([[0]], np.int32), np.array([1], np.int32)
+    per_head, _ = orc.page_scores_topk(pb.sh, pb.q, pb.kv, act, na, 4)
+    assert per_head[0, 0, 0].tolist() == [3, 5, 0, 2]          # a_p: 5, 4, 3, 2
+    assert per_head[0, 0, 1].tolist() == [1, 4, 5, 2]          # b_p: 5, 4, 4 (tie: lower page first), 2
+    pooled, sc = orc.page_scores_topk_pooled(pb.sh, pb.q, pb.kv, act, na, 4)
+    for h in range(2):
+        assert pooled[0, 0, h].tolist() == [1, 3, 4, 5]        # max: 5, 5 (pages 1, 3), 4, 4 (pages 4, 5)
+        assert sc[0, 0, h].tolist() == [5.0, 5.0, 4.0, 4.0]
+    wide, _ = orc.page_scores_topk_pooled(pb.sh, pb.q, pb.kv, act, na, 8)
+    assert wide[0, 0, 1].tolist() == [1, 3, 4, 5, 0, 2, -1, -1]
+
+
+def test_pooled_selector_brute_force_and_invariants():
+    pb = Problem(22, N=2, Hq=8, Hkv=2, d=32, B=4, g=4, kv_lens=(90, 37))
+    sh = pb.sh
+    orc.build_page_summaries(sh, pb.kv)
+    act = np.array([[1, 3, -1, -1], [0, 2, 3, -1]], np.int32)
+    na = np.array([2, 3], np.int32)
+    k = 5
+    pooled, sc = orc.page_scores_topk_pooled(sh, pb.q, pb.kv, act, na, k)
+    per_head, _ = orc.page_scores_topk(sh, pb.q, pb.kv, act, na, k)
+    G = 4
+    for s in range(2):
+        P = pb.pages(s)
+        for tok in act[s, :na[s]]:
+            for kh in range(2):
+                rows = np.stack([orc.page_scores_one(sh, pb.q, pb.kv, s, int(tok), kh * G + gi)[0] for gi in range(G)])
+                best = rows.max(axis=0)                                   # fp32 values, exact maximum
+                want = np.argsort(-best, kind="stable")[:k]                # ties: lower page first
+                for gi in range(G):
+                    assert pooled[s, tok, kh * G + gi].tolist() == want.tolist()
+                    assert sc[s, tok, kh * G + gi].tobytes() == best[want].tobytes()
+                # every pooled page is in the list of the head that attains its score (no ties in this data)
+                lists = {int(p) for gi in range(G) for p in per_head[s, tok, kh * G + gi]}
+                assert set(want.tolist()) <= lists
+    # untouched rows keep the fill value
+    assert (pooled[0, 0] == -9).all() and (pooled[1, 1] == -9).all()
+    # the union can only shrink, and is bounded by (active tokens) * k per KV head
+    up_h, uc_h = orc.page_union(sh, per_head, act, na, k, pb.kv_len)
+    up_p, uc_p = orc.page_union(sh, pooled, act, na, k, pb.kv_len)
+    for s in range(2):
+        for kh in range(2):
+            a, b = set(up_p[s, kh, :uc_p[s, kh]].tolist()), set(up_h[s, kh, :uc_h[s, kh]].tolist())
+            assert a <= b and k <= len(a) <= na[s] * k
+
+
+def test_pooled_selector_without_grouping_is_the_per_head_selector():
+    pb = Problem(23, N=1, Hq=3, Hkv=3, d=16, B=3, g=2, kv_lens=(33,))
+    orc.build_page_summaries(pb.sh, pb.kv)
+    act, na = np.array([[0, 2, -1]], np.int32), np.array([2], np.int32)
+    a, sa = orc.page_scores_topk(pb.sh, pb.q, pb.kv, act, na, 6)
+    b, sb = orc.page_scores_topk_pooled(pb.sh, pb.q, pb.kv, act, na, 6)
+    assert (a == b).all() and sa.tobytes() == sb.tobytes()
+
+
 # --- I4: union-size inequalities (Section 4.4; worst case of Section 3.1) --------------------------
 def test_union_inequalities_and_subset():
     pb = Problem(10, N=2, Hq=4, Hkv=2, d=16, B=8, g=4, kv_lens=(90, 57))
