@@ -58,6 +58,8 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c5", choices=["c1", "c2", "c3", "c4", "c5", "p1", "p2"])
     ap.add_argument("--topk", type=int, default=0, help="override the page budget per query (pages)")
+    ap.add_argument("--pooled", action="store_true",
+                    help="selector variant: one page list per (token, KV head) instead of one per query head")
     ap.add_argument("--layers", type=int, default=0, help="attention layers (default: 36 for c5, else 1)")
     ap.add_argument("--active-frac", type=float, default=None, help="override the active fraction")
     ap.add_argument("--no-extras", action="store_true", help="skip baselines, stage breakdown, cpu baseline")
@@ -229,12 +231,13 @@ class LayerRun:
     """One attention layer of the workload on the device: its own seeded pool, LoSA cache, static
     input buffers and two CUDA graphs (the whole-step call; block finalisation)."""
 
-    def __init__(self, cfg, rank, layer, dev):
+    def __init__(self, cfg, rank, layer, dev, pooled=False):
         import torch
         from paper_2604_12056_b200.layer import LosaLayer
         self.torch, self.cfg = torch, cfg
         self.w = wl.DeviceWorkload(cfg, replica=rank, layer=layer, device=dev)
-        self.layer = LosaLayer(cfg, self.w.k_pages, self.w.v_pages, self.w.page_table, self.w.kv_len, "losa", dev)
+        self.layer = LosaLayer(cfg, self.w.k_pages, self.w.v_pages, self.w.page_table, self.w.kv_len, "losa", dev,
+                               pooled=pooled)
         self.inputs = {}                       # block -> list of DeviceStepInputs (current and previous block)
         self.next_block = 0
         first = self.block_inputs(0)[0]
@@ -298,7 +301,7 @@ def run_ours(args, cfg0):
         return (n + per_block - 1) // per_block
     total_blocks = blocks_for(args.warmup + args.steps) + blocks_for(n_prof) + blocks_for(n_e2e) + 2
     cfg = wl.config(cfg0.name, n_blocks=total_blocks, m_active=cfg0.m_active, beta_active=cfg0.beta_active, topk=cfg0.topk)
-    runs = [LayerRun(cfg, D.replica_of(rank), l, dev) for l in range(L)]
+    runs = [LayerRun(cfg, D.replica_of(rank), l, dev, pooled=args.pooled) for l in range(L)]
     launches_step = launches_fin = 0
     for r in runs:
         launches_step, launches_fin = r.capture()
@@ -415,7 +418,8 @@ def run_ours(args, cfg0):
         "metric": METRIC, "value": ms_per_step * 1e3, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-        "config": {"workload": workload_name(cfg0, L), "sequences_per_gpu": cfg.batch, "layers": L,
+        "config": {"workload": workload_name(cfg0, L) + (", pooled selector (one page list per token and KV head)" if args.pooled else ""),
+                   "sequences_per_gpu": cfg.batch, "layers": L,
                    "step": "one layer-step = stages 1-6 for one layer and one denoising step; steps run in model order "
                            "(block, denoising step, layer); the last step of a block also appends the block to the cache",
                    "launch": ("CUDA graph replay of one denoising step of all layers (losa_denoise_step per layer, in order), "

@@ -212,6 +212,24 @@ int32_t losa_page_scores_topk(losa_ctx* ctx, const void* q, const losa_kv_t* kv,
                               const int32_t* step, int32_t k, int32_t* topk_pages,
                               float* topk_scores_opt, void* stream);
 
+/* Stage 2, pooled selector — one list per (token, KV head) instead of one per query head.  The
+ *   paper leaves the selector open (Section 2.3); with grouped-query attention the G heads of a KV
+ *   head read the same pages, so this variant scores a page once per KV head: the pooled score is
+ *   the largest of the G heads' U(p) (each evaluated exactly as above), the min(k, P_s) pages are
+ *   taken by (pooled score descending, page ascending), and the list is stored for every head of
+ *   the group, so topk_pages / topk_scores_opt keep the layout above and stage 3 is unchanged.  The
+ *   union of a KV head then holds at most n_active * k pages instead of n_active * G * k.  With
+ *   G = 1 the result is that of losa_page_scores_topk.  Same arguments and errors. */
+int32_t losa_page_scores_topk_pooled(losa_ctx* ctx, const void* q, const losa_kv_t* kv,
+                                     const int32_t* active_idx, const int32_t* n_active,
+                                     const int32_t* step, int32_t k, int32_t* topk_pages,
+                                     float* topk_scores_opt, void* stream);
+
+/* Selector used by losa_denoise_step / losa_denoise_step_host on this context: 0 (default) = one
+ *   list per query head, non-zero = the pooled selector.  Host-side switch; takes effect for calls
+ *   issued after it returns. */
+int32_t losa_set_pooled_selection(losa_ctx* ctx, int32_t on);
+
 /* Stage 3 — union of the selections (Section 4.2, Section 4.4).
  *   union_pages [N, H_kv, P_max] int32 out: for each sequence and KV head, the distinct logical
  *       pages selected by any active token through any of the G query heads of that KV head,

@@ -29,7 +29,8 @@ EXPORTS = [
     "losa_page_union", "losa_sparse_prefix_attn", "losa_block_attn_merge",
     "losa_update_prefix_cache", "losa_build_page_summaries", "losa_denoise_step_host",
     "losa_profile_stage4", "losa_stage4_last_ms", "losa_select_active_static",
-    "losa_denoise_step", "losa_select_active_tau",
+    "losa_denoise_step", "losa_select_active_tau", "losa_page_scores_topk_pooled",
+    "losa_set_pooled_selection",
 ]
 
 
@@ -156,6 +157,9 @@ class Context:
     def launch_count(self) -> int:
         return int(lib().losa_launch_count(self._h))
 
+    def set_pooled_selection(self, on: bool):
+        self._check("losa_set_pooled_selection", lib().losa_set_pooled_selection(self._h, C.c_int32(1 if on else 0)))
+
     def profile_stage4(self, enable: bool):
         self._check("losa_profile_stage4", lib().losa_profile_stage4(self._h, C.c_int32(1 if enable else 0)))
 
@@ -195,6 +199,12 @@ def losa_select_active_static(shape: ShapeT, x_cur, x_prev, row_width, m_per_seq
 
 def losa_page_scores_topk(ctx, q, kv, active_idx, n_active, step, k, topk_pages, topk_scores_opt=None):
     ctx._check("losa_page_scores_topk", lib().losa_page_scores_topk(
+        ctx._h, _ptr(q), C.byref(kv), _ptr(active_idx), _ptr(n_active), _ptr(step), C.c_int32(k),
+        _ptr(topk_pages), _ptr(topk_scores_opt), _stream()))
+
+
+def losa_page_scores_topk_pooled(ctx, q, kv, active_idx, n_active, step, k, topk_pages, topk_scores_opt=None):
+    ctx._check("losa_page_scores_topk_pooled", lib().losa_page_scores_topk_pooled(
         ctx._h, _ptr(q), C.byref(kv), _ptr(active_idx), _ptr(n_active), _ptr(step), C.c_int32(k),
         _ptr(topk_pages), _ptr(topk_scores_opt), _stream()))
 

@@ -188,6 +188,22 @@ int32_t losa_page_scores_topk(losa_ctx* ctx, const void* q, const losa_kv_t* kv,
   return launch_page_scores_topk(ctx, q, kv, active_idx, n_active, step, k, topk_pages, topk_scores_opt, as_stream(stream));
 }
 
+int32_t losa_page_scores_topk_pooled(losa_ctx* ctx, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
+                                     const int32_t* n_active, const int32_t* step, int32_t k, int32_t* topk_pages,
+                                     float* topk_scores_opt, void* stream) {
+  if (!ctx || !q || !active_idx || !n_active || !topk_pages || k < 1) return LOSA_ERR_INVALID_ARG;
+  int32_t rc = check_kv(ctx, kv, true);
+  if (rc != LOSA_OK) return rc;
+  if (!aligned16(q)) return LOSA_ERR_UNSUPPORTED;
+  return launch_page_scores_topk(ctx, q, kv, active_idx, n_active, step, k, topk_pages, topk_scores_opt, as_stream(stream), true);
+}
+
+int32_t losa_set_pooled_selection(losa_ctx* ctx, int32_t on) {
+  if (!ctx) return LOSA_ERR_INVALID_ARG;
+  ctx->pooled_selection = on ? 1 : 0;
+  return LOSA_OK;
+}
+
 int32_t losa_page_union(losa_ctx* ctx, const int32_t* topk_pages, const int32_t* active_idx,
                         const int32_t* n_active, int32_t k, const int32_t* kv_len, const int32_t* step,
                         int32_t* union_pages, int32_t* union_count, void* stream) {
@@ -266,7 +282,7 @@ int32_t losa_denoise_step(losa_ctx* ctx, const void* q, const void* k_blk, const
   LOSA_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_join, ctx->side_stream));
   rc = launch_select_active(ctx, q, state->q_prev, sh.n_q_heads * sh.head_dim, m_per_seq, state->step,
                             buf->active_idx, buf->n_active, nullptr, st);
-  if (rc == LOSA_OK) rc = launch_page_scores_topk(ctx, q, kv, buf->active_idx, buf->n_active, state->step, k, buf->topk_pages, nullptr, st);
+  if (rc == LOSA_OK) rc = launch_page_scores_topk(ctx, q, kv, buf->active_idx, buf->n_active, state->step, k, buf->topk_pages, nullptr, st, ctx->pooled_selection != 0);
   if (rc == LOSA_OK) rc = launch_page_union(ctx, buf->topk_pages, buf->active_idx, buf->n_active, k, kv->kv_len, state->step, buf->union_pages, buf->union_count, st);
   if (rc == LOSA_OK) rc = launch_sparse_prefix_attn(ctx, q, kv, buf->active_idx, buf->n_active, buf->union_pages, buf->union_count, state, st, true);
   if (rc != LOSA_OK) return rc;

@@ -56,6 +56,8 @@ struct losa_ctx {
   // second stream and fork/join events of the whole-step path (created on first use)
   cudaStream_t side_stream;
   cudaEvent_t ev_fork, ev_join;
+  // selector of the whole-step path: 0 = one list per query head, 1 = pooled over the heads of a KV head
+  int32_t pooled_selection;
   // optional timing of the stage-4 main kernel
   int32_t profile;
   cudaEvent_t ev_begin, ev_end;

@@ -12,7 +12,7 @@ int32_t launch_select_active(losa_ctx* c, const void* x_cur, const void* x_prev,
 int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
                                 const int32_t* active_idx, const int32_t* n_active,
                                 const int32_t* step, int32_t k, int32_t* topk_pages,
-                                float* topk_scores_opt, cudaStream_t st);
+                                float* topk_scores_opt, cudaStream_t st, bool pooled = false);
 
 int32_t launch_page_union(losa_ctx* c, const int32_t* topk_pages, const int32_t* active_idx,
                           const int32_t* n_active, int32_t k, const int32_t* kv_len,

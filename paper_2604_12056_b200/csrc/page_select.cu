@@ -225,6 +225,20 @@ page_scores_kernel(const T* __restrict__ q, const T* __restrict__ kmin, const T*
   }
 }
 
+// One score row, or (pooled selector) the element-wise maximum of the `g` consecutive rows of a KV
+// head's query heads.
+template <bool POOLED>
+struct RowView {
+  const float* base;
+  int g, stride;
+  __device__ __forceinline__ float operator[](int p) const {
+    float v = base[p];
+    if (POOLED)
+      for (int gi = 1; gi < g; ++gi) v = fmaxf(v, base[static_cast<size_t>(gi) * stride + p]);
+    return v;
+  }
+};
+
 __device__ __forceinline__ uint32_t order_bits(float x) {
   const uint32_t b = __float_as_uint(x);
   return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
@@ -237,11 +251,11 @@ __global__ void __launch_bounds__(kThreads)
 topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ kv_len,
             const int32_t* __restrict__ active_idx, const int32_t* __restrict__ n_active,
             const int32_t* __restrict__ step, int32_t* __restrict__ topk_pages,
-            float* __restrict__ topk_scores, int B, int Hq, int g, int k, int score_stride,
+            float* __restrict__ topk_scores, int B, int Hq, int g, int k, int score_stride, int pool,
             int32_t* __restrict__ status) {
   grid_dep_wait();
   extern __shared__ __align__(16) unsigned long long keys[];
-  const int h = blockIdx.x, a = blockIdx.y, s = blockIdx.z;
+  const int h = blockIdx.x * pool, a = blockIdx.y, s = blockIdx.z;   // pooled: first head of the KV head
   if (step && step[s] == 0) return;
   int na = n_active[s];
   na = na > B ? B : na;
@@ -252,7 +266,7 @@ topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ kv_len
   const int tid = threadIdx.x;
   int n = 2;
   while (n < P) n <<= 1;
-  const float* sc = scores + ((static_cast<size_t>(s) * B + a) * Hq + h) * score_stride;
+  const RowView<true> sc{scores + ((static_cast<size_t>(s) * B + a) * Hq + h) * score_stride, pool, score_stride};
   for (int p = tid; p < n; p += kThreads)
     keys[p] = (p < P) ? ((static_cast<unsigned long long>(order_bits(sc[p])) << 32) |
                          static_cast<unsigned long long>(0xffffffffu - static_cast<uint32_t>(p)))
@@ -271,14 +285,16 @@ topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ kv_len
       __syncthreads();
     }
   }
-  const size_t o = ((static_cast<size_t>(s) * B + tok) * Hq + h) * k;
-  for (int j = tid; j < k; j += kThreads) {
-    if (j < P) {
-      const unsigned long long key = keys[j];
-      topk_pages[o + j] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(key));
-      if (topk_scores) topk_scores[o + j] = unorder_bits(static_cast<uint32_t>(key >> 32));
-    } else {
-      topk_pages[o + j] = -1;
+  for (int gi = 0; gi < pool; ++gi) {                 // pooled: every head of the group gets the list
+    const size_t o = ((static_cast<size_t>(s) * B + tok) * Hq + h + gi) * k;
+    for (int j = tid; j < k; j += kThreads) {
+      if (j < P) {
+        const unsigned long long key = keys[j];
+        topk_pages[o + j] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(key));
+        if (topk_scores) topk_scores[o + j] = unorder_bits(static_cast<uint32_t>(key >> 32));
+      } else {
+        topk_pages[o + j] = -1;
+      }
     }
   }
 }
@@ -304,8 +320,8 @@ constexpr int kSelThreads = 128;
 constexpr int kSelPerThread = 8;
 constexpr int kSelSlots = 8;        // CTAs per (sequence, head): active slots are dealt out round-robin
 
-template <bool CACHED, typename F>
-__device__ __forceinline__ void for_each_key(const uint32_t (&cache)[kSelPerThread], const float* __restrict__ row,
+template <bool CACHED, typename Row, typename F>
+__device__ __forceinline__ void for_each_key(const uint32_t (&cache)[kSelPerThread], const Row& row,
                                              int P, int tid, F&& f) {
   if (CACHED) {
 #pragma unroll
@@ -318,9 +334,9 @@ __device__ __forceinline__ void for_each_key(const uint32_t (&cache)[kSelPerThre
   }
 }
 
-template <bool CACHED>
-__device__ __forceinline__ void topk_select_body(const float* __restrict__ row, int P, int kk, int k,
-                                                 int32_t* out_pages, float* out_scores) {
+template <bool CACHED, typename Row>
+__device__ __forceinline__ void topk_select_body(const Row& row, int P, int kk, int k,
+                                                 int32_t* out_pages, float* out_scores, int n_out) {
   __shared__ unsigned long long cand[kSelCap];
   __shared__ int hist[kSelBins];
   __shared__ uint32_t s_red[2][kSelThreads / 32];
@@ -335,7 +351,7 @@ __device__ __forceinline__ void topk_select_body(const float* __restrict__ row, 
     }
   }
   uint32_t lo = 0xffffffffu, hi = 0u;
-  for_each_key<CACHED>(cache, row, P, tid, [&](uint32_t ob, int) { lo = min(lo, ob); hi = max(hi, ob); });
+  for_each_key<CACHED, Row>(cache, row, P, tid, [&](uint32_t ob, int) { lo = min(lo, ob); hi = max(hi, ob); });
   lo = __reduce_min_sync(0xffffffffu, lo);
   hi = __reduce_max_sync(0xffffffffu, hi);
   if (lane == 0) { s_red[0][warp] = lo; s_red[1][warp] = hi; }
@@ -369,7 +385,7 @@ __device__ __forceinline__ void topk_select_body(const float* __restrict__ row, 
     const int shift = width > 8 ? width - 8 : 0;      // (ob - lo) >> shift is in [0, 255]
     for (int b = tid; b < kSelBins; b += kSelThreads) hist[b] = 0;
     __syncthreads();
-    for_each_key<CACHED>(cache, row, P, tid, [&](uint32_t ob, int) {
+    for_each_key<CACHED, Row>(cache, row, P, tid, [&](uint32_t ob, int) {
       if (ob >= lo && ob <= hi) atomicAdd(&hist[(ob - lo) >> shift], 1);
     });
     __syncthreads();
@@ -400,7 +416,7 @@ __device__ __forceinline__ void topk_select_body(const float* __restrict__ row, 
     __syncthreads();                                   // everyone has read s_ncand before it moves
     // take the keys above the threshold bin (and, when finishing, the threshold bin itself); the
     // order inside cand does not matter: it is sorted below
-    for_each_key<CACHED>(cache, row, P, tid, [&](uint32_t ob, int p) {
+    for_each_key<CACHED, Row>(cache, row, P, tid, [&](uint32_t ob, int p) {
       if (ob >= lo && ob <= hi) {
         const int bin = static_cast<int>((ob - lo) >> shift);
         if (bin > bstar || (finish && bin == bstar)) cand[atomicAdd(&s_ncand, 1)] = make_key(ob, p);
@@ -432,29 +448,33 @@ __device__ __forceinline__ void topk_select_body(const float* __restrict__ row, 
       __syncthreads();
     }
   }
-  for (int j = tid; j < k; j += kSelThreads) {
-    if (j < kk) {
-      const unsigned long long key = cand[j];
-      out_pages[j] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(key));
-      if (out_scores) out_scores[j] = unorder_bits(static_cast<uint32_t>(key >> 32));
-    } else {
-      out_pages[j] = -1;
+  for (int gi = 0; gi < n_out; ++gi) {               // pooled: the list goes to every head of the group
+    for (int j = tid; j < k; j += kSelThreads) {
+      if (j < kk) {
+        const unsigned long long key = cand[j];
+        out_pages[gi * k + j] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(key));
+        if (out_scores) out_scores[gi * k + j] = unorder_bits(static_cast<uint32_t>(key >> 32));
+      } else {
+        out_pages[gi * k + j] = -1;
+      }
     }
   }
 }
 
+template <bool POOLED>
 __global__ void __launch_bounds__(kSelThreads)
-topk_select_kernel(const float* __restrict__ scores, const int32_t* __restrict__ kv_len,
+topk_select_kernel(float* __restrict__ scores, const int32_t* __restrict__ kv_len,
                    const int32_t* __restrict__ active_idx, const int32_t* __restrict__ n_active,
                    const int32_t* __restrict__ step, int32_t* __restrict__ topk_pages,
-                   float* __restrict__ topk_scores, int N, int B, int Hq, int g, int k, int score_stride,
+                   float* __restrict__ topk_scores, int N, int B, int Hq, int g, int k, int score_stride, int pool,
                    int32_t* __restrict__ status) {
   grid_dep_trigger();
   grid_dep_wait();
   // A CTA serves the active slots a = j, j + kSelSlots, ... of one (sequence, head): launching a CTA
   // costs about as much as an idle CTA's whole life, and most of the B slots are idle on most steps.
-  const int qid = blockIdx.x;
-  const int h = qid % Hq, s = (qid / Hq) % N, j = qid / (Hq * N);
+  // pool > 1 (pooled selector): one list per KV head from the maximum of its `pool` heads' rows
+  const int qid = blockIdx.x, Hl = Hq / pool;
+  const int h = (qid % Hl) * pool, s = (qid / Hl) % N, j = qid / (Hl * N);
   if (step && step[s] == 0) return;
   int na = n_active[s];
   na = na > B ? B : na;
@@ -463,12 +483,29 @@ topk_select_kernel(const float* __restrict__ scores, const int32_t* __restrict__
   for (int a = j; a < na; a += kSelSlots) {
     const int tok = active_idx[s * B + a];
     if (tok < 0 || tok >= B) { if (threadIdx.x == 0) set_status(status, LOSA_ERR_BOUNDS); continue; }
-    const float* row = scores + ((static_cast<size_t>(s) * B + a) * Hq + h) * score_stride;
+    RowView<POOLED> row{scores + ((static_cast<size_t>(s) * B + a) * Hq + h) * score_stride, pool, score_stride};
     const size_t o = ((static_cast<size_t>(s) * B + tok) * Hq + h) * k;
-    if (P <= kSelThreads * kSelPerThread)
-      topk_select_body<true>(row, P, kk, k, topk_pages + o, topk_scores ? topk_scores + o : nullptr);
-    else
-      topk_select_body<false>(row, P, kk, k, topk_pages + o, topk_scores ? topk_scores + o : nullptr);
+    if (P <= kSelThreads * kSelPerThread) {
+      topk_select_body<true>(row, P, kk, k, topk_pages + o, topk_scores ? topk_scores + o : nullptr, pool);
+    } else {
+      if (POOLED && pool > 1) {
+        // the selection reads the row several times: pool once, into the group's first row (the
+        // score rows are scratch and this CTA is the only reader of these)
+        float* first = scores + ((static_cast<size_t>(s) * B + a) * Hq + h) * score_stride;
+        constexpr int U = 4;                                   // pages per thread whose loads are in flight together
+        for (int p0 = threadIdx.x; p0 < P; p0 += kSelThreads * U) {
+          float v[U];
+#pragma unroll
+          for (int u = 0; u < U; ++u) v[u] = p0 + u * kSelThreads < P ? row[p0 + u * kSelThreads] : 0.f;
+#pragma unroll
+          for (int u = 0; u < U; ++u)
+            if (p0 + u * kSelThreads < P) first[p0 + u * kSelThreads] = v[u];
+        }
+        __syncthreads();
+        row.g = 1;
+      }
+      topk_select_body<false>(row, P, kk, k, topk_pages + o, topk_scores ? topk_scores + o : nullptr, pool);
+    }
     __syncthreads();                                 // the shared state is reused by the next slot
   }
 }
@@ -574,9 +611,10 @@ int32_t topk_max_sortable(const losa_ctx* c) {
 int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
                                 const int32_t* active_idx, const int32_t* n_active,
                                 const int32_t* step, int32_t k, int32_t* topk_pages,
-                                float* topk_scores_opt, cudaStream_t st) {
+                                float* topk_scores_opt, cudaStream_t st, bool pooled) {
   const losa_shape_t& sh = c->shape;
   if (sh.max_pages_per_seq == 0) return LOSA_OK;
+  const int pool = pooled ? sh.n_q_heads / sh.n_kv_heads : 1;
   const bool bf = sh.dtype == LOSA_BF16;
   if (bf && sh.head_dim == 128) launch_scores<__nv_bfloat16, 128>(c, q, kv, active_idx, n_active, step, st);
   else if (bf) launch_scores<__nv_bfloat16, 64>(c, q, kv, active_idx, n_active, step, st);
@@ -585,22 +623,27 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
   int32_t rc = after_launch(c);
   if (rc != LOSA_OK) return rc;
 
-  const float* sc = reinterpret_cast<const float*>(c->ws + c->lay.scores);
+  float* sc = reinterpret_cast<float*>(c->ws + c->lay.scores);
   if (k <= kSelCap) {
-    const int queries = sh.batch * std::min<int>(sh.block_size, kSelSlots) * sh.n_q_heads;
-    launch_k(topk_select_kernel, queries, kSelThreads, 0, st, 
-        sc, kv->kv_len, active_idx, n_active, step, topk_pages, topk_scores_opt, sh.batch, sh.block_size,
-        sh.n_q_heads, sh.page_size, k, c->lay.score_stride, status_ptr(c));
+    const int queries = sh.batch * std::min<int>(sh.block_size, kSelSlots) * (sh.n_q_heads / pool);
+    if (pool > 1)
+      launch_k(topk_select_kernel<true>, queries, kSelThreads, 0, st,
+          sc, kv->kv_len, active_idx, n_active, step, topk_pages, topk_scores_opt, sh.batch, sh.block_size,
+          sh.n_q_heads, sh.page_size, k, c->lay.score_stride, pool, status_ptr(c));
+    else
+      launch_k(topk_select_kernel<false>, queries, kSelThreads, 0, st,
+          sc, kv->kv_len, active_idx, n_active, step, topk_pages, topk_scores_opt, sh.batch, sh.block_size,
+          sh.n_q_heads, sh.page_size, k, c->lay.score_stride, 1, status_ptr(c));
     return after_launch(c);
   }
   // budgets beyond what one warp can sort: whole-list bitonic sort, one CTA per query
   const size_t smem = static_cast<size_t>(pow2_at_least(sh.max_pages_per_seq)) * sizeof(unsigned long long);
   if (smem > 48 * 1024)
     LOSA_CUDA_TRY(c, cudaFuncSetAttribute(topk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-  dim3 grid(sh.n_q_heads, sh.block_size, sh.batch);
+  dim3 grid(sh.n_q_heads / pool, sh.block_size, sh.batch);
   launch_k(topk_kernel, grid, kThreads, smem, st, sc, kv->kv_len, active_idx, n_active, step, topk_pages,
                                             topk_scores_opt, sh.block_size, sh.n_q_heads, sh.page_size,
-                                            k, c->lay.score_stride, status_ptr(c));
+                                            k, c->lay.score_stride, pool, status_ptr(c));
   return after_launch(c);
 }
 

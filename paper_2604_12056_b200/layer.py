@@ -33,14 +33,17 @@ class LosaLayer:
     """
 
     def __init__(self, cfg, k_pages, v_pages, page_table, kv_len, mode="losa", device="cuda",
-                 share_pool_with: "LosaLayer | None" = None, tau: float = 0.0):
+                 share_pool_with: "LosaLayer | None" = None, tau: float = 0.0, pooled: bool = False):
         self.cfg, self.mode, self.device = cfg, mode, device
         self.tau = tau            # > 0: stage 1 keeps tokens until their Delta reach tau of the block's total
+        self.pooled = pooled      # stage 2 keeps one page list per (token, KV head) instead of one per query head
         N, Bk, Hq, Hkv, d = cfg.batch, cfg.block_size, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
         self.dtype = B.LOSA_BF16 if cfg.dtype == "bf16" else B.LOSA_F32
         td = B.torch_dtype(self.dtype)
         Pmax = cfg.max_pages_per_seq
         self.ctx = B.Context(N, Hq, Hkv, d, Bk, cfg.page_size, Pmax, self.dtype, cfg.sm_scale, device)
+        if pooled:
+            self.ctx.set_pooled_selection(True)
         if share_pool_with is not None:
             o = share_pool_with
             self.k_pages, self.v_pages, self.kmin, self.kmax = o.k_pages, o.v_pages, o.kmin, o.kmax
@@ -88,8 +91,9 @@ class LosaLayer:
             B.losa_select_active_tau(c, xc, xp, row_width, self.tau, None, st, self.active_idx, self.n_active, self.delta)
         else:
             B.losa_select_active(c, xc, xp, row_width, m, st, self.active_idx, self.n_active, self.delta)
-        B.losa_page_scores_topk(c, q, self.kv, self.active_idx, self.n_active, st, cfg.topk, self.topk_pages,
-                                self.topk_scores if want_scores else None)
+        scores_topk = B.losa_page_scores_topk_pooled if self.pooled else B.losa_page_scores_topk
+        scores_topk(c, q, self.kv, self.active_idx, self.n_active, st, cfg.topk, self.topk_pages,
+                    self.topk_scores if want_scores else None)
         B.losa_page_union(c, self.topk_pages, self.active_idx, self.n_active, cfg.topk, self.kv_len, st,
                           self.union_pages, self.union_count)
         B.losa_sparse_prefix_attn(c, q, self.kv, self.active_idx, self.n_active, self.union_pages,

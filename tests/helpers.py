@@ -104,8 +104,9 @@ class OracleLayer:
     attention applied to the whole block, Section 5.1 baselines); "dense": step counter pinned to
     0, i.e. dense prefix attention every step."""
 
-    def __init__(self, w, mode="losa", tau=0.0):
+    def __init__(self, w, mode="losa", tau=0.0, pooled=False):
         self.tau = tau
+        self.pooled = pooled
         cfg = w.cfg
         self.w, self.cfg, self.mode = w, cfg, mode
         self.sh = oracle_shape_of(cfg)
@@ -135,7 +136,8 @@ class OracleLayer:
             act, na, delta = orc.select_active_tau(sh, xc, xp, self.tau, None, step)
         else:
             act, na, delta = orc.select_active(sh, xc, xp, m, step)
-        orc.page_scores_topk(sh, inp.q, self.kv, act, na, cfg.topk, step, topk_pages=self.topk)
+        scores_topk = orc.page_scores_topk_pooled if self.pooled else orc.page_scores_topk
+        scores_topk(sh, inp.q, self.kv, act, na, cfg.topk, step, topk_pages=self.topk)
         up, uc = orc.page_union(sh, self.topk, act, na, cfg.topk, self.kv_len, step)
         orc.sparse_prefix_attn(sh, inp.q, self.kv, act, na, up, uc, self.o_p, self.lse_p)
         out, lse = orc.block_attn_merge(sh, inp.q, inp.k_blk, inp.v_blk, self.o_p, self.lse_p)

@@ -47,12 +47,13 @@ def compare(snap, ref, cfg, what, tau=0.0):
     assert_lse_close(snap["lse"], ref["lse"], what + " lse")
 
 
-def run_blocks(cfg, modes=("losa",), m=None, n_blocks=1, pad_nan=True, want_scores=True, fused=False, tau=0.0):
+def run_blocks(cfg, modes=("losa",), m=None, n_blocks=1, pad_nan=True, want_scores=True, fused=False, tau=0.0,
+               pooled=False):
     """Runs n_blocks blocks through GPU and oracle in lock-step, comparing after every step."""
     from paper_2604_12056_b200.layer import LosaLayer, to_device
     w = wl.Workload(cfg, pad_nan=pad_nan)
-    gpu = {md: LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len, md, tau=tau) for md in modes}
-    ora = {md: OracleLayer(w, md, tau=tau) for md in modes}
+    gpu = {md: LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len, md, tau=tau, pooled=pooled) for md in modes}
+    ora = {md: OracleLayer(w, md, tau=tau, pooled=pooled) for md in modes}
     for md in modes:     # page summaries: exact min / max on both sides
         from paper_2604_12056_b200.layer import to_host
         P = [(int(L) + cfg.page_size - 1) // cfg.page_size for L in w.kv_len]
@@ -117,7 +118,7 @@ def test_c2_reduced_bf16_all_modes():
 
 @pytest.mark.parametrize("g,d,hq,hkv,dtype", [
     (16, 64, 4, 1, "bf16"), (32, 128, 8, 2, "bf16"), (64, 128, 8, 8, "bf16"), (16, 128, 16, 1, "bf16"),
-    (32, 64, 6, 2, "f32"), (64, 128, 4, 2, "f32"), (16, 128, 2, 2, "f32"),
+    (32, 64, 6, 2, "f32"), (64, 128, 4, 2, "f32"), (16, 128, 2, 2, "f32"), (32, 128, 28, 4, "bf16"),
 ])
 def test_ragged_batch_partial_pages_and_empty_prefix(g, d, hq, hkv, dtype):
     # ragged lengths: a partial last page, an empty prefix, a single token, exact page multiples
@@ -142,6 +143,25 @@ def test_threshold_pruning_rule_whole_blocks(tau):
     # follows the active set it produces (bf16 and fp32, two sequences)
     run_blocks(wl.config("c2", kv_lens=(1500, 700), steps=4, block_size=16, topk=6), tau=tau)
     run_blocks(wl.config("c1", kv_lens=(300, 180), steps=3), tau=tau)
+
+
+@pytest.mark.parametrize("fused", [False, True])
+def test_pooled_selector_whole_blocks(fused):
+    # one page list per (token, KV head): six-call path and whole-step call, bf16 with G = 4 and fp32 with G = 3
+    run_blocks(wl.config("c2", kv_lens=(2048, 1500), steps=4), modes=("losa",) if fused else ("losa", "naive"),
+               pooled=True, fused=fused, want_scores=not fused)
+    cfg = wl.config("c2", n_q_heads=6, n_kv_heads=2, head_dim=64, page_size=16, dtype="f32",
+                    kv_lens=(5 * 16 + 3, 0, 1, 7 * 16), block_size=12, steps=3, topk=3, m_active=2)
+    run_blocks(cfg, pooled=True, fused=fused, want_scores=not fused)
+
+
+@pytest.mark.parametrize("pages,topk", [(700, 600), (1100, 8)])
+def test_pooled_selector_long_lists_and_large_budgets(pages, topk):
+    # k > 512 pages takes the whole-list sort; more than 1024 pages the selection that re-reads its
+    # row (pooled once into scratch): the pooled rows go through both
+    cfg = wl.config("c2", n_q_heads=4, n_kv_heads=2, head_dim=64, page_size=16, kv_lens=(16 * pages,),
+                    block_size=4, steps=2, topk=topk, m_active=2)
+    run_blocks(cfg, pooled=True)
 
 
 @pytest.mark.parametrize("name", ["p1", "p2"])
