@@ -626,6 +626,31 @@ def extras(args, cfg, run, flush, result, pages, block0):
             result["pages_read_per_step"][mode if mode == "naive" else "dense_measured"] = float(np.mean(pg)) if pg else None
             other.ctx.close()
 
+    # read-only HBM probe: context for the copy-measured peak the roofline is quoted against
+    probe = torch.ones(1 << 29, dtype=torch.float32, device=q_s.device)          # 2 GiB
+    ts = []
+    for _ in range(6):
+        a, b2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); probe.sum(); b2.record(); b2.synchronize()
+        ts.append(a.elapsed_time(b2))
+    result["hbm_read_probe"] = {"gbs": probe.numel() * 4 / (min(ts[1:]) * 1e-3) / 1e9,
+                                "how": "torch.sum over a 2 GiB fp32 buffer, best of 5 after one warm-up"}
+    del probe
+
+    # fingerprints of layer 0's generated tensors, so that two runs can be told to have seen the same bytes
+    import hashlib
+
+    def sha(t):
+        t = t.contiguous()
+        if t.dtype == torch.bfloat16:
+            t = t.view(torch.int16)
+        return hashlib.sha256(t.cpu().numpy().tobytes()).hexdigest()
+    first = run.block_inputs(block0)[0]
+    result["input_sha256"] = {
+        "note": f"layer 0 of this rank, after the run (blocks appended so far included); step inputs of block {block0}, step 0",
+        "k_pages": sha(layer.k_pages), "v_pages": sha(layer.v_pages), "page_table": sha(layer.page_table),
+        "kv_len": sha(layer.kv_len), "q": sha(first.q), "k_blk": sha(first.k_blk), "v_blk": sha(first.v_blk)}
+
     # the oracle on this machine's host cores (a reported baseline, not a target)
     try:
         from oracle import oracle as orc
