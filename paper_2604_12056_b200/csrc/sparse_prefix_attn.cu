@@ -328,6 +328,12 @@ __global__ void __launch_bounds__(256) attn_finish_kernel(AttnParams p, FinishPa
     qv[c] = q[row * D + lane + 32 * c];
   }
   const float Lb = f.lse_b[row];
+  // the cached prefix statistics as well: nine rows in ten are stable, and asking now saves them
+  // a second round trip (an active row overwrites these below)
+  float a[C], Lp;
+#pragma unroll
+  for (int c = 0; c < C; ++c) a[c] = p.o_p[row * D + lane + 32 * c];
+  Lp = p.lse_p[row];
   // the row's slot in the active list, if any (the list has at most B <= 64 entries)
   const int na = clamp_active(p.n_active[s], p.B);
   int slot = -1;
@@ -336,7 +342,6 @@ __global__ void __launch_bounds__(256) attn_finish_kernel(AttnParams p, FinishPa
     const unsigned hit = __ballot_sync(0xffffffffu, i < na && p.active_idx[s * p.B + i] == tok);
     if (hit) slot = base + __ffs(hit) - 1;
   }
-  float a[C], Lp;
   if (slot >= 0) {
     const int rowk = slot * p.G + gi, rg = rowk / kRowsPerGroup, r = rowk % kRowsPerGroup;
     const int sg = (s * p.Hkv + kh) * p.n_rg + rg;
@@ -351,10 +356,6 @@ __global__ void __launch_bounds__(256) attn_finish_kernel(AttnParams p, FinishPa
       p.o_p[row * D + lane + 32 * c] = a[c];
     }
     if (lane == 0) p.lse_p[row] = Lp;
-  } else {
-#pragma unroll
-    for (int c = 0; c < C; ++c) a[c] = p.o_p[row * D + lane + 32 * c];
-    Lp = p.lse_p[row];
   }
   const float Mx = fmaxf(Lp, Lb);
   const float L = Mx + logf(expf(Lp - Mx) + expf(Lb - Mx));
