@@ -280,6 +280,57 @@ def test_whole_step_call_matches_the_oracle(name, kw):
     run_blocks(cfg, n_blocks=cfg.n_blocks, fused=True)
 
 
+def test_model_step_graph_of_several_layers():
+    """The benchmark's default launch configuration in small: one CUDA graph holds one denoising step
+    of several layers (whole-step calls back to back, each layer with its own pool and state, the
+    programmatic launches running on from one layer into the next); a second graph also finalises
+    the block.  Every replayed step of every layer is compared with the oracle, over two blocks."""
+    import torch
+    from paper_2604_12056_b200.layer import LosaLayer, to_device
+    cfg = wl.config("c2", kv_lens=(1500, 640), steps=3, n_blocks=2, topk=6, m_active=2)
+    L = 3
+    ws = [wl.Workload(cfg, layer=l) for l in range(L)]
+    gpu = [LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len) for w in ws]
+    ora = [OracleLayer(w) for w in ws]
+    first = [w.start_block() for w in ws]
+    bufs = [[to_device(x) for x in (i.q, i.k_blk, i.v_blk, i.m_per_seq)] for i in first]
+    for g, b in zip(gpu, bufs):                           # warm-up outside the graph, then rewind
+        g.run_step_fused(*b)
+    torch.cuda.synchronize()
+    for g in gpu:
+        g.step.zero_()
+    graphs = []
+    for fin in (False, True):
+        gr = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(gr):
+            for g, b in zip(gpu, bufs):
+                g.run_step_fused(*b)
+                if fin:
+                    g.finalize_block(b[1], b[2])
+        graphs.append(gr)
+    for g in gpu:
+        g.step.zero_()
+    for blk in range(cfg.n_blocks):
+        steps = [first] if blk == 0 else [[w.start_block() for w in ws]]
+        steps += [[w.next_step() for w in ws] for _ in range(cfg.steps - 1)]
+        for t, inps in enumerate(steps):
+            last = t == cfg.steps - 1
+            for b, i in zip(bufs, inps):
+                for dst, src in zip(b, (i.q, i.k_blk, i.v_blk, i.m_per_seq)):
+                    dst.copy_(to_device(src))
+            graphs[1 if last else 0].replay()             # finalisation leaves the step's results in place
+            torch.cuda.synchronize()
+            for l, (g, o, i) in enumerate(zip(gpu, ora, inps)):
+                assert g.ctx.poll_status() == 0
+                snap = g.snapshot()
+                ref = o.run_step(i, finalize=last)
+                snap["delta"] = ref["delta"]
+                compare(snap, ref, cfg, f"layer {l} block {blk} step {t}")
+                if last:
+                    s2 = g.snapshot()
+                    assert (s2["kv_len"] == o.kv_len).all() and (s2["step"] == 0).all()
+
+
 def test_whole_step_call_in_a_cuda_graph_full_size():
     """The benchmark's launch configuration: the whole-step call captured in a CUDA graph and
     replayed, full-size workload, LoSA step compared with the oracle in full."""
