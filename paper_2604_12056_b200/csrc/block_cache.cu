@@ -152,6 +152,153 @@ block_attn_merge_kernel(const T* __restrict__ q, const T* __restrict__ k_blk, co
   }
 }
 
+// ---- in-block attention of the whole-step path on the tensor cores (bf16) ---------------------
+// The in-block part is a small dense contraction (B keys, all B * G rows of a KV head), and it runs
+// beside stages 1-3, where every cycle it holds an SM delays them: mma.sync tiles cut its
+// instruction count by more than an order of magnitude against the CUDA-core kernel above.
+// CTA = 64 query rows of one (sequence, KV head) (row = block token * G + head of the group), one
+// warp per 16 rows.  K_b [key][d] and V_b transposed [d][key] are staged in shared memory as bf16
+// (rows padded by 16 bytes: the fragment reads are conflict-free); Q fragments come straight from
+// global memory.  S = Q K_b^T in fp32 accumulators, softmax in registers (row statistics over the
+// four lanes that share a row), P rounded to bf16 as in stage 4, O = P V_b in fp32, normalised by
+// the fp32 sum.  BK = B rounded up to 32 or 64; keys >= B are masked, their V rows zero.
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+constexpr int kMmaRows = 64;       // query rows per CTA
+constexpr int kMmaThreads = 128;
+
+template <int D, int BK>
+__global__ void __launch_bounds__(kMmaThreads)
+block_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_blk,
+                      const __nv_bfloat16* __restrict__ v_blk, float* __restrict__ lse_out,
+                      float* __restrict__ ob_out, int B, int Hq, int Hkv, float sm_scale) {
+  grid_dep_wait();
+  constexpr int KS = D + 8;          // padded row of K_b (elements)
+  constexpr int VS = BK + 8;         // padded row of V_b^T
+  constexpr int NT = BK / 8;         // key tiles of S
+  constexpr int NO = D / 8;          // column tiles of O
+  __shared__ __align__(16) __nv_bfloat16 Ks[BK * KS];
+  __shared__ __align__(16) __nv_bfloat16 Vt[D * VS];
+  const int kh = blockIdx.y, s = blockIdx.z;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int G = Hq / Hkv, nrow = B * G;
+  // ---- stage K_b (row-major) and V_b (transposed); keys >= B are zero
+  for (int idx = tid; idx < BK * (D / 8); idx += kMmaThreads) {
+    const int t = idx % BK, ch = idx / BK;             // key fastest: the transposed stores of a warp fall into one row
+    uint4 kv = make_uint4(0u, 0u, 0u, 0u), vv = kv;
+    if (t < B) {
+      const size_t src = ((static_cast<size_t>(s) * B + t) * Hkv + kh) * D + ch * 8;
+      kv = *reinterpret_cast<const uint4*>(k_blk + src);
+      vv = *reinterpret_cast<const uint4*>(v_blk + src);
+    }
+    *reinterpret_cast<uint4*>(Ks + t * KS + ch * 8) = kv;
+    const __nv_bfloat16* ve = reinterpret_cast<const __nv_bfloat16*>(&vv);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) Vt[(ch * 8 + e) * VS + t] = ve[e];
+  }
+  // ---- this warp's 16 rows: rows g and g + 8 of the tile for this lane
+  const int g = lane >> 2, t4 = lane & 3;
+  const int lr0 = blockIdx.x * kMmaRows + warp * 16 + g, lr1 = lr0 + 8;
+  auto global_row = [&](int lr) {
+    const int c = min(lr, nrow - 1);
+    return (static_cast<size_t>(s) * B + c / G) * Hq + kh * G + c % G;
+  };
+  const size_t gr0 = global_row(lr0), gr1 = global_row(lr1);
+  const uint32_t* q0 = reinterpret_cast<const uint32_t*>(q + gr0 * D);
+  const uint32_t* q1 = reinterpret_cast<const uint32_t*>(q + gr1 * D);
+  uint32_t qa[D / 16][4];
+#pragma unroll
+  for (int ks = 0; ks < D / 16; ++ks) {
+    qa[ks][0] = q0[ks * 8 + t4];
+    qa[ks][1] = q1[ks * 8 + t4];
+    qa[ks][2] = q0[ks * 8 + 4 + t4];
+    qa[ks][3] = q1[ks * 8 + 4 + t4];
+  }
+  __syncthreads();
+  if (blockIdx.x * kMmaRows + warp * 16 >= nrow) return;       // no row of this warp exists
+  // ---- S = Q K_b^T
+  float sc[NT][4];
+#pragma unroll
+  for (int j = 0; j < NT; ++j)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) sc[j][e] = 0.f;
+#pragma unroll
+  for (int ks = 0; ks < D / 16; ++ks) {
+#pragma unroll
+    for (int j = 0; j < NT; ++j) {
+      const uint32_t* kr = reinterpret_cast<const uint32_t*>(Ks + (8 * j + g) * KS + 16 * ks);
+      mma_bf16_16816(sc[j], qa[ks], kr[t4], kr[4 + t4]);
+    }
+  }
+  // ---- softmax over the keys (natural exponent; the log-normaliser is exported in natural units)
+  float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+  for (int j = 0; j < NT; ++j) {
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const int key = 8 * j + 2 * t4 + (e & 1);
+      sc[j][e] = key < B ? sc[j][e] * sm_scale : -INFINITY;
+    }
+    m0 = fmaxf(m0, fmaxf(sc[j][0], sc[j][1]));
+    m1 = fmaxf(m1, fmaxf(sc[j][2], sc[j][3]));
+  }
+  m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 1));
+  m0 = fmaxf(m0, __shfl_xor_sync(0xffffffffu, m0, 2));
+  m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 1));
+  m1 = fmaxf(m1, __shfl_xor_sync(0xffffffffu, m1, 2));
+  float l0 = 0.f, l1 = 0.f;
+  uint32_t pa[NT][2];                // P as bf16 pairs: [j][0] row g, [j][1] row g + 8
+#pragma unroll
+  for (int j = 0; j < NT; ++j) {
+    const float p0 = expf(sc[j][0] - m0), p1 = expf(sc[j][1] - m0);
+    const float p2 = expf(sc[j][2] - m1), p3 = expf(sc[j][3] - m1);
+    l0 += p0 + p1;
+    l1 += p2 + p3;
+    pa[j][0] = pack2_bf16(p0, p1);
+    pa[j][1] = pack2_bf16(p2, p3);
+  }
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+  // ---- O = P V_b
+  float o[NO][4];
+#pragma unroll
+  for (int jn = 0; jn < NO; ++jn)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) o[jn][e] = 0.f;
+#pragma unroll
+  for (int kk = 0; kk < BK / 16; ++kk) {
+    const uint32_t a[4] = {pa[2 * kk][0], pa[2 * kk][1], pa[2 * kk + 1][0], pa[2 * kk + 1][1]};
+#pragma unroll
+    for (int jn = 0; jn < NO; ++jn) {
+      const uint32_t* vr = reinterpret_cast<const uint32_t*>(Vt + (8 * jn + g) * VS + 16 * kk);
+      mma_bf16_16816(o[jn], a, vr[t4], vr[4 + t4]);
+    }
+  }
+  const float i0 = 1.f / l0, i1 = 1.f / l1;
+  if (lr0 < nrow) {
+#pragma unroll
+    for (int jn = 0; jn < NO; ++jn)
+      *reinterpret_cast<float2*>(ob_out + gr0 * D + 8 * jn + 2 * t4) = make_float2(o[jn][0] * i0, o[jn][1] * i0);
+    if (t4 == 0) lse_out[gr0] = m0 + logf(l0);
+  }
+  if (lr1 < nrow) {
+#pragma unroll
+    for (int jn = 0; jn < NO; ++jn)
+      *reinterpret_cast<float2*>(ob_out + gr1 * D + 8 * jn + 2 * t4) = make_float2(o[jn][2] * i1, o[jn][3] * i1);
+    if (t4 == 0) lse_out[gr1] = m1 + logf(l1);
+  }
+}
+
 // Whole-step path, last kernel: one warp per (token, head) row merges the prefix statistics with
 // the in-block part (Section 2.2 / 4.3), writes the output, and keeps the row's query for the next
 // step's Eq. 1; block 0 also bumps the step counters.
@@ -353,10 +500,30 @@ int32_t launch_block_attn_merge(losa_ctx* c, const void* q, const void* k_blk, c
   return launch_merge_t<float, 64, true>(c, q, k_blk, v_blk, state, out, lse_out_opt, nullptr, st);
 }
 
+template <int D, int BK>
+int32_t launch_block_attn_mma(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk, float* lb, float* ob,
+                              cudaStream_t st) {
+  const losa_shape_t& sh = c->shape;
+  const int rows = sh.block_size * (sh.n_q_heads / sh.n_kv_heads);
+  dim3 grid((rows + kMmaRows - 1) / kMmaRows, sh.n_kv_heads, sh.batch);
+  launch_k(block_attn_mma_kernel<D, BK>, grid, kMmaThreads, 0, st,
+      static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k_blk),
+      static_cast<const __nv_bfloat16*>(v_blk), lb, ob, sh.block_size, sh.n_q_heads, sh.n_kv_heads, sh.sm_scale);
+  return after_launch(c);
+}
+
 int32_t launch_block_attn(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk, cudaStream_t st) {
   const bool bf = c->shape.dtype == LOSA_BF16;
   float* ob = reinterpret_cast<float*>(c->ws + c->lay.block_o);
   float* lb = reinterpret_cast<float*>(c->ws + c->lay.block_lse);
+  if (bf) {                                          // tensor-core path
+    const bool wide = c->shape.block_size > 32;
+    if (c->shape.head_dim == 128)
+      return wide ? launch_block_attn_mma<128, 64>(c, q, k_blk, v_blk, lb, ob, st)
+                  : launch_block_attn_mma<128, 32>(c, q, k_blk, v_blk, lb, ob, st);
+    return wide ? launch_block_attn_mma<64, 64>(c, q, k_blk, v_blk, lb, ob, st)
+                : launch_block_attn_mma<64, 32>(c, q, k_blk, v_blk, lb, ob, st);
+  }
   if (bf && c->shape.head_dim == 128) return launch_merge_t<__nv_bfloat16, 128, false>(c, q, k_blk, v_blk, nullptr, nullptr, lb, ob, st);
   if (bf) return launch_merge_t<__nv_bfloat16, 64, false>(c, q, k_blk, v_blk, nullptr, nullptr, lb, ob, st);
   if (c->shape.head_dim == 128) return launch_merge_t<float, 128, false>(c, q, k_blk, v_blk, nullptr, nullptr, lb, ob, st);
