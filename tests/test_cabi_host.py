@@ -81,11 +81,18 @@ def test_null_arguments_are_rejected_without_a_device(lib):
     for fn, nargs in (("losa_select_active", 10), ("losa_page_scores_topk", 10), ("losa_page_union", 10),
                       ("losa_sparse_prefix_attn", 9), ("losa_block_attn_merge", 8),
                       ("losa_update_prefix_cache", 8), ("losa_build_page_summaries", 3),
-                      ("losa_denoise_step_host", 11), ("losa_denoise_step", 12)):
+                      ("losa_denoise_step_host", 11), ("losa_denoise_step", 12),
+                      ("losa_page_scores_topk_pooled", 10)):
         args = [None] * nargs
         if fn in ("losa_select_active",):
             args[3] = C.c_int32(64)
         assert getattr(lib, fn)(*args) == B.LOSA_ERR_INVALID_ARG, fn
+
+
+    assert lib.losa_set_pooled_selection(None, C.c_int32(1)) == B.LOSA_ERR_INVALID_ARG
+    args = [None] * 11
+    args[3], args[4] = C.c_int32(64), C.c_double(0.5)
+    assert lib.losa_select_active_tau(*args) == B.LOSA_ERR_INVALID_ARG
 
 
 def test_missing_library_is_a_loud_error(monkeypatch):
