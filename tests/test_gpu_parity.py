@@ -273,6 +273,11 @@ def test_full_size_c3_in_the_benchmark_configuration():
     ("c2", dict(kv_lens=(2048,), steps=4)),
     ("c2", dict(kv_lens=(5 * 32 + 3, 0, 1, 7 * 32), block_size=12, steps=3, topk=3, m_active=2)),
     ("c5", dict(kv_lens=(200, 90, 64), n_blocks=2, steps=3, topk=4)),
+    # in-block attention on the tensor cores: 64 block keys (two row groups of queries), and 48 keys
+    # padded to 64 with d = 64 and two heads per KV head
+    ("c2", dict(kv_lens=(1000,), block_size=64, steps=3, topk=6, m_active=5)),
+    ("c2", dict(n_q_heads=4, n_kv_heads=2, head_dim=64, page_size=16, kv_lens=(700, 333), block_size=48, steps=3,
+                topk=5, m_active=3)),
 ])
 def test_whole_step_call_matches_the_oracle(name, kw):
     """losa_denoise_step (one call, in-block attention on a second stream) against the oracle."""
