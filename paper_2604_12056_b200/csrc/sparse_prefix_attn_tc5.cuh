@@ -221,6 +221,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     // PG pages; the first lane of a group's run waits for the group's ring slot and announces the
     // group's bytes, then every lane of the run issues its page.
     const bool is_v = warp == kTc5VWarp;
+    const unsigned long long policy = l2_evict_first_policy();
     const CUtensorMap* map = is_v ? &tmV : &tmK;
     const uint32_t ring = is_v ? vring : kring, full0 = is_v ? vfull : kfull, free0 = is_v ? vfree : kfree;
     int cursor = sg0, gbase = 0, pstart = lo;       // segment of the lane's newest item, groups before its piece, the piece's first item
@@ -287,7 +288,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         if (mine) {
           const uint32_t dst = ring + slot * SLOT + b.j * (GP * 128);
 #pragma unroll
-          for (int hf = 0; hf < HALVES; ++hf) tma_load_4d(dst + hf * HS, map, full0 + 8 * slot, hf * 64, 0, b.kh, b.phys);
+          for (int hf = 0; hf < HALVES; ++hf) tma_load_4d(dst + hf * HS, map, full0 + 8 * slot, hf * 64, 0, b.kh, b.phys, policy);
         }
         pos += cnt;
       }
