@@ -42,11 +42,11 @@ UNIT = "us/layer-step"
 L2_FLUSH_BYTES = 256 << 20
 # DRAM traffic of the stage-4 main kernel per listed (page, KV head) slice, from the ncu capture in
 # profiles/attn_tc5_kernel_c5.txt: the dense launch there moved dram__bytes_read.sum +
-# dram__bytes_write.sum = 1,087.26 MB for its 65,984 slices (16,384 of the 16,478 bytes per slice are
+# dram__bytes_write.sum = 1,085.39 MB for its 65,984 slices (16,384 of the 16,449 bytes per slice are
 # the slice's K and V).  Traffic grows in proportion to the slices, so a launch's traffic is reported
 # as slices x this figure; LoSA launches add the partial records they write (3.7-4.8 MB of DRAM
 # writes in the three LoSA launches of that capture).  Pages of 32 tokens, head dim 128, bf16 only.
-NCU_BYTES_PER_SLICE = {"losa": 1087.26e6 / 65984, "dense": 1087.26e6 / 65984}
+NCU_BYTES_PER_SLICE = {"losa": 1085.39e6 / 65984, "dense": 1085.39e6 / 65984}
 NCU_FIXED_BYTES = {"losa": 4.8e6, "dense": 0.0}
 
 
