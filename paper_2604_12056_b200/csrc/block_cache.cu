@@ -1,7 +1,8 @@
 // Stage 5 — dense in-block attention and the online-softmax merge (Section 4.3, Section 2.2);
 // stage 6 — cache maintenance (Section 4.3, Section 2.1) and the page summaries (Section 2.3).
 //
-// These stages touch O(B * H * d) data: they are latency-bound, so the kernels are plain fp32
+// These stages touch O(B * H * d) data: they are latency-bound.  In bf16 mode the in-block attention
+// runs on the tensor cores (block_attn_mma_kernel); the fp32 mode and the cache kernels are plain
 // CUDA-core code laid out for coalesced global access and conflict-free shared-memory access.
 #include "kernels.h"
 
@@ -175,10 +176,14 @@ __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
 constexpr int kMmaRows = 64;       // query rows per CTA
 constexpr int kMmaThreads = 128;
 
-template <int D, int BK>
+// MERGE = true (stage 5 of the six-call path): the in-block part is merged with the prefix
+// statistics by log-sum-exp and the attention output is written (Section 2.2 / 4.3); MERGE = false
+// (whole-step path): the normalised in-block part goes to `ob_out` and L_b to `lse_out`.
+template <int D, int BK, bool MERGE>
 __global__ void __launch_bounds__(kMmaThreads)
 block_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_blk,
-                      const __nv_bfloat16* __restrict__ v_blk, float* __restrict__ lse_out,
+                      const __nv_bfloat16* __restrict__ v_blk, const float* __restrict__ o_p,
+                      const float* __restrict__ lse_p, __nv_bfloat16* __restrict__ out, float* __restrict__ lse_out,
                       float* __restrict__ ob_out, int B, int Hq, int Hkv, float sm_scale) {
   grid_dep_wait();
   constexpr int KS = D + 8;          // padded row of K_b (elements)
@@ -284,19 +289,33 @@ block_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
       mma_bf16_16816(o[jn], a, vr[t4], vr[4 + t4]);
     }
   }
-  const float i0 = 1.f / l0, i1 = 1.f / l1;
-  if (lr0 < nrow) {
+  // rows g (accumulator halves 0, 1) and g + 8 (halves 2, 3)
+  auto finish_row = [&](int lr, size_t gr, float m, float l, int e0) {
+    if (lr >= nrow) return;
+    const float Lb = m + logf(l);
+    if (MERGE) {
+      const float Lp = lse_p[gr];
+      const float M2 = fmaxf(Lp, Lb);
+      const float L = M2 + logf(expf(Lp - M2) + expf(Lb - M2));
+      const float wp = expf(Lp - L), wb = expf(Lb - L) / l;
 #pragma unroll
-    for (int jn = 0; jn < NO; ++jn)
-      *reinterpret_cast<float2*>(ob_out + gr0 * D + 8 * jn + 2 * t4) = make_float2(o[jn][0] * i0, o[jn][1] * i0);
-    if (t4 == 0) lse_out[gr0] = m0 + logf(l0);
-  }
-  if (lr1 < nrow) {
+      for (int jn = 0; jn < NO; ++jn) {
+        const float2 pv = *reinterpret_cast<const float2*>(o_p + gr * D + 8 * jn + 2 * t4);
+        const float x = (wp > 0.f ? wp * pv.x : 0.f) + wb * o[jn][e0];
+        const float y = (wp > 0.f ? wp * pv.y : 0.f) + wb * o[jn][e0 + 1];
+        *reinterpret_cast<__nv_bfloat162*>(out + gr * D + 8 * jn + 2 * t4) = __floats2bfloat162_rn(x, y);
+      }
+      if (lse_out && t4 == 0) lse_out[gr] = L;
+    } else {
+      const float inv = 1.f / l;
 #pragma unroll
-    for (int jn = 0; jn < NO; ++jn)
-      *reinterpret_cast<float2*>(ob_out + gr1 * D + 8 * jn + 2 * t4) = make_float2(o[jn][2] * i1, o[jn][3] * i1);
-    if (t4 == 0) lse_out[gr1] = m1 + logf(l1);
-  }
+      for (int jn = 0; jn < NO; ++jn)
+        *reinterpret_cast<float2*>(ob_out + gr * D + 8 * jn + 2 * t4) = make_float2(o[jn][e0] * inv, o[jn][e0 + 1] * inv);
+      if (t4 == 0) lse_out[gr] = Lb;
+    }
+  };
+  finish_row(lr0, gr0, m0, l0, 0);
+  finish_row(lr1, gr1, m1, l1, 2);
 }
 
 // Whole-step path, last kernel: one warp per (token, head) row merges the prefix statistics with
@@ -491,41 +510,44 @@ int32_t launch_summaries_t(losa_ctx* c, losa_kv_t* kv, cudaStream_t st) {
 
 }  // namespace
 
-int32_t launch_block_attn_merge(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk,
-                                const losa_state_t* state, void* out, float* lse_out_opt, cudaStream_t st) {
-  const bool bf = c->shape.dtype == LOSA_BF16;
-  if (bf && c->shape.head_dim == 128) return launch_merge_t<__nv_bfloat16, 128, true>(c, q, k_blk, v_blk, state, out, lse_out_opt, nullptr, st);
-  if (bf) return launch_merge_t<__nv_bfloat16, 64, true>(c, q, k_blk, v_blk, state, out, lse_out_opt, nullptr, st);
-  if (c->shape.head_dim == 128) return launch_merge_t<float, 128, true>(c, q, k_blk, v_blk, state, out, lse_out_opt, nullptr, st);
-  return launch_merge_t<float, 64, true>(c, q, k_blk, v_blk, state, out, lse_out_opt, nullptr, st);
-}
-
-template <int D, int BK>
-int32_t launch_block_attn_mma(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk, float* lb, float* ob,
-                              cudaStream_t st) {
+template <int D, int BK, bool MERGE>
+int32_t launch_block_attn_mma(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk,
+                              const losa_state_t* state, void* out, float* lb, float* ob, cudaStream_t st) {
   const losa_shape_t& sh = c->shape;
   const int rows = sh.block_size * (sh.n_q_heads / sh.n_kv_heads);
   dim3 grid((rows + kMmaRows - 1) / kMmaRows, sh.n_kv_heads, sh.batch);
-  launch_k(block_attn_mma_kernel<D, BK>, grid, kMmaThreads, 0, st,
+  launch_k(block_attn_mma_kernel<D, BK, MERGE>, grid, kMmaThreads, 0, st,
       static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k_blk),
-      static_cast<const __nv_bfloat16*>(v_blk), lb, ob, sh.block_size, sh.n_q_heads, sh.n_kv_heads, sh.sm_scale);
+      static_cast<const __nv_bfloat16*>(v_blk), state ? state->o_p : nullptr, state ? state->lse_p : nullptr,
+      static_cast<__nv_bfloat16*>(out), lb, ob, sh.block_size, sh.n_q_heads, sh.n_kv_heads, sh.sm_scale);
   return after_launch(c);
+}
+
+// bf16: the tensor-core kernel, by head dimension and padded key count
+template <bool MERGE>
+int32_t dispatch_block_attn_mma(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk,
+                                const losa_state_t* state, void* out, float* lb, float* ob, cudaStream_t st) {
+  const bool wide = c->shape.block_size > 32;
+  if (c->shape.head_dim == 128)
+    return wide ? launch_block_attn_mma<128, 64, MERGE>(c, q, k_blk, v_blk, state, out, lb, ob, st)
+                : launch_block_attn_mma<128, 32, MERGE>(c, q, k_blk, v_blk, state, out, lb, ob, st);
+  return wide ? launch_block_attn_mma<64, 64, MERGE>(c, q, k_blk, v_blk, state, out, lb, ob, st)
+              : launch_block_attn_mma<64, 32, MERGE>(c, q, k_blk, v_blk, state, out, lb, ob, st);
+}
+
+int32_t launch_block_attn_merge(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk,
+                                const losa_state_t* state, void* out, float* lse_out_opt, cudaStream_t st) {
+  const bool bf = c->shape.dtype == LOSA_BF16;
+  if (bf) return dispatch_block_attn_mma<true>(c, q, k_blk, v_blk, state, out, lse_out_opt, nullptr, st);
+  if (c->shape.head_dim == 128) return launch_merge_t<float, 128, true>(c, q, k_blk, v_blk, state, out, lse_out_opt, nullptr, st);
+  return launch_merge_t<float, 64, true>(c, q, k_blk, v_blk, state, out, lse_out_opt, nullptr, st);
 }
 
 int32_t launch_block_attn(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk, cudaStream_t st) {
   const bool bf = c->shape.dtype == LOSA_BF16;
   float* ob = reinterpret_cast<float*>(c->ws + c->lay.block_o);
   float* lb = reinterpret_cast<float*>(c->ws + c->lay.block_lse);
-  if (bf) {                                          // tensor-core path
-    const bool wide = c->shape.block_size > 32;
-    if (c->shape.head_dim == 128)
-      return wide ? launch_block_attn_mma<128, 64>(c, q, k_blk, v_blk, lb, ob, st)
-                  : launch_block_attn_mma<128, 32>(c, q, k_blk, v_blk, lb, ob, st);
-    return wide ? launch_block_attn_mma<64, 64>(c, q, k_blk, v_blk, lb, ob, st)
-                : launch_block_attn_mma<64, 32>(c, q, k_blk, v_blk, lb, ob, st);
-  }
-  if (bf && c->shape.head_dim == 128) return launch_merge_t<__nv_bfloat16, 128, false>(c, q, k_blk, v_blk, nullptr, nullptr, lb, ob, st);
-  if (bf) return launch_merge_t<__nv_bfloat16, 64, false>(c, q, k_blk, v_blk, nullptr, nullptr, lb, ob, st);
+  if (bf) return dispatch_block_attn_mma<false>(c, q, k_blk, v_blk, nullptr, nullptr, lb, ob, st);
   if (c->shape.head_dim == 128) return launch_merge_t<float, 128, false>(c, q, k_blk, v_blk, nullptr, nullptr, lb, ob, st);
   return launch_merge_t<float, 64, false>(c, q, k_blk, v_blk, nullptr, nullptr, lb, ob, st);
 }
