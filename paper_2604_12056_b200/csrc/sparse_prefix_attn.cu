@@ -238,7 +238,7 @@ __device__ __forceinline__ void merge_records(const AttnParams& p, int sg, int r
     }
     Lsum += warp_sum(lj * wj);
     const int n = min(32, n_pairs - base);
-    constexpr int U = 8;                            // records whose loads are in flight together
+    constexpr int U = 4;                            // records whose loads are in flight together
     for (int i0 = 0; i0 < n; i0 += U) {
       float w[U], v[U][C];
 #pragma unroll
