@@ -305,15 +305,17 @@ struct FinishParams {
   size_t n_rows;
 };
 
+constexpr int kFinishThreads = 128;
+
 template <typename T, int D>
-__global__ void __launch_bounds__(256) attn_finish_kernel(AttnParams p, FinishParams f) {
+__global__ void __launch_bounds__(kFinishThreads) attn_finish_kernel(AttnParams p, FinishParams f) {
   grid_dep_trigger();
   grid_dep_wait();
   constexpr int C = D / 32;
   const int lane = threadIdx.x & 31;
-  const size_t row = static_cast<size_t>(blockIdx.x) * 8 + (threadIdx.x >> 5);
+  const size_t row = static_cast<size_t>(blockIdx.x) * (kFinishThreads / 32) + (threadIdx.x >> 5);
   if (blockIdx.x == 0)
-    for (int s = threadIdx.x; s < p.N; s += 256) f.step[s] += 1;
+    for (int s = threadIdx.x; s < p.N; s += kFinishThreads) f.step[s] += 1;
   if (row >= f.n_rows) return;
   const int hq = static_cast<int>(row % p.Hq), tok = static_cast<int>((row / p.Hq) % p.B);
   const int s = static_cast<int>(row / (static_cast<size_t>(p.Hq) * p.B));
@@ -623,9 +625,9 @@ int32_t launch_attn_finish(losa_ctx* c, const void* q, const int32_t* active_idx
   fp.lse_out = lse_out_opt;
   fp.step = state->step;
   fp.n_rows = static_cast<size_t>(sh.batch) * sh.block_size * sh.n_q_heads;
-  const int blocks = static_cast<int>((fp.n_rows + 7) / 8);
-  if (sh.head_dim == 128) launch_k(attn_finish_kernel<__nv_bfloat16, 128>, blocks, 256, 0, st, ap, fp);
-  else launch_k(attn_finish_kernel<__nv_bfloat16, 64>, blocks, 256, 0, st, ap, fp);
+  const int blocks = static_cast<int>((fp.n_rows + kFinishThreads / 32 - 1) / (kFinishThreads / 32));
+  if (sh.head_dim == 128) launch_k(attn_finish_kernel<__nv_bfloat16, 128>, blocks, kFinishThreads, 0, st, ap, fp);
+  else launch_k(attn_finish_kernel<__nv_bfloat16, 64>, blocks, kFinishThreads, 0, st, ap, fp);
   return after_launch(c);
 }
 
