@@ -28,13 +28,28 @@ select_active_kernel(const T* __restrict__ x_cur, const T* __restrict__ x_prev, 
   const size_t row = (static_cast<size_t>(s) * B + i) * row_width;
   constexpr int kVec = 8;
   double acc = 0.0;
-  for (int c = tid * kVec; c < row_width; c += kThreads * kVec) {
-    float a[8], b[8];
+  // two chunks per pass, all four loads requested before any is used (a row of 4,096 elements is
+  // one pass of the CTA)
+  for (int c = tid * kVec; c < row_width; c += 2 * kThreads * kVec) {
+    const int c2 = c + kThreads * kVec;
+    float a[8], b[8], a2[8], b2[8];
     load8(x_cur + row + c, a);
     load8(x_prev + row + c, b);
+    if (c2 < row_width) {
+      load8(x_cur + row + c2, a2);
+      load8(x_prev + row + c2, b2);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 8; ++j) a2[j] = b2[j] = 0.f;
+    }
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
       const double df = static_cast<double>(a[j]) - static_cast<double>(b[j]);
+      acc = fma(df, df, acc);
+    }
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const double df = static_cast<double>(a2[j]) - static_cast<double>(b2[j]);
       acc = fma(df, df, acc);
     }
   }
