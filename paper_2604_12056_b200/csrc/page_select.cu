@@ -538,14 +538,33 @@ union_kernel(const int32_t* __restrict__ topk_pages, const int32_t* __restrict__
     int na = n_active[s];
     na = na < 0 ? 0 : (na > B ? B : na);
     const int per_tok = G * k;
-    for (int idx = tid; idx < na * per_tok; idx += kThreads) {
-      const int a = idx / per_tok, rem = idx % per_tok, gi = rem / k, j = rem % k;
-      const int tok = active_idx[s * B + a];
-      if (tok < 0 || tok >= B) { set_status(status, LOSA_ERR_BOUNDS); continue; }
-      const int p = topk_pages[((static_cast<size_t>(s) * B + tok) * Hq + kh * G + gi) * k + j];
-      if (p < 0) continue;
-      if (p >= P) { set_status(status, LOSA_ERR_BOUNDS); continue; }
-      atomicOr(&bitmap[p >> 5], 1u << (p & 31));
+    // two dependent reads per entry (block position of the active slot, then the list entry): the
+    // positions are staged once, and the list entries are requested four at a time
+    __shared__ int s_tok[LOSA_MAX_BLOCK];
+    for (int a = tid; a < na; a += kThreads) s_tok[a] = active_idx[s * B + a];
+    __syncthreads();
+    constexpr int U = 4;
+    const int total = na * per_tok;
+    for (int base = tid; base < total; base += kThreads * U) {
+      int pv[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int idx = base + u * kThreads;
+        pv[u] = -1;
+        if (idx < total) {
+          const int a = idx / per_tok, rem = idx % per_tok, gi = rem / k, j = rem % k;
+          const int tok = s_tok[a];
+          if (tok < 0 || tok >= B) { set_status(status, LOSA_ERR_BOUNDS); continue; }
+          pv[u] = topk_pages[((static_cast<size_t>(s) * B + tok) * Hq + kh * G + gi) * k + j];
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int p = pv[u];
+        if (p < 0) continue;
+        if (p >= P) { set_status(status, LOSA_ERR_BOUNDS); continue; }
+        atomicOr(&bitmap[p >> 5], 1u << (p & 31));
+      }
     }
     __syncthreads();
   }
