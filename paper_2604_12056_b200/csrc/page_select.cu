@@ -53,6 +53,14 @@ template <> struct Raw8<float> {
   }
 };
 
+// A load whose issue point stays where it is written (it is requested ahead of the branch that
+// decides whether it is needed).
+__device__ __forceinline__ int ld_keep_s32(const int32_t* ptr) {
+  int v;
+  asm volatile("ld.global.nc.s32 %0, [%1];" : "=r"(v) : "l"(ptr));
+  return v;
+}
+
 template <typename T, int D>
 __global__ void __launch_bounds__(kThreads)
 page_scores_kernel(const T* __restrict__ q, const T* __restrict__ kmin, const T* __restrict__ kmax,
@@ -63,13 +71,32 @@ page_scores_kernel(const T* __restrict__ q, const T* __restrict__ kmin, const T*
   grid_dep_wait();
   constexpr int LPP = D / 8;            // lanes per page
   constexpr int GROUPS = kThreads / LPP;
+  constexpr int ITER = kPagesPerCta / GROUPS;
+  constexpr int STG = (kRowTile * (D / 8) + kThreads - 1) / kThreads;   // staging items per thread and row tile
   const int s = blockIdx.z, kh = blockIdx.y, p0 = blockIdx.x * kPagesPerCta;
+  const int tid = threadIdx.x;
+  const int grp = tid / LPP, sub = tid % LPP;
+  const int G = Hq / Hkv;
+  // First round trip: the scalars, and with them - their addresses depend on nothing else - this
+  // lane's page-table entries and the block positions of the query rows it may have to stage
+  // (entries the scalars later rule out are read and dropped).
+  int phys[ITER], tok0[STG];
+#pragma unroll
+  for (int it = 0; it < ITER; ++it) {
+    const int p = p0 + grp * ITER + it;
+    phys[it] = p < Pmax ? ld_keep_s32(page_table + static_cast<size_t>(s) * Pmax + p) : -1;
+  }
+#pragma unroll
+  for (int i = 0; i < STG; ++i) {
+    const int a = ((tid + i * kThreads) / (D / 8)) / G;
+    tok0[i] = a < B ? ld_keep_s32(active_idx + s * B + a) : 0;
+  }
   if (step && step[s] == 0) return;
   const int P = pages_of(kv_len[s], g);
   if (p0 >= P) return;
   int na = n_active[s];
   na = na < 0 ? 0 : (na > B ? B : na);
-  const int G = Hq / Hkv, rows = na * G;
+  const int rows = na * G;
   if (rows == 0) return;
 
   // positive and negative parts of the staged queries, fp32: U = sum q+ kmax + q- kmin.  A row is
@@ -77,28 +104,12 @@ page_scores_kernel(const T* __restrict__ q, const T* __restrict__ kmin, const T*
   // consecutive 16-byte words (no bank conflicts): element j = 8*c + e sits at (e/4)*(D/2) + 4*c + e%4.
   __shared__ __align__(16) float qpos[kRowTile * D];
   __shared__ __align__(16) float qneg[kRowTile * D];
-  const int tid = threadIdx.x;
-  const int grp = tid / LPP, sub = tid % LPP;
   const int np = min(kPagesPerCta, P - p0);
 
-  // Three dependent round trips to memory per CTA: (1) the scalars above, (2) this lane's physical
-  // page ids and the block positions of the query rows it will stage, (3) its share of the pages'
-  // kmin / kmax (kept in registers for every query row) and the query rows themselves.  Everything
-  // of a trip is requested before anything of it is used.
-  constexpr int ITER = kPagesPerCta / GROUPS;
-  constexpr int STG = (kRowTile * (D / 8) + kThreads - 1) / kThreads;   // staging items per thread and row tile
+  // Second round trip: this lane's share of the pages' kmin / kmax (kept in registers for every
+  // query row) and the query rows themselves.  Everything of a trip is requested before anything
+  // of it is used.
   const int nr_first = min(kRowTile, rows);
-  int phys[ITER], tok0[STG];
-#pragma unroll
-  for (int it = 0; it < ITER; ++it) {
-    const int pl = grp * ITER + it;
-    phys[it] = pl < np ? page_table[static_cast<size_t>(s) * Pmax + p0 + pl] : -1;
-  }
-#pragma unroll
-  for (int i = 0; i < STG; ++i) {
-    const int idx = tid + i * kThreads;
-    tok0[i] = idx < nr_first * (D / 8) ? active_idx[s * B + (idx / (D / 8)) / G] : 0;
-  }
   Raw8<T> klo[ITER], khi[ITER], q0[STG];
 #pragma unroll
   for (int it = 0; it < ITER; ++it) {
