@@ -38,6 +38,7 @@ int32_t make_layout(const losa_shape_t* sh, int n_ctas, WorkspaceLayout* L) {
   L->status = off;   off = align_up(off + 16, 256);
   L->counters = off; off = align_up(off + sizeof(uint32_t) * sh->batch, 256);
   L->seg_prefix = off; off = align_up(off + sizeof(int32_t) * (kMaxSegments + 1), 256);
+  L->slot_map = off; off = align_up(off + sizeof(int32_t) * sh->batch * sh->block_size, 256);
   L->delta = off;    off = align_up(off + sizeof(double) * sh->batch * sh->block_size, 256);
   L->scores = off;
   off = align_up(off + sizeof(float) * static_cast<size_t>(sh->batch) * sh->block_size * sh->n_q_heads * L->score_stride, 256);
@@ -280,15 +281,16 @@ int32_t losa_denoise_step(losa_ctx* ctx, const void* q, const void* k_blk, const
   rc = launch_block_attn(ctx, q, k_blk, v_blk, ctx->side_stream);
   if (rc != LOSA_OK) return rc;
   LOSA_CUDA_TRY(ctx, cudaEventRecord(ctx->ev_join, ctx->side_stream));
+  int32_t* slot_map = reinterpret_cast<int32_t*>(ctx->ws + ctx->lay.slot_map);
   rc = launch_select_active(ctx, q, state->q_prev, sh.n_q_heads * sh.head_dim, m_per_seq, state->step,
-                            buf->active_idx, buf->n_active, nullptr, st);
+                            buf->active_idx, buf->n_active, nullptr, st, 0.0, slot_map);
   if (rc == LOSA_OK) rc = launch_page_scores_topk(ctx, q, kv, buf->active_idx, buf->n_active, state->step, k, buf->topk_pages, nullptr, st, ctx->pooled_selection != 0);
   if (rc == LOSA_OK) rc = launch_page_union(ctx, buf->topk_pages, buf->active_idx, buf->n_active, k, kv->kv_len, state->step, buf->union_pages, buf->union_count, st);
   if (rc == LOSA_OK) rc = launch_sparse_prefix_attn(ctx, q, kv, buf->active_idx, buf->n_active, buf->union_pages, buf->union_count, state, st, true);
   if (rc != LOSA_OK) return rc;
   // join, then one pass over the rows: (merge of the partial records,) merge with the block part, commit
   LOSA_CUDA_TRY(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0));
-  if (finish_fuses_combine(ctx)) return launch_attn_finish(ctx, q, buf->active_idx, buf->n_active, state, out, lse_out_opt, st);
+  if (finish_fuses_combine(ctx)) return launch_attn_finish(ctx, q, buf->active_idx, buf->n_active, slot_map, state, out, lse_out_opt, st);
   return launch_merge_commit(ctx, q, state, out, lse_out_opt, st);
 }
 

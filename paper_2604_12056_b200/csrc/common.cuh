@@ -21,6 +21,7 @@ struct WorkspaceLayout {
   size_t status;     // int32[4]  : device status word (+ padding)
   size_t counters;   // uint32[N] : arrival counters of select_active (self-resetting)
   size_t seg_prefix; // int32[kMaxSegments + 1] : item prefix of the segments, left by the stage-4 main kernel for its combine kernel
+  size_t slot_map;   // int32[N*B] : slot of every block token in the active list of the whole-step path, -1 = stable
   size_t delta;      // double[N*B]
   size_t scores;     // float[N*B*H_q*score_stride]
   size_t partials;   // float[n_slots * kRowsPerGroup * (d + 2)]

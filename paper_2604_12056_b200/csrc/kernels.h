@@ -7,7 +7,8 @@ namespace losa {
 
 int32_t launch_select_active(losa_ctx* c, const void* x_cur, const void* x_prev, int32_t row_width,
                              const int32_t* m_per_seq, const int32_t* step, int32_t* active_idx,
-                             int32_t* n_active, float* delta_opt, cudaStream_t st, double tau = 0.0);
+                             int32_t* n_active, float* delta_opt, cudaStream_t st, double tau = 0.0,
+                             int32_t* slot_map_opt = nullptr);
 
 int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
                                 const int32_t* active_idx, const int32_t* n_active,
@@ -27,7 +28,7 @@ int32_t launch_sparse_prefix_attn(losa_ctx* c, const void* q, const losa_kv_t* k
 // launch_attn_finish merges them, merges with the in-block part, writes the output, keeps the
 // queries and bumps the step (one kernel instead of combine + merge_commit).
 bool finish_fuses_combine(const losa_ctx* c);
-int32_t launch_attn_finish(losa_ctx* c, const void* q, const int32_t* active_idx, const int32_t* n_active,
+int32_t launch_attn_finish(losa_ctx* c, const void* q, const int32_t* active_idx, const int32_t* n_active, const int32_t* slot_map,
                            losa_state_t* state, void* out, float* lse_out_opt, cudaStream_t st);
 
 int32_t launch_block_attn_merge(losa_ctx* c, const void* q, const void* k_blk, const void* v_blk,

@@ -20,7 +20,7 @@ select_active_kernel(const T* __restrict__ x_cur, const T* __restrict__ x_prev, 
                      const int32_t* __restrict__ m_per_seq, const int32_t* __restrict__ step,
                      int32_t* __restrict__ active_idx, int32_t* __restrict__ n_active,
                      float* __restrict__ delta_opt, double* __restrict__ delta_ws,
-                     unsigned int* __restrict__ counters, double tau) {
+                     unsigned int* __restrict__ counters, double tau, int32_t* __restrict__ slot_map) {
   grid_dep_trigger();
   grid_dep_wait();
   const int i = blockIdx.x, s = blockIdx.y;
@@ -125,6 +125,10 @@ select_active_kernel(const T* __restrict__ x_cur, const T* __restrict__ x_prev, 
   int32_t* out = active_idx + static_cast<size_t>(s) * B;
   if (act[0]) out[__popc(b0 & below)] = lane;
   if (act[1]) out[n0 + __popc(b1 & below)] = lane + 32;
+  if (slot_map) {                                     // the inverse map, for the kernel that finishes the step
+    if (lane < B) slot_map[s * B + lane] = act[0] ? __popc(b0 & below) : -1;
+    if (lane + 32 < B) slot_map[s * B + lane + 32] = act[1] ? n0 + __popc(b1 & below) : -1;
+  }
   for (int t = n0 + n1 + lane; t < B; t += 32) out[t] = -1;
   if (lane == 0) n_active[s] = n0 + n1;
 }
@@ -133,7 +137,7 @@ select_active_kernel(const T* __restrict__ x_cur, const T* __restrict__ x_prev, 
 
 int32_t launch_select_active(losa_ctx* c, const void* x_cur, const void* x_prev, int32_t row_width,
                              const int32_t* m_per_seq, const int32_t* step, int32_t* active_idx,
-                             int32_t* n_active, float* delta_opt, cudaStream_t st, double tau) {
+                             int32_t* n_active, float* delta_opt, cudaStream_t st, double tau, int32_t* slot_map_opt) {
   const losa_shape_t& sh = c->shape;
   dim3 grid(sh.block_size, sh.batch);
   double* dws = reinterpret_cast<double*>(c->ws + c->lay.delta);
@@ -141,11 +145,11 @@ int32_t launch_select_active(losa_ctx* c, const void* x_cur, const void* x_prev,
   if (sh.dtype == LOSA_BF16) {
     launch_k(select_active_kernel<__nv_bfloat16>, grid, kThreads, 0, st, 
         static_cast<const __nv_bfloat16*>(x_cur), static_cast<const __nv_bfloat16*>(x_prev), row_width,
-        sh.block_size, m_per_seq, step, active_idx, n_active, delta_opt, dws, ctr, tau);
+        sh.block_size, m_per_seq, step, active_idx, n_active, delta_opt, dws, ctr, tau, slot_map_opt);
   } else {
     launch_k(select_active_kernel<float>, grid, kThreads, 0, st, 
         static_cast<const float*>(x_cur), static_cast<const float*>(x_prev), row_width, sh.block_size,
-        m_per_seq, step, active_idx, n_active, delta_opt, dws, ctr, tau);
+        m_per_seq, step, active_idx, n_active, delta_opt, dws, ctr, tau, slot_map_opt);
   }
   return after_launch(c);
 }
@@ -211,11 +215,11 @@ extern "C" int32_t losa_select_active_static(const losa_shape_t* shape, const vo
   if (shape->dtype == LOSA_BF16) {
     losa::launch_k(losa::select_active_kernel<__nv_bfloat16>, grid, losa::kThreads, 0, st, 
         static_cast<const __nv_bfloat16*>(x_cur), static_cast<const __nv_bfloat16*>(x_prev), row_width,
-        shape->block_size, m_per_seq, step, active_idx, n_active, delta_opt, scratch->delta, scratch->counters, 0.0);
+        shape->block_size, m_per_seq, step, active_idx, n_active, delta_opt, scratch->delta, scratch->counters, 0.0, nullptr);
   } else {
     losa::launch_k(losa::select_active_kernel<float>, grid, losa::kThreads, 0, st, 
         static_cast<const float*>(x_cur), static_cast<const float*>(x_prev), row_width, shape->block_size,
-        m_per_seq, step, active_idx, n_active, delta_opt, scratch->delta, scratch->counters, 0.0);
+        m_per_seq, step, active_idx, n_active, delta_opt, scratch->delta, scratch->counters, 0.0, nullptr);
   }
   return cudaGetLastError() == cudaSuccess ? LOSA_OK : LOSA_ERR_CUDA;
 }

@@ -302,6 +302,7 @@ struct FinishParams {
   void* out;
   float* lse_out;
   int32_t* step;
+  const int32_t* slot_map;   // [N*B] slot of a block token in the active list, -1 = stable (null: look it up)
   size_t n_rows;
 };
 
@@ -337,12 +338,17 @@ __global__ void __launch_bounds__(kFinishThreads) attn_finish_kernel(AttnParams 
   for (int c = 0; c < C; ++c) a[c] = p.o_p[row * D + lane + 32 * c];
   Lp = p.lse_p[row];
   // the row's slot in the active list, if any (the list has at most B <= 64 entries)
-  const int na = clamp_active(p.n_active[s], p.B);
   int slot = -1;
-  for (int base = 0; base < na && slot < 0; base += 32) {
-    const int i = base + lane;
-    const unsigned hit = __ballot_sync(0xffffffffu, i < na && p.active_idx[s * p.B + i] == tok);
-    if (hit) slot = base + __ffs(hit) - 1;
+  if (f.slot_map) {
+    slot = f.slot_map[s * p.B + tok];
+    if (slot >= p.B) slot = -1;
+  } else {
+    const int na = clamp_active(p.n_active[s], p.B);
+    for (int base = 0; base < na && slot < 0; base += 32) {
+      const int i = base + lane;
+      const unsigned hit = __ballot_sync(0xffffffffu, i < na && p.active_idx[s * p.B + i] == tok);
+      if (hit) slot = base + __ffs(hit) - 1;
+    }
   }
   if (slot >= 0) {
     const int rowk = slot * p.G + gi, rg = rowk / kRowsPerGroup, r = rowk % kRowsPerGroup;
@@ -598,6 +604,7 @@ int32_t launch_sparse_prefix_attn(losa_ctx* c, const void* q, const losa_kv_t* k
 bool finish_fuses_combine(const losa_ctx* c) { return c->shape.dtype == LOSA_BF16; }
 
 int32_t launch_attn_finish(losa_ctx* c, const void* q, const int32_t* active_idx, const int32_t* n_active,
+                           const int32_t* slot_map,
                            losa_state_t* state, void* out, float* lse_out_opt, cudaStream_t st) {
   const losa_shape_t& sh = c->shape;
   AttnParams ap = {};
@@ -618,6 +625,7 @@ int32_t launch_attn_finish(losa_ctx* c, const void* q, const int32_t* active_idx
   ap.n_ctas = c->lay.n_ctas;
   FinishParams fp;
   fp.q = q;
+  fp.slot_map = slot_map;
   fp.q_prev = state->q_prev;
   fp.o_b = reinterpret_cast<const float*>(c->ws + c->lay.block_o);
   fp.lse_b = reinterpret_cast<const float*>(c->ws + c->lay.block_lse);
