@@ -126,6 +126,16 @@ int32_t losa_destroy(losa_ctx* ctx);
  * (LOSA_ERR_TIMEOUT or LOSA_ERR_BOUNDS) and clears it, or LOSA_OK. */
 int32_t losa_poll_status(losa_ctx* ctx, void* stream);
 
+/* Bound of the waits inside the bf16 stage-4 kernel (its warps hand work to one another through
+ * shared-memory barriers), in SM clock cycles; `cycles` <= 0 restores the default of about one
+ * second.  A wait that outlasts the bound makes its thread block record LOSA_ERR_TIMEOUT, wait
+ * (again within a bound) for the page copies and tensor-core instructions it had already started,
+ * release its tensor memory and return: the launch ends normally, the step's results are
+ * meaningless, and the context stays usable.  A bound of a few cycles makes every launch end this
+ * way, which is how the path is exercised without starving any barrier.  Host-side switch; takes
+ * effect for calls issued after it returns (a captured graph keeps the bound it was captured with). */
+int32_t losa_set_wait_limit(losa_ctx* ctx, int64_t cycles);
+
 /* The CUDA error code (cudaError_t or CUresult value) behind the last LOSA_ERR_CUDA, else 0. */
 int32_t losa_last_cuda_error(const losa_ctx* ctx);
 
@@ -151,13 +161,16 @@ int32_t losa_stage4_last_ms(losa_ctx* ctx, float* out_ms);
  *       active whatever m says.
  *   active_idx [N, B] int32 out: the active tokens of each sequence in ascending order, then -1.
  *       The m tokens with the largest Delta are chosen; equal Delta goes to the lower token index.
- *   n_active [N] int32 out.   delta_opt [N, B] fp32 out or NULL. */
+ *   n_active [N] int32 out.   delta_opt [N, B] fp32 out or NULL.
+ *   Inputs must be finite.  A Delta that is NaN (NaN or opposite infinities in a row) is ranked as
+ *   +inf, so that the ranking stays a total order and n_active never exceeds m; what the definition
+ *   would select in that case is left open. */
 int32_t losa_select_active(losa_ctx* ctx, const void* x_cur, const void* x_prev, int32_t row_width,
                            const int32_t* m_per_seq, const int32_t* step, int32_t* active_idx,
                            int32_t* n_active, float* delta_opt, void* stream);
 
-/* Stage 1, threshold variant (appendix: the locality heat maps select tokens "where cumulative
- * normalised MSE reaches 50% of the layer total", tau = 0.5).  Delta and the ranking are those of
+/* Stage 1, threshold variant (the rule behind the appendix's locality heat maps, which mark the
+ * tokens that carry half of a layer's total change: tau = 0.5).  Delta and the ranking are those of
  * losa_select_active; the active set is the shortest leading part of the ranking whose Delta add up
  * to at least tau times the sum of Delta over the block (both sums taken over the ranking in order,
  * in fp64).  A block whose queries did not change at all has no active token.

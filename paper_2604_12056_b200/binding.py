@@ -30,7 +30,7 @@ EXPORTS = [
     "losa_update_prefix_cache", "losa_build_page_summaries", "losa_denoise_step_host",
     "losa_profile_stage4", "losa_stage4_last_ms", "losa_select_active_static",
     "losa_denoise_step", "losa_select_active_tau", "losa_page_scores_topk_pooled",
-    "losa_set_pooled_selection",
+    "losa_set_pooled_selection", "losa_set_wait_limit",
 ]
 
 
@@ -159,6 +159,10 @@ class Context:
 
     def set_pooled_selection(self, on: bool):
         self._check("losa_set_pooled_selection", lib().losa_set_pooled_selection(self._h, C.c_int32(1 if on else 0)))
+
+    def set_wait_limit(self, cycles: int):
+        """Bound of the bf16 stage-4 kernel's internal waits in SM clock cycles; <= 0 restores the default."""
+        self._check("losa_set_wait_limit", lib().losa_set_wait_limit(self._h, C.c_int64(int(cycles))))
 
     def profile_stage4(self, enable: bool):
         self._check("losa_profile_stage4", lib().losa_profile_stage4(self._h, C.c_int32(1 if enable else 0)))

@@ -159,6 +159,12 @@ int32_t losa_stage4_last_ms(losa_ctx* ctx, float* out_ms) {
   return LOSA_OK;
 }
 
+int32_t losa_set_wait_limit(losa_ctx* ctx, int64_t cycles) {
+  if (!ctx) return LOSA_ERR_INVALID_ARG;
+  ctx->wait_cycles = cycles > 0 ? cycles : 0;
+  return LOSA_OK;
+}
+
 int32_t losa_last_cuda_error(const losa_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
 int64_t losa_launch_count(const losa_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
@@ -287,9 +293,12 @@ int32_t losa_denoise_step(losa_ctx* ctx, const void* q, const void* k_blk, const
   if (rc == LOSA_OK) rc = launch_page_scores_topk(ctx, q, kv, buf->active_idx, buf->n_active, state->step, k, buf->topk_pages, nullptr, st, ctx->pooled_selection != 0);
   if (rc == LOSA_OK) rc = launch_page_union(ctx, buf->topk_pages, buf->active_idx, buf->n_active, k, kv->kv_len, state->step, buf->union_pages, buf->union_count, st);
   if (rc == LOSA_OK) rc = launch_sparse_prefix_attn(ctx, q, kv, buf->active_idx, buf->n_active, buf->union_pages, buf->union_count, state, st, true);
+  // join (also when a launch above failed: the forked kernel must not be left reading the caller's
+  // buffers, nor a capture be left with an unjoined branch), then one pass over the rows: (merge of
+  // the partial records,) merge with the block part, commit
+  const cudaError_t joined = cudaStreamWaitEvent(st, ctx->ev_join, 0);
   if (rc != LOSA_OK) return rc;
-  // join, then one pass over the rows: (merge of the partial records,) merge with the block part, commit
-  LOSA_CUDA_TRY(ctx, cudaStreamWaitEvent(st, ctx->ev_join, 0));
+  LOSA_CUDA_TRY(ctx, joined);
   if (finish_fuses_combine(ctx)) return launch_attn_finish(ctx, q, buf->active_idx, buf->n_active, slot_map, state, out, lse_out_opt, st);
   return launch_merge_commit(ctx, q, state, out, lse_out_opt, st);
 }

@@ -438,10 +438,17 @@ __global__ void append_block_kernel(T* __restrict__ k_pages, T* __restrict__ v_p
                       blk_off, blk_stride, (static_cast<size_t>(phys) * Hkv + kh) * D, j);
 }
 
-__global__ void finalize_counters_kernel(int32_t* __restrict__ kv_len, int32_t* __restrict__ step, int N, int B) {
+// A sequence whose block did not fit its page-table row (the append kernel reported it and wrote
+// nothing beyond the row) keeps its length: later steps must not index pages past P_max.
+__global__ void finalize_counters_kernel(int32_t* __restrict__ kv_len, int32_t* __restrict__ step, int N, int B,
+                                         int g, int Pmax) {
   grid_dep_wait();
   const int s = threadIdx.x;
-  if (s < N) { kv_len[s] += B; step[s] = 0; }
+  if (s < N) {
+    const long long cap = static_cast<long long>(Pmax) * g;
+    if (static_cast<long long>(kv_len[s]) + B <= cap) kv_len[s] += B;
+    step[s] = 0;
+  }
 }
 
 template <typename T, int D, bool MERGE>
@@ -492,7 +499,8 @@ int32_t launch_update_t(losa_ctx* c, losa_kv_t* kv, losa_state_t* state, const v
       sh.n_kv_heads, sh.head_dim, sh.page_size, sh.max_pages_per_seq, kv->n_phys_pages, status_ptr(c));
   int32_t rc = after_launch(c);
   if (rc != LOSA_OK) return rc;
-  launch_k(finalize_counters_kernel, 1, std::max(32, sh.batch), 0, st, kv->kv_len, state->step, sh.batch, sh.block_size);
+  launch_k(finalize_counters_kernel, 1, std::max(32, sh.batch), 0, st, kv->kv_len, state->step, sh.batch, sh.block_size,
+           sh.page_size, sh.max_pages_per_seq);
   return after_launch(c);
 }
 

@@ -59,6 +59,10 @@ struct losa_ctx {
   cudaEvent_t ev_fork, ev_join;
   // selector of the whole-step path: 0 = one list per query head, 1 = pooled over the heads of a KV head
   int32_t pooled_selection;
+  // bound of the mbarrier waits of the bf16 stage-4 kernel in SM clock cycles (0 = the default, about a second)
+  int64_t wait_cycles;
+  // the stage-4 kernel of this context has had its shared-memory attribute set
+  int32_t attn_attr_set;
   // optional timing of the stage-4 main kernel
   int32_t profile;
   cudaEvent_t ev_begin, ev_end;

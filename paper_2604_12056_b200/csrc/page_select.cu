@@ -92,7 +92,8 @@ page_scores_kernel(const T* __restrict__ q, const T* __restrict__ kmin, const T*
     tok0[i] = a < B ? ld_keep_s32(active_idx + s * B + a) : 0;
   }
   if (step && step[s] == 0) return;
-  const int P = pages_of(kv_len[s], g);
+  int P = pages_of(kv_len[s], g);
+  if (P > Pmax) { set_status(status, LOSA_ERR_BOUNDS); P = Pmax; }    // a length beyond the page-table row
   if (p0 >= P) return;
   int na = n_active[s];
   na = na < 0 ? 0 : (na > B ? B : na);
@@ -262,7 +263,7 @@ __global__ void __launch_bounds__(kThreads)
 topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ kv_len,
             const int32_t* __restrict__ active_idx, const int32_t* __restrict__ n_active,
             const int32_t* __restrict__ step, int32_t* __restrict__ topk_pages,
-            float* __restrict__ topk_scores, int B, int Hq, int g, int k, int score_stride, int pool,
+            float* __restrict__ topk_scores, int B, int Hq, int g, int k, int Pmax, int score_stride, int pool,
             int32_t* __restrict__ status) {
   grid_dep_wait();
   extern __shared__ __align__(16) unsigned long long keys[];
@@ -273,7 +274,8 @@ topk_kernel(const float* __restrict__ scores, const int32_t* __restrict__ kv_len
   if (a >= na) return;
   int tok = active_idx[s * B + a];
   if (tok < 0 || tok >= B) { set_status(status, LOSA_ERR_BOUNDS); return; }
-  const int P = pages_of(kv_len[s], g);
+  int P = pages_of(kv_len[s], g);
+  if (P > Pmax) { set_status(status, LOSA_ERR_BOUNDS); P = Pmax; }
   const int tid = threadIdx.x;
   int n = 2;
   while (n < P) n <<= 1;
@@ -477,7 +479,7 @@ __global__ void __launch_bounds__(kSelThreads)
 topk_select_kernel(float* __restrict__ scores, const int32_t* __restrict__ kv_len,
                    const int32_t* __restrict__ active_idx, const int32_t* __restrict__ n_active,
                    const int32_t* __restrict__ step, int32_t* __restrict__ topk_pages,
-                   float* __restrict__ topk_scores, int N, int B, int Hq, int g, int k, int score_stride, int pool,
+                   float* __restrict__ topk_scores, int N, int B, int Hq, int g, int k, int Pmax, int score_stride, int pool,
                    int32_t* __restrict__ status) {
   grid_dep_trigger();
   grid_dep_wait();
@@ -489,7 +491,8 @@ topk_select_kernel(float* __restrict__ scores, const int32_t* __restrict__ kv_le
   if (step && step[s] == 0) return;
   int na = n_active[s];
   na = na > B ? B : na;
-  const int P = pages_of(kv_len[s], g);
+  int P = pages_of(kv_len[s], g);
+  if (P > Pmax) { if (threadIdx.x == 0) set_status(status, LOSA_ERR_BOUNDS); P = Pmax; }
   const int kk = min(k, P);
   for (int a = j; a < na; a += kSelSlots) {
     const int tok = active_idx[s * B + a];
@@ -659,11 +662,11 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
     if (pool > 1)
       launch_k(topk_select_kernel<true>, queries, kSelThreads, 0, st,
           sc, kv->kv_len, active_idx, n_active, step, topk_pages, topk_scores_opt, sh.batch, sh.block_size,
-          sh.n_q_heads, sh.page_size, k, c->lay.score_stride, pool, status_ptr(c));
+          sh.n_q_heads, sh.page_size, k, sh.max_pages_per_seq, c->lay.score_stride, pool, status_ptr(c));
     else
       launch_k(topk_select_kernel<false>, queries, kSelThreads, 0, st,
           sc, kv->kv_len, active_idx, n_active, step, topk_pages, topk_scores_opt, sh.batch, sh.block_size,
-          sh.n_q_heads, sh.page_size, k, c->lay.score_stride, 1, status_ptr(c));
+          sh.n_q_heads, sh.page_size, k, sh.max_pages_per_seq, c->lay.score_stride, 1, status_ptr(c));
     return after_launch(c);
   }
   // budgets beyond what one warp can sort: whole-list bitonic sort, one CTA per query
@@ -673,7 +676,7 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
   dim3 grid(sh.n_q_heads / pool, sh.block_size, sh.batch);
   launch_k(topk_kernel, grid, kThreads, smem, st, sc, kv->kv_len, active_idx, n_active, step, topk_pages,
                                             topk_scores_opt, sh.block_size, sh.n_q_heads, sh.page_size,
-                                            k, c->lay.score_stride, pool, status_ptr(c));
+                                            k, sh.max_pages_per_seq, c->lay.score_stride, pool, status_ptr(c));
   return after_launch(c);
 }
 

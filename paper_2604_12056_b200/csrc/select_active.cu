@@ -74,7 +74,10 @@ select_active_kernel(const T* __restrict__ x_cur, const T* __restrict__ x_prev, 
   __syncthreads();
   if (!s_last) return;
   __threadfence();
-  if (tid < B) s_delta[tid] = *(reinterpret_cast<volatile double*>(delta_ws) + s * B + tid);
+  if (tid < B) {
+    const double dv = *(reinterpret_cast<volatile double*>(delta_ws) + s * B + tid);
+    s_delta[tid] = dv != dv ? static_cast<double>(INFINITY) : dv;    // NaN ranks as +inf: the order below stays total
+  }
   __syncthreads();
   if (warp != 0) return;
 

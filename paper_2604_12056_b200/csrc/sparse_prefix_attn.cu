@@ -43,21 +43,9 @@ struct AttnParams {
   int32_t* status;
   int N, B, Hq, Hkv, G, Pmax, n_phys, n_rg, n_seg, n_ctas;
   float sm_scale;
-#ifdef LOSA_TRACE
-  unsigned long long* trace;   // [n_ctas][8] timestamps, development builds only
-#endif
+  long long wait_cycles;  // bound of every mbarrier wait of the bf16 main kernel, in SM clock cycles
 };
 
-#ifdef LOSA_TRACE
-__device__ __forceinline__ unsigned long long gtime() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-#define LOSA_STAMP(slot) do { if (p.trace) p.trace[blockIdx.x * 8 + (slot)] = gtime(); } while (0)
-#else
-#define LOSA_STAMP(slot) do { } while (0)
-#endif
 
 // Partial results.  A slot (CTA b, segment seg -> b + seg) holds eight records, record t for the
 // rows 16t .. 16t+15 of the row group: m[16], l[16], o[16][D] (un-normalised, relative to m).
@@ -379,7 +367,8 @@ __global__ void __launch_bounds__(kFinishThreads) attn_finish_kernel(AttnParams 
 }
 
 // ===================================================================== bf16 TMA + tensor-core kernel: shared pieces
-constexpr long long kWaitCycles = 2000000000ll;   // ~1 s: bound of every mbarrier wait
+constexpr long long kWaitCycles = 2000000000ll;   // ~1 s: default bound of every mbarrier wait
+constexpr long long kDrainCycles = 20000000ll;    // ~10 ms: bound of the waits for work already in flight when a CTA gives up
 constexpr int kSmemBudget = 232448;                // 227 KB opt-in limit per CTA
 
 constexpr int kStageIdx = 1024;     // active_idx entries (N * B) cached in shared memory when they fit
@@ -409,18 +398,25 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait.  Returns false (and raises the CTA's abort flag) when the bound runs out or
 // another warp has already given up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int32_t* status) {
+                                          int32_t* status, long long limit) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitCycles) {
+    if (clock64() - t0 > limit) {
       *abort_flag = 1;
       set_status(status, LOSA_ERR_TIMEOUT);
       return false;
     }
   }
+}
+// Wait of a CTA that has given up, for work it had already put in flight (page copies into its
+// shared memory, tensor-core instructions on its tensor memory): bounded by kDrainCycles, ignores
+// the abort flag, reports nothing (the status word already holds the reason).
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity) && clock64() - t0 < kDrainCycles) {}
 }
 // The K / V pages are read once per launch: they are marked evict-first in L2, so that the stream
 // does not push out the small arrays the following kernels read (partial records, in-block output).
@@ -508,10 +504,9 @@ int32_t ensure_tensor_maps(losa_ctx* c, const losa_kv_t* kv) {
 template <int D, int GP>
 int32_t launch_tc5(losa_ctx* c, const AttnParams& ap, cudaStream_t st, bool with_combine) {
   constexpr int smem = tc5_smem_bytes<D>();
-  static int attr_device = -1;
-  if (attr_device != c->device) {
+  if (!c->attn_attr_set) {          // a context has one shape, hence one instantiation, on one device
     LOSA_CUDA_TRY(c, cudaFuncSetAttribute(attn_tc5_kernel<D, GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    attr_device = c->device;
+    c->attn_attr_set = 1;
   }
   CUtensorMap mk, mv;
   memcpy(&mk, c->tmap_k, sizeof(mk));
@@ -529,7 +524,10 @@ template <typename T, int D, int GP>
 int32_t launch_simt(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
   const size_t smem = (static_cast<size_t>(2) * GP * D + 2 * kRowsPerGroup * D + 2 * kRowsPerGroup) * sizeof(float) +
                       (ap.n_seg + 1) * sizeof(int);
-  LOSA_CUDA_TRY(c, cudaFuncSetAttribute(attn_simt_kernel<T, D, GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  if (!c->attn_attr_set) {
+    LOSA_CUDA_TRY(c, cudaFuncSetAttribute(attn_simt_kernel<T, D, GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    c->attn_attr_set = 1;
+  }
   if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_begin, st));
   launch_k(attn_simt_kernel<T, D, GP>, ap.n_ctas, 256, smem, st, ap);
   if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_end, st));
@@ -551,10 +549,6 @@ int32_t dispatch_page(losa_ctx* c, const AttnParams& ap, cudaStream_t st, bool w
 
 }  // namespace
 
-#ifdef LOSA_TRACE
-unsigned long long* g_trace = nullptr;
-extern "C" void losa_debug_set_trace(void* p) { g_trace = static_cast<unsigned long long*>(p); }
-#endif
 
 int32_t launch_sparse_prefix_attn(losa_ctx* c, const void* q, const losa_kv_t* kv,
                                   const int32_t* active_idx, const int32_t* n_active,
@@ -594,9 +588,7 @@ int32_t launch_sparse_prefix_attn(losa_ctx* c, const void* q, const losa_kv_t* k
   ap.n_seg = c->lay.n_segments;
   ap.n_ctas = c->lay.n_ctas;
   ap.sm_scale = sh.sm_scale;
-#ifdef LOSA_TRACE
-  ap.trace = g_trace;
-#endif
+  ap.wait_cycles = c->wait_cycles > 0 ? c->wait_cycles : kWaitCycles;
   const bool with_combine = !(defer_combine && finish_fuses_combine(c));
   return sh.head_dim == 128 ? dispatch_page<128>(c, ap, st, with_combine) : dispatch_page<64>(c, ap, st, with_combine);
 }

@@ -21,16 +21,6 @@
 // mbarriers; every wait is bounded; tensor memory is returned on every path.
 #pragma once
 
-#ifdef LOSA_TRACE
-#define TC5_TR_DECL(...) long long __VA_ARGS__; long long tr_t = clock64()
-#define TC5_TR(x) do { const long long now_ = clock64(); x += now_ - tr_t; tr_t = now_; } while (0)
-#define TC5_TR_OUT(off, ...) do { if (p.trace) { const long long v_[] = {__VA_ARGS__}; for (unsigned i_ = 0; i_ < sizeof(v_) / 8; ++i_) p.trace[blockIdx.x * 32 + (off) + i_] = v_[i_]; } } while (0)
-#else
-#define TC5_TR_DECL(...) do { } while (0)
-#define TC5_TR(x) do { } while (0)
-#define TC5_TR_OUT(off, ...) do { } while (0)
-#endif
-
 constexpr int kTc5SoftmaxWarps = 8;              // two sets of four: set h takes columns 64h .. 64h+63 of every group
 constexpr int kTc5QkWarp = 8, kTc5PvWarp = 9, kTc5KWarp = 10, kTc5VWarp = 11;
 constexpr int kTc5Threads = 384;
@@ -133,7 +123,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   static_assert(D == 64 || D == 128, "head dimensions of the tensor-core path");
   static_assert(GP == 16 || GP == 32 || GP == 64, "page sizes of the tensor-core path");
   static_assert(NR >= 2 && PG <= kTc5PgMax, "ring too shallow / group too long");
-  static_assert(8 * (4 * 6 + 12) + 4 * kTc5MetaRing * kTc5PgMax + 16 <= 1024, "tail layout");
+  static_assert(8 * (4 * 6 + 14) + 4 * kTc5MetaRing * kTc5PgMax + 16 <= 1024, "tail layout");
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
@@ -144,7 +134,8 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   const uint32_t tail_s = base + 2 * NR * SLOT;
   const uint32_t kfull = tail_s, kfree = kfull + 8 * NR, vfull = kfree + 8 * NR, vfree = vfull + 8 * NR;
   const uint32_t s_full = vfree + 8 * NR, s_free = s_full + 16, p_full = s_free + 16, q_full = p_full + 16, q_free = q_full + 8, xbar = q_free + 8;
-  volatile int* meta = reinterpret_cast<volatile int*>(tail + 8 * (4 * 6 + 12));   // [kTc5MetaRing][kTc5PgMax] valid tokens per page
+  const uint32_t drain_bar = xbar + 32;            // two barriers: the issuing threads' last commit when the CTA gives up
+  volatile int* meta = reinterpret_cast<volatile int*>(tail + 8 * (4 * 6 + 14));   // [kTc5MetaRing][kTc5PgMax] valid tokens per page
   volatile int* abort_flag = meta + kTc5MetaRing * kTc5PgMax;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(abort_flag) + 1);
   int* pre = reinterpret_cast<int*>(tail + 1024);
@@ -156,10 +147,6 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   const bool staged = p.N * p.B <= kStageIdx && p.N <= kStageSeq;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-#ifdef LOSA_TRACE
-  const unsigned long long tr_g0 = gtime();
-  unsigned long long tr_g1 = 0, tr_g2 = 0;
-#endif
   if (tid == 0) {
     for (int i = 0; i < NR; ++i) {
       mbar_init(kfull + 8 * i, 1);
@@ -175,6 +162,8 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     mbar_init(q_full, kTc5SoftmaxWarps);
     mbar_init(q_free, 1);
     for (int i = 0; i < 4; ++i) mbar_init(xbar + 8 * i, 2);      // the two softmax warps of a scheduler meet here
+    mbar_init(drain_bar, 1);
+    mbar_init(drain_bar + 8, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -213,6 +202,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   auto kv_len_of = [&](int s) { return staged ? len_s[s] : p.kv_len[s]; };
   auto token_of = [&](int s, int a) { return staged ? tok_s[s * p.B + a] : p.active_idx[s * p.B + a]; };
 
+  int issued = -1;                                   // producer warps: newest group whose copies have been issued
   if (warp == kTc5KWarp || warp == kTc5VWarp) {
     // ------------------------------------------------------------------ producer warps: one for K, one for V
     // Lane j of a batch of 32 consecutive items resolves item -> logical page -> physical page (a
@@ -276,7 +266,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         const int slot = grp % NR, round = grp / NR;
         if (j0 == 0) {
           int ok = 1;
-          if (lane == 0 && round > 0) ok = mbar_wait(free0 + 8 * slot, (round - 1) & 1, abort_flag, p.status);
+          if (lane == 0 && round > 0) ok = mbar_wait(free0 + 8 * slot, (round - 1) & 1, abort_flag, p.status, p.wait_cycles);
           go = __shfl_sync(0xffffffffu, ok, 0) != 0;
           if (!go) break;
         }
@@ -290,6 +280,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
 #pragma unroll
           for (int hf = 0; hf < HALVES; ++hf) tma_load_4d(dst + hf * HS, map, full0 + 8 * slot, hf * 64, 0, b.kh, b.phys, policy);
         }
+        issued = grp;
         pos += cnt;
       }
       a = a_next;
@@ -300,18 +291,13 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     if (lane == 0) {
       int sg = sg0, item = lo, piece = 0, g = 0;
       bool ok = true;
-      TC5_TR_DECL(tr_q = 0, tr_k = 0, tr_s = 0, tr_i = 0);
       while (item < hi && ok) {
         const int seg_end = min(hi, pre[sg + 1]);
-        TC5_TR(tr_i);
-        ok = mbar_wait(q_full, piece & 1, abort_flag, p.status);
-        TC5_TR(tr_q);
+        ok = mbar_wait(q_full, piece & 1, abort_flag, p.status, p.wait_cycles);
         for (int first = item; first < seg_end && ok; first += PG, ++g) {
           const int ng = min(PG, seg_end - first), b = g & 1, use = g >> 1, slot = g % NR;
-          ok = mbar_wait(kfull + 8 * slot, (g / NR) & 1, abort_flag, p.status);
-          TC5_TR(tr_k);
-          ok = ok && (use == 0 || mbar_wait(s_free + 8 * b, (use - 1) & 1, abort_flag, p.status));
-          TC5_TR(tr_s);
+          ok = mbar_wait(kfull + 8 * slot, (g / NR) & 1, abort_flag, p.status, p.wait_cycles);
+          ok = ok && (use == 0 || mbar_wait(s_free + 8 * b, (use - 1) & 1, abort_flag, p.status, p.wait_cycles));
           if (!ok) break;
           tc5_fence_after();
           const uint32_t idesc = tc5_idesc(kRowsPerGroup, ng * GP, 0), kt = kring + slot * SLOT;
@@ -322,14 +308,12 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
           tc5_commit(s_full + 8 * b);
           tc5_commit(kfree + 8 * slot);
           if (first + PG >= seg_end) tc5_commit(q_free);        // Q may be replaced once the piece's last product has run
-          TC5_TR(tr_i);
         }
         item = seg_end;
         ++sg;
         ++piece;
         while (item < hi && pre[sg + 1] <= item) ++sg;
       }
-      TC5_TR_OUT(0, tr_q, tr_k, tr_s, tr_i, g);
     }
   } else if (warp == kTc5PvWarp) {
     // ------------------------------------------------------------------ P V issuer (one thread)
@@ -337,16 +321,12 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       const uint32_t idesc = tc5_idesc(kRowsPerGroup, D, 1);
       int sg = sg0, item = lo, g = 0;
       bool ok = true;
-      TC5_TR_DECL(tr_v = 0, tr_p = 0, tr_i = 0);
       while (item < hi && ok) {
         const int seg_end = min(hi, pre[sg + 1]);
         for (int first = item; first < seg_end && ok; first += PG, ++g) {
           const int ng = min(PG, seg_end - first), b = g & 1, use = g >> 1, slot = g % NR;
-          TC5_TR(tr_i);
-          ok = mbar_wait(vfull + 8 * slot, (g / NR) & 1, abort_flag, p.status);
-          TC5_TR(tr_v);
-          ok = ok && mbar_wait(p_full + 8 * b, use & 1, abort_flag, p.status);
-          TC5_TR(tr_p);
+          ok = mbar_wait(vfull + 8 * slot, (g / NR) & 1, abort_flag, p.status, p.wait_cycles);
+          ok = ok && mbar_wait(p_full + 8 * b, use & 1, abort_flag, p.status, p.wait_cycles);
           if (!ok) break;
           tc5_fence_after();
           const uint32_t vt = vring + slot * SLOT;
@@ -355,13 +335,11 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                        (first == item && ks == 0) ? 0u : 1u);
           tc5_commit(vfree + 8 * slot);
           tc5_commit(s_free + 8 * b);
-          TC5_TR(tr_i);
         }
         item = seg_end;
         ++sg;
         while (item < hi && pre[sg + 1] <= item) ++sg;
       }
-      TC5_TR_OUT(8, tr_v, tr_p, tr_i);
     }
   } else {
     // ------------------------------------------------------------------ softmax / epilogue warps
@@ -380,11 +358,8 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     // every wait of these warps ends with one answer for the whole warp: the tensor-memory
     // instructions that follow need all 32 lanes
     auto warp_wait = [&](uint32_t bar, uint32_t parity) {
-      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, p.status)) != 0;
+      return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, p.status, p.wait_cycles)) != 0;
     };
-#ifdef LOSA_TRACE
-    tr_g1 = gtime();
-#endif
     int n_meet = 0;
     auto pair_sync = [&]() {                                    // bounded like every other wait
       __syncwarp();
@@ -395,7 +370,6 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     };
     int sg = sg0, item = lo, piece = 0, g = 0;
     bool ok = true;
-    TC5_TR_DECL(tr_q = 0, tr_w = 0, tr_1 = 0, tr_r = 0, tr_2 = 0, tr_a = 0, tr_e = 0);
     while (item < hi && ok) {
       const int seg_end = min(hi, pre[sg + 1]);
       const int rg = sg % p.n_rg, sk = sg / p.n_rg, s = sk / p.Hkv, kh = sk % p.Hkv;
@@ -426,7 +400,6 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         __syncwarp();
         if (lane == 0) mbar_arrive(q_full, 1);
       }
-      TC5_TR(tr_q);
       float m_ref = -INFINITY, l = 0.f;                         // l: this thread's columns only
       bool o_valid = false;                                     // O holds at least one group of this piece
       for (int first = item; first < seg_end && ok; first += PG, ++g) {
@@ -436,10 +409,6 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         ok = warp_wait(s_full + 8 * b, use & 1);
         if (!ok) break;
         tc5_fence_after();
-        TC5_TR(tr_w);
-#ifdef LOSA_TRACE
-        if (g == 0) tr_g2 = gtime();
-#endif
         // pages with fewer than GP tokens (the last page of a prefix), or a group that ends inside a
         // 32-column chunk, need per-column masks; everything else takes the plain path
         bool ragged = (ncol & 31) != 0;
@@ -479,7 +448,6 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
           xmax[(b * 2 + h) * kRowsPerGroup + r] = mx_own;
           ok = pair_sync();
           const float m_new = fmaxf(mx_own, xmax[(b * 2 + (h ^ 1)) * kRowsPerGroup + r]) * scale2;
-          TC5_TR(tr_1);
           float corr = 1.f;
           if (m_new > m_ref + kTc5Tau || (m_ref == -INFINITY && m_new > -INFINITY)) {
             corr = (m_ref == -INFINITY) ? 0.f : ex2(m_ref - m_new);
@@ -504,7 +472,6 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
               tc5_wait_st();
             }
           }
-          TC5_TR(tr_r);
           // ---- pass 2: P = 2^(s - m) as bf16, written over the scores (column c of P takes the
           //      place of columns 2c, 2c+1 of S; every score of the group is in registers by now,
           //      the partner's too: it has passed the pair barrier)
@@ -528,7 +495,6 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
             tc5_wait_st();
             l += (sum[0] + sum[1]) + (sum[2] + sum[3]);
           }
-          TC5_TR(tr_2);
         }
         if (!ok) break;
         if (ragged) {
@@ -555,7 +521,6 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         __syncwarp();
         if (lane == 0) mbar_arrive(p_full + 8 * b, 1);
         o_valid = true;
-        TC5_TR(tr_a);
       }
       if (!ok) break;
       // ---- the piece's record: one 16-row tile record per 16 rows, reference maximum in base-2
@@ -582,18 +547,34 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         if (h == 0 && r < rows) { rec[rr] = m_ref; rec[kTileRows + rr] = l + xsum[r]; }
       }
       tc5_fence_before();
-      TC5_TR(tr_e);
       item = seg_end;
       ++sg;
       ++piece;
       while (item < hi && pre[sg + 1] <= item) ++sg;
     }
-#ifdef LOSA_TRACE
-    if (tid == 0) TC5_TR_OUT(16, tr_q, tr_w, tr_1, tr_r, tr_2, tr_a, tr_e, piece, hi - lo, (long long)tr_g0, (long long)tr_g1, (long long)tr_g2, (long long)gtime());
-#endif
   }
   // ---- every thread that passed the allocation meets here; tensor memory is returned on all paths
   tc5_fence_before();
   __syncthreads();
+  if (*abort_flag) {
+    // The CTA has given up (a wait ran out).  Its shared and tensor memory must not be handed on
+    // while work it started is still in flight: the producers wait, within a bound, for the newest
+    // round of copies of every ring slot (a group that was begun has had all its copies issued: the
+    // producer loop only stops between groups), the issuing threads for the products they issued.
+    if ((warp == kTc5KWarp || warp == kTc5VWarp) && lane == 0) {
+      const uint32_t full0 = warp == kTc5VWarp ? vfull : kfull;
+      for (int sl = 0; sl < NR; ++sl) {
+        if (issued < sl) continue;
+        const int gl = issued - (issued - sl) % NR;
+        mbar_drain(full0 + 8 * sl, (gl / NR) & 1);
+      }
+    }
+    if ((warp == kTc5QkWarp || warp == kTc5PvWarp) && lane == 0) {
+      const uint32_t bar = drain_bar + (warp == kTc5PvWarp ? 8 : 0);
+      tc5_commit(bar);
+      mbar_drain(bar, 0);
+    }
+    __syncthreads();
+  }
   if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(TMEM_COLS) : "memory");
 }

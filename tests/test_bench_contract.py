@@ -37,3 +37,31 @@ def test_product_arm_needs_a_gpu():
     r = run_bench("--workload", "c1", "--steps", "4", "--warmup", "3")
     assert r.returncode != 0
     assert not [ln for ln in r.stdout.splitlines() if ln.startswith("{")]      # no result line of any kind
+
+
+def test_timed_walk_always_holds_losa_steps_in_block_proportion():
+    """The K timed layer-steps are cut into ceil(K / T) dense first steps and the rest LoSA steps,
+    whatever K the caller asks for: the walk of the driver's short run (20 steps), of the default
+    run (4 blocks of 36 layers) and of a single-layer run."""
+    sys.path.insert(0, ROOT)
+    import bench
+    for K, T, L, want_layers in ((20, 8, 36, 3), (1152, 8, 36, 36), (16, 8, 1, 1), (7, 16, 1, 1), (100, 8, 36, 13)):
+        L_eff, sweeps = bench.schedule(K, T, L)
+        assert L_eff == want_layers
+        assert sum(n for _, _, n in sweeps) == K
+        dense = sum(n for _, t, n in sweeps if t == 0)
+        assert dense == -(-K // T) and dense < K
+        assert all(n == L_eff for _, _, n in sweeps[:-1]) and 1 <= sweeps[-1][2] <= L_eff
+        # model order from a block boundary: consecutive sweeps are consecutive denoising steps
+        assert [(b * T + t) for b, t, _ in sweeps] == list(range(len(sweeps)))
+    L_eff, sweeps = bench.schedule(20, 8, 36)
+    assert [(t, n) for _, t, n in sweeps] == [(0, 3), (1, 3), (2, 3), (3, 3), (4, 3), (5, 3), (6, 2)]
+
+
+def test_both_arms_name_the_workload_identically():
+    sys.path.insert(0, ROOT)
+    import bench
+    from paper_2604_12056_b200 import workloads as wl
+    src = open(os.path.join(ROOT, "bench.py")).read()
+    assert src.count("workload_name(") == 3          # the definition and one use per arm, nothing appended to the reference arm's
+    assert "36 layer(s)" in bench.workload_name(wl.config("c5"), 36)

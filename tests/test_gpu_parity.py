@@ -155,13 +155,14 @@ def test_pooled_selector_whole_blocks(fused):
     run_blocks(cfg, pooled=True, fused=fused, want_scores=not fused)
 
 
-@pytest.mark.parametrize("pages,topk", [(700, 600), (1100, 8)])
-def test_pooled_selector_long_lists_and_large_budgets(pages, topk):
+@pytest.mark.parametrize("pooled", [True, False])
+@pytest.mark.parametrize("pages,topk", [(700, 600), (1100, 8), (1100, 600)])
+def test_long_lists_and_large_budgets(pages, topk, pooled):
     # k > 512 pages takes the whole-list sort; more than 1024 pages the selection that re-reads its
-    # row (pooled once into scratch): the pooled rows go through both
+    # score row instead of keeping it in registers: per-head lists and pooled lists go through both
     cfg = wl.config("c2", n_q_heads=4, n_kv_heads=2, head_dim=64, page_size=16, kv_lens=(16 * pages,),
                     block_size=4, steps=2, topk=topk, m_active=2)
-    run_blocks(cfg, pooled=True)
+    run_blocks(cfg, pooled=pooled)
 
 
 @pytest.mark.parametrize("name", ["p1", "p2"])
@@ -210,7 +211,7 @@ def test_out_of_range_page_table_is_reported_not_fatal():
     w = wl.Workload(cfg)
     g = LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len)
     inp = w.start_block()
-    g.page_table[0, 3] = 10 ** 6          # logical page 3 now names a page outside the pool
+    g.page_table[0, 3] = g.k_pages.shape[0]          # logical page 3 now names the first page outside the pool
     g.run_step(to_device(inp.q), to_device(inp.k_blk), to_device(inp.v_blk), to_device(inp.m_per_seq))
     assert g.ctx.poll_status() == B.LOSA_ERR_BOUNDS
     assert g.ctx.poll_status() == 0       # cleared by the poll; the context stays usable
@@ -221,6 +222,94 @@ def test_out_of_range_page_table_is_reported_not_fatal():
     assert g.ctx.poll_status() == 0
     ref = OracleLayer(w).run_step(inp)
     compare(g.snapshot(), ref, cfg, "after recovery")
+
+
+def test_prefix_length_beyond_the_page_table_is_reported_not_fatal():
+    """kv_len one token past what the page-table row can hold: stages 2 and 3 clamp the page count,
+    report LOSA_ERR_BOUNDS and touch nothing outside their rows; a block that does not fit is not
+    appended and the length stays as it was."""
+    from paper_2604_12056_b200 import binding as B
+    from paper_2604_12056_b200.layer import LosaLayer, to_device, to_host
+    cfg = wl.config("c2", kv_lens=(256,), block_size=8, steps=2, topk=2, m_active=2, n_blocks=0)
+    assert cfg.max_pages_per_seq == 8
+    w = wl.Workload(cfg)
+    g = LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len)
+    i0, i1 = w.start_block(), w.next_step()
+    dev = lambda i: (to_device(i.q), to_device(i.k_blk), to_device(i.v_blk), to_device(i.m_per_seq))
+    g.run_step(*dev(i0))
+    assert g.ctx.poll_status() == 0
+    g.kv_len.fill_(8 * 32 + 1)
+    g.run_step(*dev(i1))
+    assert g.ctx.poll_status() == B.LOSA_ERR_BOUNDS
+    snap = g.snapshot()
+    assert snap["uc"].max() <= 8 and snap["topk"].max() < 8
+    g.kv_len.fill_(256)
+    g.finalize_block(*dev(i1)[1:3])                  # 256 + 8 tokens need a ninth page: refused
+    assert g.ctx.poll_status() == B.LOSA_ERR_BOUNDS
+    assert to_host(g.kv_len).tolist() == [256] and to_host(g.step).tolist() == [0]
+    # the context is still good for a whole block (index rows of stable tokens are never written:
+    # start them from the fill value the fresh oracle layer starts from)
+    g.q_prev.zero_()
+    g.topk_pages.fill_(-9)
+    o = OracleLayer(w)
+    for i in (i0, i1):
+        g.run_step(*dev(i))
+        assert g.ctx.poll_status() == 0
+        compare(g.snapshot(), o.run_step(i), cfg, "after the refused append")
+
+
+def test_non_finite_rows_never_select_more_than_m_tokens():
+    """Inputs must be finite; if they are not, a NaN change score ranks as +inf, so the ranking is
+    still a total order and at most m tokens come out (ties on +inf go to the lower index)."""
+    import torch
+    from paper_2604_12056_b200 import binding as B
+    from paper_2604_12056_b200.layer import LosaLayer
+    cfg = wl.config("c1", kv_lens=(64,), block_size=16, steps=2)
+    w = wl.Workload(cfg)
+    g = LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len)
+    x_prev = torch.zeros((1, 16, 256), device="cuda")
+    x_cur = torch.randn((1, 16, 256), device="cuda")
+    x_cur[0, 3, 7] = float("nan")
+    x_cur[0, 11, 0] = float("inf")
+    x_cur[0, 12, 5] = float("nan")
+    m = torch.tensor([2], dtype=torch.int32, device="cuda")
+    one = torch.ones(1, dtype=torch.int32, device="cuda")
+    B.losa_select_active(g.ctx, x_cur, x_prev, 256, m, one, g.active_idx, g.n_active, g.delta)
+    assert g.ctx.poll_status() == 0
+    assert g.n_active.item() == 2 and g.active_idx[0, :3].tolist() == [3, 11, -1]
+    m.fill_(5)
+    B.losa_select_active(g.ctx, x_cur, x_prev, 256, m, one, g.active_idx, g.n_active, g.delta)
+    assert g.n_active.item() == 5 and set(g.active_idx[0, :5].tolist()) >= {3, 11, 12}
+
+
+def test_expired_wait_is_reported_and_the_context_stays_usable():
+    """The bf16 stage-4 kernel bounds every wait between its warps.  With the bound set to a few
+    cycles every thread block gives up at its first wait that is not satisfied at once: it records
+    LOSA_ERR_TIMEOUT, lets the copies and tensor-core instructions it had started finish, returns
+    its tensor memory and ends normally.  No barrier is starved and nothing hangs; afterwards, with
+    the default bound, the same context computes a whole block correctly."""
+    from paper_2604_12056_b200 import binding as B
+    from paper_2604_12056_b200.layer import LosaLayer, to_device
+    cfg = wl.config("c2", kv_lens=(4096, 1500), steps=3, topk=8, m_active=3)
+    w = wl.Workload(cfg)
+    g = LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len)
+    steps = w.block_steps()
+    dev = lambda i: (to_device(i.q), to_device(i.k_blk), to_device(i.v_blk), to_device(i.m_per_seq))
+    g.ctx.set_wait_limit(1)
+    g.run_step(*dev(steps[0]))
+    assert g.ctx.poll_status() == B.LOSA_ERR_TIMEOUT
+    assert g.ctx.poll_status() == 0                       # cleared by the poll
+    g.run_step_fused(*dev(steps[0]))                      # the whole-step path reports it the same way
+    assert g.ctx.poll_status() == B.LOSA_ERR_TIMEOUT
+    g.ctx.set_wait_limit(0)                               # default bound again
+    g.step.zero_()
+    g.q_prev.zero_()
+    g.topk_pages.fill_(-9)
+    o = OracleLayer(w)
+    for t, i in enumerate(steps):
+        g.run_step(*dev(i))
+        assert g.ctx.poll_status() == 0
+        compare(g.snapshot(), o.run_step(i), cfg, f"after the expired waits, step {t}")
 
 
 def test_full_size_c3_in_the_benchmark_configuration():

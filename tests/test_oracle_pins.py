@@ -194,9 +194,11 @@ def test_topk_order_ties_and_padding():
     assert topk3[0, 0, 0].tolist() == [0, 1, 2]
 
 
-def test_fixed_order_fp32_score_matches_its_specification():
-    """The interface fixes the fp32 summation order; re-derive it with numpy float32 ops."""
-    pb = Problem(9, N=1, Hq=2, Hkv=1, d=64, B=1, g=4, kv_lens=(64,))
+@pytest.mark.parametrize("d", [64, 128])
+def test_fixed_order_fp32_score_matches_its_specification(d):
+    """The interface fixes the fp32 summation order; re-derive it in exact rational arithmetic with
+    explicit roundings, for both head dimensions (d / 8 runs, butterfly offsets d / 16 .. 1)."""
+    pb = Problem(9, N=1, Hq=2, Hkv=1, d=d, B=1, g=4, kv_lens=(64,))
     orc.build_page_summaries(pb.sh, pb.kv)
     u32, _ = orc.page_scores_one(pb.sh, pb.q, pb.kv, 0, 0, 1)
     q = pb.q[0, 0, 1].astype(np.float32)
@@ -215,16 +217,19 @@ def test_fixed_order_fp32_score_matches_its_specification():
     for p in range(16):
         ph = pb.page_table[0, p]
         lo, hi = pb.kmin[ph, 0], pb.kmax[ph, 0]
-        c = np.zeros(8, np.float32)
-        for r in range(8):
+        runs = d // 8
+        c = np.zeros(runs, np.float32)
+        for r in range(runs):
             acc = np.float32(0.0)
             for jj in range(8):
                 j = 8 * r + jj
                 acc = fma32(max(q[j], np.float32(0)), hi[j], acc)
                 acc = fma32(min(q[j], np.float32(0)), lo[j], acc)
             c[r] = acc
-        for off in (4, 2, 1):
-            c = np.array([np.float32(c[i] + c[i ^ off]) for i in range(8)], np.float32)
+        off = runs // 2
+        while off >= 1:
+            c = np.array([np.float32(c[i] + c[i ^ off]) for i in range(runs)], np.float32)
+            off //= 2
         assert np.float32(c[0] + np.float32(0.0)).tobytes() == u32[p].tobytes()
 
 
