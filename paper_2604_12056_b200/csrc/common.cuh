@@ -63,6 +63,7 @@ struct losa_ctx {
   int64_t wait_cycles;
   // the stage-4 kernel of this context has had its shared-memory attribute set
   int32_t attn_attr_set;
+  int32_t scores_attr_set;   // likewise for the page-score kernel
   // optional timing of the stage-4 main kernel
   int32_t profile;
   cudaEvent_t ev_begin, ev_end;
@@ -155,6 +156,55 @@ __device__ __forceinline__ float warp_sum(float v) {
 }
 
 __device__ __forceinline__ int pages_of(int len, int g) { return (len + g - 1) / g; }
+
+// ---- shared-memory barriers (mbarrier) -------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* ptr) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(ptr));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+
+constexpr long long kWaitCycles = 2000000000ll;   // ~1 s: default bound of every mbarrier wait
+constexpr long long kDrainCycles = 20000000ll;    // ~10 ms: bound of the waits for work already in flight when a CTA gives up
+// Bounded wait.  Returns false (and raises the CTA's abort flag) when the bound runs out or
+// another warp has already given up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int32_t* status, long long limit) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > limit) {
+      *abort_flag = 1;
+      set_status(status, LOSA_ERR_TIMEOUT);
+      return false;
+    }
+  }
+}
+// Wait of a CTA that has given up, for work it had already put in flight (page copies into its
+// shared memory, tensor-core instructions on its tensor memory): bounded by kDrainCycles, ignores
+// the abort flag, reports nothing (the status word already holds the reason).
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity) && clock64() - t0 < kDrainCycles) {}
+}
 
 // ---- balanced split of the flattened (segment, union position) list over the CTAs ------------
 // Segment seg = (s * H_kv + kh) * n_row_groups + rg holds union_count[s, kh] items when its row

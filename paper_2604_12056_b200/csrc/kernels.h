@@ -15,6 +15,10 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
                                 const int32_t* step, int32_t k, int32_t* topk_pages,
                                 float* topk_scores_opt, cudaStream_t st, bool pooled = false);
 
+// Stage 2, first half: fp32 page scores of the active queries into the workspace's score rows.
+int32_t launch_page_scores(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
+                           const int32_t* n_active, const int32_t* step, cudaStream_t st);
+
 int32_t launch_page_union(losa_ctx* c, const int32_t* topk_pages, const int32_t* active_idx,
                           const int32_t* n_active, int32_t k, const int32_t* kv_len,
                           const int32_t* step, int32_t* union_pages, int32_t* union_count,

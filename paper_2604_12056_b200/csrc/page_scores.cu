@@ -1,0 +1,536 @@
+// Stage 2, first half — QUEST page scores for the active queries (Section 2.3, Section 4.2).
+//
+// U(p) = sum_j max(q_j,0) kmax[p,j] + min(q_j,0) kmin[p,j] decides integer page ids, so it is
+// evaluated in fp32 in the one order the interface fixes: per run of 8 consecutive j a chain of 16
+// fused multiply-adds (q+ kmax, then q- kmin, j ascending) from +0; the d/8 run sums combined by the
+// butterfly c[i] += c[i ^ off], off = d/16 .. 1; finally + 0.0f.
+//
+// Persistent kernel, one CTA of eight warps per SM.  The pages of all (sequence, KV head) pairs form
+// one flat list that is cut into equal contiguous ranges, one per CTA; a CTA walks its range in
+// tiles of TP pages of one (sequence, KV head), warp w taking pages [w WP, (w+1) WP) of every tile.
+//   loading : each warp copies its own pages' kmax / kmin into its slice of a ring of shared-memory
+//             stages with asynchronous 16-byte copies (cp.async; d elements of one summary are
+//             consecutive lanes, so every copy instruction is coalesced), NS - 1 tiles ahead, the
+//             page-table entries one tile further ahead.  A warp only ever reads what it copied
+//             itself, so completion is the warp's own cp.async group count: no producer warp, no
+//             barrier, no spinning.
+//   compute : a lane owns the runs u and u + d/16 of PG pages (two runs whose sums the butterfly's
+//             first level adds) and keeps them in registers as pairs, so the two chains advance
+//             together in one packed instruction (fma.rn.f32x2): half the issue slots of the scalar
+//             form, the same roundings.  Query rows are staged once per (sequence, KV head) as
+//             positive / negative parts in the same pair layout (bf16 inputs stay bf16 in shared
+//             memory, two to a word: max(q, 0) and min(q, 0) of a bf16 are bf16; the shared-memory
+//             pipe, which also carries the shuffles, is what bounds this kernel).  The first level
+//             of the butterfly is the add of a pair's halves; the other levels run over the d/16
+//             lanes of a page as a reduce-scatter over the 2 PG (page, row) pairs a lane works on:
+//             same additions, same order, 2 PG - 1 shuffles per pass instead of 2 PG log2(d/16).
+#include "kernels.h"
+
+namespace losa {
+namespace {
+
+constexpr int kPsWarps = 8;
+constexpr int kPsThreads = kPsWarps * 32;
+constexpr int kPsRowTile = 32;                      // query rows staged at a time
+constexpr int kPsSeqStage = 4;                      // sequences whose active lists are cached in shared memory
+constexpr int kPsMaxStages = 4;
+constexpr int kPsSmemBudget = 232448;               // 227 KB opt-in limit per CTA
+
+template <typename T, int D, int PG>
+struct PsCfg {
+  static constexpr int LPP = D / 16;                      // lanes per page
+  static constexpr int GPW = 32 / LPP;                    // page groups per warp
+  static constexpr int WP = GPW * PG;                     // pages per warp and tile
+  static constexpr int TP = kPsWarps * WP;                // pages per tile
+  static constexpr int HALF_BYTES = D * static_cast<int>(sizeof(T));   // kmax (or kmin) of one page and KV head
+  static constexpr int PAGE_BYTES = 2 * HALF_BYTES;
+  static constexpr int STAGE_BYTES = TP * PAGE_BYTES;
+  static constexpr int QBUF_BYTES = 2 * kPsRowTile * D * static_cast<int>(sizeof(T));   // q+ and q- of one row tile
+  static constexpr int NP = 2 * PG;                       // (page, row) pairs a lane works on per pass
+  static constexpr int CH = HALF_BYTES / 16;              // 16-byte chunks of one summary
+  static constexpr int RPI = 32 / CH;                     // summaries one warp-wide copy instruction covers
+  static constexpr int NI = 2 * WP / RPI;                 // copy instructions per warp and tile
+  static_assert(WP <= 32 && NP >= LPP / 2 && CH <= 32, "tile / reduce-scatter shape");
+};
+
+constexpr int ps_tail_bytes(int n_seq) {
+  // prefix [n_seq + 1] | active counts [n_seq] | cached active lists
+  return 16 + 4 * (n_seq + 1) + 4 * n_seq + 4 * kPsSeqStage * LOSA_MAX_BLOCK;
+}
+
+struct PsParams {
+  const void* q;
+  const void* kmin;
+  const void* kmax;
+  const int32_t* page_table;
+  const int32_t* kv_len;
+  const int32_t* active_idx;
+  const int32_t* n_active;
+  const int32_t* step;
+  float* scores;
+  int32_t* status;
+  int N, B, Hq, Hkv, G, g, Pmax, n_phys, score_stride, n_ctas, n_stages;
+};
+
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+// waits until at most `pending` of this thread's newest copy groups are still in flight
+__device__ __forceinline__ void cp_async_wait_pending(int pending) {
+  switch (pending) {
+    case 0: asm volatile("cp.async.wait_group 0;" ::: "memory"); break;
+    case 1: asm volatile("cp.async.wait_group 1;" ::: "memory"); break;
+    case 2: asm volatile("cp.async.wait_group 2;" ::: "memory"); break;
+    default: asm volatile("cp.async.wait_group 3;" ::: "memory"); break;
+  }
+}
+
+// 8 consecutive elements from shared memory as fp32
+__device__ __forceinline__ void ld8(const __nv_bfloat16* p, float (&v)[8]) {
+  const uint4 a = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+__device__ __forceinline__ void ld8(const float* p, float (&v)[8]) {
+  const float4 a = *reinterpret_cast<const float4*>(p);
+  const float4 b = *reinterpret_cast<const float4*>(p + 4);
+  v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+}
+
+// Walk of a CTA's item range [lo, hi) in tiles: item = (sequence s, KV head kh, logical page p),
+// sequence-major, then KV head, then page; a tile never leaves its (s, kh) nor exceeds TP pages.
+struct TileWalk {
+  const int* pre;     // shared: exclusive prefix of the sequences' page counts, pre[N] = total
+  int Hkv, TP, hi;
+  int cur, s;
+  int kh, p0, np;     // the current tile
+  bool first_of_pair; // the tile is the CTA's first of this (s, kh)
+  int last_pair;
+  __device__ __forceinline__ void init(const int* pre_, int Hkv_, int TP_, int lo, int hi_) {
+    pre = pre_; Hkv = Hkv_; TP = TP_; hi = hi_; cur = lo; s = 0; last_pair = -1; np = 0;
+  }
+  __device__ __forceinline__ bool next() {
+    cur += np;
+    if (cur >= hi) return false;
+    while (static_cast<long long>(Hkv) * pre[s + 1] <= cur) ++s;
+    const int Ps = pre[s + 1] - pre[s];
+    const int off = cur - Hkv * pre[s];
+    kh = off / Ps;
+    p0 = off % Ps;
+    np = min(min(TP, Ps - p0), hi - cur);
+    const int pair = s * Hkv + kh;
+    first_of_pair = pair != last_pair;
+    last_pair = pair;
+    return true;
+  }
+};
+
+template <typename T, int D, int PG>
+__global__ void __launch_bounds__(kPsThreads, 1) page_scores_stream_kernel(PsParams p) {
+  using C = PsCfg<T, D, PG>;
+  constexpr int LPP = C::LPP, TP = C::TP, NP = C::NP, WP = C::WP;
+  extern __shared__ uint8_t ps_smem[];
+  const uint32_t raw = smem_u32(ps_smem);
+  const uint32_t base = (raw + 127u) & ~127u;
+  uint8_t* gen = ps_smem + (base - raw);
+  const int NS = p.n_stages;
+  T* qpos = reinterpret_cast<T*>(gen + static_cast<size_t>(NS) * C::STAGE_BYTES);
+  T* qneg = qpos + kPsRowTile * D;
+  int* pre = reinterpret_cast<int*>(qneg + kPsRowTile * D);
+  int* na_s = pre + p.N + 1;
+  int* tok_s = na_s + p.N;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  grid_dep_trigger();
+  grid_dep_wait();
+  if (warp == 0) {
+    // pages to score per sequence (none on a first step, none without active tokens), and their prefix
+    int run = 0;
+    for (int b0 = 0; b0 < p.N; b0 += 32) {
+      const int s = b0 + lane;
+      int c = 0, na = 0;
+      if (s < p.N) {
+        na = p.n_active[s];
+        na = na < 0 ? 0 : (na > p.B ? p.B : na);
+        const bool first_step = p.step && p.step[s] == 0;
+        int P = pages_of(p.kv_len[s], p.g);
+        if (P > p.Pmax) { set_status(p.status, LOSA_ERR_BOUNDS); P = p.Pmax; }   // a length beyond the page-table row
+        c = (first_step || na == 0 || P < 0) ? 0 : P;
+        na_s[s] = na;
+      }
+      int inc = c;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int t = __shfl_up_sync(0xffffffffu, inc, o);
+        if (lane >= o) inc += t;
+      }
+      if (s < p.N) pre[s] = run + inc - c;
+      run += __shfl_sync(0xffffffffu, inc, 31);
+    }
+    if (lane == 0) pre[p.N] = run;
+  }
+  __syncthreads();
+  const long long T_all = static_cast<long long>(p.Hkv) * pre[p.N];
+  const int lo = static_cast<int>(cta_lo(T_all, blockIdx.x, p.n_ctas));
+  const int hi = static_cast<int>(cta_lo(T_all, blockIdx.x + 1, p.n_ctas));
+  if (lo >= hi) return;                              // whole CTA
+  int s_lo = 0;
+  while (static_cast<long long>(p.Hkv) * pre[s_lo + 1] <= lo) ++s_lo;
+  for (int i = tid; i < kPsSeqStage * p.B; i += kPsThreads) {
+    const int s = s_lo + i / p.B;
+    tok_s[i] = s < p.N ? p.active_idx[s * p.B + i % p.B] : -1;
+  }
+  // block position of active slot a of sequence s
+  auto token_of = [&](int s, int a) {
+    int tok = (s >= s_lo && s < s_lo + kPsSeqStage) ? tok_s[(s - s_lo) * p.B + a] : p.active_idx[s * p.B + a];
+    if (tok < 0 || tok >= p.B) { set_status(p.status, LOSA_ERR_BOUNDS); tok = 0; }
+    return tok;
+  };
+  const T* qg = static_cast<const T*>(p.q);
+  const T* kmaxg = static_cast<const T*>(p.kmax);
+  const T* kming = static_cast<const T*>(p.kmin);
+  const int u = lane % LPP, grp = lane / LPP;
+  const uint32_t warp_off = static_cast<uint32_t>(warp) * WP * C::PAGE_BYTES;   // this warp's slice of a stage
+
+  // ---- loading pipeline of this warp: page-table entry of lane j's page (j < WP) one tile ahead of
+  //      the copies, the copies NS - 1 tiles ahead of the arithmetic
+  TileWalk w_ids, w_copy, w;
+  w_ids.init(pre, p.Hkv, TP, lo, hi);
+  w_copy.init(pre, p.Hkv, TP, lo, hi);
+  w.init(pre, p.Hkv, TP, lo, hi);
+  auto request_id = [&]() {                          // entry of this lane's page in the next tile of w_ids (0 when there is none)
+    int id = 0;
+    if (w_ids.next()) {
+      const int pl = warp * WP + lane;
+      if (lane < WP && pl < w_ids.np) {
+        id = __ldg(p.page_table + static_cast<size_t>(w_ids.s) * p.Pmax + w_ids.p0 + pl);
+        if (id < 0 || id >= p.n_phys) { set_status(p.status, LOSA_ERR_BOUNDS); id = 0; }
+      }
+    }
+    return id;
+  };
+  auto copy_tile = [&](int id, int stage) {          // the next tile of w_copy into `stage` (nothing when there is none); always one group
+    if (w_copy.next()) {
+      const uint32_t dst = base + static_cast<uint32_t>(stage) * C::STAGE_BYTES + warp_off;
+      const int c = lane % C::CH, sub = lane / C::CH;
+      constexpr int EPC = 16 / static_cast<int>(sizeof(T));
+#pragma unroll
+      for (int i = 0; i < C::NI; ++i) {
+        const int row = i * C::RPI + sub, pl = row >> 1, a = row & 1;     // page of the warp's slice, 0 = kmax / 1 = kmin
+        const int ph = __shfl_sync(0xffffffffu, id, pl);
+        if (warp * WP + pl < w_copy.np) {
+          const T* src = (a ? kming : kmaxg) + (static_cast<size_t>(ph) * p.Hkv + w_copy.kh) * D + c * EPC;
+          cp_async16(dst + pl * C::PAGE_BYTES + a * C::HALF_BYTES + c * 16, src);
+        }
+      }
+    }
+    cp_async_commit();
+  };
+  int id_next = request_id();
+  for (int i = 0; i < NS - 1; ++i) {
+    const int id = id_next;
+    id_next = request_id();
+    copy_tile(id, i);
+  }
+  __syncthreads();                                   // the cached active lists are in place
+
+  // q+ / q- of one run (8 elements j = 8 rho .. 8 rho + 7) of row r into the pair layout.  Lane
+  // u = rho % LPP works on the pair {run u, run u + LPP}; h = rho / LPP says which half this run is.
+  //   bf16: a row is D/2 words, word (jj / 4) * (4 LPP) + 4 u + jj % 4 holds element jj of both runs
+  //         (low half: run u), so a lane's four words of a chunk are one 16-byte read and the LPP
+  //         lanes of a page read consecutive 16-byte words;
+  //   fp32: a row is D floats, float (jj / 2) * (4 LPP) + 4 u + 2 (jj % 2) + h.
+  auto put_run = [&](int r, int rho, const float (&v)[8]) {
+    const int uu = rho % LPP, h = rho / LPP;
+#pragma unroll
+    for (int jj = 0; jj < 8; ++jj) {
+      const float vp = fmaxf(v[jj], 0.f), vn = fminf(v[jj], 0.f);
+      if constexpr (sizeof(T) == 2) {
+        const int at = r * D + 2 * ((jj >> 2) * (4 * LPP) + 4 * uu + (jj & 3)) + h;
+        qpos[at] = __float2bfloat16_rn(vp);          // exact: v is a bf16 value
+        qneg[at] = __float2bfloat16_rn(vn);
+      } else {
+        const int at = r * D + (jj >> 1) * (4 * LPP) + 4 * uu + 2 * (jj & 1) + h;
+        qpos[at] = vp;
+        qneg[at] = vn;
+      }
+    }
+  };
+  // rows r0 .. r0 + nr - 1 of (sequence s, KV head kh) from global memory into the staging buffers (all threads)
+  auto stage_rows = [&](int s, int kh, int r0, int nr) {
+    for (int idx = tid; idx < nr * (D / 8); idx += kPsThreads) {
+      const int r = idx / (D / 8), rho = idx % (D / 8), row = r0 + r;
+      const int tok = token_of(s, row / p.G);
+      float v[8];
+      load8(qg + ((static_cast<size_t>(s) * p.B + tok) * p.Hq + kh * p.G + row % p.G) * D + rho * 8, v);
+      put_run(r, rho, v);
+    }
+  };
+
+  // ---- reduce-scatter set-up.  After the add of a pair's halves (butterfly offset d/16) a lane
+  // holds one partial sum for each of its NP = 2 PG (page, row) pairs; the remaining offsets
+  // d/32 .. 1 pair the lanes u ^ LPP/2, u ^ LPP/4, .., u ^ 1.  As a reduce-scatter a lane keeps half
+  // of its values at every level and sends the other half, so a pass costs NP - 1 shuffles; once a
+  // single value is left the level is the plain exchange (both lanes end with the same sum).  Which
+  // half is kept is a matter of naming: a lane whose bit is set holds its pages in an order with
+  // the level's page bit flipped, or takes the pass's two rows the other way round, so that
+  // everyone keeps the low half of the array.  The additions and their order are those of the
+  // plain butterfly (fp32 addition commutes).
+  constexpr int LV = LPP == 8 ? 3 : 2;                // levels over lanes (LPP = 2^LV)
+  constexpr int LOGNP = NP == 8 ? 3 : 2;              // NP = 2^LOGNP
+  constexpr int NF = (NP >> LV) > 0 ? (NP >> LV) : 1; // complete sums a lane ends up with
+  int xperm = 0;                                      // page-order flip of this lane
+  bool rowswap = false, stores = true;                // the lane takes the rows the other way round / is not a duplicate
+#pragma unroll
+  for (int l = 0; l < LV; ++l) {
+    const int mask = (LPP / 2) >> l;
+    const bool set = (u & mask) != 0;
+    if (l < LOGNP) {
+      const int b = LOGNP - 1 - l;                    // bit of the pair index 2 i + rr this level splits on
+      if (b >= 1) { if (set) xperm ^= 1 << (b - 1); }
+      else rowswap = set;
+    } else if (set) {
+      stores = false;
+    }
+  }
+  const int slot0 = grp * PG;                        // this lane's first page within the warp's slice
+
+  for (int t = 0; w.next(); ++t) {
+    const int stage = t % NS;
+    const int rows = na_s[w.s] * p.G;
+    // ---- the tile's summaries have landed (this warp's copies of it are the oldest but NS - 2 groups)
+    cp_async_wait_pending(NS - 2);
+    __syncwarp();
+    float2 kx[PG][8], kn[PG][8];                     // {run u, run u + LPP} of kmax / kmin, element jj
+    {
+      const uint8_t* st = gen + static_cast<size_t>(stage) * C::STAGE_BYTES + warp_off;
+#pragma unroll
+      for (int i = 0; i < PG; ++i) {
+        float a0[8], a1[8], b0[8], b1[8];
+        const T* src = reinterpret_cast<const T*>(st + static_cast<size_t>(slot0 + (i ^ xperm)) * C::PAGE_BYTES) + u * 8;
+        ld8(src, a0);
+        ld8(src + 8 * LPP, a1);
+        ld8(src + D, b0);
+        ld8(src + D + 8 * LPP, b1);
+#pragma unroll
+        for (int jj = 0; jj < 8; ++jj) {
+          kx[i][jj] = make_float2(a0[jj], a1[jj]);
+          kn[i][jj] = make_float2(b0[jj], b1[jj]);
+        }
+      }
+    }
+    __syncwarp();                                    // the slice that tile t - 1 used is free: refill it
+    {
+      const int id = id_next;
+      id_next = request_id();
+      copy_tile(id, (t + NS - 1) % NS);
+    }
+    const bool warp_has_pages = warp * WP < w.np;
+    float* tile_base = p.scores + (static_cast<size_t>(w.s) * p.B * p.Hq + w.kh * p.G) * p.score_stride + w.p0 + warp * WP + slot0;
+    const int np_lane = w.np - warp * WP - slot0;    // page slot i of this lane is valid iff i < np_lane
+
+    // the chains of one pass: rows ra and rb (of the staged tile) against the PG pages in registers
+    auto fma_pass = [&](int ra, int rb, float2 (&acc)[PG][2]) {
+#pragma unroll
+      for (int i = 0; i < PG; ++i) acc[i][0] = acc[i][1] = make_float2(0.f, 0.f);
+#pragma unroll
+      for (int hf = 0; hf < 2; ++hf) {               // elements jj = 4 hf .. 4 hf + 3 of both runs
+        float2 qp0[4], qn0[4], qp1[4], qn1[4];
+        if constexpr (sizeof(T) == 2) {
+          const uint32_t* bp = reinterpret_cast<const uint32_t*>(qpos) + hf * (4 * LPP) + 4 * u;
+          const uint32_t* bn = reinterpret_cast<const uint32_t*>(qneg) + hf * (4 * LPP) + 4 * u;
+          const uint4 wp0 = *reinterpret_cast<const uint4*>(bp + ra * (D / 2)), wn0 = *reinterpret_cast<const uint4*>(bn + ra * (D / 2));
+          const uint4 wp1 = *reinterpret_cast<const uint4*>(bp + rb * (D / 2)), wn1 = *reinterpret_cast<const uint4*>(bn + rb * (D / 2));
+          const uint32_t a[4] = {wp0.x, wp0.y, wp0.z, wp0.w}, b[4] = {wn0.x, wn0.y, wn0.z, wn0.w};
+          const uint32_t c[4] = {wp1.x, wp1.y, wp1.z, wp1.w}, d[4] = {wn1.x, wn1.y, wn1.z, wn1.w};
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            qp0[e] = make_float2(__uint_as_float(a[e] << 16), __uint_as_float(a[e] & 0xffff0000u));
+            qn0[e] = make_float2(__uint_as_float(b[e] << 16), __uint_as_float(b[e] & 0xffff0000u));
+            qp1[e] = make_float2(__uint_as_float(c[e] << 16), __uint_as_float(c[e] & 0xffff0000u));
+            qn1[e] = make_float2(__uint_as_float(d[e] << 16), __uint_as_float(d[e] & 0xffff0000u));
+          }
+        } else {
+#pragma unroll
+          for (int c2 = 0; c2 < 2; ++c2) {
+            const int off = (2 * hf + c2) * (4 * LPP) + 4 * u;
+            const float4 p0 = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(qpos) + ra * D + off);
+            const float4 n0 = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(qneg) + ra * D + off);
+            const float4 p1 = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(qpos) + rb * D + off);
+            const float4 n1 = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(qneg) + rb * D + off);
+            qp0[2 * c2] = make_float2(p0.x, p0.y); qp0[2 * c2 + 1] = make_float2(p0.z, p0.w);
+            qn0[2 * c2] = make_float2(n0.x, n0.y); qn0[2 * c2 + 1] = make_float2(n0.z, n0.w);
+            qp1[2 * c2] = make_float2(p1.x, p1.y); qp1[2 * c2 + 1] = make_float2(p1.z, p1.w);
+            qn1[2 * c2] = make_float2(n1.x, n1.y); qn1[2 * c2 + 1] = make_float2(n1.z, n1.w);
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const int jj = 4 * hf + e;
+          // 2 PG independent chains advance by the q+ term, then all of them by the q- term:
+          // dependent instructions stay 2 PG issue slots apart
+#pragma unroll
+          for (int i = 0; i < PG; ++i) {
+            acc[i][0] = __ffma2_rn(qp0[e], kx[i][jj], acc[i][0]);
+            acc[i][1] = __ffma2_rn(qp1[e], kx[i][jj], acc[i][1]);
+          }
+#pragma unroll
+          for (int i = 0; i < PG; ++i) {
+            acc[i][0] = __ffma2_rn(qn0[e], kn[i][jj], acc[i][0]);
+            acc[i][1] = __ffma2_rn(qn1[e], kn[i][jj], acc[i][1]);
+          }
+        }
+      }
+    };
+    // the butterfly of one pass and its stores; offa / offb: offsets of the score rows of this lane's
+    // first and second row; has_b: the second row exists
+    auto reduce_store = [&](const float2 (&acc)[PG][2], size_t offa, size_t offb, bool has_a, bool has_b) {
+      float v[NP];
+#pragma unroll
+      for (int i = 0; i < PG; ++i)
+#pragma unroll
+        for (int rr = 0; rr < 2; ++rr) v[2 * i + rr] = __fadd_rn(acc[i][rr].x, acc[i][rr].y);      // offset d/16
+      int n = NP;
+#pragma unroll
+      for (int l = 0; l < LV; ++l) {
+        const int mask = (LPP / 2) >> l;
+        if (l < LOGNP) {
+          n >>= 1;
+#pragma unroll
+          for (int k = 0; k < NP / 2; ++k)
+            if (k < n) v[k] = __fadd_rn(v[k], __shfl_xor_sync(0xffffffffu, v[k + n], mask));
+        } else {
+          v[0] = __fadd_rn(v[0], __shfl_xor_sync(0xffffffffu, v[0], mask));
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < NF; ++k) {
+        const int i = (k >> 1) ^ xperm;
+        const bool second = (k & 1) != 0;              // of this lane's two rows (only when both are left: NF >= 2)
+        if (stores && i < np_lane && (second ? has_b : has_a))
+          tile_base[(second ? offb : offa) + i] = __fadd_rn(v[k], 0.0f);
+      }
+    };
+
+    for (int r0 = 0; r0 < rows; r0 += kPsRowTile) {
+      const int nr = min(kPsRowTile, rows - r0);
+      if (w.first_of_pair || rows > kPsRowTile) {
+        // a new (sequence, KV head), or more rows than one staging holds (every token active)
+        __syncthreads();
+        stage_rows(w.s, w.kh, r0, nr);
+        __syncthreads();
+      }
+      if (!warp_has_pages) continue;
+      int a_row = r0 / p.G, g_row = r0 % p.G;        // row r0 + r = (active slot a_row, head g_row of the KV head)
+      // offsets of the score rows of rows r and r + 1 as this lane sees them (its first row is r + 1
+      // when it takes the rows the other way round); then steps two rows on
+      auto row_offsets = [&](size_t& offa, size_t& offb) {
+        const size_t o0 = (static_cast<size_t>(a_row) * p.Hq + g_row) * p.score_stride;
+        int a1 = a_row, g1 = g_row + 1;
+        if (g1 >= p.G) { g1 = 0; ++a1; }
+        const size_t o1 = (static_cast<size_t>(a1) * p.Hq + g1) * p.score_stride;
+        offa = rowswap ? o1 : o0;
+        offb = rowswap ? o0 : o1;
+        g_row += 2;
+        while (g_row >= p.G) { g_row -= p.G; ++a_row; }
+      };
+      // rows of a pass as this lane takes them; an odd tail computes its last row twice and stores it once
+      auto pass_rows = [&](int r, int& ra, int& rb) {
+        const int r1 = min(r + 1, nr - 1);
+        ra = rowswap ? r1 : r;
+        rb = rowswap ? r : r1;
+      };
+      auto finish_pass = [&](const float2 (&acc)[PG][2], int r) {
+        size_t offa, offb;
+        row_offsets(offa, offb);
+        const bool two = r + 1 < nr;
+        reduce_store(acc, offa, offb, rowswap ? two : true, rowswap ? true : two);
+      };
+      // software pipeline over the passes: the chains of pass i + 1 are issued in the same straight
+      // line of code as the butterfly of pass i, whose shuffle latencies they hide (two passes per
+      // trip, the two accumulator sets trading places, so that nothing is copied)
+      float2 acc[PG][2], nxt[PG][2];
+      int ra, rb;
+      pass_rows(0, ra, rb);
+      fma_pass(ra, rb, acc);
+      int r = 0;
+      while (r + 4 < nr) {
+        pass_rows(r + 2, ra, rb);
+        fma_pass(ra, rb, nxt);
+        finish_pass(acc, r);
+        pass_rows(r + 4, ra, rb);
+        fma_pass(ra, rb, acc);
+        finish_pass(nxt, r + 2);
+        r += 4;
+      }
+      if (r + 2 < nr) {
+        pass_rows(r + 2, ra, rb);
+        fma_pass(ra, rb, nxt);
+        finish_pass(acc, r);
+        finish_pass(nxt, r + 2);
+      } else {
+        finish_pass(acc, r);
+      }
+    }
+  }
+  cp_async_wait_pending(0);
+}
+
+template <typename T, int D, int PG>
+int32_t launch_stream(losa_ctx* c, const PsParams& pp, cudaStream_t st) {
+  using C = PsCfg<T, D, PG>;
+  PsParams p = pp;
+  const int tail = ps_tail_bytes(p.N);
+  int ns = (kPsSmemBudget - C::QBUF_BYTES - tail - 128) / C::STAGE_BYTES;
+  ns = ns > kPsMaxStages ? kPsMaxStages : ns;
+  if (ns < 2) return LOSA_ERR_UNSUPPORTED;
+  p.n_stages = ns;
+  const int smem = 128 + ns * C::STAGE_BYTES + C::QBUF_BYTES + tail;
+  if (!c->scores_attr_set) {
+    LOSA_CUDA_TRY(c, cudaFuncSetAttribute(page_scores_stream_kernel<T, D, PG>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    c->scores_attr_set = 1;
+  }
+  launch_k(page_scores_stream_kernel<T, D, PG>, p.n_ctas, kPsThreads, smem, st, p);
+  return after_launch(c);
+}
+
+}  // namespace
+
+int32_t launch_page_scores(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
+                           const int32_t* n_active, const int32_t* step, cudaStream_t st) {
+  const losa_shape_t& sh = c->shape;
+  PsParams p;
+  p.q = q;
+  p.kmin = kv->kmin;
+  p.kmax = kv->kmax;
+  p.page_table = kv->page_table;
+  p.kv_len = kv->kv_len;
+  p.active_idx = active_idx;
+  p.n_active = n_active;
+  p.step = step;
+  p.scores = reinterpret_cast<float*>(c->ws + c->lay.scores);
+  p.status = status_ptr(c);
+  p.N = sh.batch;
+  p.B = sh.block_size;
+  p.Hq = sh.n_q_heads;
+  p.Hkv = sh.n_kv_heads;
+  p.G = sh.n_q_heads / sh.n_kv_heads;
+  p.g = sh.page_size;
+  p.Pmax = sh.max_pages_per_seq;
+  p.n_phys = kv->n_phys_pages;
+  p.score_stride = c->lay.score_stride;
+  p.n_ctas = c->n_sms;
+  p.n_stages = 0;
+  const bool bf = sh.dtype == LOSA_BF16;
+  if (bf && sh.head_dim == 128) return launch_stream<__nv_bfloat16, 128, 4>(c, p, st);
+  if (bf) return launch_stream<__nv_bfloat16, 64, 4>(c, p, st);
+  if (sh.head_dim == 128) return launch_stream<float, 128, 2>(c, p, st);
+  return launch_stream<float, 64, 2>(c, p, st);
+}
+
+}  // namespace losa

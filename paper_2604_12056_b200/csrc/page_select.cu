@@ -1,13 +1,7 @@
 // Stages 2 and 3 — QUEST page scores, top-k per active query, union per KV head
 // (Section 2.3, Section 4.2, Section 4.4).
 //
-//   page_scores_kernel : each CTA reads the min/max keys of 64 pages of one (sequence, KV head)
-//                        once and scores them against every active query of that KV head.  A page
-//                        is handled by d/8 lanes: one 16-byte vector of kmin and kmax per lane
-//                        (four pages per lane), a chain of 16 fused multiply-adds per lane and
-//                        page (q+ kmax, q- kmin), then the butterfly over the lanes as a
-//                        reduce-scatter over two query rows at a time: exactly the additions and
-//                        the order the interface fixes, so the fp32 result is reproducible bit for bit.
+//   (the page scores themselves are computed by the kernel in page_scores.cu)
 //   topk_select_kernel : one 128-thread CTA per (sequence, active token, head); threshold search over
 //                        64-bit keys (order-preserving score bits, inverted page id), see below.
 //   topk_kernel        : budgets above 512 pages: one CTA per query sorts all keys with a
@@ -22,220 +16,6 @@ namespace losa {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kPagesPerCta = 64;
-constexpr int kRowTile = 32;
-
-// Eight consecutive elements as loaded, converted to fp32 later: lets several dependent-free loads
-// be in flight before any of them is used.
-template <typename T> struct Raw8;
-template <> struct Raw8<__nv_bfloat16> {
-  uint4 u;
-  __device__ __forceinline__ void load(const __nv_bfloat16* p) { u = *reinterpret_cast<const uint4*>(p); }
-  __device__ __forceinline__ void zero() { u = make_uint4(0u, 0u, 0u, 0u); }
-  __device__ __forceinline__ void unpack(float (&v)[8]) const {
-    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      v[2 * i] = __uint_as_float(w[i] << 16);
-      v[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
-    }
-  }
-};
-template <> struct Raw8<float> {
-  float4 a, b;
-  __device__ __forceinline__ void load(const float* p) {
-    a = *reinterpret_cast<const float4*>(p);
-    b = *reinterpret_cast<const float4*>(p + 4);
-  }
-  __device__ __forceinline__ void zero() { a = make_float4(0.f, 0.f, 0.f, 0.f); b = a; }
-  __device__ __forceinline__ void unpack(float (&v)[8]) const {
-    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
-  }
-};
-
-// A load whose issue point stays where it is written (it is requested ahead of the branch that
-// decides whether it is needed).
-__device__ __forceinline__ int ld_keep_s32(const int32_t* ptr) {
-  int v;
-  asm volatile("ld.global.nc.s32 %0, [%1];" : "=r"(v) : "l"(ptr));
-  return v;
-}
-
-template <typename T, int D>
-__global__ void __launch_bounds__(kThreads)
-page_scores_kernel(const T* __restrict__ q, const T* __restrict__ kmin, const T* __restrict__ kmax,
-                   const int32_t* __restrict__ page_table, const int32_t* __restrict__ kv_len,
-                   const int32_t* __restrict__ active_idx, const int32_t* __restrict__ n_active,
-                   const int32_t* __restrict__ step, float* __restrict__ scores, int B, int Hq, int Hkv,
-                   int g, int Pmax, int n_phys, int score_stride, int32_t* __restrict__ status) {
-  grid_dep_wait();
-  constexpr int LPP = D / 8;            // lanes per page
-  constexpr int GROUPS = kThreads / LPP;
-  constexpr int ITER = kPagesPerCta / GROUPS;
-  constexpr int STG = (kRowTile * (D / 8) + kThreads - 1) / kThreads;   // staging items per thread and row tile
-  const int s = blockIdx.z, kh = blockIdx.y, p0 = blockIdx.x * kPagesPerCta;
-  const int tid = threadIdx.x;
-  const int grp = tid / LPP, sub = tid % LPP;
-  const int G = Hq / Hkv;
-  // First round trip: the scalars, and with them - their addresses depend on nothing else - this
-  // lane's page-table entries and the block positions of the query rows it may have to stage
-  // (entries the scalars later rule out are read and dropped).
-  int phys[ITER], tok0[STG];
-#pragma unroll
-  for (int it = 0; it < ITER; ++it) {
-    const int p = p0 + grp * ITER + it;
-    phys[it] = p < Pmax ? ld_keep_s32(page_table + static_cast<size_t>(s) * Pmax + p) : -1;
-  }
-#pragma unroll
-  for (int i = 0; i < STG; ++i) {
-    const int a = ((tid + i * kThreads) / (D / 8)) / G;
-    tok0[i] = a < B ? ld_keep_s32(active_idx + s * B + a) : 0;
-  }
-  if (step && step[s] == 0) return;
-  int P = pages_of(kv_len[s], g);
-  if (P > Pmax) { set_status(status, LOSA_ERR_BOUNDS); P = Pmax; }    // a length beyond the page-table row
-  if (p0 >= P) return;
-  int na = n_active[s];
-  na = na < 0 ? 0 : (na > B ? B : na);
-  const int rows = na * G;
-  if (rows == 0) return;
-
-  // positive and negative parts of the staged queries, fp32: U = sum q+ kmax + q- kmin.  A row is
-  // stored as two halves [half][lane chunk][4 floats] so that the d/8 lanes of a page read
-  // consecutive 16-byte words (no bank conflicts): element j = 8*c + e sits at (e/4)*(D/2) + 4*c + e%4.
-  __shared__ __align__(16) float qpos[kRowTile * D];
-  __shared__ __align__(16) float qneg[kRowTile * D];
-  const int np = min(kPagesPerCta, P - p0);
-
-  // Second round trip: this lane's share of the pages' kmin / kmax (kept in registers for every
-  // query row) and the query rows themselves.  Everything of a trip is requested before anything
-  // of it is used.
-  const int nr_first = min(kRowTile, rows);
-  Raw8<T> klo[ITER], khi[ITER], q0[STG];
-#pragma unroll
-  for (int it = 0; it < ITER; ++it) {
-    klo[it].zero();
-    khi[it].zero();
-    if (grp * ITER + it < np) {
-      int ph = phys[it];
-      if (ph < 0 || ph >= n_phys) { set_status(status, LOSA_ERR_BOUNDS); ph = 0; }
-      const size_t so = (static_cast<size_t>(ph) * Hkv + kh) * D + sub * 8;
-      klo[it].load(kmin + so);
-      khi[it].load(kmax + so);
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < STG; ++i) {
-    const int idx = tid + i * kThreads;
-    q0[i].zero();
-    if (idx < nr_first * (D / 8)) {
-      const int r = idx / (D / 8), ch = idx % (D / 8), gi = r % G;
-      int tok = tok0[i];
-      if (tok < 0 || tok >= B) { set_status(status, LOSA_ERR_BOUNDS); tok = 0; }
-      q0[i].load(q + ((static_cast<size_t>(s) * B + tok) * Hq + kh * G + gi) * D + ch * 8);
-    }
-  }
-  auto stage = [&](int r, int ch, const float (&v)[8]) {
-#pragma unroll
-    for (int e = 0; e < 8; ++e) {
-      const int at = r * D + (e >> 2) * (D / 2) + ch * 4 + (e & 3);
-      qpos[at] = fmaxf(v[e], 0.f);
-      qneg[at] = fminf(v[e], 0.f);
-    }
-  };
-  float lo[ITER][8], hi[ITER][8];
-  for (int r0 = 0; r0 < rows; r0 += kRowTile) {
-    const int nr = min(kRowTile, rows - r0);
-    if (r0 == 0) {
-#pragma unroll
-      for (int i = 0; i < STG; ++i) {
-        const int idx = tid + i * kThreads;
-        if (idx < nr * (D / 8)) {
-          float v[8];
-          q0[i].unpack(v);
-          stage(idx / (D / 8), idx % (D / 8), v);
-        }
-      }
-#pragma unroll
-      for (int it = 0; it < ITER; ++it) {
-        klo[it].unpack(lo[it]);
-        khi[it].unpack(hi[it]);
-      }
-    } else {
-      for (int idx = tid; idx < nr * (D / 8); idx += kThreads) {
-        const int r = idx / (D / 8), ch = idx % (D / 8);
-        const int row = r0 + r, a = row / G, gi = row % G;
-        int tok = active_idx[s * B + a];
-        if (tok < 0 || tok >= B) { set_status(status, LOSA_ERR_BOUNDS); tok = 0; }
-        float v[8];
-        load8(q + ((static_cast<size_t>(s) * B + tok) * Hq + kh * G + gi) * D + ch * 8, v);
-        stage(r, ch, v);
-      }
-    }
-    __syncthreads();
-    // Two query rows at a time: one load of a row's run feeds the chains of the ITER pages held in
-    // registers.  A lane then has NV = 2 * ITER run sums, one per (page, row) pair; every pair needs
-    // the butterfly c[i] += c[i ^ off] (off = LPP/2 .. 1) over the LPP lanes of its group.  Taken as
-    // a reduce-scatter it costs NV shuffles per lane instead of NV * log2(LPP): at each level the
-    // lane keeps the half of its values chosen by its own bit `off` and sends the other half; the
-    // additions, and their order, are those of the plain butterfly (fp32 addition commutes), so the
-    // result is the same bit for bit.  Lanes 2i and 2i+1 end with pair i = (page it = i / 2, row i % 2).
-    constexpr int NV = 2 * ITER;
-    static_assert(NV == LPP / 2, "one result per pair of lanes");
-    int a = r0 / G, gi = r0 % G;          // row r0 + r = (active token a, head gi of the KV head), gi fastest
-    for (int r = 0; r < nr; r += 2) {
-      float v[NV];
-#pragma unroll
-      for (int rr = 0; rr < 2; ++rr) {
-        const int rs = min(r + rr, nr - 1);         // an odd tail computes its last row twice and stores it once
-        float qp[8], qn[8];
-        *reinterpret_cast<float4*>(&qp[0]) = *reinterpret_cast<const float4*>(&qpos[rs * D + sub * 4]);
-        *reinterpret_cast<float4*>(&qp[4]) = *reinterpret_cast<const float4*>(&qpos[rs * D + D / 2 + sub * 4]);
-        *reinterpret_cast<float4*>(&qn[0]) = *reinterpret_cast<const float4*>(&qneg[rs * D + sub * 4]);
-        *reinterpret_cast<float4*>(&qn[4]) = *reinterpret_cast<const float4*>(&qneg[rs * D + D / 2 + sub * 4]);
-        float acc[ITER];
-#pragma unroll
-        for (int it = 0; it < ITER; ++it) acc[it] = 0.f;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-#pragma unroll
-          for (int it = 0; it < ITER; ++it) {
-            acc[it] = __fmaf_rn(qp[j], hi[it][j], acc[it]);
-            acc[it] = __fmaf_rn(qn[j], lo[it][j], acc[it]);
-          }
-        }
-#pragma unroll
-        for (int it = 0; it < ITER; ++it) v[it * 2 + rr] = acc[it];
-      }
-      {
-        int n = NV;
-#pragma unroll
-        for (int off = LPP / 2; off >= 2; off >>= 1) {
-          n >>= 1;
-          const bool up = (sub & off) != 0;
-#pragma unroll
-          for (int k = 0; k < NV / 2; ++k) {
-            if (k < n) {
-              const float send = up ? v[k] : v[k + n];
-              const float keep = up ? v[k + n] : v[k];
-              v[k] = __fadd_rn(keep, __shfl_xor_sync(0xffffffffu, send, off));
-            }
-          }
-        }
-        v[0] = __fadd_rn(v[0], __shfl_xor_sync(0xffffffffu, v[0], 1));
-      }
-      const int i = sub >> 1, it = i >> 1, rr = i & 1, pl = grp * ITER + it;
-      if ((sub & 1) == 0 && pl < np && r + rr < nr) {
-        int a2 = a, g2 = gi + rr;
-        if (g2 >= G) { g2 -= G; ++a2; }
-        scores[((static_cast<size_t>(s) * B + a2) * Hq + kh * G + g2) * score_stride + p0 + pl] = __fadd_rn(v[0], 0.0f);
-      }
-      gi += 2;
-      while (gi >= G) { gi -= G; ++a; }
-    }
-    __syncthreads();
-  }
-}
 
 // One score row, or (pooled selector) the element-wise maximum of the `g` consecutive rows of a KV
 // head's query heads.
@@ -615,18 +395,6 @@ union_kernel(const int32_t* __restrict__ topk_pages, const int32_t* __restrict__
   if (tid == 0) union_count[s * Hkv + kh] = total;
 }
 
-template <typename T, int D>
-void launch_scores(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
-                   const int32_t* n_active, const int32_t* step, cudaStream_t st) {
-  const losa_shape_t& sh = c->shape;
-  dim3 grid((sh.max_pages_per_seq + kPagesPerCta - 1) / kPagesPerCta, sh.n_kv_heads, sh.batch);
-  launch_k(page_scores_kernel<T, D>, grid, kThreads, 0, st, 
-      static_cast<const T*>(q), static_cast<const T*>(kv->kmin), static_cast<const T*>(kv->kmax),
-      kv->page_table, kv->kv_len, active_idx, n_active, step,
-      reinterpret_cast<float*>(c->ws + c->lay.scores), sh.block_size, sh.n_q_heads, sh.n_kv_heads,
-      sh.page_size, sh.max_pages_per_seq, kv->n_phys_pages, c->lay.score_stride, status_ptr(c));
-}
-
 int pow2_at_least(int x) {
   int n = 2;
   while (n < x) n <<= 1;
@@ -649,11 +417,7 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
   if (sh.max_pages_per_seq == 0) return LOSA_OK;
   const int pool = pooled ? sh.n_q_heads / sh.n_kv_heads : 1;
   const bool bf = sh.dtype == LOSA_BF16;
-  if (bf && sh.head_dim == 128) launch_scores<__nv_bfloat16, 128>(c, q, kv, active_idx, n_active, step, st);
-  else if (bf) launch_scores<__nv_bfloat16, 64>(c, q, kv, active_idx, n_active, step, st);
-  else if (sh.head_dim == 128) launch_scores<float, 128>(c, q, kv, active_idx, n_active, step, st);
-  else launch_scores<float, 64>(c, q, kv, active_idx, n_active, step, st);
-  int32_t rc = after_launch(c);
+  int32_t rc = launch_page_scores(c, q, kv, active_idx, n_active, step, st);
   if (rc != LOSA_OK) return rc;
 
   float* sc = reinterpret_cast<float*>(c->ws + c->lay.scores);

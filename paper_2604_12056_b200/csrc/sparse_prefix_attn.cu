@@ -367,57 +367,11 @@ __global__ void __launch_bounds__(kFinishThreads) attn_finish_kernel(AttnParams 
 }
 
 // ===================================================================== bf16 TMA + tensor-core kernel: shared pieces
-constexpr long long kWaitCycles = 2000000000ll;   // ~1 s: default bound of every mbarrier wait
-constexpr long long kDrainCycles = 20000000ll;    // ~10 ms: bound of the waits for work already in flight when a CTA gives up
 constexpr int kSmemBudget = 232448;                // 227 KB opt-in limit per CTA
 
 constexpr int kStageIdx = 1024;     // active_idx entries (N * B) cached in shared memory when they fit
 constexpr int kStageSeq = 64;       // ... together with n_active and kv_len of up to this many sequences
 constexpr int kTailBytes = 512 + (kMaxSegments + 1) * 4 + 4 + kStageIdx * 4 + 2 * kStageSeq * 4;   // barriers, meta, prefix, index cache
-__device__ __forceinline__ uint32_t smem_u32(const void* ptr) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(ptr));
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false (and raises the CTA's abort flag) when the bound runs out or
-// another warp has already given up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int32_t* status, long long limit) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  while (true) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > limit) {
-      *abort_flag = 1;
-      set_status(status, LOSA_ERR_TIMEOUT);
-      return false;
-    }
-  }
-}
-// Wait of a CTA that has given up, for work it had already put in flight (page copies into its
-// shared memory, tensor-core instructions on its tensor memory): bounded by kDrainCycles, ignores
-// the abort flag, reports nothing (the status word already holds the reason).
-__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
-  const long long t0 = clock64();
-  while (!mbar_try_wait(bar, parity) && clock64() - t0 < kDrainCycles) {}
-}
 // The K / V pages are read once per launch: they are marked evict-first in L2, so that the stream
 // does not push out the small arrays the following kernels read (partial records, in-block output).
 __device__ __forceinline__ unsigned long long l2_evict_first_policy() {
