@@ -41,7 +41,7 @@ int32_t make_layout(const losa_shape_t* sh, int n_ctas, WorkspaceLayout* L) {
   L->slot_map = off; off = align_up(off + sizeof(int32_t) * sh->batch * sh->block_size, 256);
   L->delta = off;    off = align_up(off + sizeof(double) * sh->batch * sh->block_size, 256);
   L->scores = off;
-  off = align_up(off + sizeof(float) * static_cast<size_t>(sh->batch) * sh->block_size * sh->n_q_heads * L->score_stride, 256);
+  off = align_up(off + 2 * sizeof(float) * static_cast<size_t>(sh->batch) * sh->block_size * sh->n_q_heads * L->score_stride, 256);
   L->partials = off;
   off = align_up(off + sizeof(float) * static_cast<size_t>(L->n_slots) * kRowsPerGroup * (sh->head_dim + 2), 256);
   const size_t rows = static_cast<size_t>(sh->batch) * sh->block_size * sh->n_q_heads;

@@ -23,7 +23,7 @@ struct WorkspaceLayout {
   size_t seg_prefix; // int32[kMaxSegments + 1] : item prefix of the segments, left by the stage-4 main kernel for its combine kernel
   size_t slot_map;   // int32[N*B] : slot of every block token in the active list of the whole-step path, -1 = stable
   size_t delta;      // double[N*B]
-  size_t scores;     // float[N*B*H_q*score_stride]
+  size_t scores;     // float[2*N*B*H_q*score_stride]: page scores, or (lower, upper) bound pairs of them
   size_t partials;   // float[n_slots * kRowsPerGroup * (d + 2)]
   size_t block_o;    // float[N*B*H_q*d]  : in-block attention output of the whole-step path
   size_t block_lse;  // float[N*B*H_q]    : its log-normaliser
@@ -64,6 +64,8 @@ struct losa_ctx {
   // the stage-4 kernel of this context has had its shared-memory attribute set
   int32_t attn_attr_set;
   int32_t scores_attr_set;   // likewise for the page-score kernel
+  int32_t bounds_attr_set;   // and for the tensor-core page-bound kernel
+  int32_t refine_attr_set;
   // optional timing of the stage-4 main kernel
   int32_t profile;
   cudaEvent_t ev_begin, ev_end;

@@ -19,6 +19,11 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
 int32_t launch_page_scores(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
                            const int32_t* n_active, const int32_t* step, cudaStream_t st);
 
+// bf16: (lower, upper) bounds of the page scores from the tensor cores, as float2 per (row, page), for
+// the selection that evaluates the exact score of the surviving candidates only.
+int32_t launch_page_bounds(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
+                           const int32_t* n_active, const int32_t* step, cudaStream_t st);
+
 int32_t launch_page_union(losa_ctx* c, const int32_t* topk_pages, const int32_t* active_idx,
                           const int32_t* n_active, int32_t k, const int32_t* kv_len,
                           const int32_t* step, int32_t* union_pages, int32_t* union_count,

@@ -130,26 +130,15 @@ struct TileWalk {
   }
 };
 
-template <typename T, int D, int PG>
-__global__ void __launch_bounds__(kPsThreads, 1) page_scores_stream_kernel(PsParams p) {
-  using C = PsCfg<T, D, PG>;
-  constexpr int LPP = C::LPP, TP = C::TP, NP = C::NP, WP = C::WP;
-  extern __shared__ uint8_t ps_smem[];
-  const uint32_t raw = smem_u32(ps_smem);
-  const uint32_t base = (raw + 127u) & ~127u;
-  uint8_t* gen = ps_smem + (base - raw);
-  const int NS = p.n_stages;
-  T* qpos = reinterpret_cast<T*>(gen + static_cast<size_t>(NS) * C::STAGE_BYTES);
-  T* qneg = qpos + kPsRowTile * D;
-  int* pre = reinterpret_cast<int*>(qneg + kPsRowTile * D);
-  int* na_s = pre + p.N + 1;
-  int* tok_s = na_s + p.N;
-
+// Common prologue of the page-score kernels (all threads of the CTA): the number of pages to score
+// per sequence (none on a first step, none without active tokens) and its exclusive prefix into
+// pre[0 .. N], the clamped active counts into na_s, this CTA's range [lo, hi) of the flat
+// (sequence, KV head, page) list, and the active lists of the first kPsSeqStage sequences of that
+// range into tok_s.  Returns false when the range is empty.  The caller synchronises the CTA before
+// reading tok_s.
+__device__ __forceinline__ bool ps_prologue(const PsParams& p, int* pre, int* na_s, int* tok_s, int& lo, int& hi, int& s_lo) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  grid_dep_trigger();
-  grid_dep_wait();
   if (warp == 0) {
-    // pages to score per sequence (none on a first step, none without active tokens), and their prefix
     int run = 0;
     for (int b0 = 0; b0 < p.N; b0 += 32) {
       const int s = b0 + lane;
@@ -176,15 +165,38 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_scores_stream_kernel(PsPar
   }
   __syncthreads();
   const long long T_all = static_cast<long long>(p.Hkv) * pre[p.N];
-  const int lo = static_cast<int>(cta_lo(T_all, blockIdx.x, p.n_ctas));
-  const int hi = static_cast<int>(cta_lo(T_all, blockIdx.x + 1, p.n_ctas));
-  if (lo >= hi) return;                              // whole CTA
-  int s_lo = 0;
+  lo = static_cast<int>(cta_lo(T_all, blockIdx.x, p.n_ctas));
+  hi = static_cast<int>(cta_lo(T_all, blockIdx.x + 1, p.n_ctas));
+  if (lo >= hi) return false;
+  s_lo = 0;
   while (static_cast<long long>(p.Hkv) * pre[s_lo + 1] <= lo) ++s_lo;
-  for (int i = tid; i < kPsSeqStage * p.B; i += kPsThreads) {
+  for (int i = tid; i < kPsSeqStage * p.B; i += blockDim.x) {
     const int s = s_lo + i / p.B;
     tok_s[i] = s < p.N ? p.active_idx[s * p.B + i % p.B] : -1;
   }
+  return true;
+}
+
+template <typename T, int D, int PG>
+__global__ void __launch_bounds__(kPsThreads, 1) page_scores_stream_kernel(PsParams p) {
+  using C = PsCfg<T, D, PG>;
+  constexpr int LPP = C::LPP, TP = C::TP, NP = C::NP, WP = C::WP;
+  extern __shared__ uint8_t ps_smem[];
+  const uint32_t raw = smem_u32(ps_smem);
+  const uint32_t base = (raw + 127u) & ~127u;
+  uint8_t* gen = ps_smem + (base - raw);
+  const int NS = p.n_stages;
+  T* qpos = reinterpret_cast<T*>(gen + static_cast<size_t>(NS) * C::STAGE_BYTES);
+  T* qneg = qpos + kPsRowTile * D;
+  int* pre = reinterpret_cast<int*>(qneg + kPsRowTile * D);
+  int* na_s = pre + p.N + 1;
+  int* tok_s = na_s + p.N;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  grid_dep_trigger();
+  grid_dep_wait();
+  int lo, hi, s_lo;
+  if (!ps_prologue(p, pre, na_s, tok_s, lo, hi, s_lo)) return;      // whole CTA: nothing in its range
   // block position of active slot a of sequence s
   auto token_of = [&](int s, int a) {
     int tok = (s >= s_lo && s < s_lo + kPsSeqStage) ? tok_s[(s - s_lo) * p.B + a] : p.active_idx[s * p.B + a];
@@ -271,6 +283,24 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_scores_stream_kernel(PsPar
       put_run(r, rho, v);
     }
   };
+  // Staging on demand (all threads, same arguments): a new (sequence, KV head), or another row tile
+  // when a pair has more rows than one staging holds (every token active).  The first tile's rows
+  // are staged before the loop, while the first copies are still in flight.
+  int staged_pair = -1, staged_r0 = -1;
+  auto ensure_rows = [&](int s, int kh, int r0, int nr) {
+    const int pair = s * p.Hkv + kh;
+    if (pair == staged_pair && r0 == staged_r0) return;
+    __syncthreads();
+    stage_rows(s, kh, r0, nr);
+    __syncthreads();
+    staged_pair = pair;
+    staged_r0 = r0;
+  };
+  {
+    TileWalk first;
+    first.init(pre, p.Hkv, TP, lo, hi);
+    if (first.next()) ensure_rows(first.s, first.kh, 0, min(kPsRowTile, na_s[first.s] * p.G));
+  }
 
   // ---- reduce-scatter set-up.  After the add of a pair's halves (butterfly offset d/16) a lane
   // holds one partial sum for each of its NP = 2 PG (page, row) pairs; the remaining offsets
@@ -419,12 +449,7 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_scores_stream_kernel(PsPar
 
     for (int r0 = 0; r0 < rows; r0 += kPsRowTile) {
       const int nr = min(kPsRowTile, rows - r0);
-      if (w.first_of_pair || rows > kPsRowTile) {
-        // a new (sequence, KV head), or more rows than one staging holds (every token active)
-        __syncthreads();
-        stage_rows(w.s, w.kh, r0, nr);
-        __syncthreads();
-      }
+      ensure_rows(w.s, w.kh, r0, nr);
       if (!warp_has_pages) continue;
       int a_row = r0 / p.G, g_row = r0 % p.G;        // row r0 + r = (active slot a_row, head g_row of the KV head)
       // offsets of the score rows of rows r and r + 1 as this lane sees them (its first row is r + 1
@@ -481,6 +506,235 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_scores_stream_kernel(PsPar
   cp_async_wait_pending(0);
 }
 
+
+// =============================================================================================
+// Tensor-core page bounds (bf16).  U(p) is the product of [q+ | q-] (rows) with [kmax | kmin]
+// (pages): a GEMM whose bf16 operands are exact (q+ and q- are q or 0).  The tensor cores accumulate
+// in an order and rounding of their own, so their result A(p) is not the fp32 value the interface
+// fixes; but |A(p) - U(p)| <= delta(p) = kMmaErrCoef * S(p), S(p) = sum_j |q+_j kmax_j| + |q-_j kmin_j|
+// (the same MMAs on the operands with their sign bits cleared): every product is exact, each of the
+// <= 2 d additions of either summation errs by at most 2^-23 of a running magnitude that never
+// exceeds S(p); 2 * 2 d * 2^-23 <= 2^-13 for d <= 128 once more, and kMmaErrCoef = 2^-13 leaves a
+// factor of four (which also covers the rounding of S and of A -+ delta themselves).  The kernel
+// writes the pair (A - delta, A + delta) per (query row, page).  The selection that follows keeps
+// every page whose upper bound reaches the k-th largest lower bound - a superset of the exact
+// top-k, ties included - and evaluates U in the fixed order for those few pages only.
+//
+// Same persistent streaming structure as the kernel above (one CTA per SM, per-warp cp.async ring).
+// A warp's slice of a tile is 16 pages = two 8-page MMA tiles; query rows are staged per
+// (sequence, KV head) as bf16 rows [q+ | q-].  The contraction index is free to permute: lane
+// (g = lane / 4, t = lane % 4) reads one 16-byte chunk (8 elements) per operand row and uses its
+// halves as the lane's k-columns of two consecutive m16n8k16 steps, for A and B alike, so every
+// fragment load is one 16-byte shared-memory read; chunk positions are XOR-swizzled by the row's
+// parity so that the two rows a quarter-warp touches fall into different banks.
+constexpr float kMmaErrCoef = 1.0f / 8192.0f;
+constexpr int kMmaWP = 16;                          // pages per warp and tile
+constexpr int kMmaTP = kPsWarps * kMmaWP;           // pages per tile
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, {%0, %1, %2, %3};"
+      : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+      : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// positive / negative part of two packed bf16 values (sign bit set <=> negative; -0 maps to +0 / -0)
+__device__ __forceinline__ uint32_t bf2_pos(uint32_t w) { return w & ~(((w >> 15) & 0x00010001u) * 0xffffu); }
+__device__ __forceinline__ uint32_t bf2_neg(uint32_t w) { return w & (((w >> 15) & 0x00010001u) * 0xffffu); }
+
+template <int D>
+struct MmaCfg {
+  static constexpr int ROW_BYTES = 4 * D;                 // [kmax | kmin] of a page, or [q+ | q-] of a query row
+  static constexpr int CPR = ROW_BYTES / 16;              // 16-byte chunks per row
+  static constexpr int CH = CPR / 2;                      // chunks of one summary
+  static constexpr int RPI = 32 / CH;                     // summaries one warp-wide copy instruction covers
+  static constexpr int NI = 2 * kMmaWP / RPI;             // copy instructions per warp and tile
+  static constexpr int STAGE_BYTES = kMmaTP * ROW_BYTES;
+  static constexpr int QBUF_BYTES = kPsRowTile * ROW_BYTES;
+};
+// byte offset of chunk c of row r in a tile of rows of `row_bytes`, with the parity swizzle
+__device__ __forceinline__ uint32_t mma_off(int r, int c, int row_bytes) {
+  return static_cast<uint32_t>(r * row_bytes + ((c ^ ((r & 1) << 2)) << 4));
+}
+
+template <int D>
+__global__ void __launch_bounds__(kPsThreads, 1) page_bounds_mma_kernel(PsParams p) {
+  using C = MmaCfg<D>;
+  using T = __nv_bfloat16;
+  constexpr int WP = kMmaWP, TP = kMmaTP;
+  extern __shared__ uint8_t ps_smem[];
+  const uint32_t raw = smem_u32(ps_smem);
+  const uint32_t base = (raw + 127u) & ~127u;
+  uint8_t* gen = ps_smem + (base - raw);
+  const int NS = p.n_stages;
+  uint8_t* qbuf = gen + static_cast<size_t>(NS) * C::STAGE_BYTES;            // [kPsRowTile][q+ | q-], swizzled chunks
+  int* pre = reinterpret_cast<int*>(qbuf + C::QBUF_BYTES);
+  int* na_s = pre + p.N + 1;
+  int* tok_s = na_s + p.N;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  grid_dep_trigger();
+  grid_dep_wait();
+  int lo, hi, s_lo;
+  if (!ps_prologue(p, pre, na_s, tok_s, lo, hi, s_lo)) return;
+  auto token_of = [&](int s, int a) {
+    int tok = (s >= s_lo && s < s_lo + kPsSeqStage) ? tok_s[(s - s_lo) * p.B + a] : p.active_idx[s * p.B + a];
+    if (tok < 0 || tok >= p.B) { set_status(p.status, LOSA_ERR_BOUNDS); tok = 0; }
+    return tok;
+  };
+  const T* qg = static_cast<const T*>(p.q);
+  const T* kmaxg = static_cast<const T*>(p.kmax);
+  const T* kming = static_cast<const T*>(p.kmin);
+  float2* bounds = reinterpret_cast<float2*>(p.scores);
+  const uint32_t warp_off = static_cast<uint32_t>(warp) * WP * C::ROW_BYTES;
+
+  TileWalk w_ids, w_copy, w;
+  w_ids.init(pre, p.Hkv, TP, lo, hi);
+  w_copy.init(pre, p.Hkv, TP, lo, hi);
+  w.init(pre, p.Hkv, TP, lo, hi);
+  auto request_id = [&]() {
+    int id = 0;
+    if (w_ids.next()) {
+      const int pl = warp * WP + lane;
+      if (lane < WP && pl < w_ids.np) {
+        id = __ldg(p.page_table + static_cast<size_t>(w_ids.s) * p.Pmax + w_ids.p0 + pl);
+        if (id < 0 || id >= p.n_phys) { set_status(p.status, LOSA_ERR_BOUNDS); id = 0; }
+      }
+    }
+    return id;
+  };
+  auto copy_tile = [&](int id, int stage) {          // always one group, empty when the walk is over
+    if (w_copy.next()) {
+      const uint32_t dst = base + static_cast<uint32_t>(stage) * C::STAGE_BYTES + warp_off;
+      const int c = lane % C::CH, sub = lane / C::CH;
+#pragma unroll
+      for (int i = 0; i < C::NI; ++i) {
+        const int row = i * C::RPI + sub, pl = row >> 1, a = row & 1;     // page of the slice, 0 = kmax / 1 = kmin
+        const int ph = __shfl_sync(0xffffffffu, id, pl);
+        if (warp * WP + pl < w_copy.np) {
+          const T* src = (a ? kming : kmaxg) + (static_cast<size_t>(ph) * p.Hkv + w_copy.kh) * D + c * 8;
+          cp_async16(dst + mma_off(pl, a * C::CH + c, C::ROW_BYTES), src);
+        } else {
+          // pages past the tile's end take part in the MMAs (their columns are not stored): keep them finite
+          *reinterpret_cast<uint4*>(gen + static_cast<size_t>(stage) * C::STAGE_BYTES + warp_off + mma_off(pl, a * C::CH + c, C::ROW_BYTES)) =
+              make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+    }
+    cp_async_commit();
+  };
+  int id_next = request_id();
+  for (int i = 0; i < NS - 1; ++i) {
+    const int id = id_next;
+    id_next = request_id();
+    copy_tile(id, i);
+  }
+  __syncthreads();                                   // the cached active lists are in place
+
+  // rows r0 .. r0 + nr - 1 of (sequence s, KV head kh) as [q+ | q-] into the staging tile; the rows
+  // up to the next multiple of 16 are cleared (they take part in the last 16-row MMA tile)
+  auto stage_rows = [&](int s, int kh, int r0, int nr) {
+    const int nr16 = (nr + 15) & ~15;
+    for (int idx = tid; idx < nr16 * C::CH; idx += kPsThreads) {
+      const int r = idx / C::CH, c = idx % C::CH, row = r0 + r;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (r < nr) {
+        const int tok = token_of(s, row / p.G);
+        v = *reinterpret_cast<const uint4*>(qg + ((static_cast<size_t>(s) * p.B + tok) * p.Hq + kh * p.G + row % p.G) * D + c * 8);
+      }
+      *reinterpret_cast<uint4*>(qbuf + mma_off(r, c, C::ROW_BYTES)) = make_uint4(bf2_pos(v.x), bf2_pos(v.y), bf2_pos(v.z), bf2_pos(v.w));
+      *reinterpret_cast<uint4*>(qbuf + mma_off(r, c + C::CH, C::ROW_BYTES)) = make_uint4(bf2_neg(v.x), bf2_neg(v.y), bf2_neg(v.z), bf2_neg(v.w));
+    }
+  };
+  // Staging on demand (all threads, same arguments): a new (sequence, KV head), or another row tile
+  // when a pair has more rows than one staging holds (every token active).  The first tile's rows
+  // are staged before the loop, while the first copies are still in flight.
+  int staged_pair = -1, staged_r0 = -1;
+  auto ensure_rows = [&](int s, int kh, int r0, int nr) {
+    const int pair = s * p.Hkv + kh;
+    if (pair == staged_pair && r0 == staged_r0) return;
+    __syncthreads();
+    stage_rows(s, kh, r0, nr);
+    __syncthreads();
+    staged_pair = pair;
+    staged_r0 = r0;
+  };
+  {
+    TileWalk first;
+    first.init(pre, p.Hkv, TP, lo, hi);
+    if (first.next()) ensure_rows(first.s, first.kh, 0, min(kPsRowTile, na_s[first.s] * p.G));
+  }
+
+  const int g = lane >> 2, t4 = lane & 3;
+  for (int t = 0; w.next(); ++t) {
+    const int stage = t % NS;
+    const int rows = na_s[w.s] * p.G;
+    cp_async_wait_pending(NS - 2);
+    __syncwarp();
+    {                                                // the slice that tile t - 1 used is free: refill it
+      const int id = id_next;
+      id_next = request_id();
+      copy_tile(id, (t + NS - 1) % NS);
+    }
+    const uint8_t* st = gen + static_cast<size_t>(stage) * C::STAGE_BYTES + warp_off;
+    const bool warp_has_pages = warp * WP < w.np;
+    for (int r0 = 0; r0 < rows; r0 += kPsRowTile) {
+      const int nr = min(kPsRowTile, rows - r0);
+      ensure_rows(w.s, w.kh, r0, nr);
+      if (!warp_has_pages) continue;
+      for (int mt = 0; mt * 16 < nr; ++mt) {
+        float c0[4] = {0.f, 0.f, 0.f, 0.f}, c1[4] = {0.f, 0.f, 0.f, 0.f};     // pages 0..7 / 8..15 of the slice
+        float m0[4] = {0.f, 0.f, 0.f, 0.f}, m1[4] = {0.f, 0.f, 0.f, 0.f};     // the same on the magnitudes
+        // chunk 4 sg + t4 of a row of parity b sits at position 4 (sg ^ b) + t4: with d = 64 b bytes,
+        // at base + d + 64 sg for even sg and base - d + 64 sg for odd sg (all four rows this lane
+        // reads have the parity of g), so every address below is a lane constant plus an immediate
+        const int dsw = (g & 1) * 64;
+        const uint8_t* a_lo_p = qbuf + (16 * mt + g) * C::ROW_BYTES + t4 * 16;
+        const uint8_t* a_hi_p = a_lo_p + 8 * C::ROW_BYTES;
+        const uint8_t* b_0_p = st + g * C::ROW_BYTES + t4 * 16;
+        const uint8_t* b_1_p = b_0_p + 8 * C::ROW_BYTES;
+#pragma unroll
+        for (int sg = 0; sg < C::CPR / 4; ++sg) {
+          const int off = 64 * sg + ((sg & 1) ? -dsw : dsw);
+          uint4 a_lo = *reinterpret_cast<const uint4*>(a_lo_p + off);
+          uint4 a_hi = *reinterpret_cast<const uint4*>(a_hi_p + off);
+          uint4 b_0 = *reinterpret_cast<const uint4*>(b_0_p + off);
+          uint4 b_1 = *reinterpret_cast<const uint4*>(b_1_p + off);
+          mma_bf16_16816(c0, a_lo.x, a_hi.x, a_lo.y, a_hi.y, b_0.x, b_0.y);
+          mma_bf16_16816(c1, a_lo.x, a_hi.x, a_lo.y, a_hi.y, b_1.x, b_1.y);
+          mma_bf16_16816(c0, a_lo.z, a_hi.z, a_lo.w, a_hi.w, b_0.z, b_0.w);
+          mma_bf16_16816(c1, a_lo.z, a_hi.z, a_lo.w, a_hi.w, b_1.z, b_1.w);
+          constexpr uint32_t kAbs = 0x7fff7fffu;
+          a_lo.x &= kAbs; a_lo.y &= kAbs; a_lo.z &= kAbs; a_lo.w &= kAbs;
+          a_hi.x &= kAbs; a_hi.y &= kAbs; a_hi.z &= kAbs; a_hi.w &= kAbs;
+          b_0.x &= kAbs; b_0.y &= kAbs; b_0.z &= kAbs; b_0.w &= kAbs;
+          b_1.x &= kAbs; b_1.y &= kAbs; b_1.z &= kAbs; b_1.w &= kAbs;
+          mma_bf16_16816(m0, a_lo.x, a_hi.x, a_lo.y, a_hi.y, b_0.x, b_0.y);
+          mma_bf16_16816(m1, a_lo.x, a_hi.x, a_lo.y, a_hi.y, b_1.x, b_1.y);
+          mma_bf16_16816(m0, a_lo.z, a_hi.z, a_lo.w, a_hi.w, b_0.z, b_0.w);
+          mma_bf16_16816(m1, a_lo.z, a_hi.z, a_lo.w, a_hi.w, b_1.z, b_1.w);
+        }
+        // c[0], c[1]: row g, pages 2 t4, 2 t4 + 1 of the 8-page tile; c[2], c[3]: row g + 8
+#pragma unroll
+        for (int hr = 0; hr < 2; ++hr) {
+          const int r = 16 * mt + g + 8 * hr;
+          if (r < nr) {
+            const int row = r0 + r, a = row / p.G, gi = row % p.G;
+            float2* dst = bounds + ((static_cast<size_t>(w.s) * p.B + a) * p.Hq + w.kh * p.G + gi) * p.score_stride + w.p0 + warp * WP + 2 * t4;
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+              const int col = warp * WP + 2 * t4 + e;
+              const float d0 = kMmaErrCoef * m0[2 * hr + e], d1 = kMmaErrCoef * m1[2 * hr + e];
+              if (col < w.np) dst[e] = make_float2(c0[2 * hr + e] - d0, c0[2 * hr + e] + d0);
+              if (col + 8 < w.np) dst[e + 8] = make_float2(c1[2 * hr + e] - d1, c1[2 * hr + e] + d1);
+            }
+          }
+        }
+      }
+    }
+  }
+  cp_async_wait_pending(0);
+}
+
 template <typename T, int D, int PG>
 int32_t launch_stream(losa_ctx* c, const PsParams& pp, cudaStream_t st) {
   using C = PsCfg<T, D, PG>;
@@ -499,10 +753,26 @@ int32_t launch_stream(losa_ctx* c, const PsParams& pp, cudaStream_t st) {
   return after_launch(c);
 }
 
-}  // namespace
+template <int D>
+int32_t launch_bounds_t(losa_ctx* c, const PsParams& pp, cudaStream_t st) {
+  using C = MmaCfg<D>;
+  PsParams p = pp;
+  const int tail = ps_tail_bytes(p.N);
+  int ns = (kPsSmemBudget - C::QBUF_BYTES - tail - 128) / C::STAGE_BYTES;
+  ns = ns > kPsMaxStages ? kPsMaxStages : ns;
+  if (ns < 2) return LOSA_ERR_UNSUPPORTED;
+  p.n_stages = ns;
+  const int smem = 128 + ns * C::STAGE_BYTES + C::QBUF_BYTES + tail;
+  if (!c->bounds_attr_set) {
+    LOSA_CUDA_TRY(c, cudaFuncSetAttribute(page_bounds_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    c->bounds_attr_set = 1;
+  }
+  launch_k(page_bounds_mma_kernel<D>, p.n_ctas, kPsThreads, smem, st, p);
+  return after_launch(c);
+}
 
-int32_t launch_page_scores(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
-                           const int32_t* n_active, const int32_t* step, cudaStream_t st) {
+PsParams make_params(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
+                     const int32_t* n_active, const int32_t* step) {
   const losa_shape_t& sh = c->shape;
   PsParams p;
   p.q = q;
@@ -526,6 +796,22 @@ int32_t launch_page_scores(losa_ctx* c, const void* q, const losa_kv_t* kv, cons
   p.score_stride = c->lay.score_stride;
   p.n_ctas = c->n_sms;
   p.n_stages = 0;
+  return p;
+}
+
+}  // namespace
+
+// bf16 only: (lower, upper) bound pairs of the page scores into the workspace's score rows (as float2)
+int32_t launch_page_bounds(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
+                           const int32_t* n_active, const int32_t* step, cudaStream_t st) {
+  const PsParams p = make_params(c, q, kv, active_idx, n_active, step);
+  return c->shape.head_dim == 128 ? launch_bounds_t<128>(c, p, st) : launch_bounds_t<64>(c, p, st);
+}
+
+int32_t launch_page_scores(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
+                           const int32_t* n_active, const int32_t* step, cudaStream_t st) {
+  const losa_shape_t& sh = c->shape;
+  const PsParams p = make_params(c, q, kv, active_idx, n_active, step);
   const bool bf = sh.dtype == LOSA_BF16;
   if (bf && sh.head_dim == 128) return launch_stream<__nv_bfloat16, 128, 4>(c, p, st);
   if (bf) return launch_stream<__nv_bfloat16, 64, 4>(c, p, st);

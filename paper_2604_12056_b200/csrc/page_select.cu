@@ -254,6 +254,285 @@ __device__ __forceinline__ void topk_select_body(const Row& row, int P, int kk, 
   }
 }
 
+
+// ---- bf16 fast path: candidates from tensor-core bounds, exact scores for the candidates only ----
+// The page score in the order the interface fixes, by four lanes (u = lane % 4; qs: [q+ (D) | q- (D)]
+// fp32 in shared memory): lane u runs the chains of runs u, u + 4(, u + 8, u + 12) - 16 fused
+// multiply-adds per run of 8 dimensions - and the butterfly c[i] += c[i ^ off], off = D/16 .. 1, is
+// taken inside the lane while off >= 4 and with two shuffles below that.  All four lanes return it.
+template <int D>
+__device__ __forceinline__ float exact_score4(const float* __restrict__ qs, const __nv_bfloat16* __restrict__ lo_p,
+                                              const __nv_bfloat16* __restrict__ hi_p, int u) {
+  constexpr int RPL = D / 32;      // runs per lane
+  uint4 lo_raw[RPL], hi_raw[RPL];  // requested together, converted run by run
+#pragma unroll
+  for (int w = 0; w < RPL; ++w) {
+    lo_raw[w] = __ldg(reinterpret_cast<const uint4*>(lo_p + 8 * (u + 4 * w)));
+    hi_raw[w] = __ldg(reinterpret_cast<const uint4*>(hi_p + 8 * (u + 4 * w)));
+  }
+  float c[RPL];
+#pragma unroll
+  for (int w = 0; w < RPL; ++w) {
+    const int t = u + 4 * w;
+    const uint32_t lw[4] = {lo_raw[w].x, lo_raw[w].y, lo_raw[w].z, lo_raw[w].w};
+    const uint32_t hw[4] = {hi_raw[w].x, hi_raw[w].y, hi_raw[w].z, hi_raw[w].w};
+    float acc = 0.f;
+#pragma unroll
+    for (int j2 = 0; j2 < 4; ++j2) {
+      const float2 qp = *reinterpret_cast<const float2*>(qs + 8 * t + 2 * j2);
+      const float2 qn = *reinterpret_cast<const float2*>(qs + D + 8 * t + 2 * j2);
+      acc = __fmaf_rn(qp.x, __uint_as_float(hw[j2] << 16), acc);
+      acc = __fmaf_rn(qn.x, __uint_as_float(lw[j2] << 16), acc);
+      acc = __fmaf_rn(qp.y, __uint_as_float(hw[j2] & 0xffff0000u), acc);
+      acc = __fmaf_rn(qn.y, __uint_as_float(lw[j2] & 0xffff0000u), acc);
+    }
+    c[w] = acc;
+  }
+  float v;
+  if constexpr (RPL == 4) v = __fadd_rn(__fadd_rn(c[0], c[2]), __fadd_rn(c[1], c[3]));   // off = 8, then off = 4
+  else v = __fadd_rn(c[0], c[1]);                                                         // off = 4
+  v = __fadd_rn(v, __shfl_xor_sync(0xffffffffu, v, 2));
+  v = __fadd_rn(v, __shfl_xor_sync(0xffffffffu, v, 1));
+  return __fadd_rn(v, 0.0f);
+}
+
+struct RefineParams {
+  float2* bounds;                 // (A - delta, A + delta) per (row, page); reused as fp32 score rows by the fallback
+  const __nv_bfloat16* q;
+  const __nv_bfloat16* kmin;
+  const __nv_bfloat16* kmax;
+  const int32_t* page_table;
+  const int32_t* kv_len;
+  const int32_t* active_idx;
+  const int32_t* n_active;
+  const int32_t* step;
+  int32_t* topk_pages;
+  float* topk_scores;
+  int32_t* status;
+  int N, B, Hq, Hkv, g, k, score_stride, Pmax, n_phys;
+};
+
+// One CTA of kSelThreads per (sequence, head, 1/8 of the active slots).  Per query: tau = lower edge
+// of the histogram bin that holds the k-th largest LOWER bound; every page whose UPPER bound reaches
+// tau is a candidate (a superset of the exact top-k, ties included: the exact score lies between the
+// bounds); exact scores in the fixed order for the candidates (four lanes each), sort, emit.  More
+// than kSelCap candidates (possible only when most pages nearly tie): exact scores for every page
+// into the score row, then the plain threshold search.
+template <int D>
+__global__ void __launch_bounds__(kSelThreads, 6)
+topk_refine_kernel(RefineParams p) {
+  grid_dep_trigger();
+  grid_dep_wait();
+  __shared__ __align__(16) float qs[2 * D];
+  __shared__ unsigned long long ckey[kSelCap];
+  __shared__ int cpage[kSelCap];
+  __shared__ int hist[kSelBins];
+  __shared__ uint32_t s_red[2][kSelThreads / 32];
+  __shared__ int s_ncand, s_bstar;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int qid = blockIdx.x;
+  const int h = qid % p.Hq, s = (qid / p.Hq) % p.N, j0 = qid / (p.Hq * p.N);
+  if (p.step && p.step[s] == 0) return;
+  int na = p.n_active[s];
+  na = na > p.B ? p.B : na;
+  int P = pages_of(p.kv_len[s], p.g);
+  if (P > p.Pmax) { if (tid == 0) set_status(p.status, LOSA_ERR_BOUNDS); P = p.Pmax; }
+  const int kk = min(p.k, P), kh = h / (p.Hq / p.Hkv);
+  const __nv_bfloat16* lo_base = p.kmin + static_cast<size_t>(kh) * D;
+  const __nv_bfloat16* hi_base = p.kmax + static_cast<size_t>(kh) * D;
+  const int u = lane & 3;
+  for (int a = j0; a < na; a += kSelSlots) {
+    const int tok = p.active_idx[s * p.B + a];
+    if (tok < 0 || tok >= p.B) { if (tid == 0) set_status(p.status, LOSA_ERR_BOUNDS); continue; }
+    float2* row2 = p.bounds + ((static_cast<size_t>(s) * p.B + a) * p.Hq + h) * p.score_stride;
+    const size_t o = ((static_cast<size_t>(s) * p.B + tok) * p.Hq + h) * p.k;
+    int32_t* out_pages = p.topk_pages + o;
+    float* out_scores = p.topk_scores ? p.topk_scores + o : nullptr;
+    // the bounds of this thread's pages: one round trip, kept in registers when the prefix has at
+    // most kSelThreads * kSelPerThread pages
+    const bool cached = P <= kSelThreads * kSelPerThread;
+    uint32_t lbc[kSelPerThread], ubc[kSelPerThread];
+    if (cached) {
+      float2 bv[kSelPerThread];
+#pragma unroll
+      for (int i = 0; i < kSelPerThread; ++i) {
+        const int pg = tid + kSelThreads * i;
+        bv[i] = pg < P ? row2[pg] : make_float2(0.f, 0.f);
+      }
+#pragma unroll
+      for (int i = 0; i < kSelPerThread; ++i) {
+        lbc[i] = order_bits(bv[i].x);
+        ubc[i] = order_bits(bv[i].y);
+      }
+    }
+    auto for_each_page = [&](auto&& f) {        // f(lower bits, upper bits, page)
+      if (cached) {
+#pragma unroll
+        for (int i = 0; i < kSelPerThread; ++i) {
+          const int pg = tid + kSelThreads * i;
+          if (pg < P) f(lbc[i], ubc[i], pg);
+        }
+      } else {
+        for (int pg = tid; pg < P; pg += kSelThreads) {
+          const float2 bv = row2[pg];
+          f(order_bits(bv.x), order_bits(bv.y), pg);
+        }
+      }
+    };
+    // the query, split into its positive and negative parts
+    for (int j = tid; j < D; j += kSelThreads) {
+      const float v = __bfloat162float(p.q[((static_cast<size_t>(s) * p.B + tok) * p.Hq + h) * D + j]);
+      qs[j] = fmaxf(v, 0.f);
+      qs[D + j] = fminf(v, 0.f);
+    }
+    if (tid == 0) s_ncand = 0;
+    for (int b = tid; b < kSelBins; b += kSelThreads) hist[b] = 0;
+    // ---- tau
+    uint32_t tau = 0u;
+    if (kk < P) {
+      uint32_t lo = 0xffffffffu, hi = 0u;
+      for_each_page([&](uint32_t lb, uint32_t, int) { lo = min(lo, lb); hi = max(hi, lb); });
+      lo = __reduce_min_sync(0xffffffffu, lo);
+      hi = __reduce_max_sync(0xffffffffu, hi);
+      if (lane == 0) { s_red[0][warp] = lo; s_red[1][warp] = hi; }
+      __syncthreads();
+#pragma unroll
+      for (int w = 0; w < kSelThreads / 32; ++w) { lo = min(lo, s_red[0][w]); hi = max(hi, s_red[1][w]); }
+      if (lo < hi) {
+        const int width = 32 - __clz(hi - lo);
+        const int shift = width > 8 ? width - 8 : 0;
+        for_each_page([&](uint32_t lb, uint32_t, int) { atomicAdd(&hist[(lb - lo) >> shift], 1); });
+        __syncthreads();
+        if (warp == 0) {
+          int c[8], tot = 0;
+#pragma unroll
+          for (int e = 0; e < 8; ++e) { c[e] = hist[8 * lane + e]; tot += c[e]; }
+          int suf = tot;
+#pragma unroll
+          for (int off = 1; off < 32; off <<= 1) {
+            const int t = __shfl_down_sync(0xffffffffu, suf, off);
+            if (lane + off < 32) suf += t;
+          }
+          const int above_lanes = suf - tot;
+          if (above_lanes < kk && kk <= suf) {
+            int run = above_lanes;
+#pragma unroll
+            for (int e = 7; e >= 0; --e) {
+              if (run < kk && kk <= run + c[e]) s_bstar = 8 * lane + e;
+              run += c[e];
+            }
+          }
+        }
+        __syncthreads();
+        tau = lo + (static_cast<uint32_t>(s_bstar) << shift);
+      } else {
+        tau = lo;
+      }
+    } else {
+      __syncthreads();
+    }
+    // ---- candidates: pages whose upper bound reaches tau
+    for_each_page([&](uint32_t, uint32_t ub, int pg) {
+      if (ub >= tau) {
+        const int i = atomicAdd(&s_ncand, 1);
+        if (i < kSelCap) cpage[i] = pg;
+      }
+    });
+    __syncthreads();
+    const int ncand = s_ncand;
+    auto phys_of = [&](int pg) {
+      int ph = __ldg(p.page_table + static_cast<size_t>(s) * p.Pmax + pg);
+      if (ph < 0 || ph >= p.n_phys) { set_status(p.status, LOSA_ERR_BOUNDS); ph = 0; }
+      return ph;
+    };
+    auto exact_at = [&](int ph) {                 // called by the four lanes of a group with the same page
+      const size_t so = static_cast<size_t>(ph) * p.Hkv * D;
+      return exact_score4<D>(qs, lo_base + so, hi_base + so, u);
+    };
+    if (ncand > kSelCap) {
+      float* row = reinterpret_cast<float*>(row2);             // the bounds are not needed any more
+      for (int p0 = 0; p0 < P; p0 += kSelThreads / 4) {          // whole warps: the shuffles need all lanes
+        const int pg = min(p0 + tid / 4, P - 1);
+        const float e = exact_at(phys_of(pg));
+        if (u == 0 && p0 + tid / 4 < P) row[pg] = e;
+      }
+      __syncthreads();
+      const RowView<false> rv{row, 1, p.score_stride};
+      topk_select_body<false>(rv, P, kk, p.k, out_pages, out_scores, 1);
+      __syncthreads();
+      continue;
+    }
+    // a group of four lanes per candidate, 32 candidates per round; the physical page ids of four
+    // rounds are requested together (one round trip instead of four)
+    constexpr int kPer = kSelThreads / 4, kAhead = 4;
+    for (int i0 = 0; i0 < ncand; i0 += kPer * kAhead) {
+      int pgs[kAhead], phs[kAhead];
+#pragma unroll
+      for (int r = 0; r < kAhead; ++r) {
+        pgs[r] = cpage[min(i0 + r * kPer + tid / 4, ncand - 1)];
+        phs[r] = phys_of(pgs[r]);
+      }
+#pragma unroll
+      for (int r = 0; r < kAhead; ++r) {
+        if (i0 + r * kPer < ncand) {                     // uniform over the CTA
+          const float e = exact_at(phs[r]);
+          const int i = i0 + r * kPer + tid / 4;
+          if (u == 0 && i < ncand) ckey[i] = make_key(order_bits(e), pgs[r]);
+        }
+      }
+    }
+    // ---- order the candidates (descending) and emit the first kk
+    __syncthreads();
+    if (ncand <= 2 * kSelThreads) {
+      // few candidates (the usual case): a candidate's position is the number of larger keys (all
+      // keys differ); every thread counts for up to two candidates, the keys are read as broadcasts
+      unsigned long long mine[2];
+      int rank[2] = {0, 0};
+#pragma unroll
+      for (int e = 0; e < 2; ++e) mine[e] = tid + e * kSelThreads < ncand ? ckey[tid + e * kSelThreads] : ~0ull;
+      for (int i = 0; i < ncand; ++i) {
+        const unsigned long long key = ckey[i];
+        rank[0] += key > mine[0] ? 1 : 0;
+        rank[1] += key > mine[1] ? 1 : 0;
+      }
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        if (tid + e * kSelThreads < ncand && rank[e] < kk) {
+          out_pages[rank[e]] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(mine[e]));
+          if (out_scores) out_scores[rank[e]] = unorder_bits(static_cast<uint32_t>(mine[e] >> 32));
+        }
+      }
+      for (int j = kk + tid; j < p.k; j += kSelThreads) out_pages[j] = -1;
+    } else {
+      int n2 = 2;
+      while (n2 < ncand) n2 <<= 1;
+      for (int i = ncand + tid; i < n2; i += kSelThreads) ckey[i] = 0ull;
+      __syncthreads();
+      for (int k2 = 2; k2 <= n2; k2 <<= 1) {
+        for (int j = k2 >> 1; j > 0; j >>= 1) {
+          for (int t = tid; t < (n2 >> 1); t += kSelThreads) {
+            const int i = ((t & ~(j - 1)) << 1) | (t & (j - 1));
+            const int x = i | j;
+            const unsigned long long ka = ckey[i], kb = ckey[x];
+            if ((ka < kb) == ((i & k2) == 0)) { ckey[i] = kb; ckey[x] = ka; }
+          }
+          __syncthreads();
+        }
+      }
+      for (int j = tid; j < p.k; j += kSelThreads) {
+        if (j < kk) {
+          const unsigned long long key = ckey[j];
+          out_pages[j] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(key));
+          if (out_scores) out_scores[j] = unorder_bits(static_cast<uint32_t>(key >> 32));
+        } else {
+          out_pages[j] = -1;
+        }
+      }
+    }
+    __syncthreads();                               // the shared state is reused by the next slot
+  }
+}
+
 template <bool POOLED>
 __global__ void __launch_bounds__(kSelThreads)
 topk_select_kernel(float* __restrict__ scores, const int32_t* __restrict__ kv_len,
@@ -417,6 +696,30 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
   if (sh.max_pages_per_seq == 0) return LOSA_OK;
   const int pool = pooled ? sh.n_q_heads / sh.n_kv_heads : 1;
   const bool bf = sh.dtype == LOSA_BF16;
+  if (bf && !pooled && k <= kSelCap) {
+    // bf16, one list per query head: bounds from the tensor cores, exact scores for the candidates only
+    int32_t rc = launch_page_bounds(c, q, kv, active_idx, n_active, step, st);
+    if (rc != LOSA_OK) return rc;
+    RefineParams rp;
+    rp.bounds = reinterpret_cast<float2*>(c->ws + c->lay.scores);
+    rp.q = static_cast<const __nv_bfloat16*>(q);
+    rp.kmin = static_cast<const __nv_bfloat16*>(kv->kmin);
+    rp.kmax = static_cast<const __nv_bfloat16*>(kv->kmax);
+    rp.page_table = kv->page_table;
+    rp.kv_len = kv->kv_len;
+    rp.active_idx = active_idx;
+    rp.n_active = n_active;
+    rp.step = step;
+    rp.topk_pages = topk_pages;
+    rp.topk_scores = topk_scores_opt;
+    rp.status = status_ptr(c);
+    rp.N = sh.batch; rp.B = sh.block_size; rp.Hq = sh.n_q_heads; rp.Hkv = sh.n_kv_heads; rp.g = sh.page_size;
+    rp.k = k; rp.score_stride = c->lay.score_stride; rp.Pmax = sh.max_pages_per_seq; rp.n_phys = kv->n_phys_pages;
+    const int queries = sh.batch * std::min<int>(sh.block_size, kSelSlots) * sh.n_q_heads;
+    if (sh.head_dim == 128) launch_k(topk_refine_kernel<128>, queries, kSelThreads, 0, st, rp);
+    else launch_k(topk_refine_kernel<64>, queries, kSelThreads, 0, st, rp);
+    return after_launch(c);
+  }
   int32_t rc = launch_page_scores(c, q, kv, active_idx, n_active, step, st);
   if (rc != LOSA_OK) return rc;
 
