@@ -235,6 +235,84 @@ void oracle_page_scores_one(const oracle_shape_t* sh, const void* q, const oracl
   }
 }
 
+/* ---------- Section 2.3: relaxed validity of a page list (selector variants with their own arithmetic) ----------
+ * The paper fixes no arithmetic for the page bound, and calls the method independent of the
+ * selector.  A selector that evaluates U(p) = sum_j max(q_j kmin_j, q_j kmax_j) in another order
+ * or precision than the fixed fp32 order cannot be compared list by list; it is checked against
+ * this rule instead, in fp64:
+ *   a list of (token, head) is VALID iff it holds exactly min(k, P_s) distinct pages of
+ *   0 .. P_s - 1 followed by -1 padding, and every listed page p has
+ *       U64(p) >= T - eps * Smax,
+ *   where T is the min(k, P_s)-th largest U64 over all pages and Smax = max_p sum_j |t_j(p)|,
+ *   t_j = the larger of q_j kmin_j and q_j kmax_j (the magnitude rounding errors scale with).
+ * With eps = 0 the only valid lists are the exact top-k sets (up to ties).  Order inside a list is
+ * not part of the rule.  Returns the number of invalid lists over the active (token, head) pairs
+ * of the sequences whose step is not 0. */
+static double page_bound_abs_f64(const float* q, const float* lo, const float* hi, int d) {
+  double acc = 0.0;
+  for (int j = 0; j < d; ++j) {
+    const double a = (double)q[j] * (double)lo[j], b = (double)q[j] * (double)hi[j];
+    acc += fabs((a > b) ? a : b);
+  }
+  return acc;
+}
+static int cmp_double_desc(const void* a, const void* b) {
+  const double x = *(const double*)a, y = *(const double*)b;
+  return (x < y) - (x > y);
+}
+int64_t oracle_check_topk_relaxed(const oracle_shape_t* sh, const void* q, const oracle_kv_t* kv,
+                                  const int32_t* active_idx, const int32_t* n_active,
+                                  const int32_t* step, int32_t k, const int32_t* topk_pages, double eps) {
+  const int B = sh->block_size, Hq = sh->n_q_heads, d = sh->head_dim, Hkv = sh->n_kv_heads, G = Hq / Hkv;
+  int64_t bad = 0;
+  for (int s = 0; s < sh->batch; ++s) {
+    if (step && step[s] == 0) continue;
+    const int P = pages_of(kv->kv_len[s], sh->page_size);
+    const int kk = k < P ? k : P;
+    for (int a = 0; a < n_active[s]; ++a) {
+      const int tok = active_idx[(int64_t)s * B + a];
+      for (int h = 0; h < Hq; ++h) {
+        const int32_t* list = topk_pages + (((int64_t)s * B + tok) * Hq + h) * k;
+        double* u = (double*)malloc(sizeof(double) * (P > 0 ? P : 1));
+        double* sorted = (double*)malloc(sizeof(double) * (P > 0 ? P : 1));
+        char* seen = (char*)calloc(P > 0 ? P : 1, 1);
+        float qv[512], lo[512], hi[512];
+        const int64_t qo = (((int64_t)s * B + tok) * Hq + h) * d;
+        for (int j = 0; j < d; ++j) qv[j] = ld_f32(q, sh->dtype, qo + j);
+        double smax = 0.0;
+        for (int p = 0; p < P; ++p) {
+          const int32_t phys = kv->page_table[(int64_t)s * sh->max_pages_per_seq + p];
+          const int64_t so = ((int64_t)phys * Hkv + h / G) * d;
+          for (int j = 0; j < d; ++j) {
+            lo[j] = ld_f32(kv->kmin, sh->dtype, so + j);
+            hi[j] = ld_f32(kv->kmax, sh->dtype, so + j);
+          }
+          u[p] = page_bound_f64(qv, lo, hi, d);
+          const double sa = page_bound_abs_f64(qv, lo, hi, d);
+          if (sa > smax) smax = sa;
+          sorted[p] = u[p];
+        }
+        qsort(sorted, P, sizeof(double), cmp_double_desc);
+        int ok = 1;
+        for (int j = 0; j < k; ++j) {
+          const int32_t p = list[j];
+          if (j < kk) {
+            if (p < 0 || p >= P || seen[p]) { ok = 0; break; }
+            seen[p] = 1;
+            if (u[p] < sorted[kk - 1] - eps * smax) { ok = 0; break; }
+          } else if (p != -1) {
+            ok = 0;
+            break;
+          }
+        }
+        bad += ok ? 0 : 1;
+        free(u); free(sorted); free(seen);
+      }
+    }
+  }
+  return bad;
+}
+
 /* ---------- Section 2.3 / 4.2: top-k pages for the active queries only ----------
  * I_{i,h} = the min(k, P_s) pages with the largest bound, ordered (bound descending, page
  * ascending).  Every (token, query head) is one query.  Sequences at step 0 are skipped. */

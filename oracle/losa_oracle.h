@@ -71,6 +71,13 @@ void oracle_page_scores_topk_pooled(const oracle_shape_t* sh, const void* q, con
                                     float* topk_scores);
 
 /* Section 4.2 / 4.4: union per (sequence, KV head). */
+/* Relaxed validity of page lists produced with another arithmetic than the fixed fp32 order: number of
+ * (active token, head) lists that are not "min(k, P) distinct in-range pages, each with fp64 bound >=
+ * the k-th largest fp64 bound - eps * (largest sum of term magnitudes)", then -1 padding. */
+int64_t oracle_check_topk_relaxed(const oracle_shape_t* sh, const void* q, const oracle_kv_t* kv,
+                                  const int32_t* active_idx, const int32_t* n_active,
+                                  const int32_t* step, int32_t k, const int32_t* topk_pages, double eps);
+
 void oracle_page_union(const oracle_shape_t* sh, const int32_t* topk_pages,
                        const int32_t* active_idx, const int32_t* n_active, int32_t k,
                        const int32_t* kv_len, const int32_t* step, int32_t* union_pages,

@@ -198,6 +198,18 @@ def page_scores_topk_pooled(sh: Shape, q, kv: KV, active_idx, n_active, k: int, 
     return topk_pages, topk_scores
 
 
+def check_topk_relaxed(sh: Shape, q, kv: KV, active_idx, n_active, k: int, topk_pages, eps: float, step=None) -> int:
+    """Number of (active token, head) lists that break the relaxed validity rule (fp64 bounds, slack
+    eps times the largest sum of term magnitudes); see losa_oracle.c."""
+    st = None if step is None else np.ascontiguousarray(step, np.int32)
+    s, kvc = sh.c(), kv.c()
+    fn = lib().oracle_check_topk_relaxed
+    fn.restype = C.c_int64
+    return int(fn(C.byref(s), _p(_chk(q, sh.elem, "q")), C.byref(kvc), _p(_chk(active_idx, np.int32, "active_idx")),
+                  _p(_chk(n_active, np.int32, "n_active")), _p(st), C.c_int32(k),
+                  _p(_chk(topk_pages, np.int32, "topk")), C.c_double(eps)))
+
+
 def page_union(sh: Shape, topk_pages, active_idx, n_active, k: int, kv_len, step=None):
     """Returns (union_pages [N,H_kv,P_max] int32, union_count [N,H_kv] int32)."""
     N, Hkv, P = sh.batch, sh.n_kv_heads, sh.max_pages_per_seq

@@ -471,3 +471,47 @@ def test_paper_stated_sizes():
     # worst case of the union (Section 3.1): min(L, B k) positions
     L, k = facts["example_L"], facts["example_k"]
     assert min(L, B * k) == facts["example_union_worst"]
+
+
+# --- relaxed validity rule for selectors with their own arithmetic (Section 2.3 leaves the selector open)
+def test_relaxed_list_rule_accepts_the_exact_lists_and_rejects_worse_ones():
+    pb = Problem(31, N=2, Hq=4, Hkv=2, d=32, B=3, g=4, kv_lens=(90, 37))
+    sh = pb.sh
+    orc.build_page_summaries(sh, pb.kv)
+    act = np.array([[0, 2, -1], [1, -1, -1]], np.int32)
+    na = np.array([2, 1], np.int32)
+    k = 5
+    topk, _ = orc.page_scores_topk(sh, pb.q, pb.kv, act, na, k)
+    assert orc.check_topk_relaxed(sh, pb.q, pb.kv, act, na, k, topk, 0.0) == 0          # exact lists pass with no slack
+    shuffled = topk.copy()
+    shuffled[0, 0, 1] = topk[0, 0, 1][::-1]                                           # order is not part of the rule
+    assert orc.check_topk_relaxed(sh, pb.q, pb.kv, act, na, k, shuffled, 0.0) == 0
+    # replace the weakest chosen page of one list by the worst page of all: invalid at any small slack
+    _, u64 = orc.page_scores_one(sh, pb.q, pb.kv, 0, 2, 3)
+    worst = int(np.argmin(u64))
+    bad = topk.copy()
+    assert worst not in bad[0, 2, 3].tolist()
+    bad[0, 2, 3, k - 1] = worst
+    assert orc.check_topk_relaxed(sh, pb.q, pb.kv, act, na, k, bad, 1e-6) == 1
+    # ... but valid once the slack covers the gap (brute force of the rule's own inequality)
+    kth = np.sort(u64)[::-1][k - 1]
+    lo, hi = pb.f(pb.kmin), pb.f(pb.kmax)
+    qv = pb.f(pb.q)[0, 2, 3].astype(np.float64)
+    smax = 0.0
+    for p in range(pb.pages(0)):
+        ph = pb.page_table[0, p]
+        t = np.maximum(qv * lo[ph, 1].astype(np.float64), qv * hi[ph, 1].astype(np.float64))
+        smax = max(smax, np.abs(t).sum())
+    need = (kth - u64[worst]) / smax
+    assert orc.check_topk_relaxed(sh, pb.q, pb.kv, act, na, k, bad, need * 1.01) == 0
+    assert orc.check_topk_relaxed(sh, pb.q, pb.kv, act, na, k, bad, need * 0.99) == 1
+    # structural violations: a repeated page, an out-of-range page, a missing entry, wrong padding
+    for edit in (lambda t: t.__setitem__((1, 1, 0, 1), t[1, 1, 0, 0]), lambda t: t.__setitem__((1, 1, 0, 0), 10),
+                 lambda t: t.__setitem__((1, 1, 0, 4), -1)):
+        t2 = topk.copy()
+        edit(t2)
+        assert orc.check_topk_relaxed(sh, pb.q, pb.kv, act, na, k, t2, 1.0) == 1
+    wide, _ = orc.page_scores_topk(sh, pb.q, pb.kv, act, na, 12)                        # k > P for sequence 1 (10 pages)
+    assert orc.check_topk_relaxed(sh, pb.q, pb.kv, act, na, 12, wide, 0.0) == 0
+    wide[1, 1, 2, 11] = 3
+    assert orc.check_topk_relaxed(sh, pb.q, pb.kv, act, na, 12, wide, 1.0) == 1
