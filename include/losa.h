@@ -238,6 +238,20 @@ int32_t losa_page_scores_topk_pooled(losa_ctx* ctx, const void* q, const losa_kv
                                      const int32_t* step, int32_t k, int32_t* topk_pages,
                                      float* topk_scores_opt, void* stream);
 
+/* Stage 2, tensor-core selector (bf16 only) - the page scores as one GEMM [q+ | q-] x [kmax | kmin] on
+ *   the tensor cores, top-k on its fp32 results.  The paper calls its method independent of the
+ *   selector (Section 2.3) and fixes no arithmetic; this variant gives up the fixed summation order of
+ *   losa_page_scores_topk, so its lists are not comparable entry by entry.  What holds instead: a
+ *   list has min(k, P_s) distinct pages of 0 .. P_s-1, then -1, and every listed page's score (in
+ *   exact arithmetic) is at least the k-th largest exact score minus 2^-11 times the largest
+ *   sum_j |t_j| over the pages (t_j the terms of U).  Lists are ordered by the tensor-core score
+ *   (descending, page ascending); topk_scores_opt receives those scores.  Same arguments and errors;
+ *   fp32 contexts return LOSA_ERR_UNSUPPORTED. */
+int32_t losa_page_scores_topk_mma(losa_ctx* ctx, const void* q, const losa_kv_t* kv,
+                                  const int32_t* active_idx, const int32_t* n_active,
+                                  const int32_t* step, int32_t k, int32_t* topk_pages,
+                                  float* topk_scores_opt, void* stream);
+
 /* Selector used by losa_denoise_step / losa_denoise_step_host on this context: 0 (default) = one
  *   list per query head, non-zero = the pooled selector.  Host-side switch; takes effect for calls
  *   issued after it returns. */

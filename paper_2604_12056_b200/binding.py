@@ -30,7 +30,7 @@ EXPORTS = [
     "losa_update_prefix_cache", "losa_build_page_summaries", "losa_denoise_step_host",
     "losa_profile_stage4", "losa_stage4_last_ms", "losa_select_active_static",
     "losa_denoise_step", "losa_select_active_tau", "losa_page_scores_topk_pooled",
-    "losa_set_pooled_selection", "losa_set_wait_limit",
+    "losa_set_pooled_selection", "losa_set_wait_limit", "losa_page_scores_topk_mma",
 ]
 
 
@@ -209,6 +209,13 @@ def losa_page_scores_topk(ctx, q, kv, active_idx, n_active, step, k, topk_pages,
 
 def losa_page_scores_topk_pooled(ctx, q, kv, active_idx, n_active, step, k, topk_pages, topk_scores_opt=None):
     ctx._check("losa_page_scores_topk_pooled", lib().losa_page_scores_topk_pooled(
+        ctx._h, _ptr(q), C.byref(kv), _ptr(active_idx), _ptr(n_active), _ptr(step), C.c_int32(k),
+        _ptr(topk_pages), _ptr(topk_scores_opt), _stream()))
+
+
+def losa_page_scores_topk_mma(ctx, q, kv, active_idx, n_active, step, k, topk_pages, topk_scores_opt=None):
+    """Stage 2 with tensor-core scores (bf16): lists valid under the relaxed rule, not entry by entry."""
+    ctx._check("losa_page_scores_topk_mma", lib().losa_page_scores_topk_mma(
         ctx._h, _ptr(q), C.byref(kv), _ptr(active_idx), _ptr(n_active), _ptr(step), C.c_int32(k),
         _ptr(topk_pages), _ptr(topk_scores_opt), _stream()))
 

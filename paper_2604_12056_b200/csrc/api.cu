@@ -202,7 +202,17 @@ int32_t losa_page_scores_topk_pooled(losa_ctx* ctx, const void* q, const losa_kv
   int32_t rc = check_kv(ctx, kv, true);
   if (rc != LOSA_OK) return rc;
   if (!aligned16(q)) return LOSA_ERR_UNSUPPORTED;
-  return launch_page_scores_topk(ctx, q, kv, active_idx, n_active, step, k, topk_pages, topk_scores_opt, as_stream(stream), true);
+  return launch_page_scores_topk(ctx, q, kv, active_idx, n_active, step, k, topk_pages, topk_scores_opt, as_stream(stream), kSelectorPooled);
+}
+
+int32_t losa_page_scores_topk_mma(losa_ctx* ctx, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
+                                  const int32_t* n_active, const int32_t* step, int32_t k, int32_t* topk_pages,
+                                  float* topk_scores_opt, void* stream) {
+  if (!ctx || !q || !active_idx || !n_active || !topk_pages || k < 1) return LOSA_ERR_INVALID_ARG;
+  int32_t rc = check_kv(ctx, kv, true);
+  if (rc != LOSA_OK) return rc;
+  if (!aligned16(q) || ctx->shape.dtype != LOSA_BF16) return LOSA_ERR_UNSUPPORTED;
+  return launch_page_scores_topk(ctx, q, kv, active_idx, n_active, step, k, topk_pages, topk_scores_opt, as_stream(stream), kSelectorMma);
 }
 
 int32_t losa_set_pooled_selection(losa_ctx* ctx, int32_t on) {
@@ -290,7 +300,7 @@ int32_t losa_denoise_step(losa_ctx* ctx, const void* q, const void* k_blk, const
   int32_t* slot_map = reinterpret_cast<int32_t*>(ctx->ws + ctx->lay.slot_map);
   rc = launch_select_active(ctx, q, state->q_prev, sh.n_q_heads * sh.head_dim, m_per_seq, state->step,
                             buf->active_idx, buf->n_active, nullptr, st, 0.0, slot_map);
-  if (rc == LOSA_OK) rc = launch_page_scores_topk(ctx, q, kv, buf->active_idx, buf->n_active, state->step, k, buf->topk_pages, nullptr, st, ctx->pooled_selection != 0);
+  if (rc == LOSA_OK) rc = launch_page_scores_topk(ctx, q, kv, buf->active_idx, buf->n_active, state->step, k, buf->topk_pages, nullptr, st, ctx->pooled_selection != 0 ? kSelectorPooled : kSelectorExact);
   if (rc == LOSA_OK) rc = launch_page_union(ctx, buf->topk_pages, buf->active_idx, buf->n_active, k, kv->kv_len, state->step, buf->union_pages, buf->union_count, st);
   if (rc == LOSA_OK) rc = launch_sparse_prefix_attn(ctx, q, kv, buf->active_idx, buf->n_active, buf->union_pages, buf->union_count, state, st, true);
   // join (also when a launch above failed: the forked kernel must not be left reading the caller's

@@ -65,6 +65,7 @@ struct losa_ctx {
   int32_t attn_attr_set;
   int32_t scores_attr_set;   // likewise for the page-score kernel
   int32_t bounds_attr_set;   // and for the tensor-core page-bound kernel
+  int32_t approx_attr_set;
   int32_t refine_attr_set;
   // optional timing of the stage-4 main kernel
   int32_t profile;

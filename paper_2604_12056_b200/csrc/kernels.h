@@ -13,7 +13,9 @@ int32_t launch_select_active(losa_ctx* c, const void* x_cur, const void* x_prev,
 int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
                                 const int32_t* active_idx, const int32_t* n_active,
                                 const int32_t* step, int32_t k, int32_t* topk_pages,
-                                float* topk_scores_opt, cudaStream_t st, bool pooled = false);
+                                float* topk_scores_opt, cudaStream_t st, int selector = 0);
+// selector: 0 = one exact list per query head, 1 = pooled over the heads of a KV head, 2 = tensor-core scores (relaxed rule, bf16)
+constexpr int kSelectorExact = 0, kSelectorPooled = 1, kSelectorMma = 2;
 
 // Stage 2, first half: fp32 page scores of the active queries into the workspace's score rows.
 int32_t launch_page_scores(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
@@ -21,8 +23,9 @@ int32_t launch_page_scores(losa_ctx* c, const void* q, const losa_kv_t* kv, cons
 
 // bf16: (lower, upper) bounds of the page scores from the tensor cores, as float2 per (row, page), for
 // the selection that evaluates the exact score of the surviving candidates only.
+// With approx_only the tensor-core value itself is written as an fp32 score row (relaxed selector).
 int32_t launch_page_bounds(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
-                           const int32_t* n_active, const int32_t* step, cudaStream_t st);
+                           const int32_t* n_active, const int32_t* step, cudaStream_t st, bool approx_only = false);
 
 int32_t launch_page_union(losa_ctx* c, const int32_t* topk_pages, const int32_t* active_idx,
                           const int32_t* n_active, int32_t k, const int32_t* kv_len,

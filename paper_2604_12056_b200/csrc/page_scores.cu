@@ -557,7 +557,8 @@ __device__ __forceinline__ uint32_t mma_off(int r, int c, int row_bytes) {
   return static_cast<uint32_t>(r * row_bytes + ((c ^ ((r & 1) << 2)) << 4));
 }
 
-template <int D>
+// APPROX: write the tensor-core score A itself as an fp32 score row (no magnitudes, no radius).
+template <int D, bool APPROX>
 __global__ void __launch_bounds__(kPsThreads, 1) page_bounds_mma_kernel(PsParams p) {
   using C = MmaCfg<D>;
   using T = __nv_bfloat16;
@@ -703,6 +704,7 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_bounds_mma_kernel(PsParams
           mma_bf16_16816(c1, a_lo.x, a_hi.x, a_lo.y, a_hi.y, b_1.x, b_1.y);
           mma_bf16_16816(c0, a_lo.z, a_hi.z, a_lo.w, a_hi.w, b_0.z, b_0.w);
           mma_bf16_16816(c1, a_lo.z, a_hi.z, a_lo.w, a_hi.w, b_1.z, b_1.w);
+          if (APPROX) continue;                          // no error radius wanted
           constexpr uint32_t kAbs = 0x7fff7fffu;
           a_lo.x &= kAbs; a_lo.y &= kAbs; a_lo.z &= kAbs; a_lo.w &= kAbs;
           a_hi.x &= kAbs; a_hi.y &= kAbs; a_hi.z &= kAbs; a_hi.w &= kAbs;
@@ -719,13 +721,18 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_bounds_mma_kernel(PsParams
           const int r = 16 * mt + g + 8 * hr;
           if (r < nr) {
             const int row = r0 + r, a = row / p.G, gi = row % p.G;
-            float2* dst = bounds + ((static_cast<size_t>(w.s) * p.B + a) * p.Hq + w.kh * p.G + gi) * p.score_stride + w.p0 + warp * WP + 2 * t4;
+            const size_t at = ((static_cast<size_t>(w.s) * p.B + a) * p.Hq + w.kh * p.G + gi) * p.score_stride + w.p0 + warp * WP + 2 * t4;
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
               const int col = warp * WP + 2 * t4 + e;
-              const float d0 = kMmaErrCoef * m0[2 * hr + e], d1 = kMmaErrCoef * m1[2 * hr + e];
-              if (col < w.np) dst[e] = make_float2(c0[2 * hr + e] - d0, c0[2 * hr + e] + d0);
-              if (col + 8 < w.np) dst[e + 8] = make_float2(c1[2 * hr + e] - d1, c1[2 * hr + e] + d1);
+              if (APPROX) {
+                if (col < w.np) p.scores[at + e] = c0[2 * hr + e];
+                if (col + 8 < w.np) p.scores[at + e + 8] = c1[2 * hr + e];
+              } else {
+                const float d0 = kMmaErrCoef * m0[2 * hr + e], d1 = kMmaErrCoef * m1[2 * hr + e];
+                if (col < w.np) bounds[at + e] = make_float2(c0[2 * hr + e] - d0, c0[2 * hr + e] + d0);
+                if (col + 8 < w.np) bounds[at + e + 8] = make_float2(c1[2 * hr + e] - d1, c1[2 * hr + e] + d1);
+              }
             }
           }
         }
@@ -753,7 +760,7 @@ int32_t launch_stream(losa_ctx* c, const PsParams& pp, cudaStream_t st) {
   return after_launch(c);
 }
 
-template <int D>
+template <int D, bool APPROX>
 int32_t launch_bounds_t(losa_ctx* c, const PsParams& pp, cudaStream_t st) {
   using C = MmaCfg<D>;
   PsParams p = pp;
@@ -763,11 +770,12 @@ int32_t launch_bounds_t(losa_ctx* c, const PsParams& pp, cudaStream_t st) {
   if (ns < 2) return LOSA_ERR_UNSUPPORTED;
   p.n_stages = ns;
   const int smem = 128 + ns * C::STAGE_BYTES + C::QBUF_BYTES + tail;
-  if (!c->bounds_attr_set) {
-    LOSA_CUDA_TRY(c, cudaFuncSetAttribute(page_bounds_mma_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    c->bounds_attr_set = 1;
+  int32_t& attr_set = APPROX ? c->approx_attr_set : c->bounds_attr_set;
+  if (!attr_set) {
+    LOSA_CUDA_TRY(c, cudaFuncSetAttribute(page_bounds_mma_kernel<D, APPROX>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    attr_set = 1;
   }
-  launch_k(page_bounds_mma_kernel<D>, p.n_ctas, kPsThreads, smem, st, p);
+  launch_k(page_bounds_mma_kernel<D, APPROX>, p.n_ctas, kPsThreads, smem, st, p);
   return after_launch(c);
 }
 
@@ -803,9 +811,10 @@ PsParams make_params(losa_ctx* c, const void* q, const losa_kv_t* kv, const int3
 
 // bf16 only: (lower, upper) bound pairs of the page scores into the workspace's score rows (as float2)
 int32_t launch_page_bounds(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
-                           const int32_t* n_active, const int32_t* step, cudaStream_t st) {
+                           const int32_t* n_active, const int32_t* step, cudaStream_t st, bool approx_only) {
   const PsParams p = make_params(c, q, kv, active_idx, n_active, step);
-  return c->shape.head_dim == 128 ? launch_bounds_t<128>(c, p, st) : launch_bounds_t<64>(c, p, st);
+  if (approx_only) return c->shape.head_dim == 128 ? launch_bounds_t<128, true>(c, p, st) : launch_bounds_t<64, true>(c, p, st);
+  return c->shape.head_dim == 128 ? launch_bounds_t<128, false>(c, p, st) : launch_bounds_t<64, false>(c, p, st);
 }
 
 int32_t launch_page_scores(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_t* active_idx,

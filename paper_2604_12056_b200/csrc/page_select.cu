@@ -691,12 +691,13 @@ int32_t topk_max_sortable(const losa_ctx* c) {
 int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
                                 const int32_t* active_idx, const int32_t* n_active,
                                 const int32_t* step, int32_t k, int32_t* topk_pages,
-                                float* topk_scores_opt, cudaStream_t st, bool pooled) {
+                                float* topk_scores_opt, cudaStream_t st, int selector) {
   const losa_shape_t& sh = c->shape;
   if (sh.max_pages_per_seq == 0) return LOSA_OK;
+  const bool pooled = selector == kSelectorPooled;
   const int pool = pooled ? sh.n_q_heads / sh.n_kv_heads : 1;
   const bool bf = sh.dtype == LOSA_BF16;
-  if (bf && !pooled && k <= kSelCap) {
+  if (bf && selector == kSelectorExact && k <= kSelCap) {
     // bf16, one list per query head: bounds from the tensor cores, exact scores for the candidates only
     int32_t rc = launch_page_bounds(c, q, kv, active_idx, n_active, step, st);
     if (rc != LOSA_OK) return rc;
@@ -720,7 +721,8 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
     else launch_k(topk_refine_kernel<64>, queries, kSelThreads, 0, st, rp);
     return after_launch(c);
   }
-  int32_t rc = launch_page_scores(c, q, kv, active_idx, n_active, step, st);
+  int32_t rc = selector == kSelectorMma ? launch_page_bounds(c, q, kv, active_idx, n_active, step, st, true)
+                                        : launch_page_scores(c, q, kv, active_idx, n_active, step, st);
   if (rc != LOSA_OK) return rc;
 
   float* sc = reinterpret_cast<float*>(c->ws + c->lay.scores);

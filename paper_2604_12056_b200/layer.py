@@ -33,10 +33,12 @@ class LosaLayer:
     """
 
     def __init__(self, cfg, k_pages, v_pages, page_table, kv_len, mode="losa", device="cuda",
-                 share_pool_with: "LosaLayer | None" = None, tau: float = 0.0, pooled: bool = False):
+                 share_pool_with: "LosaLayer | None" = None, tau: float = 0.0, pooled: bool = False,
+                 mma_selector: bool = False):
         self.cfg, self.mode, self.device = cfg, mode, device
         self.tau = tau            # > 0: stage 1 keeps tokens until their Delta reach tau of the block's total
         self.pooled = pooled      # stage 2 keeps one page list per (token, KV head) instead of one per query head
+        self.mma_selector = mma_selector   # stage 2 takes its scores from the tensor cores (relaxed list rule, bf16)
         N, Bk, Hq, Hkv, d = cfg.batch, cfg.block_size, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim
         self.dtype = B.LOSA_BF16 if cfg.dtype == "bf16" else B.LOSA_F32
         td = B.torch_dtype(self.dtype)
@@ -91,7 +93,8 @@ class LosaLayer:
             B.losa_select_active_tau(c, xc, xp, row_width, self.tau, None, st, self.active_idx, self.n_active, self.delta)
         else:
             B.losa_select_active(c, xc, xp, row_width, m, st, self.active_idx, self.n_active, self.delta)
-        scores_topk = B.losa_page_scores_topk_pooled if self.pooled else B.losa_page_scores_topk
+        scores_topk = (B.losa_page_scores_topk_mma if self.mma_selector else
+                       B.losa_page_scores_topk_pooled if self.pooled else B.losa_page_scores_topk)
         scores_topk(c, q, self.kv, self.active_idx, self.n_active, st, cfg.topk, self.topk_pages,
                     self.topk_scores if want_scores else None)
         B.losa_page_union(c, self.topk_pages, self.active_idx, self.n_active, cfg.topk, self.kv_len, st,

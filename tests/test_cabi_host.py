@@ -82,7 +82,7 @@ def test_null_arguments_are_rejected_without_a_device(lib):
                       ("losa_sparse_prefix_attn", 9), ("losa_block_attn_merge", 8),
                       ("losa_update_prefix_cache", 8), ("losa_build_page_summaries", 3),
                       ("losa_denoise_step_host", 11), ("losa_denoise_step", 12),
-                      ("losa_page_scores_topk_pooled", 10)):
+                      ("losa_page_scores_topk_pooled", 10), ("losa_page_scores_topk_mma", 10)):
         args = [None] * nargs
         if fn in ("losa_select_active",):
             args[3] = C.c_int32(64)

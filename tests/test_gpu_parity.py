@@ -165,6 +165,64 @@ def test_long_lists_and_large_budgets(pages, topk, pooled):
     run_blocks(cfg, pooled=pooled)
 
 
+@pytest.mark.parametrize("kw", [
+    dict(kv_lens=(2048, 1500), steps=4),
+    dict(n_q_heads=4, n_kv_heads=2, head_dim=64, page_size=16, kv_lens=(16 * 1100 + 5, 700), block_size=8, steps=3, topk=8,
+         m_active=3),
+    dict(kv_lens=(150,), block_size=8, steps=3, topk=64, m_active=2),
+])
+def test_tensor_core_selector_under_the_relaxed_list_rule(kw):
+    """losa_page_scores_topk_mma: page scores as a GEMM on the tensor cores.  Its lists are checked
+    against the relaxed validity rule (fp64 scores, slack 2^-11 of the largest term magnitude sum);
+    everything downstream is compared as usual, the oracle taking the GPU's own lists: the union
+    exactly, the attention within the usual tolerances."""
+    from oracle import oracle as orc
+    from paper_2604_12056_b200.layer import LosaLayer, to_device
+    cfg = wl.config("c2", **kw)
+    w = wl.Workload(cfg)
+    g = LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len, mma_selector=True)
+    o = OracleLayer(w)
+    sh, k = o.sh, cfg.topk
+    same = total = 0
+    for t, inp in enumerate(w.block_steps()):
+        g.run_step(to_device(inp.q), to_device(inp.k_blk), to_device(inp.v_blk), to_device(inp.m_per_seq))
+        snap = g.snapshot()
+        assert g.ctx.poll_status() == 0
+        act, na, _ = orc.select_active(sh, inp.q, o.q_prev, inp.m_per_seq, o.step)
+        assert (snap["act"] == act).all() and (snap["na"] == na).all()
+        if t > 0:
+            assert orc.check_topk_relaxed(sh, inp.q, o.kv, act, na, k, snap["topk"], 2.0 ** -11, o.step) == 0
+            exact = np.full_like(snap["topk"], -9)
+            orc.page_scores_topk(sh, inp.q, o.kv, act, na, k, o.step, topk_pages=exact)
+            for s in range(cfg.batch):
+                for tok in act[s, :na[s]]:
+                    total += cfg.n_q_heads
+                    same += int((np.sort(exact[s, tok], -1) == np.sort(snap["topk"][s, tok], -1)).all(-1).sum())
+        up, uc = orc.page_union(sh, snap["topk"], act, na, k, o.kv_len, o.step)
+        assert (snap["up"] == up).all() and (snap["uc"] == uc).all()
+        orc.sparse_prefix_attn(sh, inp.q, o.kv, act, na, up, uc, o.o_p, o.lse_p)
+        out, lse = orc.block_attn_merge(sh, inp.q, inp.k_blk, inp.v_blk, o.o_p, o.lse_p)
+        what = f"tensor-core selector, step {t}"
+        assert_close(snap["o_p"], o.o_p, cfg.dtype, what + " o_p")
+        assert_lse_close(snap["lse_p"], o.lse_p, what + " lse_p")
+        assert_close(snap["out"], out, cfg.dtype, what + " out")
+        assert_lse_close(snap["lse"], lse, what + " lse")
+        orc.update_prefix_cache(sh, o.kv, o.q_prev, o.step, inp.q, inp.k_blk, inp.v_blk, False)
+    assert same >= 0.9 * total          # as sets, nearly all lists are the exact ones
+
+
+def test_tensor_core_selector_needs_bf16():
+    from paper_2604_12056_b200 import binding as B
+    from paper_2604_12056_b200.layer import LosaLayer, to_device
+    cfg = wl.config("c1", kv_lens=(64,), steps=2)
+    w = wl.Workload(cfg)
+    g = LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len, mma_selector=True)
+    inp = w.start_block()
+    with pytest.raises(B.LosaError) as e:
+        g.run_step(to_device(inp.q), to_device(inp.k_blk), to_device(inp.v_blk), to_device(inp.m_per_seq))
+    assert e.value.code == B.LOSA_ERR_UNSUPPORTED
+
+
 @pytest.mark.parametrize("name", ["p1", "p2"])
 def test_paper_shaped_workloads_reduced(name):
     # the shapes of the paper's latency study (batch 1, five active tokens, budget 16 pages), shorter prefix
