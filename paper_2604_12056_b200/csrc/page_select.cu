@@ -278,13 +278,17 @@ __device__ __forceinline__ float exact_score4(const float* __restrict__ qs, cons
     const uint32_t hw[4] = {hi_raw[w].x, hi_raw[w].y, hi_raw[w].z, hi_raw[w].w};
     float acc = 0.f;
 #pragma unroll
-    for (int j2 = 0; j2 < 4; ++j2) {
-      const float2 qp = *reinterpret_cast<const float2*>(qs + 8 * t + 2 * j2);
-      const float2 qn = *reinterpret_cast<const float2*>(qs + D + 8 * t + 2 * j2);
-      acc = __fmaf_rn(qp.x, __uint_as_float(hw[j2] << 16), acc);
-      acc = __fmaf_rn(qn.x, __uint_as_float(lw[j2] << 16), acc);
-      acc = __fmaf_rn(qp.y, __uint_as_float(hw[j2] & 0xffff0000u), acc);
-      acc = __fmaf_rn(qn.y, __uint_as_float(lw[j2] & 0xffff0000u), acc);
+    for (int j4 = 0; j4 < 2; ++j4) {
+      const float4 qp = *reinterpret_cast<const float4*>(qs + 8 * t + 4 * j4);
+      const float4 qn = *reinterpret_cast<const float4*>(qs + D + 8 * t + 4 * j4);
+      acc = __fmaf_rn(qp.x, __uint_as_float(hw[2 * j4] << 16), acc);
+      acc = __fmaf_rn(qn.x, __uint_as_float(lw[2 * j4] << 16), acc);
+      acc = __fmaf_rn(qp.y, __uint_as_float(hw[2 * j4] & 0xffff0000u), acc);
+      acc = __fmaf_rn(qn.y, __uint_as_float(lw[2 * j4] & 0xffff0000u), acc);
+      acc = __fmaf_rn(qp.z, __uint_as_float(hw[2 * j4 + 1] << 16), acc);
+      acc = __fmaf_rn(qn.z, __uint_as_float(lw[2 * j4 + 1] << 16), acc);
+      acc = __fmaf_rn(qp.w, __uint_as_float(hw[2 * j4 + 1] & 0xffff0000u), acc);
+      acc = __fmaf_rn(qn.w, __uint_as_float(lw[2 * j4 + 1] & 0xffff0000u), acc);
     }
     c[w] = acc;
   }
@@ -324,7 +328,7 @@ topk_refine_kernel(RefineParams p) {
   grid_dep_trigger();
   grid_dep_wait();
   __shared__ __align__(16) float qs[2 * D];
-  __shared__ unsigned long long ckey[kSelCap];
+  __shared__ __align__(16) unsigned long long ckey[kSelCap];
   __shared__ int cpage[kSelCap];
   __shared__ int hist[kSelBins];
   __shared__ uint32_t s_red[2][kSelThreads / 32];
@@ -483,23 +487,22 @@ topk_refine_kernel(RefineParams p) {
     }
     // ---- order the candidates (descending) and emit the first kk
     __syncthreads();
-    if (ncand <= 2 * kSelThreads) {
+    if (ncand <= kSelThreads) {
       // few candidates (the usual case): a candidate's position is the number of larger keys (all
-      // keys differ); every thread counts for up to two candidates, the keys are read as broadcasts
-      unsigned long long mine[2];
-      int rank[2] = {0, 0};
-#pragma unroll
-      for (int e = 0; e < 2; ++e) mine[e] = tid + e * kSelThreads < ncand ? ckey[tid + e * kSelThreads] : ~0ull;
-      for (int i = 0; i < ncand; ++i) {
-        const unsigned long long key = ckey[i];
-        rank[0] += key > mine[0] ? 1 : 0;
-        rank[1] += key > mine[1] ? 1 : 0;
-      }
-#pragma unroll
-      for (int e = 0; e < 2; ++e) {
-        if (tid + e * kSelThreads < ncand && rank[e] < kk) {
-          out_pages[rank[e]] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(mine[e]));
-          if (out_scores) out_scores[rank[e]] = unorder_bits(static_cast<uint32_t>(mine[e] >> 32));
+      // keys differ); one candidate per thread, the keys are read as broadcasts, four at a time
+      if ((tid & ~31) < ncand) {                       // whole warps without a candidate skip the count
+        const unsigned long long mine = tid < ncand ? ckey[tid] : ~0ull;
+        int rank = 0;
+        const int n4 = ncand & ~3;
+        for (int i = 0; i < n4; i += 4) {
+          const ulonglong2 k01 = *reinterpret_cast<const ulonglong2*>(&ckey[i]);
+          const ulonglong2 k23 = *reinterpret_cast<const ulonglong2*>(&ckey[i + 2]);
+          rank += (k01.x > mine ? 1 : 0) + (k01.y > mine ? 1 : 0) + (k23.x > mine ? 1 : 0) + (k23.y > mine ? 1 : 0);
+        }
+        for (int i = n4; i < ncand; ++i) rank += ckey[i] > mine ? 1 : 0;
+        if (tid < ncand && rank < kk) {
+          out_pages[rank] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(mine));
+          if (out_scores) out_scores[rank] = unorder_bits(static_cast<uint32_t>(mine >> 32));
         }
       }
       for (int j = kk + tid; j < p.k; j += kSelThreads) out_pages[j] = -1;

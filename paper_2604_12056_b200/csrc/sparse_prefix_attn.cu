@@ -56,6 +56,33 @@ __device__ __forceinline__ float* record_base(float* partials, int slot, int w, 
 
 __device__ __forceinline__ int clamp_active(int na, int B) { return na < 0 ? 0 : (na > B ? B : na); }
 
+// C (2 or 4) consecutive elements as one vector access; a lane of the row-wise kernels below owns
+// columns lane * C .. lane * C + C - 1 of a row of D = 32 C elements.
+template <int C> __device__ __forceinline__ void ldv(const float* p, float (&v)[C]) {
+  if constexpr (C == 4) { const float4 t = *reinterpret_cast<const float4*>(p); v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
+  else { const float2 t = *reinterpret_cast<const float2*>(p); v[0] = t.x; v[1] = t.y; }
+}
+template <int C> __device__ __forceinline__ void stv(float* p, const float (&v)[C]) {
+  if constexpr (C == 4) *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+  else *reinterpret_cast<float2*>(p) = make_float2(v[0], v[1]);
+}
+template <int C> struct RawRow;                      // C elements of the I/O type, moved as they are
+template <> struct RawRow<4> { uint2 bits; };
+template <> struct RawRow<2> { uint32_t bits; };
+template <int C> __device__ __forceinline__ RawRow<C> ld_raw(const __nv_bfloat16* p) { return *reinterpret_cast<const RawRow<C>*>(p); }
+template <int C> __device__ __forceinline__ void st_raw(__nv_bfloat16* p, const RawRow<C>& r) { *reinterpret_cast<RawRow<C>*>(p) = r; }
+template <int C> __device__ __forceinline__ void st_bf16(__nv_bfloat16* p, const float (&v)[C]) {
+  RawRow<C> r;
+  if constexpr (C == 4) {
+    __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+    r.bits = make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+  } else {
+    __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]);
+    r.bits = *reinterpret_cast<uint32_t*>(&a);
+  }
+  st_raw<C>(p, r);
+}
+
 // ===================================================================== fp32 / CUDA-core kernel
 template <typename T, int D, int GP>
 __global__ void __launch_bounds__(256, 1) attn_simt_kernel(AttnParams p) {
@@ -187,7 +214,7 @@ __global__ void __launch_bounds__(256, 1) attn_simt_kernel(AttnParams p) {
 // eight records issued together.  LOG2: partial maxima in base-2 units (tensor-core kernel) or
 // natural units (fp32 kernel).
 // Merge of the partial records of row r of segment sg by one warp: returns the un-normalised
-// output columns lane + 32 c in acc, the reference maximum M and the sum of weights Lsum.
+// output columns lane * C + c in acc, the reference maximum M and the sum of weights Lsum.
 template <int D, bool LOG2>
 __device__ __forceinline__ void merge_records(const AttnParams& p, int sg, int r, int start, int end, long long T_all,
                                               int lane, float (&acc)[D / 32], float& M, float& Lsum) {
@@ -234,9 +261,10 @@ __device__ __forceinline__ void merge_records(const AttnParams& p, int sg, int r
         const int i = i0 + u;
         w[u] = (i < n) ? __shfl_sync(0xffffffffu, wj, i & 31) : 0.f;
         const unsigned long long addr = __shfl_sync(0xffffffffu, reinterpret_cast<unsigned long long>(rec), i & 31);
-        const float* src = reinterpret_cast<const float*>(addr) + 2 * kTileRows + rr * D + lane;
+        const float* src = reinterpret_cast<const float*>(addr) + 2 * kTileRows + rr * D + lane * C;
 #pragma unroll
-        for (int c = 0; c < C; ++c) v[u][c] = (w[u] != 0.f) ? src[32 * c] : 0.f;
+        for (int c = 0; c < C; ++c) v[u][c] = 0.f;
+        if (w[u] != 0.f) ldv<C>(src, v[u]);
       }
 #pragma unroll
       for (int u = 0; u < U; ++u)
@@ -272,7 +300,8 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
     const bool empty = !(Lsum > 0.f);
     const float inv = empty ? 0.f : 1.f / Lsum;
 #pragma unroll
-    for (int c = 0; c < C; ++c) p.o_p[orow * D + lane + 32 * c] = acc[c] * inv;
+    for (int c = 0; c < C; ++c) acc[c] *= inv;
+    stv<C>(p.o_p + orow * D + lane * C, acc);
     if (lane == 0) p.lse_p[orow] = empty ? -INFINITY : (LOG2 ? (M + log2f(Lsum)) * kLn2 : M + logf(Lsum));
   }
 }
@@ -309,21 +338,16 @@ __global__ void __launch_bounds__(kFinishThreads) attn_finish_kernel(AttnParams 
   const int hq = static_cast<int>(row % p.Hq), tok = static_cast<int>((row / p.Hq) % p.B);
   const int s = static_cast<int>(row / (static_cast<size_t>(p.Hq) * p.B));
   const int kh = hq / p.G, gi = hq % p.G;
-  // operands that do not depend on the row being active: requested first
+  // operands that do not depend on the row being active: requested first (one vector access each)
   const T* q = static_cast<const T*>(f.q);
   float b[C];
-  T qv[C];
-#pragma unroll
-  for (int c = 0; c < C; ++c) {
-    b[c] = f.o_b[row * D + lane + 32 * c];
-    qv[c] = q[row * D + lane + 32 * c];
-  }
+  ldv<C>(f.o_b + row * D + lane * C, b);
+  const RawRow<C> qv = ld_raw<C>(q + row * D + lane * C);
   const float Lb = f.lse_b[row];
   // the cached prefix statistics as well: nine rows in ten are stable, and asking now saves them
   // a second round trip (an active row overwrites these below)
   float a[C], Lp;
-#pragma unroll
-  for (int c = 0; c < C; ++c) a[c] = p.o_p[row * D + lane + 32 * c];
+  ldv<C>(p.o_p + row * D + lane * C, a);
   Lp = p.lse_p[row];
   // the row's slot in the active list, if any (the list has at most B <= 64 entries)
   int slot = -1;
@@ -347,10 +371,8 @@ __global__ void __launch_bounds__(kFinishThreads) attn_finish_kernel(AttnParams 
     const float inv = empty ? 0.f : 1.f / Lsum;
     Lp = empty ? -INFINITY : (M + log2f(Lsum)) * kLn2;
 #pragma unroll
-    for (int c = 0; c < C; ++c) {
-      a[c] = acc[c] * inv;
-      p.o_p[row * D + lane + 32 * c] = a[c];
-    }
+    for (int c = 0; c < C; ++c) a[c] = acc[c] * inv;
+    stv<C>(p.o_p + row * D + lane * C, a);
     if (lane == 0) p.lse_p[row] = Lp;
   }
   const float Mx = fmaxf(Lp, Lb);
@@ -358,11 +380,11 @@ __global__ void __launch_bounds__(kFinishThreads) attn_finish_kernel(AttnParams 
   const float wp = expf(Lp - L), wb = expf(Lb - L);
   T* out = static_cast<T*>(f.out);
   T* q_prev = static_cast<T*>(f.q_prev);
+  float o[C];
 #pragma unroll
-  for (int c = 0; c < C; ++c) {
-    out[row * D + lane + 32 * c] = from_f32<T>((wp > 0.f ? wp * a[c] : 0.f) + wb * b[c]);
-    q_prev[row * D + lane + 32 * c] = qv[c];
-  }
+  for (int c = 0; c < C; ++c) o[c] = (wp > 0.f ? wp * a[c] : 0.f) + wb * b[c];
+  st_bf16<C>(out + row * D + lane * C, o);
+  st_raw<C>(q_prev + row * D + lane * C, qv);
   if (f.lse_out && lane == 0) f.lse_out[row] = L;
 }
 
