@@ -48,7 +48,10 @@ L2_FLUSH_BYTES = 256 << 20
 # dram__bytes_write.sum = 1,085.39 MB for its 65,984 slices (16,384 of the 16,449 bytes per slice are
 # the slice's K and V).  Traffic grows in proportion to the slices, so a launch's traffic is reported
 # as slices x this figure; LoSA launches add the partial records they write (3.7-4.8 MB of DRAM
-# writes in the three LoSA launches of that capture).  Pages of 32 tokens, head dim 128, bf16 only.
+# writes in the three LoSA launches of that capture).  Pages of 32 tokens, head dim 128, bf16; other
+# page sizes scale by the slice size (pages of 64 with two row groups per KV head, workload c4: 537.6 MB
+# read for 16,384 slices of 32,768 bytes on the dense step, 1.001 of the slices' bytes: the second row
+# group's pass over the pages is served by the L2, see profiles/attn_tc5_kernel_c4.txt).
 NCU_BYTES_PER_SLICE = {"losa": 1085.39e6 / 65984, "dense": 1085.39e6 / 65984}
 NCU_FIXED_BYTES = {"losa": 4.8e6, "dense": 0.0}
 
@@ -466,7 +469,7 @@ def run_ours(args, cfg0):
     for r in runs:
         r.layer.ctx.profile_stage4(False)
     slice_bytes = 2 * cfg.page_size * cfg.head_dim * 2
-    scalable = cfg.head_dim == 128 and cfg.dtype == "bf16" and cfg.block_size * cfg.group <= 128
+    scalable = cfg.head_dim == 128 and cfg.dtype == "bf16"
 
     def roof(sel):
         b = sum(x for x, k in zip(k_bytes, kinds) if k in sel)

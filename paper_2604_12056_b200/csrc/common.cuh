@@ -210,8 +210,10 @@ __device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity) {
 }
 
 // ---- balanced split of the flattened (segment, union position) list over the CTAs ------------
-// Segment seg = (s * H_kv + kh) * n_row_groups + rg holds union_count[s, kh] items when its row
-// group has rows, else none.  CTA b owns items [b*T/n, (b+1)*T/n).  The partial result a CTA
+// Segment seg = rg * (N * H_kv) + (s * H_kv + kh) holds union_count[s, kh] items when its row
+// group has rows, else none.  Row-group-major: with more than 128 query rows per KV head (two row
+// groups) the two passes over a (sequence, KV head)'s pages lie half the list apart, so the CTAs b
+// and b + n/2 stream the same pages at the same time and the second read is served by the L2.  CTA b owns items [b*T/n, (b+1)*T/n).  The partial result a CTA
 // produces for a segment goes to slot b + seg, which is unique (b and seg never both stay put
 // between consecutive pieces).
 __device__ __forceinline__ int rows_in_group(int n_active, int G, int rg) {
@@ -229,7 +231,7 @@ __device__ __forceinline__ void segment_prefix(int* pre, int n_seg, int n_rg, in
     const int seg = base + lane;
     int c = 0;
     if (seg < n_seg) {
-      const int rg = seg % n_rg, sk = seg / n_rg, s = sk / H_kv;
+      const int n_sk = n_seg / n_rg, rg = seg / n_sk, sk = seg % n_sk, s = sk / H_kv;
       int na = n_active[s];
       na = na < 0 ? 0 : (na > B ? B : na);
       c = rows_in_group(na, G, rg) > 0 ? max(union_count[sk], 0) : 0;

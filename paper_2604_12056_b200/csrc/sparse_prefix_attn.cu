@@ -110,7 +110,7 @@ __global__ void __launch_bounds__(256, 1) attn_simt_kernel(AttnParams p) {
   int item = lo;
   while (item < hi) {
     const int seg_end = min(hi, pre[sg + 1]);
-    const int rg = sg % p.n_rg, sk = sg / p.n_rg, s = sk / p.Hkv, kh = sk % p.Hkv;
+    const int n_sk = p.n_seg / p.n_rg, rg = sg / n_sk, sk = sg % n_sk, s = sk / p.Hkv, kh = sk % p.Hkv;
     const int rows = rows_in_group(clamp_active(p.n_active[s], p.B), p.G, rg);
     const int len = p.kv_len[s];
     __syncthreads();
@@ -280,7 +280,7 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
   __shared__ int pre[kMaxSegments + 1];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int sg = blockIdx.x;
-  const int rg = sg % p.n_rg, sk = sg / p.n_rg, s = sk / p.Hkv, kh = sk % p.Hkv;
+  const int n_sk = p.n_seg / p.n_rg, rg = sg / n_sk, sk = sg % n_sk, s = sk / p.Hkv, kh = sk % p.Hkv;
   const int rows = rows_in_group(clamp_active(p.n_active[s], p.B), p.G, rg);
   if (blockIdx.y * 8 >= rows) return;                 // whole CTA idle: skip the prefix as well
   if (PRE) {                                          // the main kernel left the prefix in the workspace
@@ -364,7 +364,7 @@ __global__ void __launch_bounds__(kFinishThreads) attn_finish_kernel(AttnParams 
   }
   if (slot >= 0) {
     const int rowk = slot * p.G + gi, rg = rowk / kRowsPerGroup, r = rowk % kRowsPerGroup;
-    const int sg = (s * p.Hkv + kh) * p.n_rg + rg;
+    const int sg = rg * (p.n_seg / p.n_rg) + s * p.Hkv + kh;
     float acc[C], M, Lsum;
     merge_records<D, true>(p, sg, r, p.seg_prefix[sg], p.seg_prefix[sg + 1], p.seg_prefix[p.n_seg], lane, acc, M, Lsum);
     const bool empty = !(Lsum > 0.f);

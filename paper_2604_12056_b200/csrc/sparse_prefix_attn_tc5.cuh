@@ -226,7 +226,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
           pstart = pre[cursor];
         }
         const int q = i - pstart, seg_end = min(hi, pre[cursor + 1]);
-        it.sk = cursor / p.n_rg;
+        it.sk = cursor % (p.n_seg / p.n_rg);
         it.grp = gbase + q / PG;
         it.j = q % PG;
         it.ng = min(PG, seg_end - (i - it.j));
@@ -372,7 +372,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     bool ok = true;
     while (item < hi && ok) {
       const int seg_end = min(hi, pre[sg + 1]);
-      const int rg = sg % p.n_rg, sk = sg / p.n_rg, s = sk / p.Hkv, kh = sk % p.Hkv;
+      const int n_sk = p.n_seg / p.n_rg, rg = sg / n_sk, sk = sg % n_sk, s = sk / p.Hkv, kh = sk % p.Hkv;
       const int rows = rows_in_group(n_active_of(s), p.G, rg);
       const bool warp_has_rows = quarter * 32 < rows;          // the same for both warps of a pair
       // ---- the piece's Q tile: this thread's half row, two bf16 per tensor-memory column
