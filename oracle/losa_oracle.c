@@ -235,6 +235,153 @@ void oracle_page_scores_one(const oracle_shape_t* sh, const void* q, const oracl
   }
 }
 
+/* ---------- FP8 K/V pages (extension: the paper names quantised attention as orthogonal to the
+ * method, Section 6, and quotes its cached state in FP16, Section 4.5 "Memory overhead") ----------
+ * Format: E4M3 (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; largest finite value 448;
+ * no infinities).  One scale per (physical page, KV head) and tensor, a power of two:
+ *   amax = largest |x| over the page's valid tokens and d dimensions,
+ *   scale = 2^e, e = the smallest integer with amax <= 448 * 2^e, clamped to [-6, 7]  (amax = 0: e = -6),
+ *   code  = round-to-nearest-even of x / scale onto the E4M3 grid, saturated at +-448,
+ *   dequantised value = scale * value(code)   (exact in bf16 and fp16: four significant bits).
+ * Slots of a page past the prefix's end get code 0.  Appending a block re-quantises every touched
+ * page from the dequantised old values and the new rows together (the scale may have to grow). */
+double oracle_fp8_decode(uint8_t code) {
+  const int sign = code >> 7, e = (code >> 3) & 15, m = code & 7;
+  double v;
+  if (e == 15 && m == 7) return NAN;
+  if (e == 0) v = ldexp((double)m, -9);                  /* subnormal: m * 2^-3 * 2^-6 */
+  else v = ldexp(1.0 + m / 8.0, e - 7);
+  return sign ? -v : v;
+}
+uint8_t oracle_fp8_encode(double y) {
+  const uint8_t sign = (y < 0.0 || (y == 0.0 && signbit(y))) ? 0x80 : 0;
+  double a = fabs(y);
+  if (!(a == a)) return 0x7f;                             /* NaN in, NaN out (never produced from finite inputs) */
+  if (a >= 448.0) return sign | 0x7e;                     /* saturate: 0x7e = 448 */
+  double r;
+  int ex;
+  if (a < ldexp(1.0, -6)) {                               /* subnormal range, step 2^-9 */
+    r = nearbyint(ldexp(a, 9));                           /* ties to even (default rounding mode) */
+    if (r >= 8.0) return sign | 0x08;                     /* rounded up to the first normal, 2^-6 */
+    return sign | (uint8_t)r;
+  }
+  (void)frexp(a, &ex);                                    /* a = f * 2^ex, f in [0.5, 1)  =>  2^(ex-1) <= a < 2^ex */
+  int e = ex - 1;                                         /* binade of a */
+  r = nearbyint(ldexp(a, 3 - e));                         /* a / 2^(e-3): in [8, 16], ties to even */
+  if (r >= 16.0) { r = 8.0; e += 1; }
+  if (e > 8 || (e == 8 && r > 14.0)) return sign | 0x7e;
+  return sign | (uint8_t)(((e + 7) << 3) | ((int)r - 8));
+}
+static int fp8_scale_exp(double amax) {
+  if (!(amax > 0.0)) return -6;
+  int e = -6;
+  while (e < 7 && amax > ldexp(448.0, e)) ++e;
+  return e;
+}
+/* quantises n valid token rows (read through get(ctx, t, j)) of one (page, KV head) into codes[g][d] */
+typedef double (*fp8_get_fn)(const void* ctx, int t, int j);
+static float fp8_quantize_rows(fp8_get_fn get, const void* ctx, int n, int g, int d, uint8_t* codes) {
+  double amax = 0.0;
+  for (int t = 0; t < n; ++t)
+    for (int j = 0; j < d; ++j) { const double a = fabs(get(ctx, t, j)); if (a > amax) amax = a; }
+  const int e = fp8_scale_exp(amax);
+  for (int t = 0; t < g; ++t)
+    for (int j = 0; j < d; ++j) codes[(int64_t)t * d + j] = t < n ? oracle_fp8_encode(ldexp(get(ctx, t, j), -e)) : 0;
+  return (float)ldexp(1.0, e);
+}
+typedef struct { const void* base; int dtype; int64_t off, stride_tok; } fp8_src_t;
+static double fp8_get_pool(const void* c, int t, int j) {
+  const fp8_src_t* s = (const fp8_src_t*)c;
+  return ld(s->base, s->dtype, s->off + (int64_t)t * s->stride_tok + j);
+}
+void oracle_fp8_quantize_pages(const oracle_shape_t* sh, const oracle_kv_t* src, uint8_t* k_codes, uint8_t* v_codes,
+                               float* k_scale, float* v_scale) {
+  const int Hkv = sh->n_kv_heads, g = sh->page_size, d = sh->head_dim;
+  for (int s = 0; s < sh->batch; ++s) {
+    const int L = src->kv_len[s], P = pages_of(L, g);
+    for (int p = 0; p < P; ++p) {
+      const int32_t phys = src->page_table[(int64_t)s * sh->max_pages_per_seq + p];
+      const int n = (L - p * g) < g ? (L - p * g) : g;
+      for (int kh = 0; kh < Hkv; ++kh) {
+        const int64_t co = ((int64_t)phys * Hkv + kh) * g * d;
+        fp8_src_t ks = {src->k_pages, sh->dtype, kv_off(src, phys, kh, 0), src->stride_tok};
+        fp8_src_t vs = {src->v_pages, sh->dtype, kv_off(src, phys, kh, 0), src->stride_tok};
+        k_scale[(int64_t)phys * Hkv + kh] = fp8_quantize_rows(fp8_get_pool, &ks, n, g, d, k_codes + co);
+        v_scale[(int64_t)phys * Hkv + kh] = fp8_quantize_rows(fp8_get_pool, &vs, n, g, d, v_codes + co);
+      }
+    }
+  }
+}
+/* writes scale * value(code) of the valid tokens of every logical page into dst's pools (element dtype) */
+static void st_elem(void* p, int dtype, int64_t i, double v) {
+  if (dtype == 1) {                                       /* bf16: the values written here are exact in bf16 */
+    float f = (float)v;
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    ((uint16_t*)p)[i] = (uint16_t)(u >> 16);
+  } else {
+    ((float*)p)[i] = (float)v;
+  }
+}
+void oracle_fp8_dequantize_pages(const oracle_shape_t* sh, const uint8_t* k_codes, const uint8_t* v_codes,
+                                 const float* k_scale, const float* v_scale, oracle_kv_t* dst) {
+  const int Hkv = sh->n_kv_heads, g = sh->page_size, d = sh->head_dim;
+  for (int s = 0; s < sh->batch; ++s) {
+    const int L = dst->kv_len[s], P = pages_of(L, g);
+    for (int p = 0; p < P; ++p) {
+      const int32_t phys = dst->page_table[(int64_t)s * sh->max_pages_per_seq + p];
+      const int n = (L - p * g) < g ? (L - p * g) : g;
+      for (int kh = 0; kh < Hkv; ++kh) {
+        const int64_t co = ((int64_t)phys * Hkv + kh) * g * d;
+        const double ksc = k_scale[(int64_t)phys * Hkv + kh], vsc = v_scale[(int64_t)phys * Hkv + kh];
+        for (int t = 0; t < n; ++t)
+          for (int j = 0; j < d; ++j) {
+            st_elem(dst->k_pages, sh->dtype, kv_off(dst, phys, kh, t) + j, ksc * oracle_fp8_decode(k_codes[co + (int64_t)t * d + j]));
+            st_elem(dst->v_pages, sh->dtype, kv_off(dst, phys, kh, t) + j, vsc * oracle_fp8_decode(v_codes[co + (int64_t)t * d + j]));
+          }
+      }
+    }
+  }
+}
+typedef struct { const uint8_t* codes; double scale; int n_old; const void* blk; int dtype; int64_t blk_off; int blk_stride; int d; } fp8_mix_t;
+static double fp8_get_mix(const void* c, int t, int j) {
+  const fp8_mix_t* m = (const fp8_mix_t*)c;
+  if (t < m->n_old) return m->scale * oracle_fp8_decode(m->codes[(int64_t)t * m->d + j]);
+  return ld(m->blk, m->dtype, m->blk_off + (int64_t)(t - m->n_old) * m->blk_stride + j);
+}
+/* block finalisation on an FP8 cache: appends the block's rows at prefix positions L_s .. L_s+B-1 and
+ * re-quantises every touched page; kv_len[s] += B.  (Summaries and the step counter are the caller's.) */
+void oracle_fp8_append_block(const oracle_shape_t* sh, const int32_t* page_table, int32_t* kv_len,
+                             uint8_t* k_codes, uint8_t* v_codes, float* k_scale, float* v_scale,
+                             const void* k_blk, const void* v_blk) {
+  const int B = sh->block_size, Hkv = sh->n_kv_heads, g = sh->page_size, d = sh->head_dim;
+  uint8_t* tmp = (uint8_t*)malloc((size_t)g * d);
+  for (int s = 0; s < sh->batch; ++s) {
+    const int L0 = kv_len[s];
+    for (int p = L0 / g; p <= (L0 + B - 1) / g; ++p) {
+      const int32_t phys = page_table[(int64_t)s * sh->max_pages_per_seq + p];
+      const int n_old = L0 > p * g ? L0 - p * g : 0;                 /* tokens the page already holds */
+      const int last = (L0 + B) < (p + 1) * g ? (L0 + B) : (p + 1) * g;
+      const int n_new = last - (p * g + n_old);
+      const int first_blk = p * g + n_old - L0;                      /* block row of the first new token */
+      for (int kh = 0; kh < Hkv; ++kh) {
+        const int64_t co = ((int64_t)phys * Hkv + kh) * g * d, so = (int64_t)phys * Hkv + kh;
+        for (int which = 0; which < 2; ++which) {
+          uint8_t* codes = (which ? v_codes : k_codes) + co;
+          float* scale = (which ? v_scale : k_scale) + so;
+          fp8_mix_t mx = {codes, n_old ? (double)*scale : 1.0, n_old, which ? v_blk : k_blk, sh->dtype,
+                          (((int64_t)s * B + first_blk) * Hkv + kh) * d, Hkv * d, d};
+          const float sc = fp8_quantize_rows(fp8_get_mix, &mx, n_old + n_new, g, d, tmp);
+          memcpy(codes, tmp, (size_t)g * d);
+          *scale = sc;
+        }
+      }
+    }
+    kv_len[s] = L0 + B;
+  }
+  free(tmp);
+}
+
 /* ---------- Section 2.3: relaxed validity of a page list (selector variants with their own arithmetic) ----------
  * The paper fixes no arithmetic for the page bound, and calls the method independent of the
  * selector.  A selector that evaluates U(p) = sum_j max(q_j kmin_j, q_j kmax_j) in another order

@@ -71,6 +71,18 @@ void oracle_page_scores_topk_pooled(const oracle_shape_t* sh, const void* q, con
                                     float* topk_scores);
 
 /* Section 4.2 / 4.4: union per (sequence, KV head). */
+/* FP8 (E4M3) K/V pages with one power-of-two scale per (physical page, KV head) and tensor; see the
+ * definition in losa_oracle.c.  codes: [n_phys, H_kv, g, d] bytes; scales: [n_phys, H_kv] fp32. */
+double oracle_fp8_decode(uint8_t code);
+uint8_t oracle_fp8_encode(double y);
+void oracle_fp8_quantize_pages(const oracle_shape_t* sh, const oracle_kv_t* src, uint8_t* k_codes, uint8_t* v_codes,
+                               float* k_scale, float* v_scale);
+void oracle_fp8_dequantize_pages(const oracle_shape_t* sh, const uint8_t* k_codes, const uint8_t* v_codes,
+                                 const float* k_scale, const float* v_scale, oracle_kv_t* dst);
+void oracle_fp8_append_block(const oracle_shape_t* sh, const int32_t* page_table, int32_t* kv_len,
+                             uint8_t* k_codes, uint8_t* v_codes, float* k_scale, float* v_scale,
+                             const void* k_blk, const void* v_blk);
+
 /* Relaxed validity of page lists produced with another arithmetic than the fixed fp32 order: number of
  * (active token, head) lists that are not "min(k, P) distinct in-range pages, each with fp64 bound >=
  * the k-th largest fp64 bound - eps * (largest sum of term magnitudes)", then -1 padding. */

@@ -210,6 +210,46 @@ def check_topk_relaxed(sh: Shape, q, kv: KV, active_idx, n_active, k: int, topk_
                   _p(_chk(topk_pages, np.int32, "topk")), C.c_double(eps)))
 
 
+# ---- FP8 (E4M3) K/V pages, one power-of-two scale per (physical page, KV head) and tensor
+def fp8_decode(codes) -> np.ndarray:
+    fn = lib().oracle_fp8_decode
+    fn.restype, fn.argtypes = C.c_double, [C.c_uint8]
+    return np.array([fn(int(c)) for c in np.asarray(codes, np.uint8).ravel()], np.float64).reshape(np.shape(codes))
+
+
+def fp8_encode(values) -> np.ndarray:
+    fn = lib().oracle_fp8_encode
+    fn.restype, fn.argtypes = C.c_uint8, [C.c_double]
+    return np.array([fn(float(v)) for v in np.asarray(values, np.float64).ravel()], np.uint8).reshape(np.shape(values))
+
+
+def fp8_quantize_pages(sh: Shape, kv: KV):
+    """Returns (k_codes, v_codes [n_phys,H_kv,g,d] uint8, k_scale, v_scale [n_phys,H_kv] float32) of every logical page."""
+    n_phys = kv.k_pages.shape[0]
+    shape = (n_phys, sh.n_kv_heads, sh.page_size, sh.head_dim)
+    kc, vc = np.zeros(shape, np.uint8), np.zeros(shape, np.uint8)
+    ks, vs = np.ones((n_phys, sh.n_kv_heads), np.float32), np.ones((n_phys, sh.n_kv_heads), np.float32)
+    s, k = sh.c(), kv.c()
+    lib().oracle_fp8_quantize_pages(C.byref(s), C.byref(k), _p(kc), _p(vc), _p(ks), _p(vs))
+    return kc, vc, ks, vs
+
+
+def fp8_dequantize_pages(sh: Shape, k_codes, v_codes, k_scale, v_scale, kv_dst: KV):
+    """scale * value(code) of the valid tokens of every logical page into kv_dst's pools (exact in bf16 / fp32)."""
+    s, k = sh.c(), kv_dst.c()
+    lib().oracle_fp8_dequantize_pages(C.byref(s), _p(_chk(k_codes, np.uint8, "k_codes")), _p(_chk(v_codes, np.uint8, "v_codes")),
+                                      _p(_chk(k_scale, np.float32, "k_scale")), _p(_chk(v_scale, np.float32, "v_scale")), C.byref(k))
+
+
+def fp8_append_block(sh: Shape, page_table, kv_len, k_codes, v_codes, k_scale, v_scale, k_blk, v_blk):
+    """Appends the block to the FP8 cache (re-quantising every touched page) and adds B to kv_len, in place."""
+    s = sh.c()
+    lib().oracle_fp8_append_block(C.byref(s), _p(_chk(page_table, np.int32, "page_table")), _p(_chk(kv_len, np.int32, "kv_len")),
+                                  _p(_chk(k_codes, np.uint8, "k_codes")), _p(_chk(v_codes, np.uint8, "v_codes")),
+                                  _p(_chk(k_scale, np.float32, "k_scale")), _p(_chk(v_scale, np.float32, "v_scale")),
+                                  _p(_chk(k_blk, sh.elem, "k_blk")), _p(_chk(v_blk, sh.elem, "v_blk")))
+
+
 def page_union(sh: Shape, topk_pages, active_idx, n_active, k: int, kv_len, step=None):
     """Returns (union_pages [N,H_kv,P_max] int32, union_count [N,H_kv] int32)."""
     N, Hkv, P = sh.batch, sh.n_kv_heads, sh.max_pages_per_seq
