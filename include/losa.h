@@ -69,6 +69,9 @@ extern "C" {
 #define LOSA_F32   0
 #define LOSA_BF16  1
 
+#define LOSA_KV_NATIVE    0
+#define LOSA_KV_FP8_E4M3  1
+
 #define LOSA_MAX_BLOCK 64
 
 /* Problem shape of one attention layer (Section 2.1): B block tokens attend to a paged prefix. */
@@ -97,6 +100,11 @@ typedef struct {
   const int32_t* page_table;   /* [N, P_max] physical page of each logical page                  */
   int32_t*       kv_len;       /* [N] prefix tokens L_s of each sequence                         */
   int32_t        n_phys_pages; /* pages in the pool                                              */
+  int32_t        kv_format;    /* LOSA_KV_NATIVE: k_pages / v_pages hold `dtype` elements;       */
+                               /* LOSA_KV_FP8_E4M3: one byte per element (strides in bytes) and  */
+                               /* the scales below; summaries stay `dtype` (bf16 contexts only)  */
+  float*         k_scale;      /* [n_phys_pages, H_kv] power-of-two scale of each key page       */
+  float*         v_scale;      /* [n_phys_pages, H_kv] likewise for the values; NULL when native */
 } losa_kv_t;
 
 /* Per-block LoSA cache (Section 4.3 / "Memory overhead" in Section 4.5): B(d+1) scalars per head
@@ -296,6 +304,25 @@ int32_t losa_block_attn_merge(losa_ctx* ctx, const void* q, const void* k_blk, c
 int32_t losa_update_prefix_cache(losa_ctx* ctx, losa_kv_t* kv, losa_state_t* state, const void* q,
                                  const void* k_blk, const void* v_blk, int32_t finalize_block,
                                  void* stream);
+
+/* FP8 K/V pages (bf16 contexts) — an extension of the cache format; the paper names quantised
+ * attention as orthogonal to the method (Section 6) and quotes the cached state in FP16
+ * (Section 4.5, "Memory overhead").  A cache with kv_format = LOSA_KV_FP8_E4M3 stores every K / V
+ * element as one E4M3 byte (largest finite value 448) and one scale per (physical page, KV head) and
+ * tensor:  amax = largest |x| over the page's valid tokens;  scale = 2^e with e the smallest integer
+ * such that amax <= 448 * 2^e, clamped to [-6, 7];  code = round-to-nearest-even of x / scale,
+ * saturated at +-448;  the value every stage works with is scale * value(code) (exact in bf16 and
+ * fp16).  Slots of a page past the prefix's end hold code 0.  Stage 4 streams half the bytes; its
+ * arithmetic is that of the bf16 path on the dequantised values (fp16 operands, fp32 accumulation),
+ * so its results are held to the bf16 tolerances against the definition evaluated on the
+ * dequantised cache.  Stages 2, 3, 5 are unchanged (the summaries are those of the dequantised
+ * keys); block finalisation re-quantises every touched page from its dequantised old rows and the
+ * new rows together.  Inputs must satisfy |x| <= 448 * 2^7 (larger magnitudes saturate).
+ *
+ * losa_quantize_kv_pages: src is a native bf16 cache, dst an FP8 cache with the same page_table,
+ *   kv_len and n_phys_pages; writes dst's codes and scales for every logical page p < P_s of every
+ *   sequence and dst's kmin / kmax. */
+int32_t losa_quantize_kv_pages(losa_ctx* ctx, const losa_kv_t* src, losa_kv_t* dst, void* stream);
 
 /* Set-up helper — per-page min/max keys of Section 2.3 for the whole prefix: kmin/kmax of every
  * logical page p < P_s over its valid tokens. */

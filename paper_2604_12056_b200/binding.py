@@ -30,7 +30,7 @@ EXPORTS = [
     "losa_update_prefix_cache", "losa_build_page_summaries", "losa_denoise_step_host",
     "losa_profile_stage4", "losa_stage4_last_ms", "losa_select_active_static",
     "losa_denoise_step", "losa_select_active_tau", "losa_page_scores_topk_pooled",
-    "losa_set_pooled_selection", "losa_set_wait_limit", "losa_page_scores_topk_mma",
+    "losa_set_pooled_selection", "losa_set_wait_limit", "losa_page_scores_topk_mma", "losa_quantize_kv_pages",
 ]
 
 
@@ -51,7 +51,7 @@ class KvT(C.Structure):
     _fields_ = [("k_pages", C.c_void_p), ("v_pages", C.c_void_p), ("stride_page", C.c_int64),
                 ("stride_head", C.c_int64), ("stride_tok", C.c_int64), ("kmin", C.c_void_p),
                 ("kmax", C.c_void_p), ("page_table", C.c_void_p), ("kv_len", C.c_void_p),
-                ("n_phys_pages", C.c_int32)]
+                ("n_phys_pages", C.c_int32), ("kv_format", C.c_int32), ("k_scale", C.c_void_p), ("v_scale", C.c_void_p)]
 
 
 class StateT(C.Structure):
@@ -101,14 +101,21 @@ def torch_dtype(dtype: int):
     return torch.bfloat16 if dtype == LOSA_BF16 else torch.float32
 
 
-def make_kv(k_pages, v_pages, kmin, kmax, page_table, kv_len) -> KvT:
-    """losa_kv_t over a [n_phys, H_kv, g, d] pool (any strides with contiguous token rows)."""
+LOSA_KV_NATIVE, LOSA_KV_FP8_E4M3 = 0, 1
+
+
+def make_kv(k_pages, v_pages, kmin, kmax, page_table, kv_len, k_scale=None, v_scale=None) -> KvT:
+    """losa_kv_t over a [n_phys, H_kv, g, d] pool (any strides with contiguous token rows).  With
+    k_scale / v_scale ([n_phys, H_kv] fp32) the pools are uint8 tensors of E4M3 codes."""
     sp, sh_, st, sd = k_pages.stride()
     assert sd == 1 and v_pages.stride() == k_pages.stride()
+    fp8 = k_scale is not None
+    assert (k_pages.dtype == torch.uint8) == fp8
     kv = KvT(k_pages.data_ptr(), v_pages.data_ptr(), sp, sh_, st,
              0 if kmin is None else kmin.data_ptr(), 0 if kmax is None else kmax.data_ptr(),
-             page_table.data_ptr(), kv_len.data_ptr(), k_pages.shape[0])
-    kv._keep = (k_pages, v_pages, kmin, kmax, page_table, kv_len)
+             page_table.data_ptr(), kv_len.data_ptr(), k_pages.shape[0],
+             LOSA_KV_FP8_E4M3 if fp8 else LOSA_KV_NATIVE, k_scale.data_ptr() if fp8 else 0, v_scale.data_ptr() if fp8 else 0)
+    kv._keep = (k_pages, v_pages, kmin, kmax, page_table, kv_len, k_scale, v_scale)
     return kv
 
 
@@ -215,7 +222,7 @@ def losa_page_scores_topk_pooled(ctx, q, kv, active_idx, n_active, step, k, topk
 
 def losa_page_scores_topk_mma(ctx, q, kv, active_idx, n_active, step, k, topk_pages, topk_scores_opt=None):
     """Stage 2 with tensor-core scores (bf16): lists valid under the relaxed rule, not entry by entry."""
-    ctx._check("losa_page_scores_topk_mma", lib().losa_page_scores_topk_mma(
+    ctx._check("losa_page_scores_topk_mma", "losa_quantize_kv_pages", lib().losa_page_scores_topk_mma(
         ctx._h, _ptr(q), C.byref(kv), _ptr(active_idx), _ptr(n_active), _ptr(step), C.c_int32(k),
         _ptr(topk_pages), _ptr(topk_scores_opt), _stream()))
 
@@ -241,6 +248,11 @@ def losa_update_prefix_cache(ctx, kv, state, q, k_blk, v_blk, finalize_block):
     ctx._check("losa_update_prefix_cache", lib().losa_update_prefix_cache(
         ctx._h, C.byref(kv), C.byref(state), _ptr(q), _ptr(k_blk), _ptr(v_blk),
         C.c_int32(1 if finalize_block else 0), _stream()))
+
+
+def losa_quantize_kv_pages(ctx, src_kv, dst_kv):
+    """bf16 cache -> FP8 cache (codes, per-page scales, summaries of the dequantised keys)."""
+    ctx._check("losa_quantize_kv_pages", lib().losa_quantize_kv_pages(ctx._h, C.byref(src_kv), C.byref(dst_kv), _stream()))
 
 
 def losa_build_page_summaries(ctx, kv):

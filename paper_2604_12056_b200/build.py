@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(CSRC, "build")
 SO = os.path.join(HERE, "liblosa.so")
-SOURCES = ["api.cu", "select_active.cu", "page_select.cu", "page_scores.cu", "sparse_prefix_attn.cu", "block_cache.cu"]
+SOURCES = ["api.cu", "select_active.cu", "page_select.cu", "page_scores.cu", "sparse_prefix_attn.cu", "block_cache.cu", "fp8_pages.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "--expt-relaxed-constexpr"]
 

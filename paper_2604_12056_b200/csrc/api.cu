@@ -67,7 +67,11 @@ int32_t check_kv(const losa_ctx* c, const losa_kv_t* kv, bool need_summaries) {
   if (need_summaries && (!kv->kmin || !kv->kmax)) return LOSA_ERR_INVALID_ARG;
   if (kv->n_phys_pages < 1) return LOSA_ERR_INVALID_ARG;
   const losa_shape_t& sh = c->shape;
-  const int64_t es = sh.dtype == LOSA_BF16 ? 2 : 4;
+  if (kv->kv_format != LOSA_KV_NATIVE && kv->kv_format != LOSA_KV_FP8_E4M3) return LOSA_ERR_INVALID_ARG;
+  const bool fp8 = kv->kv_format == LOSA_KV_FP8_E4M3;
+  if (fp8 && (!kv->k_scale || !kv->v_scale)) return LOSA_ERR_INVALID_ARG;
+  if (fp8 && sh.dtype != LOSA_BF16) return LOSA_ERR_UNSUPPORTED;
+  const int64_t es = fp8 ? 1 : (sh.dtype == LOSA_BF16 ? 2 : 4);
   if (kv->stride_tok < sh.head_dim || kv->stride_head < 1 || kv->stride_page < 1) return LOSA_ERR_INVALID_ARG;
   if ((kv->stride_tok * es) % 16 || (kv->stride_head * es) % 16 || (kv->stride_page * es) % 16) return LOSA_ERR_UNSUPPORTED;
   if (!aligned16(kv->k_pages) || !aligned16(kv->v_pages) || (kv->kmin && !aligned16(kv->kmin)) ||
@@ -259,6 +263,16 @@ int32_t losa_update_prefix_cache(losa_ctx* ctx, losa_kv_t* kv, losa_state_t* sta
     if (rc != LOSA_OK) return rc;
   }
   return launch_update_prefix_cache(ctx, kv, state, q, k_blk, v_blk, finalize_block, as_stream(stream));
+}
+
+int32_t losa_quantize_kv_pages(losa_ctx* ctx, const losa_kv_t* src, losa_kv_t* dst, void* stream) {
+  if (!ctx || !src || !dst) return LOSA_ERR_INVALID_ARG;
+  int32_t rc = check_kv(ctx, src, false);
+  if (rc == LOSA_OK) rc = check_kv(ctx, dst, true);
+  if (rc != LOSA_OK) return rc;
+  if (src->kv_format != LOSA_KV_NATIVE || dst->kv_format != LOSA_KV_FP8_E4M3 || src->n_phys_pages != dst->n_phys_pages)
+    return LOSA_ERR_INVALID_ARG;
+  return launch_fp8_quantize(ctx, src, dst, as_stream(stream));
 }
 
 int32_t losa_build_page_summaries(losa_ctx* ctx, losa_kv_t* kv, void* stream) {

@@ -491,6 +491,14 @@ int32_t launch_update_t(losa_ctx* c, losa_kv_t* kv, losa_state_t* state, const v
         static_cast<const uint4*>(q), static_cast<uint4*>(state->q_prev), n_vec, state->step, sh.batch);
     return after_launch(c);
   }
+  if (kv->kv_format == LOSA_KV_FP8_E4M3) {
+    // FP8 pages: the touched pages are re-quantised from their dequantised old rows and the new rows
+    int32_t rc = launch_fp8_append(c, kv, k_blk, v_blk, st);
+    if (rc != LOSA_OK) return rc;
+    launch_k(finalize_counters_kernel, 1, std::max(32, sh.batch), 0, st, kv->kv_len, state->step, sh.batch, sh.block_size,
+             sh.page_size, sh.max_pages_per_seq);
+    return after_launch(c);
+  }
   dim3 grid((sh.block_size + sh.page_size - 1) / sh.page_size + 1, sh.n_kv_heads, sh.batch);
   launch_k(append_block_kernel<T>, grid, sh.head_dim, 0, st, 
       static_cast<T*>(kv->k_pages), static_cast<T*>(kv->v_pages), static_cast<T*>(kv->kmin),
@@ -577,6 +585,7 @@ int32_t launch_update_prefix_cache(losa_ctx* c, losa_kv_t* kv, losa_state_t* sta
 }
 
 int32_t launch_build_page_summaries(losa_ctx* c, losa_kv_t* kv, cudaStream_t st) {
+  if (kv->kv_format == LOSA_KV_FP8_E4M3) return launch_fp8_summaries(c, kv, st);
   return c->shape.dtype == LOSA_BF16 ? launch_summaries_t<__nv_bfloat16>(c, kv, st)
                                      : launch_summaries_t<float>(c, kv, st);
 }

@@ -53,6 +53,7 @@ struct losa_ctx {
   const void* tmap_key_v;
   int64_t tmap_strides[3];
   int32_t tmap_n_phys;
+  int32_t tmap_format;
   void* encode_fn;  // cuTensorMapEncodeTiled, resolved through the runtime
   // second stream and fork/join events of the whole-step path (created on first use)
   cudaStream_t side_stream;

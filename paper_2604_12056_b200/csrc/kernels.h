@@ -59,6 +59,13 @@ int32_t launch_update_prefix_cache(losa_ctx* c, losa_kv_t* kv, losa_state_t* sta
 
 int32_t launch_build_page_summaries(losa_ctx* c, losa_kv_t* kv, cudaStream_t st);
 
+// FP8 (E4M3) K/V pages, one power-of-two scale per (physical page, KV head) and tensor (bf16 contexts):
+// quantise a bf16 pool page by page (codes, scales, summaries of the dequantised keys); summaries of
+// an FP8 pool; block append with re-quantisation of the touched pages.
+int32_t launch_fp8_quantize(losa_ctx* c, const losa_kv_t* src, losa_kv_t* dst, cudaStream_t st);
+int32_t launch_fp8_summaries(losa_ctx* c, losa_kv_t* kv, cudaStream_t st);
+int32_t launch_fp8_append(losa_ctx* c, losa_kv_t* kv, const void* k_blk, const void* v_blk, cudaStream_t st);
+
 // Largest k and page count the top-k kernel's shared memory allows for this context.
 int32_t topk_max_sortable(const losa_ctx* c);
 

@@ -17,6 +17,8 @@
 // Every wait on an mbarrier is bounded; when a bound runs out the CTA records LOSA_ERR_TIMEOUT,
 // raises its abort flag (which ends every other wait of the CTA) and leaves through the common exit.
 #include <cuda.h>
+#include <cuda_fp16.h>
+#include <cuda_fp8.h>
 
 #include <algorithm>
 
@@ -41,6 +43,8 @@ struct AttnParams {
   float* o_p;
   float* lse_p;
   int32_t* status;
+  const float* k_scale;   // FP8 pages: [n_phys, H_kv] power-of-two scales (else null)
+  const float* v_scale;
   int N, B, Hq, Hkv, G, Pmax, n_phys, n_rg, n_seg, n_ctas;
   float sm_scale;
   long long wait_cycles;  // bound of every mbarrier wait of the bf16 main kernel, in SM clock cycles
@@ -419,6 +423,10 @@ __device__ __forceinline__ float ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+  const __half2 v = __floats2half2_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
@@ -444,13 +452,18 @@ int32_t encode_pool_map(losa_ctx* c, unsigned char* blob, const void* pool, cons
   }
   const cuuint64_t dims[4] = {static_cast<cuuint64_t>(sh.head_dim), static_cast<cuuint64_t>(sh.page_size),
                               static_cast<cuuint64_t>(sh.n_kv_heads), static_cast<cuuint64_t>(kv->n_phys_pages)};
-  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(kv->stride_tok) * 2, static_cast<cuuint64_t>(kv->stride_head) * 2,
-                                 static_cast<cuuint64_t>(kv->stride_page) * 2};
-  const cuuint32_t box[4] = {64, static_cast<cuuint32_t>(sh.page_size), 1, 1};
+  // bf16 pages: 64-element (128-byte) boxes with the 128-byte swizzle, as the MMA descriptors expect them;
+  // FP8 pages: whole rows of d bytes, unswizzled, into the staging slots (the kernel converts them)
+  const bool fp8 = kv->kv_format == LOSA_KV_FP8_E4M3;
+  const cuuint64_t es = fp8 ? 1 : 2;
+  const cuuint64_t strides[3] = {static_cast<cuuint64_t>(kv->stride_tok) * es, static_cast<cuuint64_t>(kv->stride_head) * es,
+                                 static_cast<cuuint64_t>(kv->stride_page) * es};
+  const cuuint32_t box[4] = {fp8 ? static_cast<cuuint32_t>(sh.head_dim) : 64u, static_cast<cuuint32_t>(sh.page_size), 1, 1};
   const cuuint32_t estr[4] = {1, 1, 1, 1};
   const CUresult r = reinterpret_cast<EncodeTiledFn>(c->encode_fn)(
-      reinterpret_cast<CUtensorMap*>(blob), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(pool), dims,
-      strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+      reinterpret_cast<CUtensorMap*>(blob), fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4,
+      const_cast<void*>(pool), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+      fp8 ? CU_TENSOR_MAP_SWIZZLE_NONE : CU_TENSOR_MAP_SWIZZLE_128B,
       CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   if (r != CUDA_SUCCESS) {
     c->last_cuda_error = static_cast<int32_t>(r);
@@ -462,7 +475,8 @@ int32_t encode_pool_map(losa_ctx* c, unsigned char* blob, const void* pool, cons
 int32_t ensure_tensor_maps(losa_ctx* c, const losa_kv_t* kv) {
   const bool same = c->tmap_key_k == kv->k_pages && c->tmap_key_v == kv->v_pages &&
                     c->tmap_strides[0] == kv->stride_page && c->tmap_strides[1] == kv->stride_head &&
-                    c->tmap_strides[2] == kv->stride_tok && c->tmap_n_phys == kv->n_phys_pages;
+                    c->tmap_strides[2] == kv->stride_tok && c->tmap_n_phys == kv->n_phys_pages &&
+                    c->tmap_format == kv->kv_format;
   if (same) return LOSA_OK;
   int32_t rc = encode_pool_map(c, c->tmap_k, kv->k_pages, kv);
   if (rc != LOSA_OK) return rc;
@@ -474,21 +488,24 @@ int32_t ensure_tensor_maps(losa_ctx* c, const losa_kv_t* kv) {
   c->tmap_strides[1] = kv->stride_head;
   c->tmap_strides[2] = kv->stride_tok;
   c->tmap_n_phys = kv->n_phys_pages;
+  c->tmap_format = kv->kv_format;
   return LOSA_OK;
 }
 
-template <int D, int GP>
+template <int D, int GP, bool FP8>
 int32_t launch_tc5(losa_ctx* c, const AttnParams& ap, cudaStream_t st, bool with_combine) {
-  constexpr int smem = tc5_smem_bytes<D>();
-  if (!c->attn_attr_set) {          // a context has one shape, hence one instantiation, on one device
-    LOSA_CUDA_TRY(c, cudaFuncSetAttribute(attn_tc5_kernel<D, GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    c->attn_attr_set = 1;
+  constexpr int smem = tc5_smem_bytes<D, FP8>();
+  static_assert(smem <= kSmemBudget, "shared memory of the stage-4 kernel");
+  constexpr int bit = FP8 ? 2 : 1;  // a context has one shape on one device: one instantiation per cache format
+  if (!(c->attn_attr_set & bit)) {
+    LOSA_CUDA_TRY(c, cudaFuncSetAttribute(attn_tc5_kernel<D, GP, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    c->attn_attr_set |= bit;
   }
   CUtensorMap mk, mv;
   memcpy(&mk, c->tmap_k, sizeof(mk));
   memcpy(&mv, c->tmap_v, sizeof(mv));
   if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_begin, st));
-  launch_k(attn_tc5_kernel<D, GP>, ap.n_ctas, kTc5Threads, smem, st, mk, mv, ap);
+  launch_k(attn_tc5_kernel<D, GP, FP8>, ap.n_ctas, kTc5Threads, smem, st, mk, mv, ap);
   if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_end, st));
   int32_t rc = after_launch(c);
   if (rc != LOSA_OK || !with_combine) return rc;
@@ -500,9 +517,9 @@ template <typename T, int D, int GP>
 int32_t launch_simt(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
   const size_t smem = (static_cast<size_t>(2) * GP * D + 2 * kRowsPerGroup * D + 2 * kRowsPerGroup) * sizeof(float) +
                       (ap.n_seg + 1) * sizeof(int);
-  if (!c->attn_attr_set) {
+  if (!(c->attn_attr_set & 1)) {
     LOSA_CUDA_TRY(c, cudaFuncSetAttribute(attn_simt_kernel<T, D, GP>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-    c->attn_attr_set = 1;
+    c->attn_attr_set |= 1;
   }
   if (c->profile) LOSA_CUDA_TRY(c, cudaEventRecord(c->ev_begin, st));
   launch_k(attn_simt_kernel<T, D, GP>, ap.n_ctas, 256, smem, st, ap);
@@ -516,10 +533,17 @@ int32_t launch_simt(losa_ctx* c, const AttnParams& ap, cudaStream_t st) {
 template <int D>
 int32_t dispatch_page(losa_ctx* c, const AttnParams& ap, cudaStream_t st, bool with_combine) {
   const bool bf = c->shape.dtype == LOSA_BF16;
+  if (ap.k_scale) {                 // FP8 pages (bf16 contexts only, checked by the C-ABI layer)
+    switch (c->shape.page_size) {
+      case 16: return launch_tc5<D, 16, true>(c, ap, st, with_combine);
+      case 32: return launch_tc5<D, 32, true>(c, ap, st, with_combine);
+      default: return launch_tc5<D, 64, true>(c, ap, st, with_combine);
+    }
+  }
   switch (c->shape.page_size) {
-    case 16: return bf ? launch_tc5<D, 16>(c, ap, st, with_combine) : launch_simt<float, D, 16>(c, ap, st);
-    case 32: return bf ? launch_tc5<D, 32>(c, ap, st, with_combine) : launch_simt<float, D, 32>(c, ap, st);
-    default: return bf ? launch_tc5<D, 64>(c, ap, st, with_combine) : launch_simt<float, D, 64>(c, ap, st);
+    case 16: return bf ? launch_tc5<D, 16, false>(c, ap, st, with_combine) : launch_simt<float, D, 16>(c, ap, st);
+    case 32: return bf ? launch_tc5<D, 32, false>(c, ap, st, with_combine) : launch_simt<float, D, 32>(c, ap, st);
+    default: return bf ? launch_tc5<D, 64, false>(c, ap, st, with_combine) : launch_simt<float, D, 64>(c, ap, st);
   }
 }
 
@@ -553,6 +577,9 @@ int32_t launch_sparse_prefix_attn(losa_ctx* c, const void* q, const losa_kv_t* k
   ap.o_p = state->o_p;
   ap.lse_p = state->lse_p;
   ap.status = status_ptr(c);
+  const bool fp8 = kv->kv_format == LOSA_KV_FP8_E4M3;
+  ap.k_scale = fp8 ? kv->k_scale : nullptr;
+  ap.v_scale = fp8 ? kv->v_scale : nullptr;
   ap.N = sh.batch;
   ap.B = sh.block_size;
   ap.Hq = sh.n_q_heads;

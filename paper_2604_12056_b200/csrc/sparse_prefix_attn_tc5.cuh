@@ -29,14 +29,20 @@ constexpr int kTc5PgMax = 8;                     // pages per group at the small
 constexpr int kTc5MetaRing = 16;                 // groups whose per-page token counts are kept (producer lead < 16)
 constexpr float kTc5Tau = 8.0f;                  // reference maximum moves only when it would grow by more than this (log2 units)
 constexpr int kTc5XchgBytes = (2 * 2 + 1) * kRowsPerGroup * 4;   // row maxima [group parity][set][row], row sums [row]
-constexpr int kTc5TailBytes = kTailBytes + 512 + kTc5XchgBytes;  // 1024 bytes of barriers + page meta, the segment prefix and index cache, the exchange arrays
+constexpr int kTc5ScaleBytes = 2 * kTc5MetaRing * (kTc5PgMax + 1) * 4;   // FP8 pages: per-page scales and page counts of the groups in flight, K and V
+constexpr int kTc5TailBytes = kTailBytes + 512 + kTc5XchgBytes + kTc5ScaleBytes;  // 1024 bytes of barriers + page meta, the segment prefix and index cache, the exchange arrays, the scales
+constexpr int kTc5Stg = 2;                       // FP8 pages: staging slots (bytes as they lie in memory) per tensor
 
 template <int D> constexpr int tc5_slot_bytes() { return kTc5Tok * D * 2; }
-template <int D> constexpr int tc5_ring_slots() {     // per ring (K and V have one each)
+template <int D> constexpr int tc5_stg_bytes() { return kTc5Tok * D; }
+template <int D, bool FP8> constexpr int tc5_ring_slots() {     // per ring (K and V have one each)
+  if (FP8) return 2;                                            // the staging slots take the rest
   const int n = (kSmemBudget - 1024 - kTc5TailBytes) / tc5_slot_bytes<D>() / 2;
   return n > 6 ? 6 : n;
 }
-template <int D> constexpr int tc5_smem_bytes() { return 1024 + 2 * tc5_ring_slots<D>() * tc5_slot_bytes<D>() + kTc5TailBytes; }
+template <int D, bool FP8> constexpr int tc5_smem_bytes() {
+  return 1024 + 2 * tc5_ring_slots<D, FP8>() * tc5_slot_bytes<D>() + (FP8 ? 2 * kTc5Stg * tc5_stg_bytes<D>() : 0) + kTc5TailBytes;
+}
 
 // Shared-memory matrix descriptor: 128-byte swizzle, 8-row groups 1024 bytes apart; lbo = distance
 // between 64-element blocks along the MN dimension of an MN-major operand.
@@ -44,9 +50,10 @@ __device__ __forceinline__ uint64_t tc5_desc(uint32_t saddr, uint32_t lbo) {
   return static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4) | (static_cast<uint64_t>((lbo >> 4) & 0x3FFFu) << 16) |
          (static_cast<uint64_t>(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
 }
-// Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, M x N tile, B optionally MN-major.
-__device__ __forceinline__ uint32_t tc5_idesc(int M, int N, int b_mn_major) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(b_mn_major) << 16) |
+// Instruction descriptor, kind::f16: fp32 accumulate, A and B both bf16 (fmt 1) or both fp16 (fmt 0),
+// M x N tile, B optionally MN-major.
+__device__ __forceinline__ uint32_t tc5_idesc(int M, int N, int b_mn_major, uint32_t fmt = 1u) {
+  return (1u << 4) | (fmt << 7) | (fmt << 10) | (static_cast<uint32_t>(b_mn_major) << 16) |
          (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
 }
 // D[tmem] (+)= A[tmem] . B[smem descriptor]
@@ -109,10 +116,17 @@ __device__ __forceinline__ void tc5_wait_st() { asm volatile("tcgen05.wait::st.s
 // byte offset of 16-byte chunk c (0..7) of row t in a [rows][128 B] tile with the 128-byte swizzle
 __device__ __forceinline__ uint32_t tc5_sw(int t, int c) { return static_cast<uint32_t>(t * 128 + ((c ^ (t & 7)) << 4)); }
 
-template <int D, int GP>
+// FP8: the K / V pools hold E4M3 bytes with one power-of-two scale per (page, KV head).  The page
+// copies land in staging slots as they lie in memory (half the bytes); the producer warp that issued
+// them converts a landed group to fp16 times its page's scale (exact) into the ring slot, in the
+// layout the tensor maps of the bf16 path produce, and every MMA runs on fp16 operands (Q and P are
+// converted to fp16 instead of bf16); nothing else changes.
+template <int D, int GP, bool FP8>
 __global__ void __launch_bounds__(kTc5Threads, 1)
 attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV, AttnParams p) {
-  constexpr int NR = tc5_ring_slots<D>();       // slots per ring
+  constexpr int NR = tc5_ring_slots<D, FP8>();  // slots per ring
+  constexpr int NSTG = kTc5Stg, STG = tc5_stg_bytes<D>();
+  constexpr uint32_t FMT = FP8 ? 0u : 1u;       // operand format of the MMAs: fp16 / bf16
   constexpr int SLOT = tc5_slot_bytes<D>();
   constexpr int PG = kTc5Tok / GP;              // pages per group
   constexpr int HALVES = D / 64;                // 64-column (128-byte) blocks of a K or V row
@@ -123,19 +137,22 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   static_assert(D == 64 || D == 128, "head dimensions of the tensor-core path");
   static_assert(GP == 16 || GP == 32 || GP == 64, "page sizes of the tensor-core path");
   static_assert(NR >= 2 && PG <= kTc5PgMax, "ring too shallow / group too long");
-  static_assert(8 * (4 * 6 + 14) + 4 * kTc5MetaRing * kTc5PgMax + 16 <= 1024, "tail layout");
+  static_assert(8 * (4 * 6 + 14 + 2 * kTc5Stg) + 4 * kTc5MetaRing * kTc5PgMax + 16 <= 1024, "tail layout");
 
   extern __shared__ uint8_t smem_raw[];
   const uint32_t raw = smem_u32(smem_raw);
   const uint32_t base = (raw + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - raw);
   const uint32_t kring = base, vring = base + NR * SLOT;
-  uint8_t* tail = gen + 2 * NR * SLOT;
-  const uint32_t tail_s = base + 2 * NR * SLOT;
+  constexpr int STG_ALL = FP8 ? 2 * NSTG * STG : 0;
+  const uint32_t kstg = base + 2 * NR * SLOT, vstg = kstg + NSTG * STG;          // FP8 only
+  uint8_t* tail = gen + 2 * NR * SLOT + STG_ALL;
+  const uint32_t tail_s = base + 2 * NR * SLOT + STG_ALL;
   const uint32_t kfull = tail_s, kfree = kfull + 8 * NR, vfull = kfree + 8 * NR, vfree = vfull + 8 * NR;
   const uint32_t s_full = vfree + 8 * NR, s_free = s_full + 16, p_full = s_free + 16, q_full = p_full + 16, q_free = q_full + 8, xbar = q_free + 8;
   const uint32_t drain_bar = xbar + 32;            // two barriers: the issuing threads' last commit when the CTA gives up
-  volatile int* meta = reinterpret_cast<volatile int*>(tail + 8 * (4 * 6 + 14));   // [kTc5MetaRing][kTc5PgMax] valid tokens per page
+  const uint32_t kstg_full = drain_bar + 16, vstg_full = kstg_full + 8 * NSTG;   // FP8: a staging slot's copies have landed
+  volatile int* meta = reinterpret_cast<volatile int*>(tail + 8 * (4 * 6 + 14 + 2 * kTc5Stg));   // [kTc5MetaRing][kTc5PgMax] valid tokens per page
   volatile int* abort_flag = meta + kTc5MetaRing * kTc5PgMax;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(const_cast<int*>(abort_flag) + 1);
   int* pre = reinterpret_cast<int*>(tail + 1024);
@@ -144,6 +161,8 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   int* len_s = na_s + kStageSeq;
   float* xmax = reinterpret_cast<float*>(len_s + kStageSeq);   // [2][2][128]
   float* xsum = xmax + 4 * kRowsPerGroup;                        // [128]
+  volatile float* scale_meta = xsum + kRowsPerGroup;             // FP8: [2 (K, V)][kTc5MetaRing][kTc5PgMax] page scales,
+  volatile int* ng_meta = reinterpret_cast<volatile int*>(const_cast<float*>(scale_meta) + 2 * kTc5MetaRing * kTc5PgMax);   // [2][kTc5MetaRing] pages per group
   const bool staged = p.N * p.B <= kStageIdx && p.N <= kStageSeq;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -164,6 +183,11 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     for (int i = 0; i < 4; ++i) mbar_init(xbar + 8 * i, 2);      // the two softmax warps of a scheduler meet here
     mbar_init(drain_bar, 1);
     mbar_init(drain_bar + 8, 1);
+    if (FP8)
+      for (int i = 0; i < NSTG; ++i) {
+        mbar_init(kstg_full + 8 * i, 1);
+        mbar_init(vstg_full + 8 * i, 1);
+      }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -245,6 +269,112 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       }
       return r;
     };
+    if constexpr (FP8) {
+      // ---- FP8 pages.  The copies go to staging slots (NSTG groups in flight); before a staging slot
+      // is reused, and at the end, this warp converts the groups that have landed: bytes -> fp16
+      // times the page's scale, written where the tensor maps of the bf16 path would have put them
+      // (two 128-byte-swizzled blocks per row), then announced to the MMA warps.
+      const uint32_t stg = is_v ? vstg : kstg, stg_full0 = is_v ? vstg_full : kstg_full;
+      uint8_t* stg_gen = gen + (stg - base);
+      uint8_t* ring_gen = gen + (ring - base);
+      volatile float* sc_meta = scale_meta + (is_v ? kTc5MetaRing * kTc5PgMax : 0);
+      volatile int* ngs = ng_meta + (is_v ? kTc5MetaRing : 0);
+      const float* scale_g = is_v ? p.v_scale : p.k_scale;
+      constexpr int CPRW = D / 16;                    // 16-byte chunks of a row of bytes
+      int conv = 0;                                   // groups converted so far
+      bool go = true;
+      auto convert = [&](int gc) {
+        const int ss = gc % NSTG, sr = gc % NR;
+        int ok = 1;
+        if (lane == 0) {
+          ok = mbar_wait(stg_full0 + 8 * ss, (gc / NSTG) & 1, abort_flag, p.status, p.wait_cycles);
+          if (ok && gc >= NR) ok = mbar_wait(free0 + 8 * sr, (gc / NR - 1) & 1, abort_flag, p.status, p.wait_cycles);
+        }
+        if (__shfl_sync(0xffffffffu, ok, 0) == 0) return false;
+        const int ntok = ngs[gc % kTc5MetaRing] * GP;
+        const uint8_t* src = stg_gen + ss * STG;
+        uint8_t* dst = ring_gen + sr * SLOT;
+        for (int id = lane; id < ntok * CPRW; id += 32) {
+          const int t = id / CPRW, c8 = id % CPRW;
+          const __half2 sc2 = __float2half2_rn(sc_meta[(gc % kTc5MetaRing) * kTc5PgMax + t / GP]);
+          const uint4 rawb = *reinterpret_cast<const uint4*>(src + t * D + c8 * 16);
+          const uint32_t w[4] = {rawb.x, rawb.y, rawb.z, rawb.w};
+          uint32_t h[8];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            __half2_raw lo2 = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(w[e] & 0xffffu), __NV_E4M3);
+            __half2_raw hi2 = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(w[e] >> 16), __NV_E4M3);
+            const __half2 a2 = __hmul2(*reinterpret_cast<__half2*>(&lo2), sc2), b2 = __hmul2(*reinterpret_cast<__half2*>(&hi2), sc2);
+            h[2 * e] = *reinterpret_cast<const uint32_t*>(&a2);
+            h[2 * e + 1] = *reinterpret_cast<const uint32_t*>(&b2);
+          }
+          uint8_t* row = dst + (c8 >> 2) * HS;
+          const int c = 2 * (c8 & 3);
+          *reinterpret_cast<uint4*>(row + tc5_sw(t, c)) = make_uint4(h[0], h[1], h[2], h[3]);
+          *reinterpret_cast<uint4*>(row + tc5_sw(t, c + 1)) = make_uint4(h[4], h[5], h[6], h[7]);
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMAs read the slot through the async proxy; the next copies overwrite the staging slot through it
+        __syncwarp();
+        if (lane == 0) mbar_arrive(full0 + 8 * sr, 1);
+        return true;
+      };
+      struct Ready8 { int phys, kh, valid, grp, j, ng; float scale; };
+      auto stage_b8 = [&](int i, const Item& it) {
+        const Ready r = stage_b(i, it);
+        return Ready8{r.phys, r.kh, r.valid, r.grp, r.j, r.ng, 1.f};
+      };
+      auto stage_c = [&](int i, Ready8& r) {          // the page's scale (its address needs the physical page)
+        if (i < hi) {
+          if (r.phys < 0 || r.phys >= p.n_phys || r.valid <= 0) {
+            set_status(p.status, LOSA_ERR_BOUNDS);
+            r.phys = 0;
+            r.valid = 0;
+          }
+          r.scale = __ldg(scale_g + static_cast<size_t>(r.phys) * p.Hkv + r.kh);
+        }
+      };
+      Item a = stage_a(lo + lane);
+      Ready8 b = stage_b8(lo + lane, a);
+      a = stage_a(lo + lane + 32);
+      stage_c(lo + lane, b);
+      Ready8 b1 = stage_b8(lo + lane + 32, a);
+      a = stage_a(lo + lane + 64);
+      int n_groups = 0;
+      for (int b0 = lo; b0 < hi && go; b0 += 32) {
+        const Item a_next = stage_a(b0 + lane + 96);
+        const Ready8 b2 = stage_b8(b0 + lane + 64, a);
+        stage_c(b0 + lane + 32, b1);
+        const int nb = min(32, hi - b0);
+        int pos = 0;
+        while (pos < nb && go) {
+          const int grp = __shfl_sync(0xffffffffu, b.grp, pos), j0 = __shfl_sync(0xffffffffu, b.j, pos);
+          const int ng = __shfl_sync(0xffffffffu, b.ng, pos);
+          const int cnt = min(ng - j0, nb - pos);
+          const int ss = grp % NSTG;
+          if (j0 == 0) {
+            while (go && conv + NSTG <= grp) go = convert(conv++);          // the staging slot must have been emptied
+            if (!go) break;
+          }
+          const bool mine = lane >= pos && lane < pos + cnt;
+          if (mine) {
+            if (!is_v) meta[(grp % kTc5MetaRing) * kTc5PgMax + b.j] = b.valid;
+            sc_meta[(grp % kTc5MetaRing) * kTc5PgMax + b.j] = b.scale;
+          }
+          if (j0 == 0 && lane == 0) ngs[grp % kTc5MetaRing] = ng;
+          __syncwarp();
+          if (j0 == 0 && lane == 0) mbar_expect_tx(stg_full0 + 8 * ss, ng * GP * D);
+          __syncwarp();
+          if (mine) tma_load_4d(stg + ss * STG + b.j * (GP * D), map, stg_full0 + 8 * ss, 0, 0, b.kh, b.phys, policy);
+          issued = grp;
+          n_groups = grp + 1;
+          pos += cnt;
+        }
+        a = a_next;
+        b = b1;
+        b1 = b2;
+      }
+      while (go && conv < n_groups) go = convert(conv++);
+    } else {
     Item a = stage_a(lo + lane);
     Ready b = stage_b(lo + lane, a);
     a = stage_a(lo + lane + 32);
@@ -286,6 +416,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
       a = a_next;
       b = b_next;
     }
+    }
   } else if (warp == kTc5QkWarp) {
     // ------------------------------------------------------------------ Q K^T issuer (one thread)
     if (lane == 0) {
@@ -300,7 +431,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
           ok = ok && (use == 0 || mbar_wait(s_free + 8 * b, (use - 1) & 1, abort_flag, p.status, p.wait_cycles));
           if (!ok) break;
           tc5_fence_after();
-          const uint32_t idesc = tc5_idesc(kRowsPerGroup, ng * GP, 0), kt = kring + slot * SLOT;
+          const uint32_t idesc = tc5_idesc(kRowsPerGroup, ng * GP, 0, FMT), kt = kring + slot * SLOT;
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks)
             tc5_mma_ts(tmem + COL_S + b * kTc5Tok, tmem + COL_Q + ks * 8, tc5_desc(kt + (ks >> 2) * HS + (ks & 3) * 32, 16),
@@ -318,7 +449,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   } else if (warp == kTc5PvWarp) {
     // ------------------------------------------------------------------ P V issuer (one thread)
     if (lane == 0) {
-      const uint32_t idesc = tc5_idesc(kRowsPerGroup, D, 1);
+      const uint32_t idesc = tc5_idesc(kRowsPerGroup, D, 1, FMT);
       int sg = sg0, item = lo, g = 0;
       bool ok = true;
       while (item < hi && ok) {
@@ -389,6 +520,13 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
         for (int c = 0; c < QW / 4; ++c) {
           const uint4 v = src ? __ldg(src + c) : make_uint4(0u, 0u, 0u, 0u);
           qw[4 * c] = v.x; qw[4 * c + 1] = v.y; qw[4 * c + 2] = v.z; qw[4 * c + 3] = v.w;
+        }
+        if constexpr (FP8) {                        // the MMAs of this variant take fp16 operands
+#pragma unroll
+          for (int c = 0; c < QW; ++c) {
+            const __half2 hq = __floats2half2_rn(__uint_as_float(qw[c] << 16), __uint_as_float(qw[c] & 0xffff0000u));
+            qw[c] = *reinterpret_cast<const uint32_t*>(&hq);
+          }
         }
         if (piece > 0) ok = warp_wait(q_free, (piece - 1) & 1);
         if (!ok) break;
@@ -487,7 +625,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
                   const float p0 = ex2(fmaf(__uint_as_float(sraw[32 * c + 2 * e]), scale2, -ms));
                   const float p1 = ex2(fmaf(__uint_as_float(sraw[32 * c + 2 * e + 1]), scale2, -ms));
                   sum[e & 3] += p0 + p1;
-                  w[e] = pack_bf16(p0, p1);
+                  w[e] = FP8 ? pack_f16(p0, p1) : pack_bf16(p0, p1);
                 }
                 tc5_st16(s_addr + col0 / 2 + 16 * c, w);
               }
@@ -562,11 +700,13 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
     // round of copies of every ring slot (a group that was begun has had all its copies issued: the
     // producer loop only stops between groups), the issuing threads for the products they issued.
     if ((warp == kTc5KWarp || warp == kTc5VWarp) && lane == 0) {
-      const uint32_t full0 = warp == kTc5VWarp ? vfull : kfull;
-      for (int sl = 0; sl < NR; ++sl) {
+      // (FP8 pages: the copies land in the staging slots)
+      const uint32_t full0 = FP8 ? (warp == kTc5VWarp ? vstg_full : kstg_full) : (warp == kTc5VWarp ? vfull : kfull);
+      constexpr int NSL = FP8 ? NSTG : NR;
+      for (int sl = 0; sl < NSL; ++sl) {
         if (issued < sl) continue;
-        const int gl = issued - (issued - sl) % NR;
-        mbar_drain(full0 + 8 * sl, (gl / NR) & 1);
+        const int gl = issued - (issued - sl) % NSL;
+        mbar_drain(full0 + 8 * sl, (gl / NSL) & 1);
       }
     }
     if ((warp == kTc5QkWarp || warp == kTc5PvWarp) && lane == 0) {

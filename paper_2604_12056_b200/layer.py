@@ -34,7 +34,7 @@ class LosaLayer:
 
     def __init__(self, cfg, k_pages, v_pages, page_table, kv_len, mode="losa", device="cuda",
                  share_pool_with: "LosaLayer | None" = None, tau: float = 0.0, pooled: bool = False,
-                 mma_selector: bool = False):
+                 mma_selector: bool = False, fp8_kv: bool = False):
         self.cfg, self.mode, self.device = cfg, mode, device
         self.tau = tau            # > 0: stage 1 keeps tokens until their Delta reach tau of the block's total
         self.pooled = pooled      # stage 2 keeps one page list per (token, KV head) instead of one per query head
@@ -59,6 +59,20 @@ class LosaLayer:
             self.page_table = page_table if isinstance(page_table, torch.Tensor) else to_device(page_table, device)
         self.kv_len = (kv_len.clone() if isinstance(kv_len, torch.Tensor) else to_device(kv_len, device))
         self.kv = B.make_kv(self.k_pages, self.v_pages, self.kmin, self.kmax, self.page_table, self.kv_len)
+        self.fp8_kv = fp8_kv
+        if fp8_kv:
+            # FP8 (E4M3) cache with one power-of-two scale per (page, KV head): quantised from the bf16
+            # pools by the library, which also writes the summaries of the dequantised keys; every
+            # stage then works on the FP8 cache (the bf16 pools can be released by the caller)
+            assert share_pool_with is None and self.dtype == B.LOSA_BF16
+            n_phys = self.k_pages.shape[0]
+            self.k_codes = torch.zeros(self.k_pages.shape, dtype=torch.uint8, device=device)
+            self.v_codes = torch.zeros(self.v_pages.shape, dtype=torch.uint8, device=device)
+            self.k_scale = torch.ones((n_phys, Hkv), dtype=torch.float32, device=device)
+            self.v_scale = torch.ones((n_phys, Hkv), dtype=torch.float32, device=device)
+            self.kv_native = self.kv
+            self.kv = B.make_kv(self.k_codes, self.v_codes, self.kmin, self.kmax, self.page_table, self.kv_len,
+                                self.k_scale, self.v_scale)
         self.q_prev = torch.zeros((N, Bk, Hq, d), dtype=td, device=device)
         self.o_p = torch.zeros((N, Bk, Hq, d), dtype=torch.float32, device=device)
         self.lse_p = torch.zeros((N, Bk, Hq), dtype=torch.float32, device=device)
@@ -75,7 +89,9 @@ class LosaLayer:
         self.union_count = torch.zeros((N, Hkv), dtype=torch.int32, device=device)
         self.out = torch.zeros((N, Bk, Hq, d), dtype=td, device=device)
         self.lse_out = torch.zeros((N, Bk, Hq), dtype=torch.float32, device=device)
-        if share_pool_with is None:
+        if fp8_kv:
+            B.losa_quantize_kv_pages(self.ctx, self.kv_native, self.kv)
+        elif share_pool_with is None:
             B.losa_build_page_summaries(self.ctx, self.kv)
 
     def stage_step_arg(self):

@@ -150,6 +150,37 @@ class OracleLayer:
         return res
 
 
+class OracleFp8Layer(OracleLayer):
+    """The same layer over an FP8 (E4M3) cache: the oracle quantises the workload's pools page by page
+    (its own quantiser), and every stage then runs - unchanged - on the dequantised values, which are
+    exact in the element type.  Block finalisation appends through the FP8 rule (touched pages are
+    re-quantised) and refreshes the dequantised copy and the summaries."""
+
+    def __init__(self, w, mode="losa", **kw):
+        import types
+        cfg = w.cfg
+        sh = oracle_shape_of(cfg)
+        e = w.k_pages.dtype
+        kmin = np.zeros((w.n_phys, cfg.n_kv_heads, cfg.head_dim), e)
+        kv_src = orc.KV(sh, w.k_pages, w.v_pages, kmin, kmin.copy(), w.page_table, w.kv_len.copy())
+        self.k_codes, self.v_codes, self.k_scale, self.v_scale = orc.fp8_quantize_pages(sh, kv_src)
+        deq = types.SimpleNamespace(cfg=cfg, k_pages=np.zeros_like(w.k_pages), v_pages=np.zeros_like(w.v_pages),
+                                    page_table=w.page_table, kv_len=w.kv_len.copy(), n_phys=w.n_phys)
+        kv_dst = orc.KV(sh, deq.k_pages, deq.v_pages, kmin.copy(), kmin.copy(), w.page_table, deq.kv_len)
+        orc.fp8_dequantize_pages(sh, self.k_codes, self.v_codes, self.k_scale, self.v_scale, kv_dst)
+        super().__init__(deq, mode, **kw)
+
+    def run_step(self, inp, x_sel=None, finalize=False):
+        res = super().run_step(inp, x_sel=x_sel, finalize=False)
+        if finalize:
+            orc.fp8_append_block(self.sh, self.kv.page_table, self.kv_len, self.k_codes, self.v_codes, self.k_scale,
+                                 self.v_scale, inp.k_blk, inp.v_blk)
+            orc.fp8_dequantize_pages(self.sh, self.k_codes, self.v_codes, self.k_scale, self.v_scale, self.kv)
+            orc.build_page_summaries(self.sh, self.kv)
+            self.step[:] = 0
+        return res
+
+
 def delta_gap_ok(delta_row, m, rel=1e-3):
     """The m-th and (m+1)-th largest Delta are clearly separated, or exactly equal (then the index
     tie rule decides on both sides).  Otherwise fp rounding could flip the selection."""
