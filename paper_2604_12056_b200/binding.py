@@ -222,7 +222,7 @@ def losa_page_scores_topk_pooled(ctx, q, kv, active_idx, n_active, step, k, topk
 
 def losa_page_scores_topk_mma(ctx, q, kv, active_idx, n_active, step, k, topk_pages, topk_scores_opt=None):
     """Stage 2 with tensor-core scores (bf16): lists valid under the relaxed rule, not entry by entry."""
-    ctx._check("losa_page_scores_topk_mma", "losa_quantize_kv_pages", lib().losa_page_scores_topk_mma(
+    ctx._check("losa_page_scores_topk_mma", lib().losa_page_scores_topk_mma(
         ctx._h, _ptr(q), C.byref(kv), _ptr(active_idx), _ptr(n_active), _ptr(step), C.c_int32(k),
         _ptr(topk_pages), _ptr(topk_scores_opt), _stream()))
 
