@@ -68,6 +68,8 @@ def parse_args():
                     help="selector variant: one page list per (token, KV head) instead of one per query head")
     ap.add_argument("--layers", type=int, default=0, help="attention layers (default: 36 for c5, else 1)")
     ap.add_argument("--active-frac", type=float, default=None, help="override the active fraction")
+    ap.add_argument("--kv-dtype", default="native", choices=["native", "fp8"],
+                    help="fp8: the K/V pages are stored as E4M3 bytes with one power-of-two scale per (page, KV head)")
     ap.add_argument("--no-extras", action="store_true", help="skip baselines, stage breakdown, cpu baseline")
     return ap.parse_args()
 
@@ -137,10 +139,12 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------- byte accounting
-def stage4_bytes(cfg, up, uc, na, kv_len):
+def stage4_bytes(cfg, up, uc, na, kv_len, fp8=False):
     """Algorithmic bytes of one stage-4 launch: K and V of the valid tokens of every listed page,
-    the active queries, the union list and page-table entries read, the state rows written."""
+    the active queries, the union list and page-table entries read, the state rows written (FP8
+    pages: one byte per K / V element plus the two scales of every listed page)."""
     e = 2 if cfg.dtype == "bf16" else 4
+    ekv = 1 if fp8 else e
     g, d = cfg.page_size, cfg.head_dim
     total = 0
     for s in range(cfg.batch):
@@ -153,7 +157,7 @@ def stage4_bytes(cfg, up, uc, na, kv_len):
             toks = n * g
             if n and up[s, kh, n - 1] == P - 1:    # lists ascend: only the last entry can be the partial page
                 toks -= g - tail
-            total += 2 * toks * d * e + 8 * n
+            total += 2 * toks * d * ekv + 8 * n + (8 * n if fp8 else 0)
         total += int(na[s]) * cfg.n_q_heads * (d * e + (d + 1) * 4)
     return total
 
@@ -238,13 +242,18 @@ class LayerRun:
     """One attention layer of the workload on the device: its own seeded pool, LoSA cache, static
     input buffers and two CUDA graphs (the whole-step call; block finalisation)."""
 
-    def __init__(self, cfg, rank, layer, dev, pooled=False):
+    def __init__(self, cfg, rank, layer, dev, pooled=False, fp8=False):
         import torch
         from paper_2604_12056_b200.layer import LosaLayer
         self.torch, self.cfg = torch, cfg
         self.w = wl.DeviceWorkload(cfg, replica=rank, layer=layer, device=dev)
         self.layer = LosaLayer(cfg, self.w.k_pages, self.w.v_pages, self.w.page_table, self.w.kv_len, "losa", dev,
-                               pooled=pooled)
+                               pooled=pooled, fp8_kv=fp8)
+        self.pool_mib = self.w.k_pages.numel() * (2 if fp8 else 4) / 2 ** 20
+        if fp8:                                # the library has quantised the pools: release the bf16 copies
+            torch.cuda.synchronize()
+            self.w.k_pages = self.w.v_pages = None
+            self.layer.k_pages = self.layer.v_pages = self.layer.kv_native = None
         self.inputs = {}                       # block -> list of DeviceStepInputs (current and previous block)
         self.next_block = 0
         first = self.block_inputs(0)[0]
@@ -329,7 +338,8 @@ def run_ours(args, cfg0):
     warm_blocks = max(1, -(-args.warmup // per_block))         # whole untimed blocks: at least W layer-steps
     total_blocks = warm_blocks + 4 * blocks_region + 3
     cfg = wl.config(cfg0.name, n_blocks=total_blocks, m_active=cfg0.m_active, beta_active=cfg0.beta_active, topk=cfg0.topk)
-    runs = [LayerRun(cfg, D.replica_of(rank), l, dev, pooled=args.pooled) for l in range(L)]
+    fp8 = args.kv_dtype == "fp8"
+    runs = [LayerRun(cfg, D.replica_of(rank), l, dev, pooled=args.pooled, fp8=fp8) for l in range(L)]
     launches_step = launches_fin = 0
     for r in runs:
         launches_step, launches_fin = r.capture()
@@ -421,7 +431,8 @@ def run_ours(args, cfg0):
         "metric": METRIC, "value": ms_per_step * 1e3, "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
-        "config": {"workload": workload_name(cfg0, L_model) + (", pooled selector (one page list per token and KV head)" if args.pooled else ""),
+        "config": {"workload": workload_name(cfg0, L_model) + (", pooled selector (one page list per token and KV head)" if args.pooled else "")
+                               + (", K/V pages stored as FP8 E4M3 with per-page scales" if fp8 else ""),
                    "sequences_per_gpu": cfg.batch, "layers": L_model, "layers_timed": L,
                    "step": "one layer-step = stages 1-6 for one layer and one denoising step; steps run in model order "
                            "(block, denoising step, layer) from a block boundary; the last step of a block also appends the block to the cache",
@@ -435,7 +446,7 @@ def run_ours(args, cfg0):
                    "l2": ("flushed between steps, outside the timed region: 256 MiB write, then 256 MiB read so no dirty "
                           "lines remain") if use_flush else
                          ("inputs larger than L2: consecutive layer-steps read different per-layer KV pools "
-                          f"({runs[0].w.k_pages.numel() * 4 / 2**20:.0f} MiB each), no flush")},
+                          f"({runs[0].pool_mib:.0f} MiB each), no flush")},
         "clocks": clocks, "gpu_launches": state["launches"],
         "step_us": {"losa_step_median": float(np.median(sparse_ms)) * 1e3 if sparse_ms else None,
                     "dense_first_step_median": float(np.median(dense_ms)) * 1e3 if dense_ms else None},
@@ -461,7 +472,7 @@ def run_ours(args, cfg0):
             r.layer.run_step_fused(r.q_s, r.k_s, r.v_s, r.m_s)
             k_ms.append(r.layer.ctx.stage4_last_ms())
             k_bytes.append(stage4_bytes(cfg, to_host(r.layer.union_pages), to_host(r.layer.union_count),
-                                        to_host(r.layer.n_active), to_host(r.layer.kv_len)))
+                                        to_host(r.layer.n_active), to_host(r.layer.kv_len), fp8))
             kinds.append("dense" if t == 0 else "losa")
             k_slices.append(pages_read(to_host(r.layer.union_count)))
             if t == T - 1:
@@ -469,7 +480,7 @@ def run_ours(args, cfg0):
     for r in runs:
         r.layer.ctx.profile_stage4(False)
     slice_bytes = 2 * cfg.page_size * cfg.head_dim * 2
-    scalable = cfg.head_dim == 128 and cfg.dtype == "bf16"
+    scalable = cfg.head_dim == 128 and cfg.dtype == "bf16" and not fp8     # no ncu capture of the FP8 variant is on file
 
     def roof(sel):
         b = sum(x for x, k in zip(k_bytes, kinds) if k in sel)
@@ -561,7 +572,7 @@ def run_ours(args, cfg0):
     losa_pages = [p for t, p in pages if t != 0]
     result["pages_read_per_step"] = {"losa": float(np.mean(losa_pages)) if losa_pages else None,
                                      "note": "sum over sequences and KV heads of the (page, KV head) slices listed, per layer-step"}
-    if rank == 0 and not args.no_extras:
+    if rank == 0 and not args.no_extras and not fp8:
         extras(args, cfg, runs[0], lambda v: flush(v, force=True), result, warm_blocks + 4 * blocks_region)
     missing = [k2 for k2, v in (("roofline_losa_steps", result["roofline_losa_steps"]),
                                 ("step_us.losa_step_median", result["step_us"]["losa_step_median"]),
