@@ -45,15 +45,15 @@ UNIT = "us/layer-step"
 L2_FLUSH_BYTES = 256 << 20
 # DRAM traffic of the stage-4 main kernel per listed (page, KV head) slice, from the ncu capture in
 # profiles/attn_tc5_kernel_c5.txt: the dense launch there moved dram__bytes_read.sum +
-# dram__bytes_write.sum = 1,085.39 MB for its 65,984 slices (16,384 of the 16,449 bytes per slice are
-# the slice's K and V).  Traffic grows in proportion to the slices, so a launch's traffic is reported
-# as slices x this figure; LoSA launches add the partial records they write (3.7-4.8 MB of DRAM
-# writes in the three LoSA launches of that capture).  Pages of 32 tokens, head dim 128, bf16; other
-# page sizes scale by the slice size (pages of 64 with two row groups per KV head, workload c4: 537.6 MB
-# read for 16,384 slices of 32,768 bytes on the dense step, 1.001 of the slices' bytes: the second row
-# group's pass over the pages is served by the L2, see profiles/attn_tc5_kernel_c4.txt).
-NCU_BYTES_PER_SLICE = {"losa": 1085.39e6 / 65984, "dense": 1085.39e6 / 65984}
-NCU_FIXED_BYTES = {"losa": 4.8e6, "dense": 0.0}
+# dram__bytes_write.sum = 1,077.27 + 5.16 MB for its 65,536 slices (16,384 of the 16,516 bytes per slice
+# are the slice's K and V).  Traffic grows in proportion to the slices, so a launch's traffic is reported
+# as slices x this figure; LoSA launches add the partial records they write (3.4-4.7 MB of DRAM writes
+# in the three LoSA launches of that capture).  Pages of 32 tokens, head dim 128, bf16; other page sizes
+# scale by the slice size (pages of 64 with two row groups per KV head, workload c4: 537.6 MB read for
+# 16,384 slices of 32,768 bytes on the dense step, 1.001 of the slices' bytes: the second row group's
+# pass over the pages is served by the L2, see profiles/attn_tc5_kernel_c4.txt).
+NCU_BYTES_PER_SLICE = {"losa": 1082.43e6 / 65536, "dense": 1082.43e6 / 65536}
+NCU_FIXED_BYTES = {"losa": 4.2e6, "dense": 0.0}
 
 
 def parse_args():
