@@ -291,27 +291,41 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
           if (ok && gc >= NR) ok = mbar_wait(free0 + 8 * sr, (gc / NR - 1) & 1, abort_flag, p.status, p.wait_cycles);
         }
         if (__shfl_sync(0xffffffffu, ok, 0) == 0) return false;
-        const int ntok = ngs[gc % kTc5MetaRing] * GP;
-        const uint8_t* src = stg_gen + ss * STG;
-        uint8_t* dst = ring_gen + sr * SLOT;
-        for (int id = lane; id < ntok * CPRW; id += 32) {
-          const int t = id / CPRW, c8 = id % CPRW;
-          const __half2 sc2 = __float2half2_rn(sc_meta[(gc % kTc5MetaRing) * kTc5PgMax + t / GP]);
-          const uint4 rawb = *reinterpret_cast<const uint4*>(src + t * D + c8 * 16);
-          const uint32_t w[4] = {rawb.x, rawb.y, rawb.z, rawb.w};
-          uint32_t h[8];
+        // Lane = (token within a batch of TPI, 16-byte chunk of the row); U batches are loaded before
+        // any is converted, so that the warp - alone with this work - has independent chains in flight.
+        // A byte s.eeee.mmm becomes the fp16 s.0eeee.mmm0000000 = its value / 256 (E4M3 subnormals land on
+        // fp16 subnormals), then one packed multiply by 256 * scale, exact; the quantiser never writes
+        // the NaN code.
+        constexpr int TPI = 32 / CPRW, U = (GP / TPI) < 4 ? (GP / TPI) : 4;
+        const int npg = ngs[gc % kTc5MetaRing];
+        const int tl = lane / CPRW, c8 = lane % CPRW, c = 2 * (c8 & 3);
+        const uint8_t* src = stg_gen + ss * STG + tl * D + c8 * 16;
+        uint8_t* row = ring_gen + sr * SLOT + (c8 >> 2) * HS;
+        for (int pg = 0; pg < npg; ++pg) {
+          const __half2 sc2 = __float2half2_rn(256.f * sc_meta[(gc % kTc5MetaRing) * kTc5PgMax + pg]);
+          for (int t0 = pg * GP; t0 < (pg + 1) * GP; t0 += TPI * U) {
+            uint4 rawb[U];
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            __half2_raw lo2 = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(w[e] & 0xffffu), __NV_E4M3);
-            __half2_raw hi2 = __nv_cvt_fp8x2_to_halfraw2(static_cast<__nv_fp8x2_storage_t>(w[e] >> 16), __NV_E4M3);
-            const __half2 a2 = __hmul2(*reinterpret_cast<__half2*>(&lo2), sc2), b2 = __hmul2(*reinterpret_cast<__half2*>(&hi2), sc2);
-            h[2 * e] = *reinterpret_cast<const uint32_t*>(&a2);
-            h[2 * e + 1] = *reinterpret_cast<const uint32_t*>(&b2);
+            for (int u = 0; u < U; ++u) rawb[u] = *reinterpret_cast<const uint4*>(src + (t0 + u * TPI) * D);
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+              const uint32_t w[4] = {rawb[u].x, rawb[u].y, rawb[u].z, rawb[u].w};
+              uint32_t h[8];
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                  const uint32_t x = __byte_perm(w[e], 0u, hf ? 0x3424u : 0x1404u);      // two bytes, each in the high byte of a half
+                  const uint32_t bits = ((x >> 1) & 0x3f803f80u) | (x & 0x80008000u);
+                  const __half2 v = __hmul2(*reinterpret_cast<const __half2*>(&bits), sc2);
+                  h[2 * e + hf] = *reinterpret_cast<const uint32_t*>(&v);
+                }
+              }
+              const int t = t0 + u * TPI + tl;
+              *reinterpret_cast<uint4*>(row + tc5_sw(t, c)) = make_uint4(h[0], h[1], h[2], h[3]);
+              *reinterpret_cast<uint4*>(row + tc5_sw(t, c + 1)) = make_uint4(h[4], h[5], h[6], h[7]);
+            }
           }
-          uint8_t* row = dst + (c8 >> 2) * HS;
-          const int c = 2 * (c8 & 3);
-          *reinterpret_cast<uint4*>(row + tc5_sw(t, c)) = make_uint4(h[0], h[1], h[2], h[3]);
-          *reinterpret_cast<uint4*>(row + tc5_sw(t, c + 1)) = make_uint4(h[4], h[5], h[6], h[7]);
         }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the MMAs read the slot through the async proxy; the next copies overwrite the staging slot through it
         __syncwarp();
