@@ -82,13 +82,12 @@ def test_null_arguments_are_rejected_without_a_device(lib):
                       ("losa_sparse_prefix_attn", 9), ("losa_block_attn_merge", 8),
                       ("losa_update_prefix_cache", 8), ("losa_build_page_summaries", 3),
                       ("losa_denoise_step_host", 11), ("losa_denoise_step", 12),
-                      ("losa_page_scores_topk_pooled", 10), ("losa_page_scores_topk_mma", 10)):
+                      ("losa_page_scores_topk_pooled", 10), ("losa_page_scores_topk_mma", 10),
+                      ("losa_quantize_kv_pages", 4)):
         args = [None] * nargs
         if fn in ("losa_select_active",):
             args[3] = C.c_int32(64)
         assert getattr(lib, fn)(*args) == B.LOSA_ERR_INVALID_ARG, fn
-
-
     assert lib.losa_set_pooled_selection(None, C.c_int32(1)) == B.LOSA_ERR_INVALID_ARG
     assert lib.losa_set_wait_limit(None, C.c_int64(5)) == B.LOSA_ERR_INVALID_ARG
     args = [None] * 11
