@@ -223,30 +223,49 @@ __device__ __forceinline__ int rows_in_group(int n_active, int G, int rg) {
 }
 __device__ __forceinline__ long long cta_lo(long long T, int b, int n) { return (T * b) / n; }
 
-// Exclusive prefix of segment item counts into pre[0..n_seg] (shared memory), by one warp.
+// The tensor-core kernel cuts a list in which every non-empty segment is charged segment_pad(rows)
+// items on top of its pages (placed before them): entering a segment costs a CTA about as much as
+// that many pages (drain of the pipeline, the record, the new Q tile, refill), so equal shares of
+// the charged list finish together.  A CTA's share maps back to the pages it contains; the
+// combine step finds the CTAs of a segment with the same arithmetic on the charged positions.
+constexpr int kSegPadBase = 10, kSegPadRowsPer = 8;
+__device__ __forceinline__ int segment_pad(int rows) { return rows > 0 ? kSegPadBase + rows / kSegPadRowsPer : 0; }
+
+// Exclusive prefix of segment item counts into pre[0..n_seg] (shared memory), by one warp; with
+// vpre, also the prefix of the charged counts (pages + pad of every non-empty segment).
 __device__ __forceinline__ void segment_prefix(int* pre, int n_seg, int n_rg, int H_kv, int G,
                                                const int32_t* n_active, const int32_t* union_count,
-                                               int B, int lane) {
-  int run = 0;
+                                               int B, int lane, int* vpre = nullptr) {
+  int run = 0, vrun = 0;
   for (int base = 0; base < n_seg; base += 32) {
     const int seg = base + lane;
-    int c = 0;
+    int c = 0, vc = 0;
     if (seg < n_seg) {
       const int n_sk = n_seg / n_rg, rg = seg / n_sk, sk = seg % n_sk, s = sk / H_kv;
       int na = n_active[s];
       na = na < 0 ? 0 : (na > B ? B : na);
-      c = rows_in_group(na, G, rg) > 0 ? max(union_count[sk], 0) : 0;
+      const int rows = rows_in_group(na, G, rg);
+      c = rows > 0 ? max(union_count[sk], 0) : 0;
+      vc = c > 0 ? c + segment_pad(rows) : 0;
     }
-    int inc = c;
+    int inc = c, vinc = vc;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
       const int t = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += t;
+      const int vt = __shfl_up_sync(0xffffffffu, vinc, o);
+      if (lane >= o) { inc += t; vinc += vt; }
     }
-    if (seg < n_seg) pre[seg] = run + inc - c;
+    if (seg < n_seg) {
+      pre[seg] = run + inc - c;
+      if (vpre) vpre[seg] = vrun + vinc - vc;
+    }
     run += __shfl_sync(0xffffffffu, inc, 31);
+    vrun += __shfl_sync(0xffffffffu, vinc, 31);
   }
-  if (lane == 0) pre[n_seg] = run;
+  if (lane == 0) {
+    pre[n_seg] = run;
+    if (vpre) vpre[n_seg] = vrun;
+  }
 }
 
 #endif  // __CUDACC__

@@ -300,7 +300,9 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
     if (tok < 0 || tok >= p.B) { set_status(p.status, LOSA_ERR_BOUNDS); continue; }
     const size_t orow = (static_cast<size_t>(s) * p.B + tok) * p.Hq + kh * p.G + gi;
     float acc[C], M, Lsum;
-    merge_records<D, LOG2>(p, sg, r, pre[sg], pre[sg + 1], pre[p.n_seg], lane, acc, M, Lsum);
+    // (PRE: the prefix left by the tensor-core kernel is that of the charged list; a segment's pages follow its pad)
+    const int pad = (PRE && pre[sg + 1] > pre[sg]) ? segment_pad(rows) : 0;
+    merge_records<D, LOG2>(p, sg, r, pre[sg] + pad, pre[sg + 1], pre[p.n_seg], lane, acc, M, Lsum);
     const bool empty = !(Lsum > 0.f);
     const float inv = empty ? 0.f : 1.f / Lsum;
 #pragma unroll
@@ -370,7 +372,9 @@ __global__ void __launch_bounds__(kFinishThreads) attn_finish_kernel(AttnParams 
     const int rowk = slot * p.G + gi, rg = rowk / kRowsPerGroup, r = rowk % kRowsPerGroup;
     const int sg = rg * (p.n_seg / p.n_rg) + s * p.Hkv + kh;
     float acc[C], M, Lsum;
-    merge_records<D, true>(p, sg, r, p.seg_prefix[sg], p.seg_prefix[sg + 1], p.seg_prefix[p.n_seg], lane, acc, M, Lsum);
+    const int v0 = p.seg_prefix[sg], v1 = p.seg_prefix[sg + 1];      // of the charged list: the segment's pages follow its pad
+    const int pad = v1 > v0 ? segment_pad(rows_in_group(clamp_active(p.n_active[s], p.B), p.G, rg)) : 0;
+    merge_records<D, true>(p, sg, r, v0 + pad, v1, p.seg_prefix[p.n_seg], lane, acc, M, Lsum);
     const bool empty = !(Lsum > 0.f);
     const float inv = empty ? 0.f : 1.f / Lsum;
     Lp = empty ? -INFINITY : (M + log2f(Lsum)) * kLn2;

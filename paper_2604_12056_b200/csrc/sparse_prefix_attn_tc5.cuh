@@ -30,7 +30,7 @@ constexpr int kTc5MetaRing = 16;                 // groups whose per-page token 
 constexpr float kTc5Tau = 8.0f;                  // reference maximum moves only when it would grow by more than this (log2 units)
 constexpr int kTc5XchgBytes = (2 * 2 + 1) * kRowsPerGroup * 4;   // row maxima [group parity][set][row], row sums [row]
 constexpr int kTc5ScaleBytes = 2 * kTc5MetaRing * (kTc5PgMax + 1) * 4;   // FP8 pages: per-page scales and page counts of the groups in flight, K and V
-constexpr int kTc5TailBytes = kTailBytes + 512 + kTc5XchgBytes + kTc5ScaleBytes;  // 1024 bytes of barriers + page meta, the segment prefix and index cache, the exchange arrays, the scales
+constexpr int kTc5TailBytes = kTailBytes + 512 + kTc5XchgBytes + kTc5ScaleBytes + (kMaxSegments + 1) * 4;  // 1024 bytes of barriers + page meta, the segment prefix and index cache, the exchange arrays, the scales
 constexpr int kTc5Stg = 2;                       // FP8 pages: staging slots (bytes as they lie in memory) per tensor
 
 template <int D> constexpr int tc5_slot_bytes() { return kTc5Tok * D * 2; }
@@ -163,6 +163,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   float* xsum = xmax + 4 * kRowsPerGroup;                        // [128]
   volatile float* scale_meta = xsum + kRowsPerGroup;             // FP8: [2 (K, V)][kTc5MetaRing][kTc5PgMax] page scales,
   volatile int* ng_meta = reinterpret_cast<volatile int*>(const_cast<float*>(scale_meta) + 2 * kTc5MetaRing * kTc5PgMax);   // [2][kTc5MetaRing] pages per group
+  int* vpre = const_cast<int*>(ng_meta) + 2 * kTc5MetaRing;       // prefix of the charged segment lengths (pages + pad)
   const bool staged = p.N * p.B <= kStageIdx && p.N <= kStageSeq;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -199,7 +200,7 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   grid_dep_trigger();
   grid_dep_wait();                                 // nothing above touches global memory
   if (warp == 0) {
-    segment_prefix(pre, p.n_seg, p.n_rg, p.Hkv, p.G, p.n_active, p.union_count, p.B, lane);
+    segment_prefix(pre, p.n_seg, p.n_rg, p.Hkv, p.G, p.n_active, p.union_count, p.B, lane, vpre);
   } else if (staged) {
     for (int i = tid - 32; i < p.N * p.B; i += kTc5Threads - 32) tok_s[i] = p.active_idx[i];
     for (int i = tid - 32; i < p.N; i += kTc5Threads - 32) {
@@ -212,10 +213,22 @@ attn_tc5_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__
   tc5_fence_after();
   const uint32_t tmem = *tmem_slot;
   if (blockIdx.x == 0)                             // the combine kernel reads the prefix instead of recomputing it
-    for (int i = tid; i <= p.n_seg; i += kTc5Threads) p.seg_prefix[i] = pre[i];
-  const long long T_all = pre[p.n_seg];
-  const int lo = static_cast<int>(cta_lo(T_all, blockIdx.x, p.n_ctas));
-  const int hi = static_cast<int>(cta_lo(T_all, blockIdx.x + 1, p.n_ctas));
+    for (int i = tid; i <= p.n_seg; i += kTc5Threads) p.seg_prefix[i] = vpre[i];
+  // this CTA's share of the charged list, mapped back to pages: the first page at or after a charged position
+  const long long V_all = vpre[p.n_seg];
+  auto page_at = [&](long long v) {
+    if (v >= V_all) return pre[p.n_seg];
+    int a = 0, b = p.n_seg;                          // vpre[a] <= v < vpre[b]
+    while (b - a > 1) {
+      const int mid = (a + b) >> 1;
+      if (vpre[mid] <= v) a = mid; else b = mid;
+    }
+    const int len = pre[a + 1] - pre[a], pad = vpre[a + 1] - vpre[a] - len;
+    const int off = static_cast<int>(v - vpre[a]) - pad;
+    return pre[a] + (off < 0 ? 0 : off);
+  };
+  const int lo = page_at(cta_lo(V_all, blockIdx.x, p.n_ctas));
+  const int hi = page_at(cta_lo(V_all, blockIdx.x + 1, p.n_ctas));
   if (lo >= hi) {                                  // nothing to do: give the tensor memory back
     if (warp == 0) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "n"(TMEM_COLS) : "memory");
     return;
