@@ -314,7 +314,7 @@ int32_t losa_denoise_step(losa_ctx* ctx, const void* q, const void* k_blk, const
   int32_t* slot_map = reinterpret_cast<int32_t*>(ctx->ws + ctx->lay.slot_map);
   rc = launch_select_active(ctx, q, state->q_prev, sh.n_q_heads * sh.head_dim, m_per_seq, state->step,
                             buf->active_idx, buf->n_active, nullptr, st, 0.0, slot_map);
-  if (rc == LOSA_OK) rc = launch_page_scores_topk(ctx, q, kv, buf->active_idx, buf->n_active, state->step, k, buf->topk_pages, nullptr, st, ctx->pooled_selection != 0 ? kSelectorPooled : kSelectorExact);
+  if (rc == LOSA_OK) rc = launch_page_scores_topk(ctx, q, kv, buf->active_idx, buf->n_active, state->step, k, buf->topk_pages, nullptr, st, ctx->pooled_selection != 0 ? kSelectorPooled : kSelectorExact, true);
   if (rc == LOSA_OK) rc = launch_page_union(ctx, buf->topk_pages, buf->active_idx, buf->n_active, k, kv->kv_len, state->step, buf->union_pages, buf->union_count, st);
   if (rc == LOSA_OK) rc = launch_sparse_prefix_attn(ctx, q, kv, buf->active_idx, buf->n_active, buf->union_pages, buf->union_count, state, st, true);
   // join (also when a launch above failed: the forked kernel must not be left reading the caller's

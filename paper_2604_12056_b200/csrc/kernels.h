@@ -13,7 +13,8 @@ int32_t launch_select_active(losa_ctx* c, const void* x_cur, const void* x_prev,
 int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
                                 const int32_t* active_idx, const int32_t* n_active,
                                 const int32_t* step, int32_t k, int32_t* topk_pages,
-                                float* topk_scores_opt, cudaStream_t st, int selector = 0);
+                                float* topk_scores_opt, cudaStream_t st, int selector = 0, bool after_stage1 = false);
+// after_stage1: the kernel launched just before on `st` is stage 1 of the same step (see launch_page_bounds)
 // selector: 0 = one exact list per query head, 1 = pooled over the heads of a KV head, 2 = tensor-core scores (relaxed rule, bf16)
 constexpr int kSelectorExact = 0, kSelectorPooled = 1, kSelectorMma = 2;
 
@@ -25,7 +26,11 @@ int32_t launch_page_scores(losa_ctx* c, const void* q, const losa_kv_t* kv, cons
 // the selection that evaluates the exact score of the surviving candidates only.
 // With approx_only the tensor-core value itself is written as an fp32 score row (relaxed selector).
 int32_t launch_page_bounds(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
-                           const int32_t* n_active, const int32_t* step, cudaStream_t st, bool approx_only = false);
+                           const int32_t* n_active, const int32_t* step, cudaStream_t st, bool approx_only = false,
+                           bool after_stage1 = false);
+// after_stage1: the previous kernel on `st` is stage 1 of the same step, which releases its dependents only
+// after everything before it has completed: the kernel then takes its work list and first copies (kv_len,
+// step, page table, summaries - nothing stage 1 writes) before stage 1 ends.
 
 int32_t launch_page_union(losa_ctx* c, const int32_t* topk_pages, const int32_t* active_idx,
                           const int32_t* n_active, int32_t k, const int32_t* kv_len,

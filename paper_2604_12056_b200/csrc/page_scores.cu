@@ -70,6 +70,7 @@ struct PsParams {
   float* scores;
   int32_t* status;
   int N, B, Hq, Hkv, G, g, Pmax, n_phys, score_stride, n_ctas, n_stages;
+  int early;   // the kernel before this one in the stream is stage 1 of the same step: the list and the first copies may be taken before it ends
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -136,21 +137,22 @@ struct TileWalk {
 // (sequence, KV head, page) list, and the active lists of the first kPsSeqStage sequences of that
 // range into tok_s.  Returns false when the range is empty.  The caller synchronises the CTA before
 // reading tok_s.
-__device__ __forceinline__ bool ps_prologue(const PsParams& p, int* pre, int* na_s, int* tok_s, int& lo, int& hi, int& s_lo) {
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+// The work list: pages of every sequence that is past its first step, whatever its number of
+// active tokens (a sequence without any is walked without arithmetic), so that the list - and the
+// first copies - depend on nothing stage 1 writes.  Reads bypass L1 (they may run beside the
+// previous kernel).
+__device__ __forceinline__ bool ps_list(const PsParams& p, int* pre, int& lo, int& hi, int& s_lo) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (warp == 0) {
     int run = 0;
     for (int b0 = 0; b0 < p.N; b0 += 32) {
       const int s = b0 + lane;
-      int c = 0, na = 0;
+      int c = 0;
       if (s < p.N) {
-        na = p.n_active[s];
-        na = na < 0 ? 0 : (na > p.B ? p.B : na);
-        const bool first_step = p.step && p.step[s] == 0;
-        int P = pages_of(p.kv_len[s], p.g);
+        const bool first_step = p.step && __ldcg(p.step + s) == 0;
+        int P = pages_of(__ldcg(p.kv_len + s), p.g);
         if (P > p.Pmax) { set_status(p.status, LOSA_ERR_BOUNDS); P = p.Pmax; }   // a length beyond the page-table row
-        c = (first_step || na == 0 || P < 0) ? 0 : P;
-        na_s[s] = na;
+        c = (first_step || P < 0) ? 0 : P;
       }
       int inc = c;
 #pragma unroll
@@ -170,11 +172,19 @@ __device__ __forceinline__ bool ps_prologue(const PsParams& p, int* pre, int* na
   if (lo >= hi) return false;
   s_lo = 0;
   while (static_cast<long long>(p.Hkv) * pre[s_lo + 1] <= lo) ++s_lo;
-  for (int i = tid; i < kPsSeqStage * p.B; i += blockDim.x) {
+  return true;
+}
+// What stage 1 wrote: the clamped numbers of active tokens, and the active lists of the first few
+// sequences of this CTA's range (the caller synchronises the CTA afterwards).
+__device__ __forceinline__ void ps_active(const PsParams& p, int* na_s, int* tok_s, int s_lo) {
+  for (int s = threadIdx.x; s < p.N; s += blockDim.x) {
+    const int na = p.n_active[s];
+    na_s[s] = na < 0 ? 0 : (na > p.B ? p.B : na);
+  }
+  for (int i = threadIdx.x; i < kPsSeqStage * p.B; i += blockDim.x) {
     const int s = s_lo + i / p.B;
     tok_s[i] = s < p.N ? p.active_idx[s * p.B + i % p.B] : -1;
   }
-  return true;
 }
 
 template <typename T, int D, int PG>
@@ -196,7 +206,8 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_scores_stream_kernel(PsPar
   grid_dep_trigger();
   grid_dep_wait();
   int lo, hi, s_lo;
-  if (!ps_prologue(p, pre, na_s, tok_s, lo, hi, s_lo)) return;      // whole CTA: nothing in its range
+  if (!ps_list(p, pre, lo, hi, s_lo)) return;                        // whole CTA: nothing in its range
+  ps_active(p, na_s, tok_s, s_lo);
   // block position of active slot a of sequence s
   auto token_of = [&](int s, int a) {
     int tok = (s >= s_lo && s < s_lo + kPsSeqStage) ? tok_s[(s - s_lo) * p.B + a] : p.active_idx[s * p.B + a];
@@ -530,6 +541,7 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_scores_stream_kernel(PsPar
 constexpr float kMmaErrCoef = 1.0f / 8192.0f;
 constexpr int kMmaWP = 16;                          // pages per warp and tile
 constexpr int kMmaTP = kPsWarps * kMmaWP;           // pages per tile
+constexpr int kMmaStages = 2;                       // tiles in shared memory: two leave room for the CTAs of the in-block attention, which runs beside
 
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                uint32_t b0, uint32_t b1) {
@@ -574,9 +586,13 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_bounds_mma_kernel(PsParams
   int* tok_s = na_s + p.N;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   grid_dep_trigger();
-  grid_dep_wait();
-  int lo, hi, s_lo;
-  if (!ps_prologue(p, pre, na_s, tok_s, lo, hi, s_lo)) return;
+  // When the previous kernel of the stream is known to be stage 1 of this step (whole-step path), the
+  // work list, the page-table entries and the first tiles of summaries are taken while it still
+  // runs: none of them is written by it, and it released this kernel only after everything before
+  // it had completed.  Otherwise wait first.
+  if (!p.early) grid_dep_wait();
+  int lo = 0, hi = 0, s_lo = 0;
+  const bool any = ps_list(p, pre, lo, hi, s_lo);
   auto token_of = [&](int s, int a) {
     int tok = (s >= s_lo && s < s_lo + kPsSeqStage) ? tok_s[(s - s_lo) * p.B + a] : p.active_idx[s * p.B + a];
     if (tok < 0 || tok >= p.B) { set_status(p.status, LOSA_ERR_BOUNDS); tok = 0; }
@@ -597,7 +613,7 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_bounds_mma_kernel(PsParams
     if (w_ids.next()) {
       const int pl = warp * WP + lane;
       if (lane < WP && pl < w_ids.np) {
-        id = __ldg(p.page_table + static_cast<size_t>(w_ids.s) * p.Pmax + w_ids.p0 + pl);
+        id = __ldcg(p.page_table + static_cast<size_t>(w_ids.s) * p.Pmax + w_ids.p0 + pl);
         if (id < 0 || id >= p.n_phys) { set_status(p.status, LOSA_ERR_BOUNDS); id = 0; }
       }
     }
@@ -623,12 +639,18 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_bounds_mma_kernel(PsParams
     }
     cp_async_commit();
   };
-  int id_next = request_id();
-  for (int i = 0; i < NS - 1; ++i) {
-    const int id = id_next;
+  int id_next = 0;
+  if (any) {
     id_next = request_id();
-    copy_tile(id, i);
+    for (int i = 0; i < NS - 1; ++i) {
+      const int id = id_next;
+      id_next = request_id();
+      copy_tile(id, i);
+    }
   }
+  if (p.early) grid_dep_wait();                      // every CTA, also one without work: the next kernel counts on it
+  if (!any) return;
+  ps_active(p, na_s, tok_s, s_lo);
   __syncthreads();                                   // the cached active lists are in place
 
   // rows r0 .. r0 + nr - 1 of (sequence s, KV head kh) as [q+ | q-] into the staging tile; the rows
@@ -766,7 +788,7 @@ int32_t launch_bounds_t(losa_ctx* c, const PsParams& pp, cudaStream_t st) {
   PsParams p = pp;
   const int tail = ps_tail_bytes(p.N);
   int ns = (kPsSmemBudget - C::QBUF_BYTES - tail - 128) / C::STAGE_BYTES;
-  ns = ns > kPsMaxStages ? kPsMaxStages : ns;
+  ns = ns > kMmaStages ? kMmaStages : ns;
   if (ns < 2) return LOSA_ERR_UNSUPPORTED;
   p.n_stages = ns;
   const int smem = 128 + ns * C::STAGE_BYTES + C::QBUF_BYTES + tail;
@@ -804,6 +826,7 @@ PsParams make_params(losa_ctx* c, const void* q, const losa_kv_t* kv, const int3
   p.score_stride = c->lay.score_stride;
   p.n_ctas = c->n_sms;
   p.n_stages = 0;
+  p.early = 0;
   return p;
 }
 
@@ -811,8 +834,9 @@ PsParams make_params(losa_ctx* c, const void* q, const losa_kv_t* kv, const int3
 
 // bf16 only: (lower, upper) bound pairs of the page scores into the workspace's score rows (as float2)
 int32_t launch_page_bounds(losa_ctx* c, const void* q, const losa_kv_t* kv, const int32_t* active_idx,
-                           const int32_t* n_active, const int32_t* step, cudaStream_t st, bool approx_only) {
-  const PsParams p = make_params(c, q, kv, active_idx, n_active, step);
+                           const int32_t* n_active, const int32_t* step, cudaStream_t st, bool approx_only, bool after_stage1) {
+  PsParams p = make_params(c, q, kv, active_idx, n_active, step);
+  p.early = after_stage1 ? 1 : 0;
   if (approx_only) return c->shape.head_dim == 128 ? launch_bounds_t<128, true>(c, p, st) : launch_bounds_t<64, true>(c, p, st);
   return c->shape.head_dim == 128 ? launch_bounds_t<128, false>(c, p, st) : launch_bounds_t<64, false>(c, p, st);
 }

@@ -694,7 +694,7 @@ int32_t topk_max_sortable(const losa_ctx* c) {
 int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
                                 const int32_t* active_idx, const int32_t* n_active,
                                 const int32_t* step, int32_t k, int32_t* topk_pages,
-                                float* topk_scores_opt, cudaStream_t st, int selector) {
+                                float* topk_scores_opt, cudaStream_t st, int selector, bool after_stage1) {
   const losa_shape_t& sh = c->shape;
   if (sh.max_pages_per_seq == 0) return LOSA_OK;
   const bool pooled = selector == kSelectorPooled;
@@ -702,7 +702,7 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
   const bool bf = sh.dtype == LOSA_BF16;
   if (bf && selector == kSelectorExact && k <= kSelCap) {
     // bf16, one list per query head: bounds from the tensor cores, exact scores for the candidates only
-    int32_t rc = launch_page_bounds(c, q, kv, active_idx, n_active, step, st);
+    int32_t rc = launch_page_bounds(c, q, kv, active_idx, n_active, step, st, false, after_stage1);
     if (rc != LOSA_OK) return rc;
     RefineParams rp;
     rp.bounds = reinterpret_cast<float2*>(c->ws + c->lay.scores);

@@ -21,8 +21,11 @@ select_active_kernel(const T* __restrict__ x_cur, const T* __restrict__ x_prev, 
                      int32_t* __restrict__ active_idx, int32_t* __restrict__ n_active,
                      float* __restrict__ delta_opt, double* __restrict__ delta_ws,
                      unsigned int* __restrict__ counters, double tau, int32_t* __restrict__ slot_map) {
-  grid_dep_trigger();
+  // Wait first, release afterwards: a kernel released by this one may read, before its own wait, what
+  // earlier kernels of the stream wrote (the cache's lengths, summaries and step counters), so those
+  // must have completed by then.
   grid_dep_wait();
+  grid_dep_trigger();
   const int i = blockIdx.x, s = blockIdx.y;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const size_t row = (static_cast<size_t>(s) * B + i) * row_width;
