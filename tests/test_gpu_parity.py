@@ -229,6 +229,17 @@ def test_paper_shaped_workloads_reduced(name):
     run_blocks(wl.config(name, kv_lens=(4096 + 77,), steps=4), modes=("losa", "naive", "dense"))
 
 
+def test_more_segments_than_ctas_and_very_short_segments():
+    # 24 sequences x 8 KV heads = 192 (sequence, KV head) segments for the 148 CTAs of the bf16
+    # stage-4 kernel, most of them a page or two long (shorter than the pad the work list charges per
+    # segment), some empty: CTAs whose share holds no page at all, CTAs that cross several segments
+    lens = tuple(0 if i in (3, 17) else 1 + (13 * i) % 90 for i in range(24))
+    cfg = wl.config("c2", n_q_heads=16, n_kv_heads=8, head_dim=64, page_size=16, kv_lens=lens,
+                    block_size=8, steps=3, topk=2, m_active=2)
+    run_blocks(cfg, modes=("losa", "dense"))
+    run_blocks(cfg, modes=("losa",), fused=True, want_scores=False)
+
+
 @pytest.mark.parametrize("m", [0, 1, 16])
 def test_active_count_extremes(m):
     cfg = wl.config("c2", kv_lens=(700, 333), block_size=16, steps=3, topk=4, m_active=max(m, 1))
