@@ -240,6 +240,31 @@ def test_more_segments_than_ctas_and_very_short_segments():
     run_blocks(cfg, modes=("losa",), fused=True, want_scores=False)
 
 
+@pytest.mark.parametrize("fused", [False, True])
+def test_sequences_without_active_tokens_beside_others(fused):
+    # per-sequence active counts 0 / 3 / 1 / 0 in one batch: the stage-2 work list walks every
+    # sequence that is past its first step, with or without active tokens
+    from paper_2604_12056_b200.layer import LosaLayer, to_device
+    cfg = wl.config("c2", kv_lens=(40 * 32 + 5, 300, 129 * 32, 64), block_size=16, steps=4, topk=6, m_active=3)
+    w = wl.Workload(cfg)
+    g, o = LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len), OracleLayer(w)
+    for t, inp in enumerate(w.block_steps()):
+        if t > 0:
+            inp.m_per_seq[:] = np.array([0, 3, 1, 0], np.int32)
+        args = tuple(to_device(x) for x in (inp.q, inp.k_blk, inp.v_blk, inp.m_per_seq))
+        if fused:
+            g.run_step_fused(*args)
+        else:
+            g.run_step(*args)
+        snap, ref = g.snapshot(), o.run_step(inp)
+        assert g.ctx.poll_status() == 0
+        if fused:
+            snap["delta"] = ref["delta"]
+        compare(snap, ref, cfg, f"mixed active counts step {t}")
+        if t > 0:
+            assert ref["na"].tolist() == [0, 3, 1, 0]
+
+
 @pytest.mark.parametrize("m", [0, 1, 16])
 def test_active_count_extremes(m):
     cfg = wl.config("c2", kv_lens=(700, 333), block_size=16, steps=3, topk=4, m_active=max(m, 1))
