@@ -382,6 +382,32 @@ void oracle_fp8_append_block(const oracle_shape_t* sh, const int32_t* page_table
   free(tmp);
 }
 
+/* ---------- bf16 state (extension of the cached statistics' format) ----------
+ * The paper quotes the per-block cache in FP16 (memory overhead, Section 4.5); the interface keeps it in
+ * fp32 by default.  With the bf16 state the cached prefix output o_p of a token is STORED rounded to
+ * bf16 - eight significant bits, ties to even, subnormals below 2^-126 on the 2^-133 grid - and every
+ * later use (the merge of the same step, the reuse in later steps) sees the rounded value; L_p stays as
+ * it is.  oracle_round_state_bf16 rounds, in place, the rows stage 4 has just written: those of the
+ * active tokens. */
+double oracle_round_bf16(double x) {
+  if (x == 0.0 || !(x == x) || isinf(x)) return x;
+  int ex;
+  (void)frexp(fabs(x), &ex);                              /* 2^(ex-1) <= |x| < 2^ex */
+  int e = ex - 1;
+  if (e < -126) e = -126;                                 /* subnormal range: fixed step 2^-133 */
+  const double r = nearbyint(ldexp(x, 7 - e));            /* |x| / 2^(e-7) in [128, 256): ties to even */
+  return ldexp(r, e - 7);                                 /* (256 * 2^(e-7) = 2^(e+1): the next binade, still exact) */
+}
+void oracle_round_state_bf16(const oracle_shape_t* sh, double* o_p, const int32_t* active_idx,
+                             const int32_t* n_active) {
+  const int B = sh->block_size, H = sh->n_q_heads, d = sh->head_dim;
+  for (int s = 0; s < sh->batch; ++s)
+    for (int a = 0; a < n_active[s]; ++a) {
+      double* row = o_p + ((int64_t)s * B + active_idx[(int64_t)s * B + a]) * H * d;
+      for (int64_t i = 0; i < (int64_t)H * d; ++i) row[i] = oracle_round_bf16(row[i]);
+    }
+}
+
 /* ---------- Section 2.3: relaxed validity of a page list (selector variants with their own arithmetic) ----------
  * The paper fixes no arithmetic for the page bound, and calls the method independent of the
  * selector.  A selector that evaluates U(p) = sum_j max(q_j kmin_j, q_j kmax_j) in another order

@@ -83,6 +83,12 @@ void oracle_fp8_append_block(const oracle_shape_t* sh, const int32_t* page_table
                              uint8_t* k_codes, uint8_t* v_codes, float* k_scale, float* v_scale,
                              const void* k_blk, const void* v_blk);
 
+/* bf16 state (extension; Section 4.5 quotes the cache in FP16): o_p is stored rounded to bf16 (ties to
+ * even), L_p unchanged.  Rounds the rows of the active tokens in place. */
+double oracle_round_bf16(double x);
+void oracle_round_state_bf16(const oracle_shape_t* sh, double* o_p, const int32_t* active_idx,
+                             const int32_t* n_active);
+
 /* Relaxed validity of page lists produced with another arithmetic than the fixed fp32 order: number of
  * (active token, head) lists that are not "min(k, P) distinct in-range pages, each with fp64 bound >=
  * the k-th largest fp64 bound - eps * (largest sum of term magnitudes)", then -1 padding. */

@@ -250,6 +250,21 @@ def fp8_append_block(sh: Shape, page_table, kv_len, k_codes, v_codes, k_scale, v
                                   _p(_chk(k_blk, sh.elem, "k_blk")), _p(_chk(v_blk, sh.elem, "v_blk")))
 
 
+def round_bf16(x) -> np.ndarray:
+    """Element-wise rounding to bf16 (ties to even) of float64 values, as float64."""
+    lib().oracle_round_bf16.restype = C.c_double
+    lib().oracle_round_bf16.argtypes = [C.c_double]
+    v = np.asarray(x, np.float64)
+    return np.array([lib().oracle_round_bf16(float(t)) for t in v.ravel()], np.float64).reshape(v.shape)
+
+
+def round_state_bf16(sh: Shape, o_p, active_idx, n_active):
+    """bf16 state: rounds the rows of the active tokens of o_p (float64 [N, B, H_q, d]) in place."""
+    s = sh.c()
+    lib().oracle_round_state_bf16(C.byref(s), _p(_chk(o_p, np.float64, "o_p")), _p(_chk(active_idx, np.int32, "active_idx")),
+                                  _p(_chk(n_active, np.int32, "n_active")))
+
+
 def page_union(sh: Shape, topk_pages, active_idx, n_active, k: int, kv_len, step=None):
     """Returns (union_pages [N,H_kv,P_max] int32, union_count [N,H_kv] int32)."""
     N, Hkv, P = sh.batch, sh.n_kv_heads, sh.max_pages_per_seq
