@@ -109,11 +109,17 @@ typedef struct {
 
 /* Per-block LoSA cache (Section 4.3 / "Memory overhead" in Section 4.5): B(d+1) scalars per head
  * and sequence, plus the previous step's queries and a step counter. Host struct, device pointers. */
+#define LOSA_STATE_F32  0
+#define LOSA_STATE_BF16 1
 typedef struct {
   void*    q_prev;  /* [N, B, H_q, d] queries of the previous step (dtype)                       */
-  float*   o_p;     /* [N, B, H_q, d] cached prefix attention output                             */
-  float*   lse_p;   /* [N, B, H_q]    cached prefix log-normaliser L_p                            */
+  void*    o_p;     /* [N, B, H_q, d] cached prefix attention output: fp32, or bf16 (o_p_format)  */
+  float*   lse_p;   /* [N, B, H_q]    cached prefix log-normaliser L_p (fp32)                     */
   int32_t* step;    /* [N] denoising steps done for the current block; 0 = no valid cache        */
+  int32_t  o_p_format;  /* LOSA_STATE_F32 (0, the default) or LOSA_STATE_BF16: o_p is STORED rounded to
+                           bf16 (ties to even) and every use - the merge of the same step, the reuse in
+                           later steps - sees the stored value (the paper quotes this cache in FP16,
+                           Section 4.5); bf16 contexts only                                       */
 } losa_state_t;
 
 typedef struct losa_ctx losa_ctx;

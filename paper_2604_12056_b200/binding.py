@@ -55,7 +55,8 @@ class KvT(C.Structure):
 
 
 class StateT(C.Structure):
-    _fields_ = [("q_prev", C.c_void_p), ("o_p", C.c_void_p), ("lse_p", C.c_void_p), ("step", C.c_void_p)]
+    _fields_ = [("q_prev", C.c_void_p), ("o_p", C.c_void_p), ("lse_p", C.c_void_p), ("step", C.c_void_p),
+                ("o_p_format", C.c_int32)]
 
 
 class StepBuffersT(C.Structure):
@@ -119,8 +120,14 @@ def make_kv(k_pages, v_pages, kmin, kmax, page_table, kv_len, k_scale=None, v_sc
     return kv
 
 
+LOSA_STATE_F32, LOSA_STATE_BF16 = 0, 1
+
+
 def make_state(q_prev, o_p, lse_p, step) -> StateT:
-    st = StateT(q_prev.data_ptr(), o_p.data_ptr(), lse_p.data_ptr(), step.data_ptr())
+    """o_p: float32, or bfloat16 for the bf16 state (stored rounded; bf16 contexts only)."""
+    import torch
+    fmt = LOSA_STATE_BF16 if o_p.dtype == torch.bfloat16 else LOSA_STATE_F32
+    st = StateT(q_prev.data_ptr(), o_p.data_ptr(), lse_p.data_ptr(), step.data_ptr(), fmt)
     st._keep = (q_prev, o_p, lse_p, step)
     return st
 

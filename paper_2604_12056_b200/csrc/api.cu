@@ -62,6 +62,13 @@ int current_sm_count() {
   return 148;
 }
 
+// The cached prefix output is fp32, or - in bf16 contexts - stored rounded to bf16.
+int32_t check_state_format(const losa_ctx* c, const losa_state_t* st) {
+  if (st->o_p_format != LOSA_STATE_F32 && st->o_p_format != LOSA_STATE_BF16) return LOSA_ERR_INVALID_ARG;
+  if (st->o_p_format == LOSA_STATE_BF16 && c->shape.dtype != LOSA_BF16) return LOSA_ERR_UNSUPPORTED;
+  return LOSA_OK;
+}
+
 int32_t check_kv(const losa_ctx* c, const losa_kv_t* kv, bool need_summaries) {
   if (!kv || !kv->k_pages || !kv->v_pages || !kv->page_table || !kv->kv_len) return LOSA_ERR_INVALID_ARG;
   if (need_summaries && (!kv->kmin || !kv->kmax)) return LOSA_ERR_INVALID_ARG;
@@ -239,6 +246,7 @@ int32_t losa_sparse_prefix_attn(losa_ctx* ctx, const void* q, const losa_kv_t* k
   if (!ctx || !q || !active_idx || !n_active || !union_pages || !union_count || !state || !state->o_p || !state->lse_p)
     return LOSA_ERR_INVALID_ARG;
   int32_t rc = check_kv(ctx, kv, false);
+  if (rc == LOSA_OK) rc = check_state_format(ctx, state);
   if (rc != LOSA_OK) return rc;
   if (!aligned16(q) || !aligned16(state->o_p)) return LOSA_ERR_UNSUPPORTED;
   return launch_sparse_prefix_attn(ctx, q, kv, active_idx, n_active, union_pages, union_count, state, as_stream(stream));
@@ -247,7 +255,9 @@ int32_t losa_sparse_prefix_attn(losa_ctx* ctx, const void* q, const losa_kv_t* k
 int32_t losa_block_attn_merge(losa_ctx* ctx, const void* q, const void* k_blk, const void* v_blk,
                               const losa_state_t* state, void* out, float* lse_out_opt, void* stream) {
   if (!ctx || !q || !k_blk || !v_blk || !state || !state->o_p || !state->lse_p || !out) return LOSA_ERR_INVALID_ARG;
-  if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out)) return LOSA_ERR_UNSUPPORTED;
+  const int32_t rc = check_state_format(ctx, state);
+  if (rc != LOSA_OK) return rc;
+  if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out) || !aligned16(state->o_p)) return LOSA_ERR_UNSUPPORTED;
   return launch_block_attn_merge(ctx, q, k_blk, v_blk, state, out, lse_out_opt, as_stream(stream));
 }
 
@@ -291,6 +301,7 @@ int32_t losa_denoise_step(losa_ctx* ctx, const void* q, const void* k_blk, const
   if (!buf->active_idx || !buf->n_active || !buf->topk_pages || !buf->union_pages || !buf->union_count)
     return LOSA_ERR_INVALID_ARG;
   int32_t rc = check_kv(ctx, kv, true);
+  if (rc == LOSA_OK) rc = check_state_format(ctx, state);
   if (rc != LOSA_OK) return rc;
   if (!aligned16(q) || !aligned16(k_blk) || !aligned16(v_blk) || !aligned16(out) || !aligned16(state->q_prev) ||
       !aligned16(state->o_p))

@@ -182,7 +182,7 @@ constexpr int kMmaThreads = 128;
 template <int D, int BK, bool MERGE>
 __global__ void __launch_bounds__(kMmaThreads)
 block_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ k_blk,
-                      const __nv_bfloat16* __restrict__ v_blk, const float* __restrict__ o_p,
+                      const __nv_bfloat16* __restrict__ v_blk, const void* __restrict__ o_p, int o_p_bf16,
                       const float* __restrict__ lse_p, __nv_bfloat16* __restrict__ out, float* __restrict__ lse_out,
                       float* __restrict__ ob_out, int B, int Hq, int Hkv, float sm_scale) {
   grid_dep_wait();
@@ -300,7 +300,9 @@ block_attn_mma_kernel(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* 
       const float wp = expf(Lp - L), wb = expf(Lb - L) / l;
 #pragma unroll
       for (int jn = 0; jn < NO; ++jn) {
-        const float2 pv = *reinterpret_cast<const float2*>(o_p + gr * D + 8 * jn + 2 * t4);
+        float2 pv;                                   // the cached prefix output as it is stored (fp32 or bf16)
+        if (o_p_bf16) pv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(static_cast<const __nv_bfloat16*>(o_p) + gr * D + 8 * jn + 2 * t4));
+        else pv = *reinterpret_cast<const float2*>(static_cast<const float*>(o_p) + gr * D + 8 * jn + 2 * t4);
         const float x = (wp > 0.f ? wp * pv.x : 0.f) + wb * o[jn][e0];
         const float y = (wp > 0.f ? wp * pv.y : 0.f) + wb * o[jn][e0 + 1];
         *reinterpret_cast<__nv_bfloat162*>(out + gr * D + 8 * jn + 2 * t4) = __floats2bfloat162_rn(x, y);
@@ -462,7 +464,7 @@ int32_t launch_merge_t(losa_ctx* c, const void* q, const void* k_blk, const void
   dim3 grid((sh.block_size + kTokTile - 1) / kTokTile, sh.n_kv_heads, sh.batch);
   launch_k(block_attn_merge_kernel<T, D, MERGE>, grid, kBaThreads, smem, st, 
       static_cast<const T*>(q), static_cast<const T*>(k_blk), static_cast<const T*>(v_blk),
-      state ? state->o_p : nullptr, state ? state->lse_p : nullptr, static_cast<T*>(out), lse_out, ob_out,
+      state ? static_cast<const float*>(state->o_p) : nullptr, state ? state->lse_p : nullptr, static_cast<T*>(out), lse_out, ob_out,
       sh.block_size, sh.n_q_heads, sh.n_kv_heads, sh.sm_scale);
   return after_launch(c);
 }
@@ -474,7 +476,7 @@ int32_t launch_merge_commit_t(losa_ctx* c, const void* q, losa_state_t* state, v
   const size_t n_rows = static_cast<size_t>(sh.batch) * sh.block_size * sh.n_q_heads;
   const int blocks = static_cast<int>((n_rows + kThreads / 32 - 1) / (kThreads / 32));
   launch_k(merge_commit_kernel<T, D>, blocks, kThreads, 0, st, 
-      static_cast<const T*>(q), static_cast<T*>(state->q_prev), state->o_p, state->lse_p,
+      static_cast<const T*>(q), static_cast<T*>(state->q_prev), static_cast<const float*>(state->o_p), state->lse_p,
       reinterpret_cast<const float*>(c->ws + c->lay.block_o), reinterpret_cast<const float*>(c->ws + c->lay.block_lse),
       static_cast<T*>(out), lse_out, state->step, sh.batch, n_rows);
   return after_launch(c);
@@ -534,7 +536,8 @@ int32_t launch_block_attn_mma(losa_ctx* c, const void* q, const void* k_blk, con
   dim3 grid((rows + kMmaRows - 1) / kMmaRows, sh.n_kv_heads, sh.batch);
   launch_k(block_attn_mma_kernel<D, BK, MERGE>, grid, kMmaThreads, 0, st,
       static_cast<const __nv_bfloat16*>(q), static_cast<const __nv_bfloat16*>(k_blk),
-      static_cast<const __nv_bfloat16*>(v_blk), state ? state->o_p : nullptr, state ? state->lse_p : nullptr,
+      static_cast<const __nv_bfloat16*>(v_blk), state ? state->o_p : nullptr,
+      (state && state->o_p_format == LOSA_STATE_BF16) ? 1 : 0, state ? state->lse_p : nullptr,
       static_cast<__nv_bfloat16*>(out), lb, ob, sh.block_size, sh.n_q_heads, sh.n_kv_heads, sh.sm_scale);
   return after_launch(c);
 }

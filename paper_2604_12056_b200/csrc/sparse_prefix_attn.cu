@@ -40,7 +40,8 @@ struct AttnParams {
   const int32_t* union_count;
   float* partials;
   int32_t* seg_prefix;  // workspace copy of the segment prefix (written by the bf16 main kernel, read by its combine kernel)
-  float* o_p;
+  void* o_p;                // cached prefix output, fp32 or bf16 (o_p_bf16)
+  int o_p_bf16;
   float* lse_p;
   int32_t* status;
   const float* k_scale;   // FP8 pages: [n_phys, H_kv] power-of-two scales (else null)
@@ -85,6 +86,32 @@ template <int C> __device__ __forceinline__ void st_bf16(__nv_bfloat16* p, const
     r.bits = *reinterpret_cast<uint32_t*>(&a);
   }
   st_raw<C>(p, r);
+}
+
+// C elements of the cached prefix output (fp32 or bf16 storage) at element offset i
+template <int C> __device__ __forceinline__ void ld_state(const void* base, int bf16, size_t i, float (&v)[C]) {
+  if (bf16) {
+    const RawRow<C> r = ld_raw<C>(static_cast<const __nv_bfloat16*>(base) + i);
+    if constexpr (C == 4) {
+      v[0] = __uint_as_float(r.bits.x << 16); v[1] = __uint_as_float(r.bits.x & 0xffff0000u);
+      v[2] = __uint_as_float(r.bits.y << 16); v[3] = __uint_as_float(r.bits.y & 0xffff0000u);
+    } else {
+      v[0] = __uint_as_float(r.bits << 16); v[1] = __uint_as_float(r.bits & 0xffff0000u);
+    }
+  } else {
+    ldv<C>(static_cast<const float*>(base) + i, v);
+  }
+}
+// ... stored; with bf16 storage v comes back holding the stored (rounded) values, which is what every
+// later use must see
+template <int C> __device__ __forceinline__ void st_state(void* base, int bf16, size_t i, float (&v)[C]) {
+  if (bf16) {
+#pragma unroll
+    for (int c = 0; c < C; ++c) v[c] = __bfloat162float(__float2bfloat16_rn(v[c]));
+    st_bf16<C>(static_cast<__nv_bfloat16*>(base) + i, v);
+  } else {
+    stv<C>(static_cast<float*>(base) + i, v);
+  }
 }
 
 // ===================================================================== fp32 / CUDA-core kernel
@@ -307,7 +334,7 @@ __global__ void __launch_bounds__(256) attn_combine_kernel(AttnParams p) {
     const float inv = empty ? 0.f : 1.f / Lsum;
 #pragma unroll
     for (int c = 0; c < C; ++c) acc[c] *= inv;
-    stv<C>(p.o_p + orow * D + lane * C, acc);
+    st_state<C>(p.o_p, p.o_p_bf16, orow * D + lane * C, acc);
     if (lane == 0) p.lse_p[orow] = empty ? -INFINITY : (LOG2 ? (M + log2f(Lsum)) * kLn2 : M + logf(Lsum));
   }
 }
@@ -353,7 +380,7 @@ __global__ void __launch_bounds__(kFinishThreads) attn_finish_kernel(AttnParams 
   // the cached prefix statistics as well: nine rows in ten are stable, and asking now saves them
   // a second round trip (an active row overwrites these below)
   float a[C], Lp;
-  ldv<C>(p.o_p + row * D + lane * C, a);
+  ld_state<C>(p.o_p, p.o_p_bf16, row * D + lane * C, a);
   Lp = p.lse_p[row];
   // the row's slot in the active list, if any (the list has at most B <= 64 entries)
   int slot = -1;
@@ -380,7 +407,7 @@ __global__ void __launch_bounds__(kFinishThreads) attn_finish_kernel(AttnParams 
     Lp = empty ? -INFINITY : (M + log2f(Lsum)) * kLn2;
 #pragma unroll
     for (int c = 0; c < C; ++c) a[c] = acc[c] * inv;
-    stv<C>(p.o_p + row * D + lane * C, a);
+    st_state<C>(p.o_p, p.o_p_bf16, row * D + lane * C, a);
     if (lane == 0) p.lse_p[row] = Lp;
   }
   const float Mx = fmaxf(Lp, Lb);
@@ -579,6 +606,7 @@ int32_t launch_sparse_prefix_attn(losa_ctx* c, const void* q, const losa_kv_t* k
   ap.partials = reinterpret_cast<float*>(c->ws + c->lay.partials);
   ap.seg_prefix = reinterpret_cast<int32_t*>(c->ws + c->lay.seg_prefix);
   ap.o_p = state->o_p;
+  ap.o_p_bf16 = state->o_p_format == LOSA_STATE_BF16 ? 1 : 0;
   ap.lse_p = state->lse_p;
   ap.status = status_ptr(c);
   const bool fp8 = kv->kv_format == LOSA_KV_FP8_E4M3;
@@ -612,6 +640,7 @@ int32_t launch_attn_finish(losa_ctx* c, const void* q, const int32_t* active_idx
   ap.partials = reinterpret_cast<float*>(c->ws + c->lay.partials);
   ap.seg_prefix = reinterpret_cast<int32_t*>(c->ws + c->lay.seg_prefix);
   ap.o_p = state->o_p;
+  ap.o_p_bf16 = state->o_p_format == LOSA_STATE_BF16 ? 1 : 0;
   ap.lse_p = state->lse_p;
   ap.status = status_ptr(c);
   ap.N = sh.batch;

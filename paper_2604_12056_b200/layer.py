@@ -34,7 +34,7 @@ class LosaLayer:
 
     def __init__(self, cfg, k_pages, v_pages, page_table, kv_len, mode="losa", device="cuda",
                  share_pool_with: "LosaLayer | None" = None, tau: float = 0.0, pooled: bool = False,
-                 mma_selector: bool = False, fp8_kv: bool = False):
+                 mma_selector: bool = False, fp8_kv: bool = False, state_bf16: bool = False):
         self.cfg, self.mode, self.device = cfg, mode, device
         self.tau = tau            # > 0: stage 1 keeps tokens until their Delta reach tau of the block's total
         self.pooled = pooled      # stage 2 keeps one page list per (token, KV head) instead of one per query head
@@ -74,7 +74,8 @@ class LosaLayer:
             self.kv = B.make_kv(self.k_codes, self.v_codes, self.kmin, self.kmax, self.page_table, self.kv_len,
                                 self.k_scale, self.v_scale)
         self.q_prev = torch.zeros((N, Bk, Hq, d), dtype=td, device=device)
-        self.o_p = torch.zeros((N, Bk, Hq, d), dtype=torch.float32, device=device)
+        # cached prefix output: fp32, or stored rounded to bf16 (bf16 contexts only)
+        self.o_p = torch.zeros((N, Bk, Hq, d), dtype=torch.bfloat16 if state_bf16 else torch.float32, device=device)
         self.lse_p = torch.zeros((N, Bk, Hq), dtype=torch.float32, device=device)
         self.step = torch.zeros(N, dtype=torch.int32, device=device)
         self.zero_step = torch.zeros(N, dtype=torch.int32, device=device)
@@ -138,6 +139,6 @@ class LosaLayer:
         """Host copies of every intermediate of the last step."""
         return dict(act=to_host(self.active_idx), na=to_host(self.n_active), delta=to_host(self.delta),
                     topk=to_host(self.topk_pages), topk_scores=to_host(self.topk_scores),
-                    up=to_host(self.union_pages), uc=to_host(self.union_count), o_p=to_host(self.o_p),
+                    up=to_host(self.union_pages), uc=to_host(self.union_count), o_p=to_host(self.o_p.float()),
                     lse_p=to_host(self.lse_p), out=to_host(self.out), lse=to_host(self.lse_out),
                     step=to_host(self.step), kv_len=to_host(self.kv_len))

@@ -104,9 +104,10 @@ class OracleLayer:
     attention applied to the whole block, Section 5.1 baselines); "dense": step counter pinned to
     0, i.e. dense prefix attention every step."""
 
-    def __init__(self, w, mode="losa", tau=0.0, pooled=False):
+    def __init__(self, w, mode="losa", tau=0.0, pooled=False, state_bf16=False):
         self.tau = tau
         self.pooled = pooled
+        self.state_bf16 = state_bf16      # the cached prefix output is stored rounded to bf16
         cfg = w.cfg
         self.w, self.cfg, self.mode = w, cfg, mode
         self.sh = oracle_shape_of(cfg)
@@ -140,6 +141,8 @@ class OracleLayer:
         scores_topk(sh, inp.q, self.kv, act, na, cfg.topk, step, topk_pages=self.topk)
         up, uc = orc.page_union(sh, self.topk, act, na, cfg.topk, self.kv_len, step)
         orc.sparse_prefix_attn(sh, inp.q, self.kv, act, na, up, uc, self.o_p, self.lse_p)
+        if self.state_bf16:
+            orc.round_state_bf16(sh, self.o_p, act, na)
         out, lse = orc.block_attn_merge(sh, inp.q, inp.k_blk, inp.v_blk, self.o_p, self.lse_p)
         res = dict(act=act, na=na, delta=delta, topk=self.topk.copy(), up=up, uc=uc,
                    o_p=self.o_p.copy(), lse_p=self.lse_p.copy(), out=out, lse=lse,

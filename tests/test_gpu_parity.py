@@ -48,12 +48,13 @@ def compare(snap, ref, cfg, what, tau=0.0):
 
 
 def run_blocks(cfg, modes=("losa",), m=None, n_blocks=1, pad_nan=True, want_scores=True, fused=False, tau=0.0,
-               pooled=False):
+               pooled=False, state_bf16=False):
     """Runs n_blocks blocks through GPU and oracle in lock-step, comparing after every step."""
     from paper_2604_12056_b200.layer import LosaLayer, to_device
     w = wl.Workload(cfg, pad_nan=pad_nan)
-    gpu = {md: LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len, md, tau=tau, pooled=pooled) for md in modes}
-    ora = {md: OracleLayer(w, md, tau=tau, pooled=pooled) for md in modes}
+    gpu = {md: LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len, md, tau=tau, pooled=pooled,
+                         state_bf16=state_bf16) for md in modes}
+    ora = {md: OracleLayer(w, md, tau=tau, pooled=pooled, state_bf16=state_bf16) for md in modes}
     for md in modes:     # page summaries: exact min / max on both sides
         from paper_2604_12056_b200.layer import to_host
         P = [(int(L) + cfg.page_size - 1) // cfg.page_size for L in w.kv_len]
@@ -263,6 +264,29 @@ def test_sequences_without_active_tokens_beside_others(fused):
         compare(snap, ref, cfg, f"mixed active counts step {t}")
         if t > 0:
             assert ref["na"].tolist() == [0, 3, 1, 0]
+
+
+@pytest.mark.parametrize("fused", [False, True])
+def test_state_stored_in_bf16(fused):
+    # the cached prefix output stored rounded to bf16: the oracle rounds the rows stage 4 writes, and
+    # the merge of the same step and the reuse in later steps see the rounded values on both sides
+    cfg = wl.config("c2", kv_lens=(33 * 32 + 7, 500), block_size=16, steps=4, topk=6, m_active=3, n_blocks=2)
+    gpu, _ = run_blocks(cfg, modes=("losa",) if fused else ("losa", "dense"), n_blocks=2, fused=fused, want_scores=False,
+                        state_bf16=True)
+    import torch
+    assert gpu["losa"].o_p.dtype == torch.bfloat16
+
+
+def test_bf16_state_needs_a_bf16_context():
+    from paper_2604_12056_b200 import binding as B
+    from paper_2604_12056_b200.layer import LosaLayer, to_device
+    cfg = wl.config("c1")
+    w = wl.Workload(cfg)
+    g = LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len, state_bf16=True)
+    inp = w.start_block()
+    with pytest.raises(B.LosaError) as e:
+        g.run_step(*(to_device(x) for x in (inp.q, inp.k_blk, inp.v_blk, inp.m_per_seq)))
+    assert e.value.code == B.LOSA_ERR_UNSUPPORTED
 
 
 @pytest.mark.parametrize("m", [0, 1, 16])
