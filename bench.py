@@ -68,6 +68,8 @@ def parse_args():
                     help="selector variant: one page list per (token, KV head) instead of one per query head")
     ap.add_argument("--layers", type=int, default=0, help="attention layers (default: 36 for c5, else 1)")
     ap.add_argument("--active-frac", type=float, default=None, help="override the active fraction")
+    ap.add_argument("--selector", default="exact", choices=["exact", "mma"],
+                    help="mma: stage 2 takes its page scores from a tensor-core GEMM; lists valid under the relaxed rule")
     ap.add_argument("--state-dtype", default="f32", choices=["f32", "bf16"],
                     help="bf16: the cached prefix output of the per-block state is stored rounded to bf16")
     ap.add_argument("--kv-dtype", default="native", choices=["native", "fp8"],
@@ -244,13 +246,13 @@ class LayerRun:
     """One attention layer of the workload on the device: its own seeded pool, LoSA cache, static
     input buffers and two CUDA graphs (the whole-step call; block finalisation)."""
 
-    def __init__(self, cfg, rank, layer, dev, pooled=False, fp8=False, state_bf16=False):
+    def __init__(self, cfg, rank, layer, dev, pooled=False, fp8=False, state_bf16=False, mma=False):
         import torch
         from paper_2604_12056_b200.layer import LosaLayer
         self.torch, self.cfg = torch, cfg
         self.w = wl.DeviceWorkload(cfg, replica=rank, layer=layer, device=dev)
         self.layer = LosaLayer(cfg, self.w.k_pages, self.w.v_pages, self.w.page_table, self.w.kv_len, "losa", dev,
-                               pooled=pooled, fp8_kv=fp8, state_bf16=state_bf16)
+                               pooled=pooled, fp8_kv=fp8, state_bf16=state_bf16, mma_selector=mma)
         self.pool_mib = self.w.k_pages.numel() * (2 if fp8 else 4) / 2 ** 20
         if fp8:                                # the library has quantised the pools: release the bf16 copies
             torch.cuda.synchronize()
@@ -341,8 +343,8 @@ def run_ours(args, cfg0):
     total_blocks = warm_blocks + 4 * blocks_region + 3
     cfg = wl.config(cfg0.name, n_blocks=total_blocks, m_active=cfg0.m_active, beta_active=cfg0.beta_active, topk=cfg0.topk)
     fp8 = args.kv_dtype == "fp8"
-    runs = [LayerRun(cfg, D.replica_of(rank), l, dev, pooled=args.pooled, fp8=fp8, state_bf16=args.state_dtype == "bf16")
-            for l in range(L)]
+    runs = [LayerRun(cfg, D.replica_of(rank), l, dev, pooled=args.pooled, fp8=fp8, state_bf16=args.state_dtype == "bf16",
+                     mma=args.selector == "mma") for l in range(L)]
     launches_step = launches_fin = 0
     for r in runs:
         launches_step, launches_fin = r.capture()
@@ -436,7 +438,8 @@ def run_ours(args, cfg0):
         "vs_baseline": None, "dtype": cfg.dtype, "data": "synthetic",
         "config": {"workload": workload_name(cfg0, L_model) + (", pooled selector (one page list per token and KV head)" if args.pooled else "")
                                + (", K/V pages stored as FP8 E4M3 with per-page scales" if fp8 else "")
-                               + (", cached prefix output stored as bf16" if args.state_dtype == "bf16" else ""),
+                               + (", cached prefix output stored as bf16" if args.state_dtype == "bf16" else "")
+                               + (", tensor-core page scores (relaxed list rule)" if args.selector == "mma" else ""),
                    "sequences_per_gpu": cfg.batch, "layers": L_model, "layers_timed": L,
                    "step": "one layer-step = stages 1-6 for one layer and one denoising step; steps run in model order "
                            "(block, denoising step, layer) from a block boundary; the last step of a block also appends the block to the cache",

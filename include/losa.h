@@ -271,6 +271,18 @@ int32_t losa_page_scores_topk_mma(losa_ctx* ctx, const void* q, const losa_kv_t*
  *   issued after it returns. */
 int32_t losa_set_pooled_selection(losa_ctx* ctx, int32_t on);
 
+/* Selector of stage 2 inside losa_denoise_step / losa_denoise_step_host, by name:
+ *   LOSA_SELECTOR_EXACT  one list per query head in the fixed fp32 order (losa_page_scores_topk; default)
+ *   LOSA_SELECTOR_POOLED one list per KV head (losa_page_scores_topk_pooled; the same as
+ *                        losa_set_pooled_selection(ctx, 1))
+ *   LOSA_SELECTOR_MMA    page scores as a GEMM on the tensor cores, lists valid under the relaxed rule
+ *                        (losa_page_scores_topk_mma; bf16 contexts, else LOSA_ERR_UNSUPPORTED)
+ * Host-only; LOSA_ERR_INVALID_ARG for another value. */
+#define LOSA_SELECTOR_EXACT  0
+#define LOSA_SELECTOR_POOLED 1
+#define LOSA_SELECTOR_MMA    2
+int32_t losa_set_step_selector(losa_ctx* ctx, int32_t selector);
+
 /* Stage 3 — union of the selections (Section 4.2, Section 4.4).
  *   union_pages [N, H_kv, P_max] int32 out: for each sequence and KV head, the distinct logical
  *       pages selected by any active token through any of the G query heads of that KV head,

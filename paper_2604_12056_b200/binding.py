@@ -30,7 +30,7 @@ EXPORTS = [
     "losa_update_prefix_cache", "losa_build_page_summaries", "losa_denoise_step_host",
     "losa_profile_stage4", "losa_stage4_last_ms", "losa_select_active_static",
     "losa_denoise_step", "losa_select_active_tau", "losa_page_scores_topk_pooled",
-    "losa_set_pooled_selection", "losa_set_wait_limit", "losa_page_scores_topk_mma", "losa_quantize_kv_pages",
+    "losa_set_pooled_selection", "losa_set_step_selector", "losa_set_wait_limit", "losa_page_scores_topk_mma", "losa_quantize_kv_pages",
 ]
 
 
@@ -170,6 +170,10 @@ class Context:
 
     def launch_count(self) -> int:
         return int(lib().losa_launch_count(self._h))
+
+    def set_step_selector(self, selector: int):
+        """0 = exact per-head lists, 1 = pooled per KV head, 2 = tensor-core scores (relaxed list rule)."""
+        self._check("losa_set_step_selector", lib().losa_set_step_selector(self._h, C.c_int32(selector)))
 
     def set_pooled_selection(self, on: bool):
         self._check("losa_set_pooled_selection", lib().losa_set_pooled_selection(self._h, C.c_int32(1 if on else 0)))

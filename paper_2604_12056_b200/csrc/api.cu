@@ -232,6 +232,15 @@ int32_t losa_set_pooled_selection(losa_ctx* ctx, int32_t on) {
   return LOSA_OK;
 }
 
+int32_t losa_set_step_selector(losa_ctx* ctx, int32_t selector) {
+  if (!ctx) return LOSA_ERR_INVALID_ARG;
+  if (selector != LOSA_SELECTOR_EXACT && selector != LOSA_SELECTOR_POOLED && selector != LOSA_SELECTOR_MMA)
+    return LOSA_ERR_INVALID_ARG;
+  if (selector == LOSA_SELECTOR_MMA && ctx->shape.dtype != LOSA_BF16) return LOSA_ERR_UNSUPPORTED;
+  ctx->pooled_selection = selector;                  // the codes are those of launch_page_scores_topk
+  return LOSA_OK;
+}
+
 int32_t losa_page_union(losa_ctx* ctx, const int32_t* topk_pages, const int32_t* active_idx,
                         const int32_t* n_active, int32_t k, const int32_t* kv_len, const int32_t* step,
                         int32_t* union_pages, int32_t* union_count, void* stream) {
@@ -325,7 +334,7 @@ int32_t losa_denoise_step(losa_ctx* ctx, const void* q, const void* k_blk, const
   int32_t* slot_map = reinterpret_cast<int32_t*>(ctx->ws + ctx->lay.slot_map);
   rc = launch_select_active(ctx, q, state->q_prev, sh.n_q_heads * sh.head_dim, m_per_seq, state->step,
                             buf->active_idx, buf->n_active, nullptr, st, 0.0, slot_map);
-  if (rc == LOSA_OK) rc = launch_page_scores_topk(ctx, q, kv, buf->active_idx, buf->n_active, state->step, k, buf->topk_pages, nullptr, st, ctx->pooled_selection != 0 ? kSelectorPooled : kSelectorExact, true);
+  if (rc == LOSA_OK) rc = launch_page_scores_topk(ctx, q, kv, buf->active_idx, buf->n_active, state->step, k, buf->topk_pages, nullptr, st, ctx->pooled_selection, true);
   if (rc == LOSA_OK) rc = launch_page_union(ctx, buf->topk_pages, buf->active_idx, buf->n_active, k, kv->kv_len, state->step, buf->union_pages, buf->union_count, st);
   if (rc == LOSA_OK) rc = launch_sparse_prefix_attn(ctx, q, kv, buf->active_idx, buf->n_active, buf->union_pages, buf->union_count, state, st, true);
   // join (also when a launch above failed: the forked kernel must not be left reading the caller's

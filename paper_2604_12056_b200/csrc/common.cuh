@@ -58,7 +58,8 @@ struct losa_ctx {
   // second stream and fork/join events of the whole-step path (created on first use)
   cudaStream_t side_stream;
   cudaEvent_t ev_fork, ev_join;
-  // selector of the whole-step path: 0 = one list per query head, 1 = pooled over the heads of a KV head
+  // selector of the whole-step path: 0 = one list per query head, 1 = pooled over the heads of a KV head,
+  // 2 = tensor-core scores under the relaxed list rule (the codes of launch_page_scores_topk)
   int32_t pooled_selection;
   // bound of the mbarrier waits of the bf16 stage-4 kernel in SM clock cycles (0 = the default, about a second)
   int64_t wait_cycles;

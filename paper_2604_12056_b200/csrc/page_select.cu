@@ -724,7 +724,7 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
     else launch_k(topk_refine_kernel<64>, queries, kSelThreads, 0, st, rp);
     return after_launch(c);
   }
-  int32_t rc = selector == kSelectorMma ? launch_page_bounds(c, q, kv, active_idx, n_active, step, st, true)
+  int32_t rc = selector == kSelectorMma ? launch_page_bounds(c, q, kv, active_idx, n_active, step, st, true, after_stage1)
                                         : launch_page_scores(c, q, kv, active_idx, n_active, step, st);
   if (rc != LOSA_OK) return rc;
 

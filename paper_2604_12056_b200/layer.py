@@ -46,6 +46,8 @@ class LosaLayer:
         self.ctx = B.Context(N, Hq, Hkv, d, Bk, cfg.page_size, Pmax, self.dtype, cfg.sm_scale, device)
         if pooled:
             self.ctx.set_pooled_selection(True)
+        if mma_selector and self.dtype == B.LOSA_BF16:
+            self.ctx.set_step_selector(2)              # the whole-step call takes the tensor-core selector as well
         if share_pool_with is not None:
             o = share_pool_with
             self.k_pages, self.v_pages, self.kmin, self.kmax = o.k_pages, o.v_pages, o.kmin, o.kmax

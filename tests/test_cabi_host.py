@@ -90,6 +90,7 @@ def test_null_arguments_are_rejected_without_a_device(lib):
         assert getattr(lib, fn)(*args) == B.LOSA_ERR_INVALID_ARG, fn
     assert lib.losa_set_pooled_selection(None, C.c_int32(1)) == B.LOSA_ERR_INVALID_ARG
     assert lib.losa_set_wait_limit(None, C.c_int64(5)) == B.LOSA_ERR_INVALID_ARG
+    assert lib.losa_set_step_selector(None, C.c_int32(2)) == B.LOSA_ERR_INVALID_ARG
     args = [None] * 11
     args[3], args[4] = C.c_int32(64), C.c_double(0.5)
     assert lib.losa_select_active_tau(*args) == B.LOSA_ERR_INVALID_ARG

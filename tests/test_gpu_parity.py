@@ -172,7 +172,8 @@ def test_long_lists_and_large_budgets(pages, topk, pooled):
          m_active=3),
     dict(kv_lens=(150,), block_size=8, steps=3, topk=64, m_active=2),
 ])
-def test_tensor_core_selector_under_the_relaxed_list_rule(kw):
+@pytest.mark.parametrize("fused", [False, True])
+def test_tensor_core_selector_under_the_relaxed_list_rule(kw, fused):
     """losa_page_scores_topk_mma: page scores as a GEMM on the tensor cores.  Its lists are checked
     against the relaxed validity rule (fp64 scores, slack 2^-11 of the largest term magnitude sum);
     everything downstream is compared as usual, the oracle taking the GPU's own lists: the union
@@ -186,7 +187,11 @@ def test_tensor_core_selector_under_the_relaxed_list_rule(kw):
     sh, k = o.sh, cfg.topk
     same = total = 0
     for t, inp in enumerate(w.block_steps()):
-        g.run_step(to_device(inp.q), to_device(inp.k_blk), to_device(inp.v_blk), to_device(inp.m_per_seq))
+        args = (to_device(inp.q), to_device(inp.k_blk), to_device(inp.v_blk), to_device(inp.m_per_seq))
+        if fused:                                  # the whole-step call with losa_set_step_selector(ctx, LOSA_SELECTOR_MMA)
+            g.run_step_fused(*args)
+        else:
+            g.run_step(*args)
         snap = g.snapshot()
         assert g.ctx.poll_status() == 0
         act, na, _ = orc.select_active(sh, inp.q, o.q_prev, inp.m_per_seq, o.step)
