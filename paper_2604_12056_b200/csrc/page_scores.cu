@@ -55,7 +55,7 @@ struct PsCfg {
 
 constexpr int ps_tail_bytes(int n_seq) {
   // prefix [n_seq + 1] | active counts [n_seq] | cached active lists
-  return 16 + 4 * (n_seq + 1) + 4 * n_seq + 4 * kPsSeqStage * LOSA_MAX_BLOCK;
+  return 16 + 4 * (n_seq + 1) + 4 * n_seq + 4 * kPsSeqStage * LOSA_MAX_BLOCK + 4 * n_seq;   // ... | pages per sequence
 }
 
 struct PsParams {
@@ -131,6 +131,31 @@ struct TileWalk {
   }
 };
 
+// The same walk over a list that counts TILES: a (sequence, KV head) with P pages has nt = ceil(P / TP)
+// tiles of ceil(P / nt) pages each (the last one shorter), so every CTA gets whole tiles and the
+// CTAs differ by at most one tile - a tile costs about the same whatever it holds (a chain of
+// dependent latencies), and a range cut in the middle of tiles has one or two more of them.
+struct TileWalkEven {
+  const int* pre;     // shared: exclusive prefix of the sequences' tile counts per KV head
+  const int* pages;   // shared: pages per sequence
+  int Hkv, TP, hi;
+  int cur, s;
+  int kh, p0, np;     // the current tile
+  __device__ __forceinline__ void init(const int* pre_, const int* pages_, int Hkv_, int TP_, int lo, int hi_) {
+    pre = pre_; pages = pages_; Hkv = Hkv_; TP = TP_; hi = hi_; cur = lo - 1; s = 0; np = 0;
+  }
+  __device__ __forceinline__ bool next() {
+    if (++cur >= hi) return false;
+    while (static_cast<long long>(Hkv) * pre[s + 1] <= cur) ++s;
+    const int nt = pre[s + 1] - pre[s], off = cur - Hkv * pre[s], P = pages[s];
+    kh = off / nt;
+    const int ts = (P + nt - 1) / nt;
+    p0 = (off % nt) * ts;
+    np = min(ts, P - p0);
+    return true;
+  }
+};
+
 // Common prologue of the page-score kernels (all threads of the CTA): the number of pages to score
 // per sequence (none on a first step, none without active tokens) and its exclusive prefix into
 // pre[0 .. N], the clamped active counts into na_s, this CTA's range [lo, hi) of the flat
@@ -141,7 +166,10 @@ struct TileWalk {
 // active tokens (a sequence without any is walked without arithmetic), so that the list - and the
 // first copies - depend on nothing stage 1 writes.  Reads bypass L1 (they may run beside the
 // previous kernel).
-__device__ __forceinline__ bool ps_list(const PsParams& p, int* pre, int& lo, int& hi, int& s_lo) {
+// tile_pages > 0: the list counts tiles of at most that many pages (TileWalkEven) and pages_s
+// receives the page count of every sequence.
+__device__ __forceinline__ bool ps_list(const PsParams& p, int* pre, int& lo, int& hi, int& s_lo, int tile_pages = 0,
+                                        int* pages_s = nullptr) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   if (warp == 0) {
     int run = 0;
@@ -153,6 +181,8 @@ __device__ __forceinline__ bool ps_list(const PsParams& p, int* pre, int& lo, in
         int P = pages_of(__ldcg(p.kv_len + s), p.g);
         if (P > p.Pmax) { set_status(p.status, LOSA_ERR_BOUNDS); P = p.Pmax; }   // a length beyond the page-table row
         c = (first_step || P < 0) ? 0 : P;
+        if (pages_s) pages_s[s] = c;
+        if (tile_pages > 0) c = (c + tile_pages - 1) / tile_pages;
       }
       int inc = c;
 #pragma unroll
@@ -584,6 +614,7 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_bounds_mma_kernel(PsParams
   int* pre = reinterpret_cast<int*>(qbuf + C::QBUF_BYTES);
   int* na_s = pre + p.N + 1;
   int* tok_s = na_s + p.N;
+  int* pages_s = tok_s + kPsSeqStage * LOSA_MAX_BLOCK;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   grid_dep_trigger();
   // When the previous kernel of the stream is known to be stage 1 of this step (whole-step path), the
@@ -592,7 +623,7 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_bounds_mma_kernel(PsParams
   // it had completed.  Otherwise wait first.
   if (!p.early) grid_dep_wait();
   int lo = 0, hi = 0, s_lo = 0;
-  const bool any = ps_list(p, pre, lo, hi, s_lo);
+  const bool any = ps_list(p, pre, lo, hi, s_lo, TP, pages_s);
   auto token_of = [&](int s, int a) {
     int tok = (s >= s_lo && s < s_lo + kPsSeqStage) ? tok_s[(s - s_lo) * p.B + a] : p.active_idx[s * p.B + a];
     if (tok < 0 || tok >= p.B) { set_status(p.status, LOSA_ERR_BOUNDS); tok = 0; }
@@ -604,10 +635,10 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_bounds_mma_kernel(PsParams
   float2* bounds = reinterpret_cast<float2*>(p.scores);
   const uint32_t warp_off = static_cast<uint32_t>(warp) * WP * C::ROW_BYTES;
 
-  TileWalk w_ids, w_copy, w;
-  w_ids.init(pre, p.Hkv, TP, lo, hi);
-  w_copy.init(pre, p.Hkv, TP, lo, hi);
-  w.init(pre, p.Hkv, TP, lo, hi);
+  TileWalkEven w_ids, w_copy, w;
+  w_ids.init(pre, pages_s, p.Hkv, TP, lo, hi);
+  w_copy.init(pre, pages_s, p.Hkv, TP, lo, hi);
+  w.init(pre, pages_s, p.Hkv, TP, lo, hi);
   auto request_id = [&]() {
     int id = 0;
     if (w_ids.next()) {
@@ -682,8 +713,8 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_bounds_mma_kernel(PsParams
     staged_r0 = r0;
   };
   {
-    TileWalk first;
-    first.init(pre, p.Hkv, TP, lo, hi);
+    TileWalkEven first;
+    first.init(pre, pages_s, p.Hkv, TP, lo, hi);
     if (first.next()) ensure_rows(first.s, first.kh, 0, min(kPsRowTile, na_s[first.s] * p.G));
   }
 
