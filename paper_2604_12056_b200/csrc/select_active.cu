@@ -27,6 +27,9 @@ select_active_kernel(const T* __restrict__ x_cur, const T* __restrict__ x_prev, 
   grid_dep_wait();
   grid_dep_trigger();
   const int i = blockIdx.x, s = blockIdx.y;
+  // what the sequence's last CTA needs at the very end: asked for now, so that it is not one more round trip there
+  const int m_given = m_per_seq ? m_per_seq[s] : -1;
+  const int step_now = step ? step[s] : 1;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const size_t row = (static_cast<size_t>(s) * B + i) * row_width;
   constexpr int kVec = 8;
@@ -84,8 +87,8 @@ select_active_kernel(const T* __restrict__ x_cur, const T* __restrict__ x_prev, 
   __syncthreads();
   if (warp != 0) return;
 
-  int m = m_per_seq ? m_per_seq[s] : -1;
-  const bool first_step = step && step[s] == 0;
+  int m = m_given;
+  const bool first_step = step_now == 0;
   if (m < 0 || m > B || first_step) m = B;
   // token t = lane (+32): rank under (Delta descending, token ascending)
   int rank[2] = {B, B};
