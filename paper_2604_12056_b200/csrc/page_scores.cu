@@ -71,6 +71,7 @@ struct PsParams {
   int32_t* status;
   int N, B, Hq, Hkv, G, g, Pmax, n_phys, score_stride, n_ctas, n_stages;
   int early;   // the kernel before this one in the stream is stage 1 of the same step: the list and the first copies may be taken before it ends
+  int tile_pages;   // tensor-core bounds kernel: pages per tile of this launch (16 .. 128, chosen on the host)
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
@@ -604,7 +605,7 @@ template <int D, bool APPROX>
 __global__ void __launch_bounds__(kPsThreads, 1) page_bounds_mma_kernel(PsParams p) {
   using C = MmaCfg<D>;
   using T = __nv_bfloat16;
-  constexpr int WP = kMmaWP, TP = kMmaTP;
+  constexpr int WP = kMmaWP;                         // (a tile holds p.tile_pages <= kMmaTP pages)
   extern __shared__ uint8_t ps_smem[];
   const uint32_t raw = smem_u32(ps_smem);
   const uint32_t base = (raw + 127u) & ~127u;
@@ -623,7 +624,8 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_bounds_mma_kernel(PsParams
   // it had completed.  Otherwise wait first.
   if (!p.early) grid_dep_wait();
   int lo = 0, hi = 0, s_lo = 0;
-  const bool any = ps_list(p, pre, lo, hi, s_lo, TP, pages_s);
+  const int tile = p.tile_pages;                     // at most TP
+  const bool any = ps_list(p, pre, lo, hi, s_lo, tile, pages_s);
   auto token_of = [&](int s, int a) {
     int tok = (s >= s_lo && s < s_lo + kPsSeqStage) ? tok_s[(s - s_lo) * p.B + a] : p.active_idx[s * p.B + a];
     if (tok < 0 || tok >= p.B) { set_status(p.status, LOSA_ERR_BOUNDS); tok = 0; }
@@ -636,9 +638,9 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_bounds_mma_kernel(PsParams
   const uint32_t warp_off = static_cast<uint32_t>(warp) * WP * C::ROW_BYTES;
 
   TileWalkEven w_ids, w_copy, w;
-  w_ids.init(pre, pages_s, p.Hkv, TP, lo, hi);
-  w_copy.init(pre, pages_s, p.Hkv, TP, lo, hi);
-  w.init(pre, pages_s, p.Hkv, TP, lo, hi);
+  w_ids.init(pre, pages_s, p.Hkv, tile, lo, hi);
+  w_copy.init(pre, pages_s, p.Hkv, tile, lo, hi);
+  w.init(pre, pages_s, p.Hkv, tile, lo, hi);
   auto request_id = [&]() {
     int id = 0;
     if (w_ids.next()) {
@@ -714,7 +716,7 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_bounds_mma_kernel(PsParams
   };
   {
     TileWalkEven first;
-    first.init(pre, pages_s, p.Hkv, TP, lo, hi);
+    first.init(pre, pages_s, p.Hkv, tile, lo, hi);
     if (first.next()) ensure_rows(first.s, first.kh, 0, min(kPsRowTile, na_s[first.s] * p.G));
   }
 
@@ -858,6 +860,7 @@ PsParams make_params(losa_ctx* c, const void* q, const losa_kv_t* kv, const int3
   p.n_ctas = c->n_sms;
   p.n_stages = 0;
   p.early = 0;
+  p.tile_pages = 0;
   return p;
 }
 
@@ -868,6 +871,20 @@ int32_t launch_page_bounds(losa_ctx* c, const void* q, const losa_kv_t* kv, cons
                            const int32_t* n_active, const int32_t* step, cudaStream_t st, bool approx_only, bool after_stage1) {
   PsParams p = make_params(c, q, kv, active_idx, n_active, step);
   p.early = after_stage1 ? 1 : 0;
+  // Pages per tile: a tile costs a fixed part plus a part per page (about 0.8 us + 2 us per 128 pages),
+  // and the kernel lasts as many tiles as its busiest CTA gets; of the sizes 16, 32 .. 128 the one that
+  // makes (rounds) x (cost of a tile) least, on the assumption that every prefix has its longest
+  // length (the real lengths live on the device): short prefixes get small tiles so that every CTA has one.
+  {
+    const losa_shape_t& sh = c->shape;
+    float best = 3.0e38f;
+    for (int tp = kMmaTP; tp >= 16; tp -= 16) {
+      const long long tiles = static_cast<long long>(sh.batch) * sh.n_kv_heads * ((sh.max_pages_per_seq + tp - 1) / tp);
+      const long long rounds = (tiles + p.n_ctas - 1) / p.n_ctas;
+      const float cost = static_cast<float>(rounds) * (0.8f + 2.0f * static_cast<float>(tp) / 128.f);
+      if (cost < best) { best = cost; p.tile_pages = tp; }
+    }
+  }
   if (approx_only) return c->shape.head_dim == 128 ? launch_bounds_t<128, true>(c, p, st) : launch_bounds_t<64, true>(c, p, st);
   return c->shape.head_dim == 128 ? launch_bounds_t<128, false>(c, p, st) : launch_bounds_t<64, false>(c, p, st);
 }
