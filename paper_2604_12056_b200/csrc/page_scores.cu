@@ -562,7 +562,10 @@ __global__ void __launch_bounds__(kPsThreads, 1) page_scores_stream_kernel(PsPar
 // every page whose upper bound reaches the k-th largest lower bound - a superset of the exact
 // top-k, ties included - and evaluates U in the fixed order for those few pages only.
 //
-// Same persistent streaming structure as the kernel above (one CTA per SM, per-warp cp.async ring).
+// Same persistent streaming structure as the kernel above (one CTA per SM, per-warp cp.async ring),
+// but its work list counts whole tiles: a (sequence, KV head) with P pages is cut into
+// ceil(P / tile) tiles of equal size, tile <= 128 pages chosen per launch (see launch_page_bounds),
+// because a tile costs this kernel about the same whatever it holds.
 // A warp's slice of a tile is 16 pages = two 8-page MMA tiles; query rows are staged per
 // (sequence, KV head) as bf16 rows [q+ | q-].  The contraction index is free to permute: lane
 // (g = lane / 4, t = lane % 4) reads one 16-byte chunk (8 elements) per operand row and uses its
