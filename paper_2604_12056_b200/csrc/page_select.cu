@@ -322,12 +322,18 @@ struct RefineParams {
 // bounds); exact scores in the fixed order for the candidates (four lanes each), sort, emit.  More
 // than kSelCap candidates (possible only when most pages nearly tie): exact scores for every page
 // into the score row, then the plain threshold search.
-template <int D>
-__global__ void __launch_bounds__(kSelThreads, 6)
+// POOLED (one list per KV head, Section 4.2's selector with the group's maximum as the page score):
+// a CTA serves the G heads of a KV head at once.  max over the heads of the lower (upper) bounds is
+// a lower (upper) bound of the pooled score, so the same search applies to those; a candidate's
+// exact score is the largest of its G exact scores; the list goes to every head of the group.
+constexpr int kMaxPool = 16;     // heads per KV head the interface admits
+
+template <int D, bool POOLED>
+__global__ void __launch_bounds__(kSelThreads, POOLED ? 4 : 6)
 topk_refine_kernel(RefineParams p) {
   grid_dep_trigger();
   grid_dep_wait();
-  __shared__ __align__(16) float qs[2 * D];
+  __shared__ __align__(16) float qs[(POOLED ? kMaxPool : 1) * 2 * D];
   __shared__ __align__(16) unsigned long long ckey[kSelCap];
   __shared__ int cpage[kSelCap];
   __shared__ int hist[kSelBins];
@@ -335,7 +341,8 @@ topk_refine_kernel(RefineParams p) {
   __shared__ int s_ncand, s_bstar;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int qid = blockIdx.x;
-  const int h = qid % p.Hq, s = (qid / p.Hq) % p.N, j0 = qid / (p.Hq * p.N);
+  const int pool = POOLED ? p.Hq / p.Hkv : 1, Hl = p.Hq / pool;
+  const int h = (qid % Hl) * pool, s = (qid / Hl) % p.N, j0 = qid / (Hl * p.N);   // pooled: h = the group's first head
   if (p.step && p.step[s] == 0) return;
   int na = p.n_active[s];
   na = na > p.B ? p.B : na;
@@ -355,6 +362,30 @@ topk_refine_kernel(RefineParams p) {
     // the bounds of this thread's pages: one round trip, kept in registers when the prefix has at
     // most kSelThreads * kSelPerThread pages
     const bool cached = P <= kSelThreads * kSelPerThread;
+    if constexpr (POOLED) {
+      if (!cached) {
+        // the passes below read the row several times: pool once, into the group's first row (the
+        // rows are scratch, this CTA is their only reader, and a thread reads back only what it wrote)
+        constexpr int U = 4;                                   // pages per thread whose loads are in flight together
+        for (int p0 = tid; p0 < P; p0 += kSelThreads * U) {
+          float2 v[U];
+#pragma unroll
+          for (int e = 0; e < U; ++e) v[e] = p0 + e * kSelThreads < P ? row2[p0 + e * kSelThreads] : make_float2(0.f, 0.f);
+          for (int gi = 1; gi < pool; ++gi) {
+            float2 w[U];
+#pragma unroll
+            for (int e = 0; e < U; ++e)
+              w[e] = p0 + e * kSelThreads < P ? row2[static_cast<size_t>(gi) * p.score_stride + p0 + e * kSelThreads]
+                                              : make_float2(0.f, 0.f);
+#pragma unroll
+            for (int e = 0; e < U; ++e) { v[e].x = fmaxf(v[e].x, w[e].x); v[e].y = fmaxf(v[e].y, w[e].y); }
+          }
+#pragma unroll
+          for (int e = 0; e < U; ++e)
+            if (p0 + e * kSelThreads < P) row2[p0 + e * kSelThreads] = v[e];
+        }
+      }
+    }
     uint32_t lbc[kSelPerThread], ubc[kSelPerThread];
     if (cached) {
       float2 bv[kSelPerThread];
@@ -362,6 +393,21 @@ topk_refine_kernel(RefineParams p) {
       for (int i = 0; i < kSelPerThread; ++i) {
         const int pg = tid + kSelThreads * i;
         bv[i] = pg < P ? row2[pg] : make_float2(0.f, 0.f);
+      }
+      if constexpr (POOLED) {
+        for (int gi = 1; gi < pool; ++gi) {
+          float2 bg[kSelPerThread];
+#pragma unroll
+          for (int i = 0; i < kSelPerThread; ++i) {
+            const int pg = tid + kSelThreads * i;
+            bg[i] = pg < P ? row2[static_cast<size_t>(gi) * p.score_stride + pg] : make_float2(0.f, 0.f);
+          }
+#pragma unroll
+          for (int i = 0; i < kSelPerThread; ++i) {
+            bv[i].x = fmaxf(bv[i].x, bg[i].x);
+            bv[i].y = fmaxf(bv[i].y, bg[i].y);
+          }
+        }
       }
 #pragma unroll
       for (int i = 0; i < kSelPerThread; ++i) {
@@ -378,16 +424,17 @@ topk_refine_kernel(RefineParams p) {
         }
       } else {
         for (int pg = tid; pg < P; pg += kSelThreads) {
-          const float2 bv = row2[pg];
+          const float2 bv = row2[pg];                  // pooled: already the group's maximum
           f(order_bits(bv.x), order_bits(bv.y), pg);
         }
       }
     };
     // the query, split into its positive and negative parts
-    for (int j = tid; j < D; j += kSelThreads) {
+    for (int j = tid; j < pool * D; j += kSelThreads) {       // the group's heads are consecutive in q
       const float v = __bfloat162float(p.q[((static_cast<size_t>(s) * p.B + tok) * p.Hq + h) * D + j]);
-      qs[j] = fmaxf(v, 0.f);
-      qs[D + j] = fminf(v, 0.f);
+      const int gi = j / D, d = j % D;
+      qs[gi * 2 * D + d] = fmaxf(v, 0.f);
+      qs[gi * 2 * D + D + d] = fminf(v, 0.f);
     }
     if (tid == 0) s_ncand = 0;
     for (int b = tid; b < kSelBins; b += kSelThreads) hist[b] = 0;
@@ -451,7 +498,10 @@ topk_refine_kernel(RefineParams p) {
     };
     auto exact_at = [&](int ph) {                 // called by the four lanes of a group with the same page
       const size_t so = static_cast<size_t>(ph) * p.Hkv * D;
-      return exact_score4<D>(qs, lo_base + so, hi_base + so, u);
+      float e = exact_score4<D>(qs, lo_base + so, hi_base + so, u);
+      if constexpr (POOLED)
+        for (int gi = 1; gi < pool; ++gi) e = fmaxf(e, exact_score4<D>(qs + gi * 2 * D, lo_base + so, hi_base + so, u));
+      return e;
     };
     if (ncand > kSelCap) {
       float* row = reinterpret_cast<float*>(row2);             // the bounds are not needed any more
@@ -462,7 +512,7 @@ topk_refine_kernel(RefineParams p) {
       }
       __syncthreads();
       const RowView<false> rv{row, 1, p.score_stride};
-      topk_select_body<false>(rv, P, kk, p.k, out_pages, out_scores, 1);
+      topk_select_body<false>(rv, P, kk, p.k, out_pages, out_scores, pool);
       __syncthreads();
       continue;
     }
@@ -501,11 +551,14 @@ topk_refine_kernel(RefineParams p) {
         }
         for (int i = n4; i < ncand; ++i) rank += ckey[i] > mine ? 1 : 0;
         if (tid < ncand && rank < kk) {
-          out_pages[rank] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(mine));
-          if (out_scores) out_scores[rank] = unorder_bits(static_cast<uint32_t>(mine >> 32));
+          for (int gi = 0; gi < pool; ++gi) {
+            out_pages[gi * p.k + rank] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(mine));
+            if (out_scores) out_scores[gi * p.k + rank] = unorder_bits(static_cast<uint32_t>(mine >> 32));
+          }
         }
       }
-      for (int j = kk + tid; j < p.k; j += kSelThreads) out_pages[j] = -1;
+      for (int gi = 0; gi < pool; ++gi)
+        for (int j = kk + tid; j < p.k; j += kSelThreads) out_pages[gi * p.k + j] = -1;
     } else {
       int n2 = 2;
       while (n2 < ncand) n2 <<= 1;
@@ -522,13 +575,15 @@ topk_refine_kernel(RefineParams p) {
           __syncthreads();
         }
       }
-      for (int j = tid; j < p.k; j += kSelThreads) {
-        if (j < kk) {
-          const unsigned long long key = ckey[j];
-          out_pages[j] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(key));
-          if (out_scores) out_scores[j] = unorder_bits(static_cast<uint32_t>(key >> 32));
-        } else {
-          out_pages[j] = -1;
+      for (int gi = 0; gi < pool; ++gi) {
+        for (int j = tid; j < p.k; j += kSelThreads) {
+          if (j < kk) {
+            const unsigned long long key = ckey[j];
+            out_pages[gi * p.k + j] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(key));
+            if (out_scores) out_scores[gi * p.k + j] = unorder_bits(static_cast<uint32_t>(key >> 32));
+          } else {
+            out_pages[gi * p.k + j] = -1;
+          }
         }
       }
     }
@@ -700,8 +755,9 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
   const bool pooled = selector == kSelectorPooled;
   const int pool = pooled ? sh.n_q_heads / sh.n_kv_heads : 1;
   const bool bf = sh.dtype == LOSA_BF16;
-  if (bf && selector == kSelectorExact && k <= kSelCap) {
-    // bf16, one list per query head: bounds from the tensor cores, exact scores for the candidates only
+  if (bf && (selector == kSelectorExact || pooled) && k <= kSelCap) {
+    // bf16, exact lists (per query head, or per KV head from the group's maximum): bounds from the
+    // tensor cores, exact scores for the candidates only
     int32_t rc = launch_page_bounds(c, q, kv, active_idx, n_active, step, st, false, after_stage1);
     if (rc != LOSA_OK) return rc;
     RefineParams rp;
@@ -719,9 +775,14 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
     rp.status = status_ptr(c);
     rp.N = sh.batch; rp.B = sh.block_size; rp.Hq = sh.n_q_heads; rp.Hkv = sh.n_kv_heads; rp.g = sh.page_size;
     rp.k = k; rp.score_stride = c->lay.score_stride; rp.Pmax = sh.max_pages_per_seq; rp.n_phys = kv->n_phys_pages;
-    const int queries = sh.batch * std::min<int>(sh.block_size, kSelSlots) * sh.n_q_heads;
-    if (sh.head_dim == 128) launch_k(topk_refine_kernel<128>, queries, kSelThreads, 0, st, rp);
-    else launch_k(topk_refine_kernel<64>, queries, kSelThreads, 0, st, rp);
+    const int queries = sh.batch * std::min<int>(sh.block_size, kSelSlots) * (sh.n_q_heads / pool);
+    if (pool > 1) {
+      if (sh.head_dim == 128) launch_k(topk_refine_kernel<128, true>, queries, kSelThreads, 0, st, rp);
+      else launch_k(topk_refine_kernel<64, true>, queries, kSelThreads, 0, st, rp);
+    } else {
+      if (sh.head_dim == 128) launch_k(topk_refine_kernel<128, false>, queries, kSelThreads, 0, st, rp);
+      else launch_k(topk_refine_kernel<64, false>, queries, kSelThreads, 0, st, rp);
+    }
     return after_launch(c);
   }
   int32_t rc = selector == kSelectorMma ? launch_page_bounds(c, q, kv, active_idx, n_active, step, st, true, after_stage1)

@@ -157,10 +157,10 @@ def test_pooled_selector_whole_blocks(fused):
 
 
 @pytest.mark.parametrize("pooled", [True, False])
-@pytest.mark.parametrize("pages,topk", [(700, 600), (1100, 8), (1100, 600)])
+@pytest.mark.parametrize("pages,topk", [(700, 600), (1100, 8), (1300, 8), (1100, 600)])
 def test_long_lists_and_large_budgets(pages, topk, pooled):
     # k > 512 pages takes the whole-list sort; more than 1024 pages the selection that re-reads its
-    # score row instead of keeping it in registers: per-head lists and pooled lists go through both
+    # row of scores or bounds instead of keeping it in registers: per-head lists and pooled lists go through both
     cfg = wl.config("c2", n_q_heads=4, n_kv_heads=2, head_dim=64, page_size=16, kv_lens=(16 * pages,),
                     block_size=4, steps=2, topk=topk, m_active=2)
     run_blocks(cfg, pooled=pooled)
