@@ -641,3 +641,37 @@ def test_full_size_c5_layer_in_the_benchmark_configuration():
     phys = int(to_host(g.page_table)[5, 1024])
     np.testing.assert_array_equal(to_host(g.k_pages[phys, 3]), to_host(kb[5, :, 3]))
     np.testing.assert_array_equal(to_host(g.kmax[phys, 3]), to_host(kb[5, :, 3]).max(0))
+
+
+def test_full_size_c5_layer_with_pooled_lists():
+    """The same layer with one page list per (token, KV head): the LoSA step of the whole-step call
+    (bounds from the tensor cores, pooled over the four heads of a KV head, candidates refined with
+    exact scores) compared with the oracle in full.  The dense step only supplies the cached state."""
+    import torch
+    from paper_2604_12056_b200.layer import LosaLayer
+    cfg = wl.config("c5", n_blocks=2)
+    dw = wl.DeviceWorkload(cfg, replica=0, layer=5)
+    g = LosaLayer(cfg, dw.k_pages, dw.v_pages, dw.page_table, dw.kv_len, pooled=True)
+    d0, d1 = dw.start_block(), dw.next_step()
+    g.run_step_fused(d0.q, d0.k_blk, d0.v_blk, d0.m_per_seq)
+    torch.cuda.synchronize()
+    s0 = g.snapshot()
+    g.run_step_fused(d1.q, d1.k_blk, d1.v_blk, d1.m_per_seq)
+    torch.cuda.synchronize()
+    s1 = g.snapshot()
+    assert g.ctx.poll_status() == 0
+    o = OracleLayer(dw.host_copy(), pooled=True)
+    h0, h1 = d0.host_copy(), d1.host_copy()
+    o.o_p[:] = s0["o_p"]
+    o.lse_p[:] = s0["lse_p"]
+    o.q_prev[:] = h0.q
+    o.step[:] = 1
+    ref = o.run_step(h1)
+    s1["delta"] = ref["delta"]
+    compare(s1, ref, cfg, "c5 layer, pooled lists, LoSA step")
+    G = cfg.n_q_heads // cfg.n_kv_heads
+    lists = s1["topk"].reshape(cfg.batch, cfg.block_size, cfg.n_kv_heads, G, cfg.topk)
+    for s in range(cfg.batch):
+        for tok in ref["act"][s, :ref["na"][s]]:
+            assert (lists[s, tok] == lists[s, tok, :, :1]).all()      # one list per KV head
+    assert ref["uc"].sum() < 8 * 8 * 1024 // 4
