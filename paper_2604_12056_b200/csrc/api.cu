@@ -39,6 +39,9 @@ int32_t make_layout(const losa_shape_t* sh, int n_ctas, WorkspaceLayout* L) {
   L->counters = off; off = align_up(off + sizeof(uint32_t) * sh->batch, 256);
   L->seg_prefix = off; off = align_up(off + sizeof(int32_t) * (kMaxSegments + 1), 256);
   L->slot_map = off; off = align_up(off + sizeof(int32_t) * sh->batch * sh->block_size, 256);
+  L->union_bits = off;
+  off = align_up(off + sizeof(uint32_t) * static_cast<size_t>(sh->batch) * sh->n_kv_heads * ((sh->max_pages_per_seq + 31) / 32), 256);
+  L->union_tickets = off; off = align_up(off + sizeof(uint32_t) * sh->batch * sh->n_kv_heads, 256);
   L->delta = off;    off = align_up(off + sizeof(double) * sh->batch * sh->block_size, 256);
   L->scores = off;
   off = align_up(off + 2 * sizeof(float) * static_cast<size_t>(sh->batch) * sh->block_size * sh->n_q_heads * L->score_stride, 256);
@@ -126,7 +129,7 @@ int32_t losa_create(const losa_shape_t* shape, void* workspace, size_t workspace
   if (rc == LOSA_OK && workspace_bytes < c->lay.total) rc = LOSA_ERR_INVALID_ARG;
   if (rc == LOSA_OK && shape->max_pages_per_seq > topk_max_sortable(c)) rc = LOSA_ERR_UNSUPPORTED;
   if (rc != LOSA_OK) { delete c; return rc; }
-  // status word and arrival counters start at zero
+  // status word, arrival counters and page bitmaps start at zero
   e = cudaMemset(c->ws, 0, c->lay.delta);
   if (e != cudaSuccess) { delete c; return LOSA_ERR_CUDA; }
   *out = c;
@@ -334,8 +337,9 @@ int32_t losa_denoise_step(losa_ctx* ctx, const void* q, const void* k_blk, const
   int32_t* slot_map = reinterpret_cast<int32_t*>(ctx->ws + ctx->lay.slot_map);
   rc = launch_select_active(ctx, q, state->q_prev, sh.n_q_heads * sh.head_dim, m_per_seq, state->step,
                             buf->active_idx, buf->n_active, nullptr, st, 0.0, slot_map);
-  if (rc == LOSA_OK) rc = launch_page_scores_topk(ctx, q, kv, buf->active_idx, buf->n_active, state->step, k, buf->topk_pages, nullptr, st, ctx->pooled_selection, true);
-  if (rc == LOSA_OK) rc = launch_page_union(ctx, buf->topk_pages, buf->active_idx, buf->n_active, k, kv->kv_len, state->step, buf->union_pages, buf->union_count, st);
+  bool union_done = false;                              // stage 3 written by the selection kernel itself
+  if (rc == LOSA_OK) rc = launch_page_scores_topk(ctx, q, kv, buf->active_idx, buf->n_active, state->step, k, buf->topk_pages, nullptr, st, ctx->pooled_selection, true, buf->union_pages, buf->union_count, &union_done);
+  if (rc == LOSA_OK && !union_done) rc = launch_page_union(ctx, buf->topk_pages, buf->active_idx, buf->n_active, k, kv->kv_len, state->step, buf->union_pages, buf->union_count, st);
   if (rc == LOSA_OK) rc = launch_sparse_prefix_attn(ctx, q, kv, buf->active_idx, buf->n_active, buf->union_pages, buf->union_count, state, st, true);
   // join (also when a launch above failed: the forked kernel must not be left reading the caller's
   // buffers, nor a capture be left with an unjoined branch), then one pass over the rows: (merge of

@@ -22,6 +22,8 @@ struct WorkspaceLayout {
   size_t counters;   // uint32[N] : arrival counters of select_active (self-resetting)
   size_t seg_prefix; // int32[kMaxSegments + 1] : item prefix of the segments, left by the stage-4 main kernel for its combine kernel
   size_t slot_map;   // int32[N*B] : slot of every block token in the active list of the whole-step path, -1 = stable
+  size_t union_bits;    // uint32[N*H_kv*ceil(P_max/32)] : page bitmaps of the selection that also writes the union (all zero between launches)
+  size_t union_tickets; // uint32[N*H_kv] : its arrival counters (self-resetting)
   size_t delta;      // double[N*B]
   size_t scores;     // float[2*N*B*H_q*score_stride]: page scores, or (lower, upper) bound pairs of them
   size_t partials;   // float[n_slots * kRowsPerGroup * (d + 2)]

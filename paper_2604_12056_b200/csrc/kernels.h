@@ -13,7 +13,11 @@ int32_t launch_select_active(losa_ctx* c, const void* x_cur, const void* x_prev,
 int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
                                 const int32_t* active_idx, const int32_t* n_active,
                                 const int32_t* step, int32_t k, int32_t* topk_pages,
-                                float* topk_scores_opt, cudaStream_t st, int selector = 0, bool after_stage1 = false);
+                                float* topk_scores_opt, cudaStream_t st, int selector = 0, bool after_stage1 = false,
+                                int32_t* union_pages = nullptr, int32_t* union_count = nullptr, bool* union_done = nullptr);
+// union_pages / union_count / union_done (all three or none): where the selection can also write stage 3's
+// union (the bf16 candidate refinement, bitmaps of at most 256 words), it does so and sets *union_done;
+// otherwise *union_done is false and the caller launches stage 3 itself.
 // after_stage1: the kernel launched just before on `st` is stage 1 of the same step (see launch_page_bounds)
 // selector: 0 = one exact list per query head, 1 = pooled over the heads of a KV head, 2 = tensor-core scores (relaxed rule, bf16)
 constexpr int kSelectorExact = 0, kSelectorPooled = 1, kSelectorMma = 2;

@@ -6,6 +6,8 @@
 //                        64-bit keys (order-preserving score bits, inverted page id), see below.
 //   topk_kernel        : budgets above 512 pages: one CTA per query sorts all keys with a
 //                        shared-memory bitonic network.
+//   topk_refine_kernel : bf16, k <= 512 (the default): candidates from tensor-core bounds, exact scores
+//                        for those only; in the whole-step call it also writes stage 3's union.
 //   union_kernel       : one CTA per (sequence, KV head) ORs the selected ids into a bitmap and
 //                        emits the set bits in ascending order with a popcount scan.
 #include <algorithm>
@@ -314,7 +316,58 @@ struct RefineParams {
   float* topk_scores;
   int32_t* status;
   int N, B, Hq, Hkv, g, k, score_stride, Pmax, n_phys;
+  // stage 3 inside this kernel (whole-step call): the lists are ORed into one bitmap per (sequence, KV
+  // head) as they are emitted, and the last CTA of a (sequence, KV head) to finish writes the union.
+  // union_bits == nullptr: lists only.
+  uint32_t* union_bits;           // [N][Hkv][W] words, all zero between launches
+  unsigned int* union_tickets;    // [N][Hkv] arrival counters, self-resetting
+  int32_t* union_pages;
+  int32_t* union_count;
+  int W;                          // words per bitmap, ceil(Pmax / 32) <= kSelBins
 };
+
+// The set bits of a bitmap in shared memory, ascending, then -1 up to Pmax; the count.  All NT threads
+// of the CTA call it; s_warp: NT / 32 ints of shared memory.
+template <int NT>
+__device__ __forceinline__ void union_emit(const uint32_t* bitmap, int W, int Pmax, int32_t* __restrict__ out,
+                                           int32_t* __restrict__ count, int* s_warp) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // each thread owns a contiguous run of words; exclusive scan of the per-thread popcounts
+  const int per = (W + NT - 1) / NT;
+  const int w0 = tid * per, w1 = min(W, w0 + per);
+  int cnt = 0;
+  for (int w = w0; w < w1; ++w) cnt += __popc(bitmap[w]);
+  int inc = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xffffffffu, inc, o);
+    if (lane >= o) inc += t;
+  }
+  if (lane == 31) s_warp[warp] = inc;
+  __syncthreads();
+  int base = 0, total = 0;
+#pragma unroll
+  for (int w = 0; w < NT / 32; ++w) {
+    if (w < warp) base += s_warp[w];
+    total += s_warp[w];
+  }
+  int pos = base + inc - cnt;
+  for (int w = w0; w < w1; ++w) {
+    uint32_t v = bitmap[w];
+    while (v) {
+      const int b = __ffs(v) - 1;
+      v &= v - 1;
+      out[pos++] = w * 32 + b;
+    }
+  }
+  for (int t = total + tid; t < Pmax; t += NT) out[t] = -1;
+  if (tid == 0) *count = total;
+}
+
+__device__ __forceinline__ uint32_t prefix_word(int w, int P) {   // word w of the bitmap "pages 0 .. P-1"
+  const int lo = w * 32;
+  return (P >= lo + 32) ? 0xffffffffu : (P > lo ? ((1u << (P - lo)) - 1u) : 0u);
+}
 
 // One CTA of kSelThreads per (sequence, head, 1/8 of the active slots).  Per query: tau = lower edge
 // of the histogram bin that holds the k-th largest LOWER bound; every page whose UPPER bound reaches
@@ -343,12 +396,28 @@ topk_refine_kernel(RefineParams p) {
   const int qid = blockIdx.x;
   const int pool = POOLED ? p.Hq / p.Hkv : 1, Hl = p.Hq / pool;
   const int h = (qid % Hl) * pool, s = (qid / Hl) % p.N, j0 = qid / (Hl * p.N);   // pooled: h = the group's first head
-  if (p.step && p.step[s] == 0) return;
-  int na = p.n_active[s];
+  const int kh = h / (p.Hq / p.Hkv);
+  const bool first_step = p.step && p.step[s] == 0;
+  int na = first_step ? 0 : p.n_active[s];
   na = na > p.B ? p.B : na;
+  if (na <= 0) {
+    // no lists for this sequence: on the first step of a block the union is the whole prefix, with
+    // no active token it is empty; written by the first CTA of the (sequence, KV head)
+    if (!p.union_bits || j0 != 0 || h != kh * (p.Hq / p.Hkv)) return;
+    const int P0 = first_step ? min(pages_of(p.kv_len[s], p.g), p.Pmax) : 0;
+    uint32_t* bm = reinterpret_cast<uint32_t*>(hist);
+    for (int w = tid; w < p.W; w += kSelThreads) bm[w] = prefix_word(w, P0);
+    __syncthreads();
+    union_emit<kSelThreads>(bm, p.W, p.Pmax, p.union_pages + (static_cast<size_t>(s) * p.Hkv + kh) * p.Pmax,
+                            p.union_count + s * p.Hkv + kh, reinterpret_cast<int*>(s_red[0]));
+    return;
+  }
+  if (j0 >= na) return;                                  // no slot for this CTA
   int P = pages_of(p.kv_len[s], p.g);
   if (P > p.Pmax) { if (tid == 0) set_status(p.status, LOSA_ERR_BOUNDS); P = p.Pmax; }
-  const int kk = min(p.k, P), kh = h / (p.Hq / p.Hkv);
+  const int kk = min(p.k, P);
+  uint32_t* bits = p.union_bits ? p.union_bits + (static_cast<size_t>(s) * p.Hkv + kh) * p.W : nullptr;
+  auto mark = [&](int pg) { if (bits) atomicOr(&bits[pg >> 5], 1u << (pg & 31)); };
   const __nv_bfloat16* lo_base = p.kmin + static_cast<size_t>(kh) * D;
   const __nv_bfloat16* hi_base = p.kmax + static_cast<size_t>(kh) * D;
   const int u = lane & 3;
@@ -514,6 +583,8 @@ topk_refine_kernel(RefineParams p) {
       const RowView<false> rv{row, 1, p.score_stride};
       topk_select_body<false>(rv, P, kk, p.k, out_pages, out_scores, pool);
       __syncthreads();
+      if (bits)
+        for (int j = tid; j < kk; j += kSelThreads) mark(out_pages[j]);     // this CTA's own stores
       continue;
     }
     // a group of four lanes per candidate, 32 candidates per round; the physical page ids of four
@@ -551,10 +622,12 @@ topk_refine_kernel(RefineParams p) {
         }
         for (int i = n4; i < ncand; ++i) rank += ckey[i] > mine ? 1 : 0;
         if (tid < ncand && rank < kk) {
+          const int pg = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(mine));
           for (int gi = 0; gi < pool; ++gi) {
-            out_pages[gi * p.k + rank] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(mine));
+            out_pages[gi * p.k + rank] = pg;
             if (out_scores) out_scores[gi * p.k + rank] = unorder_bits(static_cast<uint32_t>(mine >> 32));
           }
+          mark(pg);
         }
       }
       for (int gi = 0; gi < pool; ++gi)
@@ -581,6 +654,7 @@ topk_refine_kernel(RefineParams p) {
             const unsigned long long key = ckey[j];
             out_pages[gi * p.k + j] = static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(key));
             if (out_scores) out_scores[gi * p.k + j] = unorder_bits(static_cast<uint32_t>(key >> 32));
+            if (gi == 0) mark(static_cast<int32_t>(0xffffffffu - static_cast<uint32_t>(key)));
           } else {
             out_pages[gi * p.k + j] = -1;
           }
@@ -589,6 +663,25 @@ topk_refine_kernel(RefineParams p) {
     }
     __syncthreads();                               // the shared state is reused by the next slot
   }
+  if (!bits) return;
+  // ---- stage 3: the last CTA of this (sequence, KV head) writes the union
+  __syncthreads();                                 // every thread's marks precede ...
+  if (tid == 0) {
+    __threadfence();                               // ... this fence (cumulative), which precedes the ticket
+    // CTAs of this (sequence, KV head) that hold a slot: all of them arrive here
+    const unsigned int n_grp = static_cast<unsigned int>((p.Hq / p.Hkv / pool) * min(na, static_cast<int>(gridDim.x) / (Hl * p.N)));
+    s_bstar = atomicInc(&p.union_tickets[s * p.Hkv + kh], n_grp - 1) == n_grp - 1 ? 1 : 0;
+  }
+  __syncthreads();
+  if (!s_bstar) return;
+  __threadfence();
+  uint32_t* bm = reinterpret_cast<uint32_t*>(hist);
+  for (int w = tid; w < p.W; w += kSelThreads) {
+    bm[w] = atomicExch(bits + w, 0u);              // the marks were made in L2; all zero again for the next launch
+  }
+  __syncthreads();
+  union_emit<kSelThreads>(bm, p.W, p.Pmax, p.union_pages + (static_cast<size_t>(s) * p.Hkv + kh) * p.Pmax,
+                          p.union_count + s * p.Hkv + kh, reinterpret_cast<int*>(s_red[0]));
 }
 
 template <bool POOLED>
@@ -651,18 +744,13 @@ union_kernel(const int32_t* __restrict__ topk_pages, const int32_t* __restrict__
   grid_dep_wait();
   extern __shared__ uint32_t bitmap[];
   __shared__ int s_warp[kThreads / 32];
-  const int kh = blockIdx.x, s = blockIdx.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int kh = blockIdx.x, s = blockIdx.y, tid = threadIdx.x;
   const int P = min(pages_of(kv_len[s], g), Pmax);
   const int W = (Pmax + 31) / 32;
   const int G = Hq / Hkv;
   const bool all = step && step[s] == 0;
   for (int w = tid; w < W; w += kThreads) {
-    uint32_t v = 0;
-    if (all) {
-      const int lo = w * 32;
-      v = (P >= lo + 32) ? 0xffffffffu : (P > lo ? ((1u << (P - lo)) - 1u) : 0u);
-    }
-    bitmap[w] = v;
+    bitmap[w] = all ? prefix_word(w, P) : 0u;
   }
   __syncthreads();
   if (!all) {
@@ -699,37 +787,8 @@ union_kernel(const int32_t* __restrict__ topk_pages, const int32_t* __restrict__
     }
     __syncthreads();
   }
-  // each thread owns a contiguous run of words; exclusive scan of the per-thread popcounts
-  const int per = (W + kThreads - 1) / kThreads;
-  const int w0 = tid * per, w1 = min(W, w0 + per);
-  int cnt = 0;
-  for (int w = w0; w < w1; ++w) cnt += __popc(bitmap[w]);
-  int inc = cnt;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int t = __shfl_up_sync(0xffffffffu, inc, o);
-    if (lane >= o) inc += t;
-  }
-  if (lane == 31) s_warp[warp] = inc;
-  __syncthreads();
-  int base = 0, total = 0;
-#pragma unroll
-  for (int w = 0; w < kThreads / 32; ++w) {
-    if (w < warp) base += s_warp[w];
-    total += s_warp[w];
-  }
-  int pos = base + inc - cnt;
-  int32_t* out = union_pages + (static_cast<size_t>(s) * Hkv + kh) * Pmax;
-  for (int w = w0; w < w1; ++w) {
-    uint32_t v = bitmap[w];
-    while (v) {
-      const int b = __ffs(v) - 1;
-      v &= v - 1;
-      out[pos++] = w * 32 + b;
-    }
-  }
-  for (int t = total + tid; t < Pmax; t += kThreads) out[t] = -1;
-  if (tid == 0) union_count[s * Hkv + kh] = total;
+  union_emit<kThreads>(bitmap, W, Pmax, union_pages + (static_cast<size_t>(s) * Hkv + kh) * Pmax,
+                       union_count + s * Hkv + kh, s_warp);
 }
 
 int pow2_at_least(int x) {
@@ -749,7 +808,9 @@ int32_t topk_max_sortable(const losa_ctx* c) {
 int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
                                 const int32_t* active_idx, const int32_t* n_active,
                                 const int32_t* step, int32_t k, int32_t* topk_pages,
-                                float* topk_scores_opt, cudaStream_t st, int selector, bool after_stage1) {
+                                float* topk_scores_opt, cudaStream_t st, int selector, bool after_stage1,
+                                int32_t* union_pages, int32_t* union_count, bool* union_done) {
+  if (union_done) *union_done = false;
   const losa_shape_t& sh = c->shape;
   if (sh.max_pages_per_seq == 0) return LOSA_OK;
   const bool pooled = selector == kSelectorPooled;
@@ -775,6 +836,13 @@ int32_t launch_page_scores_topk(losa_ctx* c, const void* q, const losa_kv_t* kv,
     rp.status = status_ptr(c);
     rp.N = sh.batch; rp.B = sh.block_size; rp.Hq = sh.n_q_heads; rp.Hkv = sh.n_kv_heads; rp.g = sh.page_size;
     rp.k = k; rp.score_stride = c->lay.score_stride; rp.Pmax = sh.max_pages_per_seq; rp.n_phys = kv->n_phys_pages;
+    rp.W = (sh.max_pages_per_seq + 31) / 32;
+    const bool with_union = union_pages && union_count && union_done && rp.W <= kSelBins;
+    rp.union_bits = with_union ? reinterpret_cast<uint32_t*>(c->ws + c->lay.union_bits) : nullptr;
+    rp.union_tickets = reinterpret_cast<unsigned int*>(c->ws + c->lay.union_tickets);
+    rp.union_pages = union_pages;
+    rp.union_count = union_count;
+    if (with_union) *union_done = true;
     const int queries = sh.batch * std::min<int>(sh.block_size, kSelSlots) * (sh.n_q_heads / pool);
     if (pool > 1) {
       if (sh.head_dim == 128) launch_k(topk_refine_kernel<128, true>, queries, kSelThreads, 0, st, rp);

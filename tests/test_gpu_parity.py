@@ -271,6 +271,36 @@ def test_sequences_without_active_tokens_beside_others(fused):
             assert ref["na"].tolist() == [0, 3, 1, 0]
 
 
+@pytest.mark.parametrize("pooled", [False, True])
+@pytest.mark.parametrize("fused", [False, True])
+def test_sequences_on_different_steps_in_one_batch(fused, pooled):
+    # the step counter is per sequence: after two steps, sequences 0 and 2 are put back on a first step
+    # (every token active, union = whole prefix) while 1 and 3 go on with lists; then all continue
+    from paper_2604_12056_b200.layer import LosaLayer, to_device
+    cfg = wl.config("c2", kv_lens=(40 * 32 + 5, 300, 70 * 32, 64), block_size=16, steps=5, topk=6, m_active=3)
+    w = wl.Workload(cfg)
+    g, o = LosaLayer(cfg, w.k_pages, w.v_pages, w.page_table, w.kv_len, pooled=pooled), OracleLayer(w, pooled=pooled)
+    for t, inp in enumerate(w.block_steps()):
+        if t == 2:
+            g.step[0] = 0
+            g.step[2] = 0
+            o.step[[0, 2]] = 0
+        args = tuple(to_device(x) for x in (inp.q, inp.k_blk, inp.v_blk, inp.m_per_seq))
+        if fused:
+            g.run_step_fused(*args)
+        else:
+            g.run_step(*args)
+        snap, ref = g.snapshot(), o.run_step(inp)
+        assert g.ctx.poll_status() == 0
+        if fused:
+            snap["delta"] = ref["delta"]
+        compare(snap, ref, cfg, f"staggered steps, step {t}")
+        if t == 2:
+            assert ref["na"].tolist() == [16, 3, 16, 3]
+            P = [(L + 31) // 32 for L in cfg.kv_lens]
+            assert (ref["uc"][0] == P[0]).all() and (ref["uc"][2] == P[2]).all() and (ref["uc"][1] <= P[1]).all()
+
+
 @pytest.mark.parametrize("fused", [False, True])
 def test_state_stored_in_bf16(fused):
     # the cached prefix output stored rounded to bf16: the oracle rounds the rows stage 4 writes, and
