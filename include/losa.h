@@ -360,7 +360,8 @@ typedef struct {
  * out / lse_out_opt what stage 5 produces; q_prev and step are updated as by stage 6.
  * Being one call, it may schedule freely inside: the in-block attention of stage 5 (which needs
  * nothing from stages 1-4) runs on a second stream owned by the context and is joined before a
- * final merge kernel that also keeps the queries.  All work is ordered after prior work on
+ * final merge kernel that also keeps the queries; where stage 2 runs the candidate refinement
+ * (bf16, k <= 512) that kernel also writes stage 3's union.  All work is ordered after prior work on
  * `stream` and complete when `stream` reaches the end of the call's work; the call can be captured
  * in a CUDA graph after one un-captured call on the context (which creates the second stream). */
 int32_t losa_denoise_step(losa_ctx* ctx, const void* q, const void* k_blk, const void* v_blk, void* out,
