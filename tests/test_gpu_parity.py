@@ -166,6 +166,15 @@ def test_long_lists_and_large_budgets(pages, topk, pooled):
     run_blocks(cfg, pooled=pooled)
 
 
+def test_whole_step_call_beyond_the_bitmap_of_the_selection_kernel():
+    # more than 8,192 pages per sequence: the whole-step call's selection kernel leaves stage 3 to the
+    # union kernel (its bitmap holds 256 words); lists, union and attention as usual
+    cfg = wl.config("c2", n_q_heads=4, n_kv_heads=2, head_dim=64, page_size=16, kv_lens=(16 * 8300 + 3,),
+                    block_size=4, steps=2, topk=8, m_active=2)
+    assert cfg.max_pages_per_seq > 8192
+    run_blocks(cfg, modes=("losa",), fused=True, want_scores=False)
+
+
 @pytest.mark.parametrize("kw", [
     dict(kv_lens=(2048, 1500), steps=4),
     dict(n_q_heads=4, n_kv_heads=2, head_dim=64, page_size=16, kv_lens=(16 * 1100 + 5, 700), block_size=8, steps=3, topk=8,
